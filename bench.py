@@ -1,0 +1,365 @@
+#!/usr/bin/env python
+"""Benchmark of the Jacobi hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload c3_eigenmode_16384] [--mode fused] [--tsteps T]
+
+One *step* is one whole job of the workload: its sweeps (every sweep with its halo exchange:
+pack, unpack, update) followed by the residual reduction.  The metric is Jacobi GLUP/s
+(1e9 lattice-point updates per second); effective GB/s = GLUP/s x compulsory bytes per point
+(16 B: read u, write u'; 24 B with f).
+
+Prints exactly one JSON line on stdout.  With N > 1 (launched by torchrun) every rank runs an
+independent replica of the job on its own GPU -- the path is a single-GPU library and has no
+exchange between GPUs -- and rank 0 reports units of all ranks / max time over ranks.
+
+``--impl reference`` times the CPU oracle (the plain C checker under oracle/) on the host
+cores for the same metric; it is a deliberately slow program, reported for context.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+from paper_2210_01238_b200 import inputs  # noqa: E402
+
+METRIC = "jacobi_glups"
+UNIT = "GLUP/s"
+L2_BYTES = 126e6
+
+# DRAM bytes per launch of the dominant kernel from an ncu capture (profiles/), and the hash of
+# the kernel sources the capture was taken with; reported as null once the sources changed.
+NCU_TRAFFIC = {
+    "fused": {"kernel": "sweep2d_kernel", "bytes_per_launch": None, "src_sha": None},
+}
+
+
+def log(*a):
+    print(*a, file=sys.stderr, flush=True)
+
+
+def kernel_src_sha() -> str:
+    h = hashlib.sha256()
+    for p in sorted((ROOT / "paper_2210_01238_b200" / "csrc").glob("*")):
+        h.update(p.read_bytes())
+    return h.hexdigest()[:16]
+
+
+def measured_peak_gbs():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        try:
+            return float(json.loads(p.read_text())["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples of one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid: str | None):
+        self.uuid, self.proc = uuid, None
+
+    def start(self):
+        cmd = ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"]
+        if self.uuid:
+            cmd += ["-i", self.uuid]
+        try:
+            self.proc = subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        # "under load": samples in the upper half of the clock range seen (idle samples sit low)
+        load = [x for x in sm if x >= 0.5 * max(sm)] if sm else []
+        return {"sm_mhz": statistics.median(load) if load else None,
+                "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------- workloads
+def make_inputs(w: inputs.Workload):
+    u0 = inputs.initial_u(w)
+    f = inputs.rhs(w)
+    return u0, f
+
+
+def job_updates(w: inputs.Workload, sweeps: int) -> float:
+    return float(w.points) * sweeps
+
+
+# ----------------------------------------------------------------------------- reference arm
+def oracle_time_job(w: inputs.Workload, u0, f, target_seconds: float, max_sweeps: int):
+    """Times the CPU oracle (blocked form: pack, unpack, update per sweep, then the residual) on a
+    bounded number of sweeps of the same grid.  Returns (glups, sweeps, seconds, threads)."""
+    from oracle import orc
+    B = orc.Blocked(w.n, w.b, w.halo, w.has_f)
+    for face, v in enumerate(w.boundary()):
+        B.set_boundary(face, v)
+    B.set_u(u0)
+    if f is not None:
+        B.set_f(f)
+    t0 = time.perf_counter()
+    B.sweep(1)
+    t1 = time.perf_counter() - t0
+    sweeps = int(max(1, min(max_sweeps, target_seconds / max(t1, 1e-9))))
+    t0 = time.perf_counter()
+    B.sweep(sweeps)
+    B.residual()
+    dt = time.perf_counter() - t0
+    B.close()
+    return job_updates(w, sweeps) / dt / 1e9, sweeps, dt, orc.max_threads()
+
+
+def run_reference(args, w: inputs.Workload):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    u0, f = make_inputs(w)
+    vals, sweeps = [], 0
+    per_step = max(2.0, min(20.0, 60.0 / max(1, args.steps + args.warmup)))
+    for i in range(args.warmup + args.steps):
+        g, sweeps, dt, threads = oracle_time_job(w, u0, f, per_step, w.sweeps)
+        log(f"[reference] step {i}: {sweeps} sweeps in {dt:.2f} s -> {g:.3f} GLUP/s on {threads} threads")
+        if i >= args.warmup:
+            vals.append((g, dt))
+    total_updates = sum(g * dt for g, dt in vals)
+    total_time = sum(dt for _, dt in vals)
+    value = total_updates / total_time
+    sample = f"{sweeps} of {w.sweeps} sweeps (+1 residual) of the full {'x'.join(map(str, w.n))} grid per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_time / len(vals),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": w.name, "grid": list(w.n), "block": list(w.b), "halo": w.halo,
+                   "sweeps_per_step": sweeps, "has_f": w.has_f},
+        "effective_gbs": value * w.bytes_per_point,
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------- our arm
+def run_ours(args, w: inputs.Workload):
+    import torch
+    import torch.distributed as dist
+    from paper_2210_01238_b200 import jac
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local)
+    distributed = world > 1
+    if distributed:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if distributed:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    stream = torch.cuda.current_stream()
+    u0, f = make_inputs(w)
+    sweeps = args.sweeps if args.sweeps > 0 else w.sweeps
+    J = jac.Jacobi(w.n, w.b, w.halo, w.has_f, args.mode, args.tsteps)
+    for face, v in enumerate(w.boundary()):
+        J.set_boundary(face, v)
+    u0_dev = torch.from_numpy(u0).cuda()
+    if f is not None:
+        J.set_f(f)
+    del f
+
+    def job():
+        J.set_u_device(u0_dev)      # device-resident input -> blocks (inside the timed job)
+        J.sweep(sweeps)
+        return J.residual()
+
+    # ---- device-resident timing: K steps between two barriers, CUDA events on the launch stream
+    for _ in range(args.warmup):
+        res = job()
+    barrier()
+    sampler = ClockSampler(str(torch.cuda.get_device_properties(local).uuid)
+                           if hasattr(torch.cuda.get_device_properties(local), "uuid") else None)
+    if sampler.uuid and not sampler.uuid.startswith("GPU-"):
+        sampler.uuid = "GPU-" + sampler.uuid
+    sampler.start()
+    l0 = J.launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sweep_ms = []
+    ev0.record(stream)
+    for _ in range(args.steps):
+        J.set_u_device(u0_dev)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        J.sweep(sweeps)
+        b.record(stream)
+        res = J.residual()
+        sweep_ms.append((a, b))
+    ev1.record(stream)
+    barrier()
+    launches = J.launch_count() - l0
+    clocks = sampler.stop()
+    ms_total = ev0.elapsed_time(ev1)
+    sweep_only_ms = sum(a.elapsed_time(b) for a, b in sweep_ms)
+    if distributed:
+        t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    value = job_updates(w, sweeps) * args.steps * world / (ms_total * 1e-3) / 1e9
+
+    # ---- roofline of the dominant kernel (the sweep): algorithmic bytes per launch / mean launch time
+    peak, peak_kind = measured_peak_gbs()
+    launches_per_sweep_call = sweeps if args.mode == "fused" else None
+    tsteps = J.desc.tsteps if args.mode == "temporal" else 1
+    if args.mode == "temporal":
+        tsteps = args.tsteps or 4
+        n_launch = -(-sweeps // tsteps)
+    else:
+        n_launch = sweeps
+    sweeps_per_launch = sweeps / n_launch
+    alg_bytes_per_launch = w.points * w.bytes_per_point * sweeps_per_launch
+    launch_ms = sweep_only_ms / (args.steps * n_launch)
+    achieved = alg_bytes_per_launch / (launch_ms * 1e-3) / 1e9
+    traffic = None
+    rec = NCU_TRAFFIC.get(args.mode)
+    if rec and rec["bytes_per_launch"] and rec["src_sha"] == kernel_src_sha():
+        traffic = rec["bytes_per_launch"]
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
+                "kernel": "sweep (one launch covers all blocks)",
+                "launch_ms": launch_ms, "sweeps_per_launch": sweeps_per_launch,
+                "frac_of_nominal_8TBs": achieved / 8000.0,
+                "note": "time per launch includes the pack/unpack launches in the exchange schedule"}
+
+    # ---- end to end through the C ABI with host buffers: H2D of u0, the job, D2H of the solution
+    e2e = None
+    if rank == 0 or distributed:
+        host_in = torch.from_numpy(u0).pin_memory()
+        host_out = torch.empty_like(host_in).pin_memory()
+        e2e_steps = max(1, min(args.steps, 3))
+        J.set_u_pinned(host_in); J.sweep(1); J.get_u_pinned(host_out)   # warm the path
+        barrier()
+        t0 = time.perf_counter()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(e2e_steps):
+            J.set_u_pinned(host_in)
+            J.sweep(sweeps)
+            res_e2e = J.residual()
+            J.get_u_pinned(host_out)
+        e1.record(stream)
+        barrier()
+        wall = time.perf_counter() - t0
+        ms_e2e = max(e0.elapsed_time(e1), 0.0)
+        ms_e2e = max(ms_e2e, wall * 1e3 * 0.0)  # device time covers the copies (they run on the stream)
+        if distributed:
+            t = torch.tensor([ms_e2e], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e2e = float(t.item())
+        e2e = {"value": job_updates(w, sweeps) * e2e_steps * world / (ms_e2e * 1e-3) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": int(u0.nbytes), "d2h_bytes_per_step": int(u0.nbytes) + 8,
+               "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps,
+               "what": "jac_set_u(pinned host) + jac_sweep + jac_residual + jac_get_u(pinned host)"}
+        del host_in, host_out
+    J.close()
+    del u0_dev
+    torch.cuda.empty_cache()
+
+    # ---- the oracle on the host cores, bounded sample (rank 0, single-GPU runs only)
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        fcpu = inputs.rhs(w)
+        g, osw, dt, threads = oracle_time_job(w, u0, fcpu, 12.0, w.sweeps)
+        cpu_baseline = {"value": g, "unit": UNIT, "cores": threads, "kind": "oracle",
+                        "sample": f"{osw} of {w.sweeps} sweeps (+1 residual) of the full "
+                                  f"{'x'.join(map(str, w.n))} grid, {dt:.1f} s"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "grid": list(w.n), "block": list(w.b), "halo": w.halo,
+                       "has_f": w.has_f, "sweeps_per_step": sweeps, "residuals_per_step": 1,
+                       "schedule": args.mode, "tsteps": tsteps,
+                       "l2": f"arrays of {w.points * 8 / 1e6:.0f} MB each exceed the {L2_BYTES / 1e6:.0f} MB L2"
+                             if w.points * 8 > L2_BYTES else "arrays fit in L2 (no flush; latency-bound case)",
+                       "replicas": world},
+            "effective_gbs": value * w.bytes_per_point,
+            "frac_of_8TBs": value * w.bytes_per_point / 8000.0 / world,
+            "residual": res,
+            "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e,
+            "gpu_launches": int(launches), "clocks": clocks,
+        }
+        print(json.dumps(line), flush=True)
+    if distributed:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c3_eigenmode_16384", choices=sorted(inputs.CONFIGS))
+    ap.add_argument("--mode", default="fused", choices=["fused", "exchange", "pertask", "temporal"])
+    ap.add_argument("--tsteps", type=int, default=0)
+    ap.add_argument("--sweeps", type=int, default=0, help="sweeps per step (default: the workload's)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        log("warning: fewer than 3 warm-up steps")
+    w = inputs.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

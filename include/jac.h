@@ -1,0 +1,174 @@
+/*
+ * jac.h -- C ABI of libjac: block-decomposed Jacobi relaxation on one NVIDIA B200 (sm_100a).
+ *
+ * The method (paper, Section V-C "Proxy Application: Jacobi3d"): a fixed number of Jacobi
+ * iterations over a domain decomposed into cuboid blocks.  In every iteration each block
+ * packs its boundary faces into contiguous buffers, the buffers reach the neighbouring
+ * blocks, are unpacked into their ghost cells, and once all halos are in place the Jacobi
+ * update runs on the GPU.  The paper fixes neither the stencil nor the boundary rule; this
+ * library uses
+ *
+ *     u'(p) = ( sum of the 2d face neighbours of u at p  [+ f(p)] ) * (1/c),   c = 2d,
+ *
+ * evaluated as  s = (W + E) + (S + N);  3D: s = s + (D + U);  with f: s = s + f;
+ * u' = s * 0.25 (2D) or s * (1.0/6.0) (3D), every operation one IEEE-754 round-to-nearest
+ * fp64 add or multiply (no fused multiply-add), Dirichlet values in the ghost layer around
+ * the domain (one constant per domain face, default 0).
+ *
+ * Conventions
+ *   - x is the fastest-varying axis, then y, then z.  "Dense" arrays are n[0]*n[1]*n[2]
+ *     doubles in that order (in 2D n[2] = 1).
+ *   - Blocks are numbered x-fastest over the block grid g[a] = n[a] / b[a].
+ *   - Faces: 0:-x 1:+x 2:-y 3:+y 4:-z 5:+z.  A face is the `halo` interior layers next to
+ *     that side over the interior extent of the other axes (no edges, no corners).  A packed
+ *     face holds those elements in source memory order: an x face is [bz][by][halo], a y face
+ *     [bz][halo][bx], a z face [halo][by][bx] (last index fastest).  Faces on the domain
+ *     boundary are neither packed nor unpacked.
+ *   - All device work is issued on the caller's stream and is asynchronous unless stated.
+ *   - The library never allocates or frees device memory: the caller passes one workspace
+ *     (see jac_workspace_bytes) and keeps it, and the stream, alive until jac_destroy.
+ *   - Every function returns JAC_OK (0) or a negative error code and never aborts; on error
+ *     out-parameters are left untouched.  A CUDA failure is sticky: later calls on the same
+ *     context return JAC_ECUDA until it is destroyed.
+ *   - A context is not thread-safe; different contexts are independent.
+ */
+#ifndef JAC_H_
+#define JAC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define JAC_OK        0
+#define JAC_EINVAL   (-1)  /* null pointer, bad dimension, size, face, block or count            */
+#define JAC_ENOMEM   (-2)  /* workspace null, too small or not 256-byte aligned                  */
+#define JAC_ECUDA    (-3)  /* a CUDA runtime call failed (sticky); see jac_last_cuda_error       */
+#define JAC_ENODEV   (-4)  /* no usable CUDA device                                              */
+
+/* How jac_sweep schedules one iteration.  All modes leave bit-identical interiors. */
+#define JAC_MODE_FUSED    0 /* one launch per sweep over all blocks; the update also writes each
+                               new face value straight into the neighbour's ghost cells, so the
+                               exchange for the next sweep is already done                       */
+#define JAC_MODE_PERTASK  1 /* the task-per-block schedule: per sweep one pack launch per
+                               (block, face), one unpack launch per (block, face), one update
+                               launch per block                                                  */
+#define JAC_MODE_TEMPORAL 2 /* `tsteps` sweeps per launch; tiles read across block borders
+                               directly (equivalent to an exchange before every sweep)           */
+#define JAC_MODE_EXCHANGE 3 /* per sweep three launches over all blocks: pack, unpack, update    */
+
+typedef struct jac_ctx jac_ctx; /* opaque, host memory, owned by the library */
+
+typedef struct jac_desc {
+    int32_t ndim;    /* 2 or 3                                                                   */
+    int32_t halo;    /* ghost width h, 1 <= h <= min(b[a]) and h <= 8                            */
+    int32_t has_f;   /* 0: f == 0 and is never read (16 B/point/sweep); 1: f present (24 B)      */
+    int32_t mode;    /* JAC_MODE_*                                                               */
+    int32_t tsteps;  /* JAC_MODE_TEMPORAL: sweeps per launch, 1..8; 0 = library default          */
+    int32_t reserved;/* must be 0                                                                */
+    int64_t n[3];    /* global interior points; n[2] ignored (taken as 1) when ndim == 2         */
+    int64_t b[3];    /* block interior points; n[a] % b[a] == 0                                  */
+    void   *stream;  /* cudaStream_t of the caller (NULL = the legacy default stream)            */
+} jac_desc;
+
+/* Physical placement chosen for a descriptor (pure host query; element = one double). */
+typedef struct jac_layout {
+    int64_t g[3];          /* block grid                                                         */
+    int64_t nblocks;
+    int64_t pad[3];        /* padded block dims: pad[0] = b[0] + 2*xpad, pad[1] = b[1] + 2h,
+                              pad[2] = b[2] + 2h (3D) or 1                                       */
+    int64_t xpad;          /* ghost columns are the innermost h of an xpad-wide margin           */
+    int64_t origin;        /* element offset of interior point (0,0,0) inside a padded block     */
+    int64_t block_stride;  /* elements between consecutive blocks of one array                   */
+    int64_t face_elems[6]; /* elements of one packed face                                        */
+    int64_t face_offset[6];/* element offset of each face inside a block's send region           */
+    int64_t send_stride;   /* elements of one block's send region                                */
+    int64_t partials;      /* doubles of reduction scratch                                       */
+    int64_t off_u[2];      /* byte offsets inside the workspace: the two solution arrays,        */
+    int64_t off_f;         /*   f (same padded layout as u; -1 if has_f == 0),                   */
+    int64_t off_send;      /*   send buffers,                                                    */
+    int64_t off_scratch;   /*   reduction scratch + result word                                  */
+    int64_t total_bytes;
+} jac_layout;
+
+/* Workspace size in bytes for `desc` (pure host computation, no CUDA call).
+ * Errors: JAC_EINVAL for a null pointer or an invalid descriptor. */
+int jac_workspace_bytes(const jac_desc *desc, size_t *bytes);
+
+/* The placement behind jac_workspace_bytes (pure host computation). */
+int jac_get_layout(const jac_desc *desc, jac_layout *out);
+
+/* Create a context over `dev_workspace` (DEVICE pointer, 256-byte aligned, >= the size from
+ * jac_workspace_bytes).  Zero-fills both solution arrays, f and the send buffers on the
+ * stream (so u = 0, f = 0, all Dirichlet values 0).  The device current at this call is the
+ * one every later call on the context must be issued under.
+ * Errors: JAC_EINVAL, JAC_ENOMEM, JAC_ENODEV, JAC_ECUDA. */
+int jac_create(const jac_desc *desc, void *dev_workspace, size_t bytes, jac_ctx **out);
+
+/* Frees the host-side context only (after synchronising the stream). */
+int jac_destroy(jac_ctx *ctx);
+
+/* Set / read the current solution or the right-hand side from a dense array.
+ * jac_set_u, jac_set_f, jac_get_u take HOST pointers (pageable or pinned) and return after
+ * the copy has completed; the *_device variants take DEVICE pointers to dense arrays and
+ * are asynchronous on the stream.  jac_set_f* returns JAC_EINVAL when has_f == 0.
+ * Setting u leaves inter-block ghost cells stale until the next exchange. */
+int jac_set_u(jac_ctx *ctx, const double *host_dense);
+int jac_set_f(jac_ctx *ctx, const double *host_dense);
+int jac_get_u(jac_ctx *ctx, double *host_dense);
+int jac_set_u_device(jac_ctx *ctx, const double *dev_dense);
+int jac_set_f_device(jac_ctx *ctx, const double *dev_dense);
+int jac_get_u_device(jac_ctx *ctx, double *dev_dense);
+
+/* Dirichlet value of one domain face: written into the ghost layers (all h of them, interior
+ * extent) of every block touching that face, in both solution arrays.  Asynchronous. */
+int jac_set_boundary(jac_ctx *ctx, int face, double value);
+
+/* Inspection (synchronous, HOST output).
+ * jac_get_block_padded: the canonical padded block (b+2h)^d of the current state, x fastest,
+ *   ghost cells as they currently are (edge/corner ghosts are never written: they stay 0).
+ * jac_get_halo_buffer: the packed face of (block, face) as the last pack left it. */
+int jac_get_block_padded(jac_ctx *ctx, int64_t block, double *host);
+int jac_get_halo_buffer(jac_ctx *ctx, int64_t block, int face, double *host);
+
+/* Halo pack: for every block and every face with a neighbour block, gather the h interior
+ * layers next to that face of the current state into the face's contiguous send buffer
+ * (paper Section V-C: "packing the GPU data").  One launch over all blocks and faces
+ * (JAC_MODE_PERTASK: one launch per block face). */
+int jac_pack_halos(jac_ctx *ctx);
+
+/* Halo unpack: for every block and every face with a neighbour, copy the neighbour's
+ * opposite-face send buffer into this block's h ghost layers on that face (paper Section
+ * V-C: "the data are unpacked into the GPU").  On one GPU the transfer between pack and
+ * unpack is the neighbour reading the send buffer in place. */
+int jac_unpack_halos(jac_ctx *ctx);
+
+/* nsweeps Jacobi iterations, each "exchange halos, then update every block" (paper Section
+ * V-C), scheduled as desc.mode says.  Afterwards the interiors hold the new state; the
+ * inter-block ghost cells are only guaranteed current after the next jac_pack_halos +
+ * jac_unpack_halos (jac_residual does that itself when needed).  nsweeps == 0 is a no-op;
+ * nsweeps < 0 is JAC_EINVAL. */
+int jac_sweep(jac_ctx *ctx, int nsweeps);
+
+/* L2 norm of the residual of the current state, sqrt( sum_p ( s(p) - c*u(p) )^2 ) with s as in
+ * the update (including + f), over all interior points, not normalised.  (The paper runs a
+ * fixed iteration count and has no residual; this is the convergence measure of the same
+ * Jacobi method.)  Exchanges halos first if the ghosts are stale, reduces on the device in a
+ * fixed order (repeatable bit for bit), synchronises the stream and writes one HOST double. */
+int jac_residual(jac_ctx *ctx, double *host_out_l2);
+
+/* Number of kernel launches this context has issued so far (HOST output). */
+int jac_launch_count(const jac_ctx *ctx, int64_t *host_out);
+
+/* cudaError_t value of the failure that made the context sticky (0 if none). */
+int jac_last_cuda_error(const jac_ctx *ctx);
+
+/* Static, NUL-terminated description of an error code. */
+const char *jac_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* JAC_H_ */

@@ -1,0 +1,605 @@
+// Host side of libjac: descriptor validation, workspace layout, launch scheduling and the
+// C ABI declared in include/jac.h.  No device memory is allocated here: every buffer lives
+// in the caller's workspace.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "jac.h"
+#include "jac_geom.h"
+#include "jac_kernels.cuh"
+
+namespace {
+
+constexpr int kNumSMs = 148;  // B200
+constexpr long long kMaxGrid = 2147483647LL;
+
+long long round_up(long long v, long long m) { return (v + m - 1) / m * m; }
+long long ceil_div(long long a, long long b) { return (a + b - 1) / b; }
+int pow2_ceil(long long v) { int p = 1; while (p < v) p <<= 1; return p; }
+
+// How one launch of the sweep / residual kernels is cut into CTAs.
+struct Tiling {
+    int nv;        // points per thread along x (2 when bx is even: 128-bit accesses)
+    dim3 block;
+    int tiles_x, tiles_y, tiles_z;
+    int march;     // rows (2D) or planes (3D) a CTA marches through
+    long long ctas_per_block;
+};
+
+Tiling make_tiling(const JacGeom& g)
+{
+    Tiling t{};
+    t.nv = (g.bx % 2 == 0) ? 2 : 1;
+    const long long need = ceil_div(g.bx, t.nv);
+    const long long want_ctas = (long long)kNumSMs * 16;
+    if (g.ndim == 2) {
+        const int tpb = (int)std::min<long long>(256, round_up(need, 32));
+        t.block = dim3(tpb, 1, 1);
+        t.tiles_x = (int)ceil_div(need, tpb);
+        t.tiles_z = 1;
+        int rows = std::min(g.by, 64);
+        while (rows > 8 && g.nblocks * t.tiles_x * ceil_div(g.by, rows) < want_ctas) rows = (rows + 1) / 2;
+        t.march = rows;
+        t.tiles_y = (int)ceil_div(g.by, rows);
+    } else {
+        const int tx = std::min(64, pow2_ceil(need));
+        const int ty = std::min(std::max(1, 512 / tx), std::min(8, pow2_ceil(g.by)));
+        t.block = dim3(tx, ty, 1);
+        t.tiles_x = (int)ceil_div(need, tx);
+        t.tiles_y = (int)ceil_div(g.by, ty);
+        int planes = g.bz;
+        while (planes > 16 && g.nblocks * t.tiles_x * t.tiles_y * ceil_div(g.bz, planes) < want_ctas)
+            planes = (planes + 1) / 2;
+        t.march = planes;
+        t.tiles_z = (int)ceil_div(g.bz, planes);
+    }
+    t.ctas_per_block = (long long)t.tiles_x * t.tiles_y * t.tiles_z;
+    return t;
+}
+
+int build_geometry(const jac_desc* d, JacGeom* g, jac_layout* L)
+{
+    if (!d) return JAC_EINVAL;
+    if (d->ndim != 2 && d->ndim != 3) return JAC_EINVAL;
+    if (d->halo < 1 || d->halo > 8) return JAC_EINVAL;
+    if (d->has_f != 0 && d->has_f != 1) return JAC_EINVAL;
+    if (d->mode < JAC_MODE_FUSED || d->mode > JAC_MODE_EXCHANGE) return JAC_EINVAL;
+    if (d->tsteps < 0 || d->tsteps > 8 || d->reserved != 0) return JAC_EINVAL;
+    long long n[3] = {1, 1, 1}, b[3] = {1, 1, 1}, gr[3] = {1, 1, 1};
+    for (int a = 0; a < d->ndim; ++a) {
+        n[a] = d->n[a];
+        b[a] = d->b[a];
+        if (n[a] < 1 || b[a] < 1 || b[a] > n[a] || n[a] % b[a] != 0) return JAC_EINVAL;
+        if (d->halo > b[a]) return JAC_EINVAL;
+        if (b[a] > (1LL << 30) || n[a] > (1LL << 40)) return JAC_EINVAL;
+        gr[a] = n[a] / b[a];
+        if (gr[a] > (1LL << 30)) return JAC_EINVAL;
+    }
+    std::memset(g, 0, sizeof(*g));
+    g->ndim = d->ndim;
+    g->h = d->halo;
+    g->xpad = (int)round_up(d->halo, 4);
+    g->nfaces = 2 * d->ndim;
+    g->bx = (int)b[0]; g->by = (int)b[1]; g->bz = (int)b[2];
+    g->gx = (int)gr[0]; g->gy = (int)gr[1]; g->gz = (int)gr[2];
+    g->nx = n[0]; g->ny = n[1]; g->nz = n[2];
+    const long long hz = (d->ndim == 3) ? d->halo : 0;
+    const long long PY = b[1] + 2 * d->halo, PZ = b[2] + 2 * hz;
+    g->PX = b[0] + 2 * g->xpad;
+    g->PXY = g->PX * PY;
+    g->block_stride = round_up(g->PXY * PZ, 16);
+    g->origin = (hz * PY + d->halo) * g->PX + g->xpad;
+    g->nblocks = gr[0] * gr[1] * gr[2];
+    if (g->nblocks > (1LL << 40) / std::max<long long>(1, g->block_stride)) return JAC_EINVAL;
+    const long long h = d->halo;
+    g->face_elems[0] = g->face_elems[1] = h * b[1] * b[2];
+    g->face_elems[2] = g->face_elems[3] = h * b[0] * b[2];
+    g->face_elems[4] = g->face_elems[5] = (d->ndim == 3) ? h * b[0] * b[1] : 0;
+    long long off = 0;
+    for (int fc = 0; fc < 6; ++fc) {
+        g->face_off[fc] = off;
+        off += round_up(g->face_elems[fc], 16);  // every face buffer starts on a 128-byte line
+    }
+    g->send_stride = off;
+
+    const Tiling t = make_tiling(*g);
+    const long long ctas = g->nblocks * t.ctas_per_block;
+    if (ctas > kMaxGrid) return JAC_EINVAL;
+    long long max_face = 0;
+    for (int fc = 0; fc < 6; ++fc) max_face = std::max(max_face, g->face_elems[fc]);
+    if (g->nblocks * g->nfaces * ceil_div(max_face, 1024) > kMaxGrid) return JAC_EINVAL;
+
+    if (L) {
+        std::memset(L, 0, sizeof(*L));
+        for (int a = 0; a < 3; ++a) L->g[a] = gr[a];
+        L->nblocks = g->nblocks;
+        L->pad[0] = g->PX; L->pad[1] = PY; L->pad[2] = PZ;
+        L->xpad = g->xpad;
+        L->origin = g->origin;
+        L->block_stride = g->block_stride;
+        for (int fc = 0; fc < 6; ++fc) {
+            L->face_elems[fc] = g->face_elems[fc];
+            L->face_offset[fc] = g->face_off[fc];
+        }
+        L->send_stride = g->send_stride;
+        L->partials = round_up(ctas, 32);
+        const long long arr_bytes = round_up(g->nblocks * g->block_stride * 8, 256);
+        long long o = 0;
+        L->off_u[0] = o; o += arr_bytes;
+        L->off_u[1] = o; o += arr_bytes;
+        if (d->has_f) { L->off_f = o; o += arr_bytes; } else L->off_f = -1;
+        L->off_send = o; o += round_up(g->nblocks * g->send_stride * 8, 256);
+        L->off_scratch = o; o += round_up((L->partials + 32) * 8, 256);
+        L->total_bytes = o;
+    }
+    return JAC_OK;
+}
+
+}  // namespace
+
+struct jac_ctx {
+    jac_desc desc;
+    JacGeom g;
+    jac_layout L;
+    Tiling tile;
+    char* ws;
+    double* u[2];
+    double* f;
+    double* send;
+    double* partials;
+    double* result;
+    int cur;            // which of u[] holds the current state
+    bool ghosts_fresh;  // inter-block ghosts of u[cur] equal the neighbours' current faces
+    bool packed_current;  // the send buffers hold the faces of the current state
+    cudaStream_t stream;
+    int device;
+    int cuda_err;       // sticky
+    long long launches;
+};
+
+namespace {
+
+#define JAC_CK(ctx, call)                                  \
+    do {                                                   \
+        cudaError_t e_ = (call);                           \
+        if (e_ != cudaSuccess) {                           \
+            (ctx)->cuda_err = (int)e_;                     \
+            return JAC_ECUDA;                              \
+        }                                                  \
+    } while (0)
+
+int check_launch(jac_ctx* c)
+{
+    c->launches++;
+    JAC_CK(c, cudaGetLastError());
+    return JAC_OK;
+}
+
+// ---- kernel dispatch ---------------------------------------------------------------
+template <int NV, bool HAS_F, int OP>
+void launch_sweep_t(jac_ctx* c, const double* u, double* un, long long blk0, long long nblk)
+{
+    const Tiling& t = c->tile;
+    const unsigned grid = (unsigned)(nblk * t.ctas_per_block);
+    if (c->g.ndim == 2)
+        jac::sweep2d_kernel<NV, HAS_F, OP><<<grid, t.block, 0, c->stream>>>(
+            u, un, c->f, c->partials, c->g, blk0, t.tiles_x, t.tiles_y, t.march);
+    else
+        jac::sweep3d_kernel<NV, HAS_F, OP><<<grid, t.block, 0, c->stream>>>(
+            u, un, c->f, c->partials, c->g, blk0, t.tiles_x, t.tiles_y, t.tiles_z, t.march);
+}
+
+template <int OP>
+int launch_sweep(jac_ctx* c, const double* u, double* un, long long blk0, long long nblk)
+{
+    const bool f = c->desc.has_f != 0;
+    if (c->tile.nv == 2) {
+        if (f) launch_sweep_t<2, true, OP>(c, u, un, blk0, nblk);
+        else launch_sweep_t<2, false, OP>(c, u, un, blk0, nblk);
+    } else {
+        if (f) launch_sweep_t<1, true, OP>(c, u, un, blk0, nblk);
+        else launch_sweep_t<1, false, OP>(c, u, un, blk0, nblk);
+    }
+    return check_launch(c);
+}
+
+int halo_chunks(const jac_ctx* c, int face_lo, int face_hi)
+{
+    long long m = 1;
+    for (int fc = face_lo; fc < face_hi; ++fc) m = std::max(m, c->g.face_elems[fc]);
+    return (int)ceil_div(m, 256 * 4);
+}
+
+// pack or unpack all faces of all blocks in one launch
+template <bool UNPACK>
+int launch_halo_all(jac_ctx* c)
+{
+    const int chunks = halo_chunks(c, 0, c->g.nfaces);
+    const unsigned grid = (unsigned)(c->g.nblocks * c->g.nfaces * chunks);
+    jac::halo_kernel<UNPACK><<<grid, 256, 0, c->stream>>>(c->u[c->cur], c->send, c->g, 0, chunks);
+    return check_launch(c);
+}
+
+bool has_neighbour(const JacGeom& g, long long blk, int face)
+{
+    const long long co[3] = {blk % g.gx, (blk / g.gx) % g.gy, blk / ((long long)g.gx * g.gy)};
+    const int ga[3] = {g.gx, g.gy, g.gz};
+    const int a = face >> 1;
+    return (face & 1) ? co[a] + 1 < ga[a] : co[a] > 0;
+}
+
+// one launch per (block, face) that has a neighbour: the task-per-block schedule
+template <bool UNPACK>
+int launch_halo_pertask(jac_ctx* c)
+{
+    for (long long blk = 0; blk < c->g.nblocks; ++blk)
+        for (int face = 0; face < c->g.nfaces; ++face) {
+            if (!has_neighbour(c->g, blk, face)) continue;
+            const int chunks = halo_chunks(c, face, face + 1);
+            jac::halo_kernel<UNPACK><<<(unsigned)chunks, 256, 0, c->stream>>>(
+                c->u[c->cur], c->send, c->g, blk * c->g.nfaces + face, chunks);
+            const int rc = check_launch(c);
+            if (rc) return rc;
+        }
+    return JAC_OK;
+}
+
+int do_pack(jac_ctx* c)
+{
+    return c->desc.mode == JAC_MODE_PERTASK ? launch_halo_pertask<false>(c) : launch_halo_all<false>(c);
+}
+int do_unpack(jac_ctx* c)
+{
+    return c->desc.mode == JAC_MODE_PERTASK ? launch_halo_pertask<true>(c) : launch_halo_all<true>(c);
+}
+
+int do_exchange(jac_ctx* c)
+{
+    int rc = do_pack(c);
+    if (rc) return rc;
+    c->packed_current = true;
+    rc = do_unpack(c);
+    if (rc) return rc;
+    c->ghosts_fresh = true;
+    return JAC_OK;
+}
+
+// ---- strided box copies between a dense array and the padded blocks ------------------
+cudaError_t copy_box(void* dst, size_t dpitch, size_t drows, const void* src, size_t spitch,
+                     size_t srows, size_t width_bytes, size_t height, size_t depth,
+                     cudaMemcpyKind kind, cudaStream_t st)
+{
+    cudaMemcpy3DParms p;
+    std::memset(&p, 0, sizeof(p));
+    p.srcPtr = make_cudaPitchedPtr(const_cast<void*>(src), spitch, width_bytes, srows);
+    p.dstPtr = make_cudaPitchedPtr(dst, dpitch, width_bytes, drows);
+    p.extent = make_cudaExtent(width_bytes, height, depth);
+    p.kind = kind;
+    return cudaMemcpy3DAsync(&p, st);
+}
+
+// host dense <-> interiors of all blocks of `arr`
+int copy_dense_host(jac_ctx* c, double* arr, double* host, bool to_device)
+{
+    const JacGeom& g = c->g;
+    const size_t PY = (size_t)(g.PXY / g.PX);
+    for (long long blk = 0; blk < g.nblocks; ++blk) {
+        const long long bxi = blk % g.gx, byi = (blk / g.gx) % g.gy, bzi = blk / ((long long)g.gx * g.gy);
+        double* dev = arr + blk * g.block_stride + g.origin;
+        double* hp = host + ((bzi * g.bz) * g.ny + byi * g.by) * g.nx + bxi * g.bx;
+        cudaError_t e;
+        if (to_device)
+            e = copy_box(dev, g.PX * 8, PY, hp, g.nx * 8, g.ny, (size_t)g.bx * 8, g.by, g.bz,
+                         cudaMemcpyHostToDevice, c->stream);
+        else
+            e = copy_box(hp, g.nx * 8, g.ny, dev, g.PX * 8, PY, (size_t)g.bx * 8, g.by, g.bz,
+                         cudaMemcpyDeviceToHost, c->stream);
+        JAC_CK(c, e);
+    }
+    JAC_CK(c, cudaStreamSynchronize(c->stream));
+    return JAC_OK;
+}
+
+template <bool TO_BLOCKS>
+int copy_dense_device(jac_ctx* c, double* arr, double* dense)
+{
+    const long long total = c->g.nx * c->g.ny * c->g.nz;
+    const unsigned grid = (unsigned)std::min<long long>(ceil_div(total, 256), (long long)kNumSMs * 32);
+    jac::dense_copy_kernel<TO_BLOCKS><<<grid, 256, 0, c->stream>>>(arr, dense, c->g);
+    return check_launch(c);
+}
+
+int usable(jac_ctx* c)
+{
+    if (!c) return JAC_EINVAL;
+    if (c->cuda_err) return JAC_ECUDA;
+    return JAC_OK;
+}
+
+int default_tsteps(const jac_desc& d) { return d.tsteps > 0 ? d.tsteps : 4; }
+
+}  // namespace
+
+// =====================================================================================
+// C ABI
+// =====================================================================================
+extern "C" {
+
+int jac_workspace_bytes(const jac_desc* desc, size_t* bytes)
+{
+    if (!desc || !bytes) return JAC_EINVAL;
+    JacGeom g;
+    jac_layout L;
+    const int rc = build_geometry(desc, &g, &L);
+    if (rc) return rc;
+    *bytes = (size_t)L.total_bytes;
+    return JAC_OK;
+}
+
+int jac_get_layout(const jac_desc* desc, jac_layout* out)
+{
+    if (!desc || !out) return JAC_EINVAL;
+    JacGeom g;
+    jac_layout L;
+    const int rc = build_geometry(desc, &g, &L);
+    if (rc) return rc;
+    *out = L;
+    return JAC_OK;
+}
+
+int jac_create(const jac_desc* desc, void* dev_workspace, size_t bytes, jac_ctx** out)
+{
+    if (!desc || !out) return JAC_EINVAL;
+    JacGeom g;
+    jac_layout L;
+    int rc = build_geometry(desc, &g, &L);
+    if (rc) return rc;
+    if (desc->mode == JAC_MODE_TEMPORAL && desc->ndim != 2) return JAC_EINVAL;
+    if (!dev_workspace || bytes < (size_t)L.total_bytes || ((uintptr_t)dev_workspace & 255u))
+        return JAC_ENOMEM;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        cudaGetLastError();
+        return JAC_ENODEV;
+    }
+    jac_ctx* c = new (std::nothrow) jac_ctx();
+    if (!c) return JAC_ENOMEM;
+    c->desc = *desc;
+    c->g = g;
+    c->L = L;
+    c->tile = make_tiling(g);
+    c->ws = static_cast<char*>(dev_workspace);
+    c->u[0] = reinterpret_cast<double*>(c->ws + L.off_u[0]);
+    c->u[1] = reinterpret_cast<double*>(c->ws + L.off_u[1]);
+    c->f = desc->has_f ? reinterpret_cast<double*>(c->ws + L.off_f) : nullptr;
+    c->send = reinterpret_cast<double*>(c->ws + L.off_send);
+    c->partials = reinterpret_cast<double*>(c->ws + L.off_scratch);
+    c->result = c->partials + L.partials;
+    c->cur = 0;
+    c->ghosts_fresh = false;
+    c->packed_current = false;
+    c->stream = static_cast<cudaStream_t>(desc->stream);
+    c->device = dev;
+    c->cuda_err = 0;
+    c->launches = 0;
+    const cudaError_t e = cudaMemsetAsync(c->ws, 0, (size_t)L.total_bytes, c->stream);
+    if (e != cudaSuccess) {
+        delete c;
+        return JAC_ECUDA;
+    }
+    *out = c;
+    return JAC_OK;
+}
+
+int jac_destroy(jac_ctx* ctx)
+{
+    if (!ctx) return JAC_EINVAL;
+    cudaStreamSynchronize(ctx->stream);
+    delete ctx;
+    return JAC_OK;
+}
+
+int jac_set_u(jac_ctx* c, const double* host_dense)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    if (!host_dense) return JAC_EINVAL;
+    c->ghosts_fresh = false;
+    c->packed_current = false;
+    return copy_dense_host(c, c->u[c->cur], const_cast<double*>(host_dense), true);
+}
+
+int jac_set_f(jac_ctx* c, const double* host_dense)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    if (!host_dense || !c->f) return JAC_EINVAL;
+    return copy_dense_host(c, c->f, const_cast<double*>(host_dense), true);
+}
+
+int jac_get_u(jac_ctx* c, double* host_dense)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    if (!host_dense) return JAC_EINVAL;
+    return copy_dense_host(c, c->u[c->cur], host_dense, false);
+}
+
+int jac_set_u_device(jac_ctx* c, const double* dev_dense)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    if (!dev_dense) return JAC_EINVAL;
+    c->ghosts_fresh = false;
+    c->packed_current = false;
+    return copy_dense_device<true>(c, c->u[c->cur], const_cast<double*>(dev_dense));
+}
+
+int jac_set_f_device(jac_ctx* c, const double* dev_dense)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    if (!dev_dense || !c->f) return JAC_EINVAL;
+    return copy_dense_device<true>(c, c->f, const_cast<double*>(dev_dense));
+}
+
+int jac_get_u_device(jac_ctx* c, double* dev_dense)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    if (!dev_dense) return JAC_EINVAL;
+    return copy_dense_device<false>(c, c->u[c->cur], dev_dense);
+}
+
+int jac_set_boundary(jac_ctx* c, int face, double value)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    if (face < 0 || face >= c->g.nfaces) return JAC_EINVAL;
+    c->g.bval[face] = value;
+    const int axis = face >> 1;
+    const long long on_face = c->g.nblocks / (axis == 0 ? c->g.gx : axis == 1 ? c->g.gy : c->g.gz);
+    const int chunks = (int)std::min<long long>(ceil_div(c->g.face_elems[face], 256), 64);
+    jac::fill_boundary_kernel<<<(unsigned)(on_face * chunks), 256, 0, c->stream>>>(
+        c->u[0], c->u[1], c->g, face, value, chunks);
+    return check_launch(c);
+}
+
+int jac_get_block_padded(jac_ctx* c, int64_t block, double* host)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    if (!host || block < 0 || block >= c->g.nblocks) return JAC_EINVAL;
+    const JacGeom& g = c->g;
+    const long long h = g.h, hz = (g.ndim == 3) ? g.h : 0;
+    const size_t PY = (size_t)(g.PXY / g.PX);
+    const double* src = c->u[c->cur] + block * g.block_stride + g.origin - (hz * g.PXY + h * g.PX + h);
+    const size_t w = (size_t)(g.bx + 2 * h), ht = (size_t)(g.by + 2 * h), dp = (size_t)(g.bz + 2 * hz);
+    JAC_CK(c, copy_box(host, w * 8, ht, src, g.PX * 8, PY, w * 8, ht, dp, cudaMemcpyDeviceToHost, c->stream));
+    JAC_CK(c, cudaStreamSynchronize(c->stream));
+    return JAC_OK;
+}
+
+int jac_get_halo_buffer(jac_ctx* c, int64_t block, int face, double* host)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    if (!host || block < 0 || block >= c->g.nblocks || face < 0 || face >= c->g.nfaces) return JAC_EINVAL;
+    const double* src = c->send + block * c->g.send_stride + c->g.face_off[face];
+    JAC_CK(c, cudaMemcpyAsync(host, src, (size_t)c->g.face_elems[face] * 8, cudaMemcpyDeviceToHost, c->stream));
+    JAC_CK(c, cudaStreamSynchronize(c->stream));
+    return JAC_OK;
+}
+
+int jac_pack_halos(jac_ctx* c)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    rc = do_pack(c);
+    if (rc) return rc;
+    c->packed_current = true;
+    return JAC_OK;
+}
+
+int jac_unpack_halos(jac_ctx* c)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    rc = do_unpack(c);
+    if (rc) return rc;
+    // ghosts are current only if the buffers were packed from the current state
+    c->ghosts_fresh = c->packed_current;
+    return JAC_OK;
+}
+
+int jac_sweep(jac_ctx* c, int nsweeps)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    if (nsweeps < 0) return JAC_EINVAL;
+    if (nsweeps == 0) return JAC_OK;
+    const JacGeom& g = c->g;
+    switch (c->desc.mode) {
+        case JAC_MODE_FUSED:
+            if (!c->ghosts_fresh && (rc = do_exchange(c))) return rc;
+            for (int s = 0; s < nsweeps; ++s) {
+                if ((rc = launch_sweep<jac::OP_UPDATE_PUSH>(c, c->u[c->cur], c->u[c->cur ^ 1], 0, g.nblocks)))
+                    return rc;
+                c->cur ^= 1;
+                c->packed_current = false;
+            }
+            c->ghosts_fresh = true;
+            break;
+        case JAC_MODE_EXCHANGE:
+            for (int s = 0; s < nsweeps; ++s) {
+                if ((rc = do_exchange(c))) return rc;
+                if ((rc = launch_sweep<jac::OP_UPDATE>(c, c->u[c->cur], c->u[c->cur ^ 1], 0, g.nblocks)))
+                    return rc;
+                c->cur ^= 1;
+                c->ghosts_fresh = false;
+                c->packed_current = false;
+            }
+            break;
+        case JAC_MODE_PERTASK:
+            for (int s = 0; s < nsweeps; ++s) {
+                if ((rc = do_exchange(c))) return rc;
+                for (long long blk = 0; blk < g.nblocks; ++blk)
+                    if ((rc = launch_sweep<jac::OP_UPDATE>(c, c->u[c->cur], c->u[c->cur ^ 1], blk, 1)))
+                        return rc;
+                c->cur ^= 1;
+                c->ghosts_fresh = false;
+                c->packed_current = false;
+            }
+            break;
+        case JAC_MODE_TEMPORAL:
+            (void)default_tsteps;
+            return JAC_EINVAL;
+        default:
+            return JAC_EINVAL;
+    }
+    return JAC_OK;
+}
+
+int jac_residual(jac_ctx* c, double* host_out_l2)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    if (!host_out_l2) return JAC_EINVAL;
+    if (!c->ghosts_fresh && (rc = do_exchange(c))) return rc;
+    if ((rc = launch_sweep<jac::OP_RESIDUAL>(c, c->u[c->cur], nullptr, 0, c->g.nblocks))) return rc;
+    const long long nparts = c->g.nblocks * c->tile.ctas_per_block;
+    jac::reduce_partials_kernel<<<1, 1024, 0, c->stream>>>(c->partials, nparts, c->result);
+    if ((rc = check_launch(c))) return rc;
+    double sum = 0.0;
+    JAC_CK(c, cudaMemcpyAsync(&sum, c->result, sizeof(double), cudaMemcpyDeviceToHost, c->stream));
+    JAC_CK(c, cudaStreamSynchronize(c->stream));
+    *host_out_l2 = std::sqrt(sum);
+    return JAC_OK;
+}
+
+int jac_launch_count(const jac_ctx* c, int64_t* host_out)
+{
+    if (!c || !host_out) return JAC_EINVAL;
+    *host_out = c->launches;
+    return JAC_OK;
+}
+
+int jac_last_cuda_error(const jac_ctx* c) { return c ? c->cuda_err : 0; }
+
+const char* jac_strerror(int code)
+{
+    switch (code) {
+        case JAC_OK: return "ok";
+        case JAC_EINVAL: return "invalid argument";
+        case JAC_ENOMEM: return "workspace missing, too small or misaligned";
+        case JAC_ECUDA: return "CUDA runtime error";
+        case JAC_ENODEV: return "no usable CUDA device";
+        default: return "unknown error code";
+    }
+}
+
+}  // extern "C"

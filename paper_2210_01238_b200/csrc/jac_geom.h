@@ -1,0 +1,27 @@
+// Geometry shared by the host code and the kernels of libjac (plain data, passed by value).
+//
+// Physical placement of one block (element = one double):
+//
+//   row    = [ xpad margin | bx interior | xpad margin ]      PX  = bx + 2*xpad
+//   plane  = (h + by + h) rows                                PXY = PX * (by + 2h)
+//   block  = (h + bz + h) planes in 3D, 1 plane in 2D         block_stride (multiple of 16)
+//
+// xpad is h rounded up to a multiple of 4, so the first interior point of every row sits on
+// a 32-byte sector boundary and the ghost columns are the innermost h cells of the margin.
+// `origin` is the offset of interior point (0,0,0).  u, u' and f all use this placement, so
+// one offset addresses all three.
+#pragma once
+#include <stdint.h>
+
+struct JacGeom {
+    int ndim, h, xpad, nfaces;
+    int bx, by, bz;  // block interior
+    int gx, gy, gz;  // block grid
+    long long nx, ny, nz;
+    long long PX, PXY, block_stride, origin;
+    long long nblocks;
+    long long face_elems[6];
+    long long face_off[6];
+    long long send_stride;
+    double bval[6];
+};

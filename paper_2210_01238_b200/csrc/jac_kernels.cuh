@@ -1,0 +1,377 @@
+// Device code of libjac: Jacobi update (2D 5-point / 3D 7-point), halo pack / unpack,
+// residual reduction, dense <-> block copies.  sm_100a, fp64, no tensor cores: the work is
+// bound by HBM bandwidth, so the kernels are organised around coalesced 128-bit accesses,
+// register reuse along the marching axis and single launches over all blocks.
+//
+// Arithmetic contract (same as the header): s = (W + E) + (S + N); 3D: s = s + (D + U);
+// with f: s = s + f; u' = s * 0.25 or s * (1/6).  Every operation is an explicit
+// round-to-nearest intrinsic, so the compiler cannot contract an FMA.
+#pragma once
+#include <cuda_runtime.h>
+
+#include "jac_geom.h"
+
+namespace jac {
+
+enum : int { OP_UPDATE = 0, OP_UPDATE_PUSH = 1, OP_RESIDUAL = 2 };
+
+__device__ __forceinline__ double add_rn(double a, double b) { return __dadd_rn(a, b); }
+__device__ __forceinline__ double sub_rn(double a, double b) { return __dsub_rn(a, b); }
+__device__ __forceinline__ double mul_rn(double a, double b) { return __dmul_rn(a, b); }
+
+// NV consecutive doubles held by one thread (NV = 1 or 2; NV = 2 uses one 128-bit access).
+template <int NV> struct Vec { double v[NV]; };
+
+template <int NV> __device__ __forceinline__ Vec<NV> load_vec(const double* p);
+template <> __device__ __forceinline__ Vec<1> load_vec<1>(const double* p) {
+    Vec<1> r; r.v[0] = *p; return r;
+}
+template <> __device__ __forceinline__ Vec<2> load_vec<2>(const double* p) {
+    const double2 t = *reinterpret_cast<const double2*>(p);
+    Vec<2> r; r.v[0] = t.x; r.v[1] = t.y; return r;
+}
+template <int NV> __device__ __forceinline__ void store_vec(double* p, const Vec<NV>& a);
+template <> __device__ __forceinline__ void store_vec<1>(double* p, const Vec<1>& a) { *p = a.v[0]; }
+template <> __device__ __forceinline__ void store_vec<2>(double* p, const Vec<2>& a) {
+    *reinterpret_cast<double2*>(p) = make_double2(a.v[0], a.v[1]);
+}
+
+// Sum of a per-thread value over the CTA in a fixed order: lanes by shuffle, then warps in
+// index order by thread 0.  Returns the total in thread 0.
+__device__ __forceinline__ double block_sum(double v) {
+    __shared__ double warp_part[32];
+    const int tid = threadIdx.x + blockDim.x * (threadIdx.y + blockDim.y * threadIdx.z);
+    const int nthreads = blockDim.x * blockDim.y * blockDim.z;
+    const int lane = tid & 31, warp = tid >> 5;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v = add_rn(v, __shfl_down_sync(0xffffffffu, v, off));
+    if (lane == 0) warp_part[warp] = v;
+    __syncthreads();
+    double total = 0.0;
+    if (tid == 0) {
+        const int nwarps = (nthreads + 31) >> 5;
+        for (int w = 0; w < nwarps; ++w) total = add_rn(total, warp_part[w]);
+    }
+    return total;
+}
+
+// ---------------------------------------------------------------------------------------
+// 2D: one CTA owns a strip of `rows` rows x (blockDim.x * NV) columns of one block and
+// marches along y.  The rows j-1, j, j+1 of a thread's own columns live in registers; the
+// west/east neighbours of the strip are read through L1 (those sectors were just fetched by
+// the neighbouring lanes' vector loads).  DRAM sees each interior point once.
+//
+// OP_UPDATE       u' <- update(u)
+// OP_UPDATE_PUSH  same, and every new value within h of a block face that has a neighbour is
+//                 also stored into that neighbour's ghost cell of u' (the exchange for the
+//                 next sweep, done while the value is in a register)
+// OP_RESIDUAL     per-CTA partial of sum r^2, r = s - 4u
+// ---------------------------------------------------------------------------------------
+template <int NV, bool HAS_F, int OP>
+__global__ void __launch_bounds__(256)
+sweep2d_kernel(const double* __restrict__ u, double* __restrict__ un, const double* __restrict__ f,
+               double* __restrict__ partials, const JacGeom g, const long long blk0,
+               const int tiles_x, const int tiles_y, const int rows)
+{
+    const long long t = blockIdx.x;
+    const int xt = (int)(t % tiles_x);
+    const int yt = (int)((t / tiles_x) % tiles_y);
+    const long long blk = blk0 + t / ((long long)tiles_x * tiles_y);
+    const int x = (xt * blockDim.x + threadIdx.x) * NV;
+    const int j0 = yt * rows;
+    const int j1 = min(g.by, j0 + rows);
+    const long long PX = g.PX;
+    double acc = 0.0;
+
+    if (x < g.bx) {
+        const long long base = blk * g.block_stride + g.origin + x;
+        const double* ub = u + base;
+        const double* fb = HAS_F ? f + base : nullptr;
+        double* ob = (OP == OP_RESIDUAL) ? nullptr : un + base;
+
+        const int bxi = (int)(blk % g.gx), byi = (int)(blk / g.gx);
+        const bool nb_mx = bxi > 0, nb_px = bxi + 1 < g.gx;
+        const bool nb_my = byi > 0, nb_py = byi + 1 < g.gy;
+        const long long bs = g.block_stride;
+
+        Vec<NV> S = load_vec<NV>(ub + (long long)(j0 - 1) * PX);
+        Vec<NV> Cc = load_vec<NV>(ub + (long long)j0 * PX);
+#pragma unroll 4
+        for (int j = j0; j < j1; ++j) {
+            const long long ro = (long long)j * PX;
+            const Vec<NV> N = load_vec<NV>(ub + ro + PX);
+            const double w = ub[ro - 1];
+            const double e = ub[ro + NV];
+            Vec<NV> ff;
+            if (HAS_F) ff = load_vec<NV>(fb + ro);
+            Vec<NV> o;
+#pragma unroll
+            for (int q = 0; q < NV; ++q) {
+                const double W = (q == 0) ? w : Cc.v[q - 1];
+                const double E = (q == NV - 1) ? e : Cc.v[q + 1];
+                double s = add_rn(add_rn(W, E), add_rn(S.v[q], N.v[q]));
+                if (HAS_F) s = add_rn(s, ff.v[q]);
+                if (OP == OP_RESIDUAL) {
+                    const double r = sub_rn(s, mul_rn(4.0, Cc.v[q]));
+                    acc = add_rn(acc, mul_rn(r, r));
+                } else {
+                    o.v[q] = mul_rn(s, 0.25);
+                }
+            }
+            if (OP != OP_RESIDUAL) store_vec<NV>(ob + ro, o);
+            if (OP == OP_UPDATE_PUSH) {
+                // my interior column c < h is the left neighbour's ghost column bx + c;
+                // my column c >= bx - h is the right neighbour's ghost column c - bx
+#pragma unroll
+                for (int q = 0; q < NV; ++q) {
+                    const int c = x + q;
+                    if (nb_mx && c < g.h) ob[ro + q - bs + g.bx] = o.v[q];
+                    if (nb_px && c >= g.bx - g.h) ob[ro + q + bs - g.bx] = o.v[q];
+                }
+                if (nb_my && j < g.h)
+                    store_vec<NV>(ob - bs * g.gx + (long long)(g.by + j) * PX, o);
+                if (nb_py && j >= g.by - g.h)
+                    store_vec<NV>(ob + bs * g.gx + (long long)(j - g.by) * PX, o);
+            }
+            S = Cc;
+            Cc = N;
+        }
+    }
+    if (OP == OP_RESIDUAL) {
+        const double total = block_sum(acc);
+        if (threadIdx.x == 0) partials[blockIdx.x] = total;
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// 3D: one CTA owns (blockDim.x * NV) x blockDim.y columns of one block over a range of
+// `planes` z-planes and marches along z.  Planes k-1, k, k+1 of a thread's own column are
+// in registers (DRAM traffic: one load per point); the y and x neighbours of plane k come
+// through L1, which holds the plane since it was fetched as "k+1" one step earlier.
+// ---------------------------------------------------------------------------------------
+template <int NV, bool HAS_F, int OP>
+__global__ void __launch_bounds__(512)
+sweep3d_kernel(const double* __restrict__ u, double* __restrict__ un, const double* __restrict__ f,
+               double* __restrict__ partials, const JacGeom g, const long long blk0,
+               const int tiles_x, const int tiles_y, const int tiles_z, const int planes)
+{
+    const long long t = blockIdx.x;
+    const int xt = (int)(t % tiles_x);
+    const int yt = (int)((t / tiles_x) % tiles_y);
+    const int zt = (int)((t / ((long long)tiles_x * tiles_y)) % tiles_z);
+    const long long blk = blk0 + t / ((long long)tiles_x * tiles_y * tiles_z);
+    const int x = (xt * blockDim.x + threadIdx.x) * NV;
+    const int y = yt * blockDim.y + threadIdx.y;
+    const int k0 = zt * planes;
+    const int k1 = min(g.bz, k0 + planes);
+    const long long PX = g.PX, PXY = g.PXY;
+    const double c6 = 1.0 / 6.0;
+    double acc = 0.0;
+
+    if (x < g.bx && y < g.by) {
+        const long long base = blk * g.block_stride + g.origin + (long long)y * PX + x;
+        const double* ub = u + base;
+        const double* fb = HAS_F ? f + base : nullptr;
+        double* ob = (OP == OP_RESIDUAL) ? nullptr : un + base;
+
+        const int bxi = (int)(blk % g.gx);
+        const int byi = (int)((blk / g.gx) % g.gy);
+        const int bzi = (int)(blk / ((long long)g.gx * g.gy));
+        const bool nb_mx = bxi > 0, nb_px = bxi + 1 < g.gx;
+        const bool nb_my = byi > 0, nb_py = byi + 1 < g.gy;
+        const bool nb_mz = bzi > 0, nb_pz = bzi + 1 < g.gz;
+        const long long bs = g.block_stride;
+        const long long bsy = bs * g.gx, bsz = bs * g.gx * g.gy;
+
+        Vec<NV> D = load_vec<NV>(ub + (long long)(k0 - 1) * PXY);
+        Vec<NV> Cc = load_vec<NV>(ub + (long long)k0 * PXY);
+#pragma unroll 2
+        for (int k = k0; k < k1; ++k) {
+            const long long po = (long long)k * PXY;
+            const Vec<NV> U = load_vec<NV>(ub + po + PXY);
+            const Vec<NV> S = load_vec<NV>(ub + po - PX);
+            const Vec<NV> N = load_vec<NV>(ub + po + PX);
+            const double w = ub[po - 1];
+            const double e = ub[po + NV];
+            Vec<NV> ff;
+            if (HAS_F) ff = load_vec<NV>(fb + po);
+            Vec<NV> o;
+#pragma unroll
+            for (int q = 0; q < NV; ++q) {
+                const double W = (q == 0) ? w : Cc.v[q - 1];
+                const double E = (q == NV - 1) ? e : Cc.v[q + 1];
+                double s = add_rn(add_rn(W, E), add_rn(S.v[q], N.v[q]));
+                s = add_rn(s, add_rn(D.v[q], U.v[q]));
+                if (HAS_F) s = add_rn(s, ff.v[q]);
+                if (OP == OP_RESIDUAL) {
+                    const double r = sub_rn(s, mul_rn(6.0, Cc.v[q]));
+                    acc = add_rn(acc, mul_rn(r, r));
+                } else {
+                    o.v[q] = mul_rn(s, c6);
+                }
+            }
+            if (OP != OP_RESIDUAL) store_vec<NV>(ob + po, o);
+            if (OP == OP_UPDATE_PUSH) {
+#pragma unroll
+                for (int q = 0; q < NV; ++q) {
+                    const int c = x + q;
+                    if (nb_mx && c < g.h) ob[po + q - bs + g.bx] = o.v[q];
+                    if (nb_px && c >= g.bx - g.h) ob[po + q + bs - g.bx] = o.v[q];
+                }
+                if (nb_my && y < g.h) store_vec<NV>(ob + po - bsy + (long long)g.by * PX, o);
+                if (nb_py && y >= g.by - g.h) store_vec<NV>(ob + po + bsy - (long long)g.by * PX, o);
+                if (nb_mz && k < g.h) store_vec<NV>(ob + po - bsz + (long long)g.bz * PXY, o);
+                if (nb_pz && k >= g.bz - g.h) store_vec<NV>(ob + po + bsz - (long long)g.bz * PXY, o);
+            }
+            D = Cc;
+            Cc = U;
+        }
+    }
+    if (OP == OP_RESIDUAL) {
+        const double total = block_sum(acc);
+        if (threadIdx.x == 0 && threadIdx.y == 0) partials[blockIdx.x] = total;
+    }
+}
+
+// Second pass of the residual: one CTA adds the per-CTA partials in a fixed order.
+__global__ void __launch_bounds__(1024)
+reduce_partials_kernel(const double* __restrict__ partials, const long long n, double* __restrict__ out)
+{
+    double acc = 0.0;
+    for (long long i = threadIdx.x; i < n; i += blockDim.x) acc = add_rn(acc, partials[i]);
+    const double total = block_sum(acc);
+    if (threadIdx.x == 0) *out = total;
+}
+
+// ---------------------------------------------------------------------------------------
+// Halo pack / unpack.  One launch covers `npairs` consecutive (block, face) pairs starting at
+// pair0 (pair = block * nfaces + face); each pair is cut into chunks of blockDim.x * EPT
+// elements.  Pairs whose face lies on the domain boundary do nothing.
+//
+// Element e of a packed face (source memory order):
+//   x face: e = (k*by + j)*h + c      y face: e = (k*h + r)*bx + i      z face: e = (p*by + j)*bx + i
+// Pack reads the interior strip next to the face; unpack writes the ghost strip of the same
+// face from the neighbour's opposite-face buffer.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ long long neighbour_block(const JacGeom& g, long long blk, int face)
+{
+    const int bxi = (int)(blk % g.gx);
+    const int byi = (int)((blk / g.gx) % g.gy);
+    const int bzi = (int)(blk / ((long long)g.gx * g.gy));
+    switch (face) {
+        case 0: return bxi > 0 ? blk - 1 : -1;
+        case 1: return bxi + 1 < g.gx ? blk + 1 : -1;
+        case 2: return byi > 0 ? blk - g.gx : -1;
+        case 3: return byi + 1 < g.gy ? blk + g.gx : -1;
+        case 4: return bzi > 0 ? blk - (long long)g.gx * g.gy : -1;
+        default: return bzi + 1 < g.gz ? blk + (long long)g.gx * g.gy : -1;
+    }
+}
+
+// offset (relative to the block's interior origin) of element e of the strip on `face`;
+// lo = first layer of the strip along the face's axis (interior-relative)
+__device__ __forceinline__ long long strip_offset(const JacGeom& g, int face, long long e, int lo)
+{
+    const int axis = face >> 1;
+    long long x, y, z;
+    if (axis == 0) {
+        x = e % g.h + lo; const long long t = e / g.h; y = t % g.by; z = t / g.by;
+    } else if (axis == 1) {
+        x = e % g.bx; const long long t = e / g.bx; y = t % g.h + lo; z = t / g.h;
+    } else {
+        x = e % g.bx; const long long t = e / g.bx; y = t % g.by; z = t / g.by + lo;
+    }
+    return z * g.PXY + y * g.PX + x;
+}
+
+template <bool UNPACK>
+__global__ void __launch_bounds__(256)
+halo_kernel(double* __restrict__ u, double* __restrict__ send, const JacGeom g,
+            const long long pair0, const int chunks)
+{
+    const long long t = blockIdx.x;
+    const long long pair = pair0 + t / chunks;
+    const int chunk = (int)(t % chunks);
+    const long long blk = pair / g.nfaces;
+    const int face = (int)(pair % g.nfaces);
+    const long long nb = neighbour_block(g, blk, face);
+    if (nb < 0) return;
+    const long long n = g.face_elems[face];
+    const int axis = face >> 1;
+    const int ext = axis == 0 ? g.bx : (axis == 1 ? g.by : g.bz);
+    double* ub = u + blk * g.block_stride + g.origin;
+    constexpr int EPT = 4;
+    const long long e0 = (long long)chunk * blockDim.x * EPT + threadIdx.x;
+    if (!UNPACK) {
+        double* buf = send + blk * g.send_stride + g.face_off[face];
+        const int lo = (face & 1) ? ext - g.h : 0;
+#pragma unroll
+        for (int q = 0; q < EPT; ++q) {
+            const long long e = e0 + (long long)q * blockDim.x;
+            if (e < n) buf[e] = ub[strip_offset(g, face, e, lo)];
+        }
+    } else {
+        const double* buf = send + nb * g.send_stride + g.face_off[face ^ 1];
+        const int lo = (face & 1) ? ext : -g.h;
+#pragma unroll
+        for (int q = 0; q < EPT; ++q) {
+            const long long e = e0 + (long long)q * blockDim.x;
+            if (e < n) ub[strip_offset(g, face, e, lo)] = buf[e];
+        }
+    }
+}
+
+// Dirichlet value into the ghost strip of `face` of every block on that domain face, in both
+// solution arrays.  grid = (chunks, blocks on the face).
+__global__ void __launch_bounds__(256)
+fill_boundary_kernel(double* __restrict__ u0, double* __restrict__ u1, const JacGeom g,
+                     const int face, const double value, const int chunks)
+{
+    const int axis = face >> 1;
+    const long long t = blockIdx.x;
+    const long long m = t / chunks;  // index among the blocks on this face
+    const int chunk = (int)(t % chunks);
+    // enumerate blocks with the face's axis coordinate fixed at 0 or g-1
+    long long c[3];
+    const int ga[3] = {g.gx, g.gy, g.gz};
+    long long rem = m;
+    for (int a = 0; a < 3; ++a) {
+        if (a == axis) { c[a] = (face & 1) ? ga[a] - 1 : 0; continue; }
+        c[a] = rem % ga[a];
+        rem /= ga[a];
+    }
+    const long long blk = (c[2] * g.gy + c[1]) * g.gx + c[0];
+    const int ext = axis == 0 ? g.bx : (axis == 1 ? g.by : g.bz);
+    const int lo = (face & 1) ? ext : -g.h;
+    const long long n = g.face_elems[face];
+    const long long base = blk * g.block_stride + g.origin;
+    for (long long e = (long long)chunk * blockDim.x + threadIdx.x; e < n;
+         e += (long long)chunks * blockDim.x) {
+        const long long off = base + strip_offset(g, face, e, lo);
+        u0[off] = value;
+        u1[off] = value;
+    }
+}
+
+// Dense array (x fastest over the global interior) <-> block interiors.
+template <bool TO_BLOCKS>
+__global__ void __launch_bounds__(256)
+dense_copy_kernel(double* __restrict__ blocks, double* __restrict__ dense, const JacGeom g)
+{
+    const long long total = g.nx * g.ny * g.nz;
+    for (long long p = (long long)blockIdx.x * blockDim.x + threadIdx.x; p < total;
+         p += (long long)gridDim.x * blockDim.x) {
+        const long long gi = p % g.nx;
+        const long long t = p / g.nx;
+        const long long gj = t % g.ny;
+        const long long gk = t / g.ny;
+        const long long bxi = gi / g.bx, byi = gj / g.by, bzi = gk / g.bz;
+        const long long blk = (bzi * g.gy + byi) * g.gx + bxi;
+        const long long off = blk * g.block_stride + g.origin + (gk - bzi * g.bz) * g.PXY +
+                              (gj - byi * g.by) * g.PX + (gi - bxi * g.bx);
+        if (TO_BLOCKS) blocks[off] = dense[p];
+        else dense[p] = blocks[off];
+    }
+}
+
+}  // namespace jac

@@ -1,0 +1,273 @@
+"""ctypes binding of ``libjac.so`` -- argument marshalling only.
+
+Every step of the hot path (sweep, pack, unpack, residual) runs in the library's CUDA
+kernels; PyTorch is used here for nothing but device memory and the stream.  There is no
+CPU fallback: if the shared library is missing, or a call is made without a CUDA device,
+an exception is raised.
+
+    from paper_2210_01238_b200 import jac
+    J = jac.Jacobi(n=(4096, 4096), b=(512, 512), halo=1, has_f=True)
+    J.set_f(f); J.sweep(10); r = J.residual(); u = J.get_u()
+"""
+from __future__ import annotations
+
+import ctypes as C
+from pathlib import Path
+
+import numpy as np
+
+_PKG = Path(__file__).resolve().parent
+LIB_PATH = _PKG / "libjac.so"
+
+MODE_FUSED, MODE_PERTASK, MODE_TEMPORAL, MODE_EXCHANGE = 0, 1, 2, 3
+MODES = {"fused": MODE_FUSED, "pertask": MODE_PERTASK, "temporal": MODE_TEMPORAL,
+         "exchange": MODE_EXCHANGE}
+
+OK, EINVAL, ENOMEM, ECUDA, ENODEV = 0, -1, -2, -3, -4
+
+EXPORTS = [
+    "jac_workspace_bytes", "jac_get_layout", "jac_create", "jac_destroy",
+    "jac_set_u", "jac_set_f", "jac_get_u", "jac_set_u_device", "jac_set_f_device",
+    "jac_get_u_device", "jac_set_boundary", "jac_get_block_padded", "jac_get_halo_buffer",
+    "jac_pack_halos", "jac_unpack_halos", "jac_sweep", "jac_residual", "jac_launch_count",
+    "jac_last_cuda_error", "jac_strerror",
+]
+
+
+class Desc(C.Structure):
+    _fields_ = [("ndim", C.c_int32), ("halo", C.c_int32), ("has_f", C.c_int32),
+                ("mode", C.c_int32), ("tsteps", C.c_int32), ("reserved", C.c_int32),
+                ("n", C.c_int64 * 3), ("b", C.c_int64 * 3), ("stream", C.c_void_p)]
+
+
+class Layout(C.Structure):
+    _fields_ = [("g", C.c_int64 * 3), ("nblocks", C.c_int64), ("pad", C.c_int64 * 3),
+                ("xpad", C.c_int64), ("origin", C.c_int64), ("block_stride", C.c_int64),
+                ("face_elems", C.c_int64 * 6), ("face_offset", C.c_int64 * 6),
+                ("send_stride", C.c_int64), ("partials", C.c_int64), ("off_u", C.c_int64 * 2),
+                ("off_f", C.c_int64), ("off_send", C.c_int64), ("off_scratch", C.c_int64),
+                ("total_bytes", C.c_int64)]
+
+
+class JacError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        self.code = code
+        super().__init__(f"{what}: {strerror(code)} ({code})")
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """The loaded shared library.  Raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not LIB_PATH.exists():
+            raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2210_01238_b200.build`")
+        L = C.CDLL(str(LIB_PATH))
+        dp, vp = C.POINTER(C.c_double), C.c_void_p
+        L.jac_workspace_bytes.argtypes = [C.POINTER(Desc), C.POINTER(C.c_size_t)]
+        L.jac_get_layout.argtypes = [C.POINTER(Desc), C.POINTER(Layout)]
+        L.jac_create.argtypes = [C.POINTER(Desc), vp, C.c_size_t, C.POINTER(vp)]
+        L.jac_destroy.argtypes = [vp]
+        for name in ("jac_set_u", "jac_set_f", "jac_get_u", "jac_set_u_device",
+                     "jac_set_f_device", "jac_get_u_device"):
+            getattr(L, name).argtypes = [vp, vp]
+        L.jac_set_boundary.argtypes = [vp, C.c_int, C.c_double]
+        L.jac_get_block_padded.argtypes = [vp, C.c_int64, vp]
+        L.jac_get_halo_buffer.argtypes = [vp, C.c_int64, C.c_int, vp]
+        L.jac_pack_halos.argtypes = [vp]
+        L.jac_unpack_halos.argtypes = [vp]
+        L.jac_sweep.argtypes = [vp, C.c_int]
+        L.jac_residual.argtypes = [vp, dp]
+        L.jac_launch_count.argtypes = [vp, C.POINTER(C.c_int64)]
+        L.jac_last_cuda_error.argtypes = [vp]
+        L.jac_strerror.argtypes = [C.c_int]
+        L.jac_strerror.restype = C.c_char_p
+        for name in EXPORTS:
+            if name != "jac_strerror":
+                getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().jac_strerror(int(code)).decode()
+
+
+def make_desc(n, b, halo=1, has_f=False, mode=MODE_FUSED, tsteps=0, stream=0) -> Desc:
+    ndim = len(n)
+    d = Desc()
+    d.ndim, d.halo, d.has_f = ndim, int(halo), int(bool(has_f))
+    d.mode = MODES[mode] if isinstance(mode, str) else int(mode)
+    d.tsteps, d.reserved = int(tsteps), 0
+    for a in range(3):
+        d.n[a] = int(n[a]) if a < ndim else 1
+        d.b[a] = int(b[a]) if a < ndim else 1
+    d.stream = stream or None
+    return d
+
+
+def workspace_bytes(desc: Desc) -> int:
+    out = C.c_size_t(0)
+    rc = lib().jac_workspace_bytes(C.byref(desc), C.byref(out))
+    if rc:
+        raise JacError(rc, "jac_workspace_bytes")
+    return out.value
+
+
+def get_layout(desc: Desc) -> Layout:
+    out = Layout()
+    rc = lib().jac_get_layout(C.byref(desc), C.byref(out))
+    if rc:
+        raise JacError(rc, "jac_get_layout")
+    return out
+
+
+def _host_ptr(a: np.ndarray):
+    assert a.dtype == np.float64 and a.flags["C_CONTIGUOUS"]
+    return a.ctypes.data
+
+
+class Jacobi:
+    """One context of the library over a torch-owned workspace on the current CUDA device.
+
+    n, b: global / block interior points in (x, y[, z]) order.  Dense arrays are numpy float64
+    of shape (ny, nx) / (nz, ny, nx), or torch CUDA float64 tensors of that shape for the
+    ``*_device`` calls.
+    """
+
+    def __init__(self, n, b, halo=1, has_f=False, mode="fused", tsteps=0, stream=None):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("paper_2210_01238_b200.jac needs a CUDA device; there is no CPU path")
+        self._torch = torch
+        self.n, self.b = tuple(int(x) for x in n), tuple(int(x) for x in b)
+        self.ndim = len(self.n)
+        self.stream = stream if stream is not None else torch.cuda.current_stream()
+        self.desc = make_desc(n, b, halo, has_f, mode, tsteps, self.stream.cuda_stream)
+        self.layout = get_layout(self.desc)
+        nbytes = workspace_bytes(self.desc)
+        with torch.cuda.stream(self.stream):
+            self.workspace = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        self._ctx = C.c_void_p()
+        self._call("jac_create", lib().jac_create(C.byref(self.desc), self.workspace.data_ptr(),
+                                                  nbytes, C.byref(self._ctx)))
+
+    # ---- plumbing
+    def _call(self, what: str, rc: int):
+        if rc:
+            detail = ""
+            if rc == ECUDA and self._ctx:
+                detail = f" [cudaError {lib().jac_last_cuda_error(self._ctx)}]"
+            raise JacError(rc, what + detail)
+
+    def close(self):
+        if getattr(self, "_ctx", None):
+            lib().jac_destroy(self._ctx)
+            self._ctx = C.c_void_p()
+            self.workspace = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    @property
+    def dense_shape(self):
+        return tuple(reversed(self.n))
+
+    @property
+    def nblocks(self) -> int:
+        return int(self.layout.nblocks)
+
+    def _dev_ptr(self, t):
+        assert t.is_cuda and t.dtype == self._torch.float64 and t.is_contiguous()
+        assert tuple(t.shape) == self.dense_shape
+        return t.data_ptr()
+
+    # ---- data in / out
+    def set_u(self, dense: np.ndarray):
+        d = np.ascontiguousarray(dense, dtype=np.float64)
+        assert d.shape == self.dense_shape
+        self._call("jac_set_u", lib().jac_set_u(self._ctx, _host_ptr(d)))
+
+    def set_f(self, dense: np.ndarray):
+        d = np.ascontiguousarray(dense, dtype=np.float64)
+        assert d.shape == self.dense_shape
+        self._call("jac_set_f", lib().jac_set_f(self._ctx, _host_ptr(d)))
+
+    def get_u(self, out: np.ndarray | None = None) -> np.ndarray:
+        if out is None:
+            out = np.empty(self.dense_shape, dtype=np.float64)
+        assert out.shape == self.dense_shape
+        self._call("jac_get_u", lib().jac_get_u(self._ctx, _host_ptr(out)))
+        return out
+
+    def set_u_device(self, t):
+        self._call("jac_set_u_device", lib().jac_set_u_device(self._ctx, self._dev_ptr(t)))
+
+    def set_f_device(self, t):
+        self._call("jac_set_f_device", lib().jac_set_f_device(self._ctx, self._dev_ptr(t)))
+
+    def get_u_device(self, out=None):
+        if out is None:
+            with self._torch.cuda.stream(self.stream):
+                out = self._torch.empty(self.dense_shape, dtype=self._torch.float64, device="cuda")
+        self._call("jac_get_u_device", lib().jac_get_u_device(self._ctx, self._dev_ptr(out)))
+        return out
+
+    def set_u_pinned(self, t):
+        """``t``: pinned host torch tensor of the dense shape (asynchronous DMA source)."""
+        assert not t.is_cuda and t.dtype == self._torch.float64 and t.is_contiguous()
+        self._call("jac_set_u", lib().jac_set_u(self._ctx, t.data_ptr()))
+
+    def get_u_pinned(self, t):
+        assert not t.is_cuda and t.dtype == self._torch.float64 and t.is_contiguous()
+        self._call("jac_get_u", lib().jac_get_u(self._ctx, t.data_ptr()))
+        return t
+
+    def set_boundary(self, face: int, value: float):
+        self._call("jac_set_boundary", lib().jac_set_boundary(self._ctx, int(face), float(value)))
+
+    def get_block_padded(self, blk: int) -> np.ndarray:
+        h = self.desc.halo
+        out = np.empty(tuple(x + 2 * h for x in reversed(self.b)), dtype=np.float64)
+        self._call("jac_get_block_padded",
+                   lib().jac_get_block_padded(self._ctx, int(blk), _host_ptr(out)))
+        return out
+
+    def get_halo_buffer(self, blk: int, face: int) -> np.ndarray:
+        dims = list(self.b)
+        dims[face // 2] = self.desc.halo
+        out = np.empty(tuple(reversed(dims)), dtype=np.float64)
+        self._call("jac_get_halo_buffer",
+                   lib().jac_get_halo_buffer(self._ctx, int(blk), int(face), _host_ptr(out)))
+        return out
+
+    # ---- the hot path
+    def pack_halos(self):
+        self._call("jac_pack_halos", lib().jac_pack_halos(self._ctx))
+
+    def unpack_halos(self):
+        self._call("jac_unpack_halos", lib().jac_unpack_halos(self._ctx))
+
+    def sweep(self, nsweeps: int = 1):
+        self._call("jac_sweep", lib().jac_sweep(self._ctx, int(nsweeps)))
+
+    def residual(self) -> float:
+        out = C.c_double(0.0)
+        self._call("jac_residual", lib().jac_residual(self._ctx, C.byref(out)))
+        return out.value
+
+    def launch_count(self) -> int:
+        out = C.c_int64(0)
+        self._call("jac_launch_count", lib().jac_launch_count(self._ctx, C.byref(out)))
+        return out.value

@@ -1,0 +1,193 @@
+"""GPU library vs CPU oracle, element by element, on small shapes that span several tiles and
+ragged tails: sweep (every schedule), pack, unpack, residual, boundary values, data in/out.
+Bars: halos and ghosts bit-exact; sweep bit-exact (the bar the library is held to is
+max|du| <= 1e-12 max|u|; identical operation order makes it 0); residual rel. error <= 1e-10."""
+import numpy as np
+import pytest
+
+from paper_2210_01238_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+SWEEP_TOL = 1e-12
+RESID_TOL = 1e-10
+BVALS = [0.5, -1.0, 2.0, 3.0, -0.25, 1.5]
+
+# (n, b, halo): single block, many tiny blocks, odd widths (scalar path), rows longer than one
+# CTA tile (x tiles), more rows than one strip (y tiles), halo 1..4
+SHAPES_2D = [((12, 8), (12, 8), 1), ((12, 8), (4, 4), 1), ((12, 8), (1, 1), 1), ((15, 9), (5, 3), 1),
+             ((15, 9), (5, 3), 3), ((64, 48), (16, 8), 4), ((640, 72), (640, 72), 1),
+             ((1100, 200), (550, 100), 2), ((130, 210), (130, 70), 1), ((36, 24), (12, 8), 2)]
+SHAPES_3D = [((6, 4, 8), (3, 2, 4), 1), ((6, 4, 8), (1, 1, 1), 1), ((6, 4, 8), (6, 4, 8), 2),
+             ((20, 12, 40), (10, 12, 20), 1), ((132, 20, 36), (132, 10, 18), 1),
+             ((24, 18, 12), (8, 6, 4), 3), ((48, 40, 20), (24, 20, 10), 2)]
+MODES = ["fused", "exchange", "pertask"]
+
+
+@pytest.fixture(scope="module")
+def jac():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2210_01238_b200 import jac as _jac
+    _jac.lib()  # raises if the library was not built
+    return _jac
+
+
+def _random_problem(n, seed=0):
+    rng = np.random.default_rng(seed)
+    shape = tuple(reversed(n))
+    return rng.uniform(-1, 1, shape), rng.uniform(-1, 1, shape)
+
+
+def _setup_pair(jac, orc, n, b, h, has_f, mode, seed=0, tsteps=0):
+    ndim = len(n)
+    u0, f = _random_problem(n, seed)
+    J = jac.Jacobi(n, b, h, has_f, mode, tsteps)
+    B = orc.Blocked(n, b, h, has_f)
+    for face in range(2 * ndim):
+        J.set_boundary(face, BVALS[face])
+        B.set_boundary(face, BVALS[face])
+    J.set_u(u0)
+    B.set_u(u0)
+    if has_f:
+        J.set_f(f)
+        B.set_f(f)
+    return J, B
+
+
+def _assert_sweep_close(got, want):
+    scale = np.max(np.abs(want))
+    assert np.max(np.abs(got - want)) <= SWEEP_TOL * scale
+    assert np.array_equal(got, want), "same operation order should give identical bits"
+
+
+@pytest.mark.parametrize("n,b,h", SHAPES_2D + SHAPES_3D)
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("has_f", [False, True])
+def test_sweep_matches_oracle(jac, orc, n, b, h, mode, has_f):
+    J, B = _setup_pair(jac, orc, n, b, h, has_f, mode)
+    for nsw in (1, 2, 4):
+        J.sweep(nsw)
+        B.sweep(nsw)
+        _assert_sweep_close(J.get_u(), B.get_u())
+    r_gpu, r_cpu = J.residual(), B.residual()
+    assert abs(r_gpu - r_cpu) <= RESID_TOL * r_cpu
+    # a residual call must not disturb the state
+    J.sweep(1)
+    B.sweep(1)
+    _assert_sweep_close(J.get_u(), B.get_u())
+    J.close()
+    B.close()
+
+
+@pytest.mark.parametrize("n,b,h", SHAPES_2D + SHAPES_3D)
+@pytest.mark.parametrize("mode", ["fused", "pertask"])
+def test_pack_and_unpack_are_bit_exact(jac, orc, n, b, h, mode):
+    ndim = len(n)
+    J = jac.Jacobi(n, b, h, False, mode)
+    B = orc.Blocked(n, b, h, False)
+    dense = inputs.uniform_field(n, inputs.HALO_BENCH_SEED)
+    for face in range(2 * ndim):
+        J.set_boundary(face, BVALS[face])
+        B.set_boundary(face, BVALS[face])
+    J.set_u(dense)
+    B.set_u(dense)
+    J.pack_halos()
+    B.pack()
+    for blk in range(B.nblocks):
+        for face in range(2 * ndim):
+            if B.neighbour(blk, face) >= 0:
+                assert np.array_equal(J.get_halo_buffer(blk, face), B.get_halo_buffer(blk, face)), (blk, face)
+    J.unpack_halos()
+    B.unpack()
+    for blk in range(B.nblocks):
+        assert np.array_equal(J.get_block_padded(blk), B.get_block_padded(blk)), blk
+    J.close()
+    B.close()
+
+
+def test_ghosts_after_a_fused_sweep_are_current(jac, orc):
+    """The fused schedule writes new face values straight into the neighbours' ghosts: after the
+    sweep the padded blocks must equal the oracle's after sweep + pack + unpack."""
+    for n, b, h in [((36, 24), (12, 8), 2), ((24, 18, 12), (8, 6, 4), 3), ((15, 9), (5, 3), 1)]:
+        J, B = _setup_pair(jac, orc, n, b, h, True, "fused", seed=3)
+        J.sweep(3)
+        B.sweep(3)
+        B.pack()
+        B.unpack()
+        for blk in range(B.nblocks):
+            assert np.array_equal(J.get_block_padded(blk), B.get_block_padded(blk)), (n, blk)
+        J.close()
+        B.close()
+
+
+def test_device_resident_set_and_get(jac, orc):
+    import torch
+    n, b = (130, 70), (26, 14)
+    u0, f = _random_problem(n, 5)
+    J = jac.Jacobi(n, b, 1, True)
+    J.set_u_device(torch.from_numpy(u0).cuda())
+    J.set_f_device(torch.from_numpy(f).cuda())
+    assert np.array_equal(J.get_u_device().cpu().numpy(), u0)
+    assert np.array_equal(J.get_u(), u0)
+    B = orc.Blocked(n, b, 1, True)
+    B.set_u(u0)
+    B.set_f(f)
+    J.sweep(3)
+    B.sweep(3)
+    _assert_sweep_close(J.get_u_device().cpu().numpy(), B.get_u())
+    J.close()
+
+
+def test_residual_is_repeatable_and_matches_norm_of_f_at_zero(jac):
+    n, b = (96, 80), (32, 16)
+    _, f = _random_problem(n, 6)
+    J = jac.Jacobi(n, b, 1, True)
+    J.set_f(f)
+    r = [J.residual() for _ in range(3)]
+    assert r[0] == r[1] == r[2]
+    assert r[0] == pytest.approx(np.linalg.norm(f), rel=1e-13)
+    J.close()
+
+
+def test_empty_and_error_paths(jac):
+    import ctypes as C
+    J = jac.Jacobi((8, 8), (4, 4))
+    J.sweep(0)
+    with pytest.raises(jac.JacError):
+        J.sweep(-1)
+    with pytest.raises(jac.JacError):
+        J.set_boundary(4, 1.0)       # no z faces in 2D
+    with pytest.raises(jac.JacError):
+        J.get_halo_buffer(99, 0)
+    with pytest.raises(jac.JacError):
+        J.set_f(np.zeros((8, 8)))    # created without f
+    assert jac.lib().jac_residual(J._ctx, None) == jac.EINVAL
+    # undersized / misaligned workspace
+    import torch
+    d = jac.make_desc((8, 8), (4, 4))
+    need = jac.workspace_bytes(d)
+    ws = torch.empty(need + 512, dtype=torch.uint8, device="cuda")
+    ctx = C.c_void_p()
+    assert jac.lib().jac_create(C.byref(d), ws.data_ptr(), need - 1, C.byref(ctx)) == jac.ENOMEM
+    assert jac.lib().jac_create(C.byref(d), ws.data_ptr() + 8, need, C.byref(ctx)) == jac.ENOMEM
+    assert not ctx.value
+    J.close()
+
+
+def test_launch_counts_per_schedule(jac):
+    """fused: one launch per sweep (after one initial exchange); exchange: three; per-task: one per
+    block face with a neighbour, twice, plus one per block."""
+    n, b = (32, 24), (8, 8)   # 4 x 3 blocks, interior faces: 2*(3*3 + 4*2) = 34
+    counts = {}
+    for mode in MODES:
+        J = jac.Jacobi(n, b, 1, False, mode)
+        J.set_u(np.zeros((24, 32)))
+        c0 = J.launch_count()
+        J.sweep(5)
+        counts[mode] = J.launch_count() - c0
+        J.close()
+    assert counts["fused"] == 2 + 5
+    assert counts["exchange"] == 3 * 5
+    assert counts["pertask"] == 5 * (2 * 34 + 12)
