@@ -32,12 +32,14 @@ def needs_build() -> bool:
     return any(p.stat().st_mtime > t for p in [*SOURCES, *HEADERS, Path(__file__)])
 
 
-def build(force: bool = False, verbose: bool = False) -> Path:
-    if not force and not needs_build():
+def build(force: bool = False, verbose: bool = False, out: Path | None = None, defines=()) -> Path:
+    """Compile the library.  ``out``/``defines`` build a variant (-DNAME=VALUE) somewhere else."""
+    LIB = Path(out) if out else globals()["LIB"]
+    if not force and not out and not needs_build():
         return LIB
     nvcc = os.environ.get("NVCC", "nvcc")
     tmp = LIB.with_suffix(f".{os.getpid()}.tmp")
-    cmd = [nvcc, *NVCC_FLAGS, f"-I{ROOT / 'include'}", f"-I{CSRC}"]
+    cmd = [nvcc, *NVCC_FLAGS, f"-I{ROOT / 'include'}", f"-I{CSRC}", *[f"-D{d}" for d in defines]]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += ["-o", str(tmp), *map(str, SOURCES)]

@@ -68,7 +68,7 @@ int build_geometry(const jac_desc* d, JacGeom* g, jac_layout* L)
     if (d->halo < 1 || d->halo > 8) return JAC_EINVAL;
     if (d->has_f != 0 && d->has_f != 1) return JAC_EINVAL;
     if (d->mode < JAC_MODE_FUSED || d->mode > JAC_MODE_EXCHANGE) return JAC_EINVAL;
-    if (d->tsteps < 0 || d->tsteps > 8 || d->reserved != 0) return JAC_EINVAL;
+    if (d->tsteps < 0 || d->tsteps > 4 || d->reserved != 0) return JAC_EINVAL;
     long long n[3] = {1, 1, 1}, b[3] = {1, 1, 1}, gr[3] = {1, 1, 1};
     for (int a = 0; a < d->ndim; ++a) {
         n[a] = d->n[a];
@@ -322,6 +322,34 @@ int usable(jac_ctx* c)
 
 int default_tsteps(const jac_desc& d) { return d.tsteps > 0 ? d.tsteps : 4; }
 
+// T sweeps in one launch (2D, register-streaming temporal blocking)
+template <int T>
+int launch_temporal(jac_ctx* c, const double* u, double* un)
+{
+    const JacGeom& g = c->g;
+    const int strips_x = (int)ceil_div(g.nx, 120);
+    int rows = 256;
+    while (rows > 32 && (long long)strips_x * ceil_div(g.ny, rows) < (long long)kNumSMs * 48) rows /= 2;
+    const int strips_y = (int)ceil_div(g.ny, rows);
+    const unsigned grid = (unsigned)ceil_div((long long)strips_x * strips_y, jac::kTemporalWarps);
+    const int threads = jac::kTemporalWarps * 32;
+    if (c->desc.has_f)
+        jac::temporal2d_kernel<T, true><<<grid, threads, 0, c->stream>>>(u, un, c->f, g, strips_x, strips_y, rows);
+    else
+        jac::temporal2d_kernel<T, false><<<grid, threads, 0, c->stream>>>(u, un, c->f, g, strips_x, strips_y, rows);
+    return check_launch(c);
+}
+
+int launch_temporal_n(jac_ctx* c, int t, const double* u, double* un)
+{
+    switch (t) {
+        case 1: return launch_temporal<1>(c, u, un);
+        case 2: return launch_temporal<2>(c, u, un);
+        case 3: return launch_temporal<3>(c, u, un);
+        default: return launch_temporal<4>(c, u, un);
+    }
+}
+
 }  // namespace
 
 // =====================================================================================
@@ -358,7 +386,7 @@ int jac_create(const jac_desc* desc, void* dev_workspace, size_t bytes, jac_ctx*
     jac_layout L;
     int rc = build_geometry(desc, &g, &L);
     if (rc) return rc;
-    if (desc->mode == JAC_MODE_TEMPORAL && desc->ndim != 2) return JAC_EINVAL;
+    if (desc->mode == JAC_MODE_TEMPORAL && (desc->ndim != 2 || desc->b[0] % 4 != 0)) return JAC_EINVAL;
     if (!dev_workspace || bytes < (size_t)L.total_bytes || ((uintptr_t)dev_workspace & 255u))
         return JAC_ENOMEM;
     int dev = -1;
@@ -555,9 +583,18 @@ int jac_sweep(jac_ctx* c, int nsweeps)
                 c->packed_current = false;
             }
             break;
-        case JAC_MODE_TEMPORAL:
-            (void)default_tsteps;
-            return JAC_EINVAL;
+        case JAC_MODE_TEMPORAL: {
+            const int T = default_tsteps(c->desc);
+            for (int left = nsweeps; left > 0;) {
+                const int t = std::min(T, left);
+                if ((rc = launch_temporal_n(c, t, c->u[c->cur], c->u[c->cur ^ 1]))) return rc;
+                c->cur ^= 1;
+                left -= t;
+            }
+            c->ghosts_fresh = false;
+            c->packed_current = false;
+            break;
+        }
         default:
             return JAC_EINVAL;
     }

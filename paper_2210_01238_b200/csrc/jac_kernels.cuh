@@ -374,4 +374,262 @@ dense_copy_kernel(double* __restrict__ blocks, double* __restrict__ dense, const
     }
 }
 
+// ---------------------------------------------------------------------------------------
+// 2D temporal blocking: T sweeps per launch, in registers.
+//
+// A warp owns a strip 128 columns wide (4 consecutive points per lane) and streams it along
+// y.  Input row r enters at level 0; level s (s = 1..T) trails it and produces its row
+// r - 2s + 1 from rows r-2s, r-2s+1, r-2s+2 of level s-1, so a T-deep pipeline of 3-row
+// windows lives in registers (3*4*T doubles per lane).  Each level lags the one below by two
+// rows, so within one step no level waits for another (they are evaluated top level first):
+// the fp64 pipe always has 4*T independent points to work on.  West/east neighbours come from
+// the adjacent lanes by shuffle, so warps never synchronise with each other.  The two edge
+// lanes of a warp lose one point of validity per level; lanes 1..30 (120 columns) are exact
+// after T <= 4 levels and are the ones stored.  Strips read across block borders directly
+// (the neighbour's interior is the halo), which is what an exchange before every sweep would
+// deliver; Dirichlet values are injected for rows/columns outside the domain at every level.
+//
+// Input rows are fetched with cp.async into a per-warp shared-memory ring DEPTH rows deep, so
+// the loads in flight cost no registers.  Requires bx % 4 == 0.
+// ---------------------------------------------------------------------------------------
+#ifndef JAC_TW
+#define JAC_TW 4      // warps per CTA (independent strips)
+#endif
+#ifndef JAC_TD
+#define JAC_TD 8      // input rows in flight per warp
+#endif
+#ifndef JAC_TCOPY
+#define JAC_TCOPY 2   // 0: each lane copies its own 32 B (.cg); 1: same through L1 (.ca);
+#endif                // 2: each copy instruction covers 512 contiguous bytes of the row
+#ifndef JAC_TOCC
+#define JAC_TOCC 3    // CTAs per SM the register allocation aims for
+#endif
+constexpr int kTemporalWarps = JAC_TW;
+constexpr int kTemporalDepth = JAC_TD;
+
+struct RowCursor {
+    long long off;  // element offset of the row within the array, relative to a lane's column base
+    int j;          // row index inside its block (negative while still below the domain)
+    __device__ __forceinline__ void init(long long gy, const JacGeom& g, long long block_row_stride) {
+        if (gy < 0) { j = (int)gy; off = gy * g.PX; }
+        else {
+            const long long byi = gy / g.by;
+            j = (int)(gy - byi * g.by);
+            off = byi * block_row_stride + (long long)j * g.PX;
+        }
+    }
+    __device__ __forceinline__ void advance(const JacGeom& g, long long block_row_stride) {
+        ++j;
+        off += g.PX;
+        if (j == g.by) { j = 0; off += block_row_stride - (long long)g.by * g.PX; }
+    }
+};
+
+struct Row4 { double v[4]; };
+
+__device__ __forceinline__ Row4 load_row4(const double* p) {
+    const double2 a = *reinterpret_cast<const double2*>(p);
+    const double2 b = *reinterpret_cast<const double2*>(p + 2);
+    Row4 r; r.v[0] = a.x; r.v[1] = a.y; r.v[2] = b.x; r.v[3] = b.y; return r;
+}
+__device__ __forceinline__ void store_row4(double* p, const Row4& r) {
+    *reinterpret_cast<double2*>(p) = make_double2(r.v[0], r.v[1]);
+    *reinterpret_cast<double2*>(p + 2) = make_double2(r.v[2], r.v[3]);
+}
+__device__ __forceinline__ Row4 fill_row4(double c) { Row4 r; r.v[0] = r.v[1] = r.v[2] = r.v[3] = c; return r; }
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+    const unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
+#if JAC_TCOPY == 1
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem_src) : "memory");
+#else
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem_src) : "memory");
+#endif
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+}
+
+template <int T>
+struct TemporalCtx {
+    const double* ub;     // u + this lane's column base (its 4 points)
+    const double* fb;
+    double* ob;
+    const double* src_a;  // copy sources: the lane's own 4 points (JAC_TCOPY 0/1), or the two
+    const double* src_b;  //   16-byte chunks it copies for the warp (JAC_TCOPY 2)
+    bool copy_a, copy_b;  // chunk lies inside the domain
+    double2* ring;        // the warp's ring: [stage][64 double2]
+    long long brs;        // elements between vertically adjacent blocks
+    long long ny;
+    long long r0;         // first input row of the strip
+    long long in_end;     // one past the last input row that is needed
+    long long Y0, Y1;     // output rows of this strip
+    double cx;            // Dirichlet value for this lane if it is outside the domain in x
+    double c_my, c_py;    // Dirichlet values below / above the domain
+    int lane;
+    bool xout, edge_x, store_lane;
+};
+
+// start the copy of input row r into its ring stage (nothing to copy outside the domain)
+template <int T>
+__device__ __forceinline__ void issue_row(const TemporalCtx<T>& c, long long r, const RowCursor& cur) {
+    if (r >= 0 && r < c.ny && r < c.in_end) {
+        double2* st = c.ring + (int)((r - c.r0) % kTemporalDepth) * 64;
+#if JAC_TCOPY == 2
+        if (c.copy_a) cp_async16(st + c.lane, c.src_a + cur.off);
+        if (c.copy_b) cp_async16(st + 32 + c.lane, c.src_b + cur.off);
+#else
+        if (c.copy_a) {
+            cp_async16(st + 2 * c.lane, c.src_a + cur.off);
+            cp_async16(st + 2 * c.lane + 1, c.src_a + cur.off + 2);
+        }
+#endif
+    }
+    cp_async_commit();
+}
+
+// input row r for this lane once its copy has landed (Dirichlet value outside the domain)
+template <int T>
+__device__ __forceinline__ Row4 take_row(const TemporalCtx<T>& c, long long r) {
+    if (r < 0) return fill_row4(c.xout ? c.cx : c.c_my);
+    if (r >= c.ny) return fill_row4(c.xout ? c.cx : c.c_py);
+    if (c.xout) return fill_row4(c.cx);
+    const double2* st = c.ring + (int)((r - c.r0) % kTemporalDepth) * 64 + 2 * c.lane;
+    const double2 a = st[0], b = st[1];
+    Row4 o; o.v[0] = a.x; o.v[1] = a.y; o.v[2] = b.x; o.v[3] = b.y;
+    return o;
+}
+
+__host__ __device__ constexpr int slot3(int ph, int d) { return (((ph + d) % 3) + 3) % 3; }
+
+// one pipeline step: input row r arrives (phase PH = (r - r0) mod 3), every level advances one row
+template <int T, bool HAS_F, int PH>
+__device__ __forceinline__ void temporal_step(Row4 (&win)[T][3], const TemporalCtx<T>& c, const JacGeom& g,
+                                              long long r, RowCursor& load_cur, RowCursor (&lvl_cur)[T])
+{
+    cp_async_wait<kTemporalDepth - 1>();
+#if JAC_TCOPY == 2
+    __syncwarp();                                    // other lanes' chunks of row r have landed too
+#endif
+    win[0][PH] = take_row<T>(c, r);
+#if JAC_TCOPY == 2
+    __syncwarp();                                    // everyone has read the stage before it is refilled
+#endif
+    issue_row<T>(c, r + kTemporalDepth, load_cur);   // refills the stage just read
+    load_cur.advance(g, c.brs);
+#pragma unroll
+    for (int s = T; s >= 1; --s) {
+        const int d = -2 * s + 1;              // level s produces row r + d
+        const long long rs = r + d;
+        const Row4& S = win[s - 1][slot3(PH, d - 1)];
+        const Row4& M = win[s - 1][slot3(PH, d)];
+        const Row4& N = win[s - 1][slot3(PH, d + 1)];
+        const double w = __shfl_up_sync(0xffffffffu, M.v[3], 1);
+        const double e = __shfl_down_sync(0xffffffffu, M.v[0], 1);
+        const bool row_in = rs >= 0 && rs < c.ny;
+        Row4 ff;
+        if (HAS_F) {
+            if (row_in && !c.xout) ff = load_row4(c.fb + lvl_cur[s - 1].off);
+            else ff = fill_row4(0.0);
+        }
+        Row4 o;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const double W = (q == 0) ? w : M.v[q - 1];
+            const double E = (q == 3) ? e : M.v[q + 1];
+            double sum = add_rn(add_rn(W, E), add_rn(S.v[q], N.v[q]));
+            if (HAS_F) sum = add_rn(sum, ff.v[q]);
+            o.v[q] = mul_rn(sum, 0.25);
+        }
+        if (!row_in) o = fill_row4(rs < 0 ? c.c_my : c.c_py);
+        if (c.edge_x && c.xout) o = fill_row4(c.cx);
+        if (s < T) {
+            win[s][slot3(PH, d)] = o;
+        } else if (c.store_lane && rs >= c.Y0 && rs < c.Y1) {
+            store_row4(c.ob + lvl_cur[T - 1].off, o);
+        }
+        lvl_cur[s - 1].advance(g, c.brs);
+    }
+}
+
+// element offset of global column gx (row 0 of block row 0); gx must be inside the domain
+__device__ __forceinline__ long long column_base(const JacGeom& g, long long gx) {
+    const long long bxi = gx / g.bx;
+    return bxi * g.block_stride + g.origin + (gx - bxi * g.bx);
+}
+
+template <int T, bool HAS_F>
+__global__ void __launch_bounds__(kTemporalWarps * 32, JAC_TOCC)
+temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const double* __restrict__ f,
+                  const JacGeom g, const int strips_x, const int strips_y, const int rows_per_strip)
+{
+    __shared__ double2 ring_mem[kTemporalWarps][kTemporalDepth][64];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long wid = (long long)blockIdx.x * kTemporalWarps + warp;
+    if (wid >= (long long)strips_x * strips_y) return;   // whole warps only; warps never meet at a barrier
+    const int sx = (int)(wid % strips_x), sy = (int)(wid / strips_x);
+
+    TemporalCtx<T> c;
+    c.lane = lane;
+    const long long X0 = (long long)sx * 120 - 4;
+    const long long gx = X0 + 4 * lane;
+    c.xout = gx < 0 || gx >= g.nx;
+    c.cx = gx < 0 ? g.bval[0] : g.bval[1];
+    c.c_my = g.bval[2];
+    c.c_py = g.bval[3];
+    c.edge_x = (sx == 0) || (X0 + 128 > g.nx);
+    c.store_lane = lane >= 1 && lane <= 30 && !c.xout;
+    const long long col = c.xout ? g.origin : column_base(g, gx);
+    c.ub = u + col;
+    c.fb = HAS_F ? f + col : nullptr;
+    c.ob = un + col;
+#if JAC_TCOPY == 2
+    const long long xa = X0 + 2 * lane, xb = X0 + 64 + 2 * lane;
+    c.copy_a = xa >= 0 && xa < g.nx;
+    c.copy_b = xb >= 0 && xb < g.nx;
+    c.src_a = u + (c.copy_a ? column_base(g, xa) : g.origin);
+    c.src_b = u + (c.copy_b ? column_base(g, xb) : g.origin);
+#else
+    c.copy_a = !c.xout;
+    c.copy_b = false;
+    c.src_a = c.ub;
+    c.src_b = c.ub;
+#endif
+    c.ring = &ring_mem[warp][0][0];
+    c.brs = g.block_stride * g.gx;
+    c.ny = g.ny;
+    c.Y0 = (long long)sy * rows_per_strip;
+    c.Y1 = min(g.ny, c.Y0 + rows_per_strip);
+    c.r0 = c.Y0 - T;
+    c.in_end = c.Y1 + T;
+    const long long r_end = c.Y1 + 2 * T - 1;   // the top level trails the input by 2T - 1 rows
+
+    Row4 win[T][3];
+#pragma unroll
+    for (int s = 0; s < T; ++s)
+#pragma unroll
+        for (int k = 0; k < 3; ++k) win[s][k] = fill_row4(0.0);
+
+    RowCursor load_cur;
+    load_cur.init(c.r0, g, c.brs);
+    RowCursor lvl_cur[T];
+#pragma unroll
+    for (int s = 1; s <= T; ++s) lvl_cur[s - 1].init(c.r0 - 2 * s + 1, g, c.brs);
+
+    // fill the ring with the first DEPTH rows
+#pragma unroll 1
+    for (int k = 0; k < kTemporalDepth; ++k) {
+        issue_row<T>(c, c.r0 + k, load_cur);
+        load_cur.advance(g, c.brs);
+    }
+
+    for (long long r = c.r0; r < r_end; r += 3) {
+        temporal_step<T, HAS_F, 0>(win, c, g, r, load_cur, lvl_cur);
+        if (r + 1 < r_end) temporal_step<T, HAS_F, 1>(win, c, g, r + 1, load_cur, lvl_cur);
+        if (r + 2 < r_end) temporal_step<T, HAS_F, 2>(win, c, g, r + 2, load_cur, lvl_cur);
+    }
+    cp_async_wait<0>();
+}
+
 }  // namespace jac

@@ -12,12 +12,14 @@ an exception is raised.
 from __future__ import annotations
 
 import ctypes as C
+import os
 from pathlib import Path
 
 import numpy as np
 
 _PKG = Path(__file__).resolve().parent
-LIB_PATH = _PKG / "libjac.so"
+# JAC_LIB selects another build of the same library (e.g. one compiled with different tile sizes)
+LIB_PATH = Path(os.environ["JAC_LIB"]) if os.environ.get("JAC_LIB") else _PKG / "libjac.so"
 
 MODE_FUSED, MODE_PERTASK, MODE_TEMPORAL, MODE_EXCHANGE = 0, 1, 2, 3
 MODES = {"fused": MODE_FUSED, "pertask": MODE_PERTASK, "temporal": MODE_TEMPORAL,

@@ -191,3 +191,35 @@ def test_launch_counts_per_schedule(jac):
     assert counts["fused"] == 2 + 5
     assert counts["exchange"] == 3 * 5
     assert counts["pertask"] == 5 * (2 * 34 + 12)
+
+
+# temporal blocking: widths that leave ragged strips (120 columns per warp), several row strips,
+# blocks narrower and wider than a strip, every depth, sweep counts that leave a remainder
+TEMPORAL_SHAPES = [((8, 8), (4, 4)), ((120, 40), (60, 20)), ((124, 33), (124, 33)),
+                   ((256, 100), (64, 25)), ((1100, 200), (220, 50)), ((36, 24), (12, 8)),
+                   ((480, 96), (4, 1)), ((2048, 300), (1024, 150))]
+
+
+@pytest.mark.parametrize("n,b", TEMPORAL_SHAPES)
+@pytest.mark.parametrize("tsteps", [1, 2, 3, 4])
+@pytest.mark.parametrize("has_f", [False, True])
+def test_temporal_blocking_matches_oracle(jac, orc, n, b, tsteps, has_f):
+    J, B = _setup_pair(jac, orc, n, b, 1, has_f, "temporal", seed=2, tsteps=tsteps)
+    for nsw in (1, 4, 7):
+        J.sweep(nsw)
+        B.sweep(nsw)
+        _assert_sweep_close(J.get_u(), B.get_u())
+    r_gpu, r_cpu = J.residual(), B.residual()
+    assert abs(r_gpu - r_cpu) <= RESID_TOL * r_cpu
+    J.sweep(5)
+    B.sweep(5)
+    _assert_sweep_close(J.get_u(), B.get_u())
+    J.close()
+    B.close()
+
+
+def test_temporal_mode_rejects_unsupported_shapes(jac):
+    with pytest.raises(jac.JacError):
+        jac.Jacobi((12, 8), (6, 4), mode="temporal")          # bx % 4 != 0
+    with pytest.raises(jac.JacError):
+        jac.Jacobi((8, 8, 8), (4, 4, 4), mode="temporal")     # 3D
