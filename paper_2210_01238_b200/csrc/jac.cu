@@ -386,7 +386,9 @@ int jac_create(const jac_desc* desc, void* dev_workspace, size_t bytes, jac_ctx*
     jac_layout L;
     int rc = build_geometry(desc, &g, &L);
     if (rc) return rc;
-    if (desc->mode == JAC_MODE_TEMPORAL && (desc->ndim != 2 || desc->b[0] % 4 != 0)) return JAC_EINVAL;
+    if (desc->mode == JAC_MODE_TEMPORAL &&
+        (desc->ndim != 2 || desc->b[0] % 4 != 0 || desc->n[1] >= (1LL << 30)))
+        return JAC_EINVAL;
     if (!dev_workspace || bytes < (size_t)L.total_bytes || ((uintptr_t)dev_workspace & 255u))
         return JAC_ENOMEM;
     int dev = -1;

@@ -388,9 +388,11 @@ dense_copy_kernel(double* __restrict__ blocks, double* __restrict__ dense, const
 // after T <= 4 levels and are the ones stored.  Strips read across block borders directly
 // (the neighbour's interior is the halo), which is what an exchange before every sweep would
 // deliver; Dirichlet values are injected for rows/columns outside the domain at every level.
+// Steps that touch no domain boundary run a variant without any of those fix-ups.
 //
 // Input rows are fetched with cp.async into a per-warp shared-memory ring DEPTH rows deep, so
-// the loads in flight cost no registers.  Requires bx % 4 == 0.
+// the loads in flight cost no registers; each copy instruction of a warp covers 512
+// contiguous bytes of the row.  Requires bx % 4 == 0 and ny < 2^30.
 // ---------------------------------------------------------------------------------------
 #ifndef JAC_TW
 #define JAC_TW 4      // warps per CTA (independent strips)
@@ -398,9 +400,6 @@ dense_copy_kernel(double* __restrict__ blocks, double* __restrict__ dense, const
 #ifndef JAC_TD
 #define JAC_TD 8      // input rows in flight per warp
 #endif
-#ifndef JAC_TCOPY
-#define JAC_TCOPY 2   // 0: each lane copies its own 32 B (.cg); 1: same through L1 (.ca);
-#endif                // 2: each copy instruction covers 512 contiguous bytes of the row
 #ifndef JAC_TOCC
 #define JAC_TOCC 3    // CTAs per SM the register allocation aims for
 #endif
@@ -410,11 +409,11 @@ constexpr int kTemporalDepth = JAC_TD;
 struct RowCursor {
     long long off;  // element offset of the row within the array, relative to a lane's column base
     int j;          // row index inside its block (negative while still below the domain)
-    __device__ __forceinline__ void init(long long gy, const JacGeom& g, long long block_row_stride) {
-        if (gy < 0) { j = (int)gy; off = gy * g.PX; }
+    __device__ __forceinline__ void init(int gy, const JacGeom& g, long long block_row_stride) {
+        if (gy < 0) { j = gy; off = (long long)gy * g.PX; }
         else {
-            const long long byi = gy / g.by;
-            j = (int)(gy - byi * g.by);
+            const int byi = gy / g.by;
+            j = gy - byi * g.by;
             off = byi * block_row_stride + (long long)j * g.PX;
         }
     }
@@ -440,62 +439,57 @@ __device__ __forceinline__ Row4 fill_row4(double c) { Row4 r; r.v[0] = r.v[1] = 
 
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
     const unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
-#if JAC_TCOPY == 1
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem_src) : "memory");
-#else
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem_src) : "memory");
-#endif
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
 }
 
-template <int T>
+// Per-lane constants of a strip.  A ring stage holds one row as 64 chunks of 16 bytes in
+// natural order (chunk k = columns 2k, 2k+1 of the strip).  One copy instruction of the warp
+// moves chunks `lane` (or `32 + lane`): 512 contiguous bytes on both sides, which the memory
+// pipeline turns into four full-line requests (a permuted shared-memory destination was
+// measured to split it into per-lane sector requests and to triple the L2 request count).
+// A lane then reads its own 4 points from chunks 2*lane and 2*lane + 1.
 struct TemporalCtx {
-    const double* ub;     // u + this lane's column base (its 4 points)
-    const double* fb;
-    double* ob;
-    const double* src_a;  // copy sources: the lane's own 4 points (JAC_TCOPY 0/1), or the two
-    const double* src_b;  //   16-byte chunks it copies for the warp (JAC_TCOPY 2)
-    bool copy_a, copy_b;  // chunk lies inside the domain
-    double2* ring;        // the warp's ring: [stage][64 double2]
+    const double* fb;     // f + this lane's column base (its 4 points)
+    double* ob;           // u' + this lane's column base
+    const double* src_a;  // u + column base of chunk `lane`
+    const double* src_b;  // u + column base of chunk `32 + lane`
+    double2* dst_a;       // ring positions (stage 0) of the two chunks this lane copies
+    double2* dst_b;
+    const double2* mine;  // ring position (stage 0) of this lane's first chunk
     long long brs;        // elements between vertically adjacent blocks
-    long long ny;
-    long long r0;         // first input row of the strip
-    long long in_end;     // one past the last input row that is needed
-    long long Y0, Y1;     // output rows of this strip
+    int ny;
+    int r0;               // first input row of the strip
+    int in_end;           // one past the last input row that is needed
+    int Y0, Y1;           // output rows of this strip
     double cx;            // Dirichlet value for this lane if it is outside the domain in x
     double c_my, c_py;    // Dirichlet values below / above the domain
-    int lane;
+    bool copy_a, copy_b;  // chunk lies inside the domain
     bool xout, edge_x, store_lane;
 };
 
 // start the copy of input row r into its ring stage (nothing to copy outside the domain)
-template <int T>
-__device__ __forceinline__ void issue_row(const TemporalCtx<T>& c, long long r, const RowCursor& cur) {
+__device__ __forceinline__ void issue_row(const TemporalCtx& c, int r, const RowCursor& cur) {
     if (r >= 0 && r < c.ny && r < c.in_end) {
-        double2* st = c.ring + (int)((r - c.r0) % kTemporalDepth) * 64;
-#if JAC_TCOPY == 2
-        if (c.copy_a) cp_async16(st + c.lane, c.src_a + cur.off);
-        if (c.copy_b) cp_async16(st + 32 + c.lane, c.src_b + cur.off);
-#else
-        if (c.copy_a) {
-            cp_async16(st + 2 * c.lane, c.src_a + cur.off);
-            cp_async16(st + 2 * c.lane + 1, c.src_a + cur.off + 2);
-        }
-#endif
+        const int st = ((r - c.r0) % kTemporalDepth) * 64;
+        if (c.copy_a) cp_async16(c.dst_a + st, c.src_a + cur.off);
+        if (c.copy_b) cp_async16(c.dst_b + st, c.src_b + cur.off);
     }
     cp_async_commit();
 }
 
-// input row r for this lane once its copy has landed (Dirichlet value outside the domain)
-template <int T>
-__device__ __forceinline__ Row4 take_row(const TemporalCtx<T>& c, long long r) {
-    if (r < 0) return fill_row4(c.xout ? c.cx : c.c_my);
-    if (r >= c.ny) return fill_row4(c.xout ? c.cx : c.c_py);
-    if (c.xout) return fill_row4(c.cx);
-    const double2* st = c.ring + (int)((r - c.r0) % kTemporalDepth) * 64 + 2 * c.lane;
+// input row r for this lane once its copy has landed
+template <bool EDGE>
+__device__ __forceinline__ Row4 take_row(const TemporalCtx& c, int r) {
+    if (EDGE) {   // Dirichlet value outside the domain
+        if (r < 0) return fill_row4(c.xout ? c.cx : c.c_my);
+        if (r >= c.ny) return fill_row4(c.xout ? c.cx : c.c_py);
+        if (c.xout) return fill_row4(c.cx);
+    }
+    const double2* st = c.mine + ((r - c.r0) % kTemporalDepth) * 64;
     const double2 a = st[0], b = st[1];
     Row4 o; o.v[0] = a.x; o.v[1] = a.y; o.v[2] = b.x; o.v[3] = b.y;
     return o;
@@ -503,35 +497,40 @@ __device__ __forceinline__ Row4 take_row(const TemporalCtx<T>& c, long long r) {
 
 __host__ __device__ constexpr int slot3(int ph, int d) { return (((ph + d) % 3) + 3) % 3; }
 
-// one pipeline step: input row r arrives (phase PH = (r - r0) mod 3), every level advances one row
-template <int T, bool HAS_F, int PH>
-__device__ __forceinline__ void temporal_step(Row4 (&win)[T][3], const TemporalCtx<T>& c, const JacGeom& g,
-                                              long long r, RowCursor& load_cur, RowCursor (&lvl_cur)[T])
+// One pipeline step: input row r arrives (phase PH = (r - r0) mod 3) and every level advances
+// one row.  EDGE = false is for steps in which no row and no column involved lies outside the
+// domain: no Dirichlet fix-up is compiled in.
+template <int T, bool HAS_F, int PH, bool EDGE>
+__device__ __forceinline__ void temporal_step(Row4 (&win)[T][3], const TemporalCtx& c, const JacGeom& g,
+                                              int r, RowCursor& load_cur, RowCursor& out_cur)
 {
     cp_async_wait<kTemporalDepth - 1>();
-#if JAC_TCOPY == 2
-    __syncwarp();                                    // other lanes' chunks of row r have landed too
-#endif
-    win[0][PH] = take_row<T>(c, r);
-#if JAC_TCOPY == 2
+    __syncwarp();                                    // the other lanes' chunks of row r have landed too
+    win[0][PH] = take_row<EDGE>(c, r);
     __syncwarp();                                    // everyone has read the stage before it is refilled
-#endif
-    issue_row<T>(c, r + kTemporalDepth, load_cur);   // refills the stage just read
+    issue_row(c, r + kTemporalDepth, load_cur);
     load_cur.advance(g, c.brs);
 #pragma unroll
     for (int s = T; s >= 1; --s) {
         const int d = -2 * s + 1;              // level s produces row r + d
-        const long long rs = r + d;
+        const int rs = r + d;
         const Row4& S = win[s - 1][slot3(PH, d - 1)];
         const Row4& M = win[s - 1][slot3(PH, d)];
         const Row4& N = win[s - 1][slot3(PH, d + 1)];
         const double w = __shfl_up_sync(0xffffffffu, M.v[3], 1);
         const double e = __shfl_down_sync(0xffffffffu, M.v[0], 1);
-        const bool row_in = rs >= 0 && rs < c.ny;
         Row4 ff;
         if (HAS_F) {
-            if (row_in && !c.xout) ff = load_row4(c.fb + lvl_cur[s - 1].off);
-            else ff = fill_row4(0.0);
+            // f of row rs: the output cursor points at row r - 2T + 1, i.e. (T - s) * 2 rows below rs
+            const bool ok = EDGE ? (rs >= 0 && rs < c.ny && !c.xout) : true;
+            if (ok) {
+                RowCursor fc = out_cur;
+#pragma unroll
+                for (int k = 0; k < 2 * (T - s); ++k) fc.advance(g, c.brs);
+                ff = load_row4(c.fb + fc.off);
+            } else {
+                ff = fill_row4(0.0);
+            }
         }
         Row4 o;
 #pragma unroll
@@ -542,21 +541,34 @@ __device__ __forceinline__ void temporal_step(Row4 (&win)[T][3], const TemporalC
             if (HAS_F) sum = add_rn(sum, ff.v[q]);
             o.v[q] = mul_rn(sum, 0.25);
         }
-        if (!row_in) o = fill_row4(rs < 0 ? c.c_my : c.c_py);
-        if (c.edge_x && c.xout) o = fill_row4(c.cx);
+        if (EDGE) {
+            if (rs < 0) o = fill_row4(c.c_my);
+            if (rs >= c.ny) o = fill_row4(c.c_py);
+            if (c.xout) o = fill_row4(c.cx);
+        }
         if (s < T) {
             win[s][slot3(PH, d)] = o;
         } else if (c.store_lane && rs >= c.Y0 && rs < c.Y1) {
-            store_row4(c.ob + lvl_cur[T - 1].off, o);
+            store_row4(c.ob + out_cur.off, o);
         }
-        lvl_cur[s - 1].advance(g, c.brs);
     }
+    out_cur.advance(g, c.brs);
 }
 
 // element offset of global column gx (row 0 of block row 0); gx must be inside the domain
 __device__ __forceinline__ long long column_base(const JacGeom& g, long long gx) {
     const long long bxi = gx / g.bx;
     return bxi * g.block_stride + g.origin + (gx - bxi * g.bx);
+}
+
+template <int T, bool HAS_F, int PH>
+__device__ __forceinline__ void temporal_step_any(Row4 (&win)[T][3], const TemporalCtx& c, const JacGeom& g,
+                                                  int r, RowCursor& load_cur, RowCursor& out_cur)
+{
+    // warp-uniform: does this step see a row outside [0, ny) or a column outside [0, nx)?
+    const bool edge = c.edge_x || (r - 2 * T < 0) || (r >= c.ny);
+    if (edge) temporal_step<T, HAS_F, PH, true>(win, c, g, r, load_cur, out_cur);
+    else temporal_step<T, HAS_F, PH, false>(win, c, g, r, load_cur, out_cur);
 }
 
 template <int T, bool HAS_F>
@@ -570,8 +582,7 @@ temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
     if (wid >= (long long)strips_x * strips_y) return;   // whole warps only; warps never meet at a barrier
     const int sx = (int)(wid % strips_x), sy = (int)(wid / strips_x);
 
-    TemporalCtx<T> c;
-    c.lane = lane;
+    TemporalCtx c;
     const long long X0 = (long long)sx * 120 - 4;
     const long long gx = X0 + 4 * lane;
     c.xout = gx < 0 || gx >= g.nx;
@@ -581,29 +592,24 @@ temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
     c.edge_x = (sx == 0) || (X0 + 128 > g.nx);
     c.store_lane = lane >= 1 && lane <= 30 && !c.xout;
     const long long col = c.xout ? g.origin : column_base(g, gx);
-    c.ub = u + col;
     c.fb = HAS_F ? f + col : nullptr;
     c.ob = un + col;
-#if JAC_TCOPY == 2
     const long long xa = X0 + 2 * lane, xb = X0 + 64 + 2 * lane;
     c.copy_a = xa >= 0 && xa < g.nx;
     c.copy_b = xb >= 0 && xb < g.nx;
     c.src_a = u + (c.copy_a ? column_base(g, xa) : g.origin);
     c.src_b = u + (c.copy_b ? column_base(g, xb) : g.origin);
-#else
-    c.copy_a = !c.xout;
-    c.copy_b = false;
-    c.src_a = c.ub;
-    c.src_b = c.ub;
-#endif
-    c.ring = &ring_mem[warp][0][0];
+    double2* ring = &ring_mem[warp][0][0];
+    c.dst_a = ring + lane;        // chunk k = lane
+    c.dst_b = ring + 32 + lane;   // chunk k = 32 + lane
+    c.mine = ring + 2 * lane;     // chunks 2*lane and 2*lane + 1
     c.brs = g.block_stride * g.gx;
-    c.ny = g.ny;
-    c.Y0 = (long long)sy * rows_per_strip;
-    c.Y1 = min(g.ny, c.Y0 + rows_per_strip);
+    c.ny = (int)g.ny;
+    c.Y0 = sy * rows_per_strip;
+    c.Y1 = min(c.ny, c.Y0 + rows_per_strip);
     c.r0 = c.Y0 - T;
     c.in_end = c.Y1 + T;
-    const long long r_end = c.Y1 + 2 * T - 1;   // the top level trails the input by 2T - 1 rows
+    const int r_end = c.Y1 + 2 * T - 1;   // the top level trails the input by 2T - 1 rows
 
     Row4 win[T][3];
 #pragma unroll
@@ -611,23 +617,21 @@ temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
 #pragma unroll
         for (int k = 0; k < 3; ++k) win[s][k] = fill_row4(0.0);
 
-    RowCursor load_cur;
+    RowCursor load_cur, out_cur;
     load_cur.init(c.r0, g, c.brs);
-    RowCursor lvl_cur[T];
-#pragma unroll
-    for (int s = 1; s <= T; ++s) lvl_cur[s - 1].init(c.r0 - 2 * s + 1, g, c.brs);
+    out_cur.init(c.r0 - 2 * T + 1, g, c.brs);   // row produced by the top level in the first step
 
     // fill the ring with the first DEPTH rows
 #pragma unroll 1
     for (int k = 0; k < kTemporalDepth; ++k) {
-        issue_row<T>(c, c.r0 + k, load_cur);
+        issue_row(c, c.r0 + k, load_cur);
         load_cur.advance(g, c.brs);
     }
 
-    for (long long r = c.r0; r < r_end; r += 3) {
-        temporal_step<T, HAS_F, 0>(win, c, g, r, load_cur, lvl_cur);
-        if (r + 1 < r_end) temporal_step<T, HAS_F, 1>(win, c, g, r + 1, load_cur, lvl_cur);
-        if (r + 2 < r_end) temporal_step<T, HAS_F, 2>(win, c, g, r + 2, load_cur, lvl_cur);
+    for (int r = c.r0; r < r_end; r += 3) {
+        temporal_step_any<T, HAS_F, 0>(win, c, g, r, load_cur, out_cur);
+        if (r + 1 < r_end) temporal_step_any<T, HAS_F, 1>(win, c, g, r + 1, load_cur, out_cur);
+        if (r + 2 < r_end) temporal_step_any<T, HAS_F, 2>(win, c, g, r + 2, load_cur, out_cur);
     }
     cp_async_wait<0>();
 }
