@@ -47,6 +47,7 @@ extern "C" {
 #define JAC_ENOMEM   (-2)  /* workspace null, too small or not 256-byte aligned                  */
 #define JAC_ECUDA    (-3)  /* a CUDA runtime call failed (sticky); see jac_last_cuda_error       */
 #define JAC_ENODEV   (-4)  /* no usable CUDA device                                              */
+#define JAC_ELIMIT   (-5)  /* problem larger than the fixed scratch of jac_residual_dense_static */
 
 /* How jac_sweep schedules one iteration.  All modes leave bit-identical interiors. */
 #define JAC_MODE_FUSED    0 /* one launch per sweep over all blocks; the update also writes each
@@ -159,6 +160,33 @@ int jac_sweep(jac_ctx *ctx, int nsweeps);
  * Jacobi method.)  Exchanges halos first if the ghosts are stale, reduces on the device in a
  * fixed order (repeatable bit for bit), synchronises the stream and writes one HOST double. */
 int jac_residual(jac_ctx *ctx, double *host_out_l2);
+
+/* Residual norm of a DENSE grid without a context, a workspace or any allocation.
+ * (The paper has no counterpart: this is a convenience of this library.)
+ *
+ * For callers that cannot allocate device memory -- code living inside another framework's
+ * memory pool, a monitoring hook that must not stall the solver it watches (cudaMalloc
+ * synchronises the device), a process whose device memory is already full -- and that hold
+ * nothing but the solver's dense arrays.  Computes sqrt( sum_p ( s(p) - c*u(p) )^2 ), s as in the
+ * update, over the n[0]*n[1](*n[2]) points of `dev_u` (DEVICE pointer, dense, x fastest; n[2] is
+ * ignored when ndim == 2).  `dev_f` is a DEVICE pointer of the same shape or NULL for f == 0.
+ * `host_bvals` is a HOST array of 2*ndim Dirichlet values in face order, or NULL for all zero.
+ * `stream` is a cudaStream_t (NULL = legacy default stream).  Writes one HOST double after
+ * synchronising the stream.  Inputs are only read; nothing is retained after the call.
+ *
+ * The only scratch is a fixed ~0.5 MB array inside the library image, held by every GPU that
+ * loads the library until the process exits.  Hence:
+ *   - at most 2^29 points (a 4 GiB fp64 grid); more returns JAC_ELIMIT and does nothing;
+ *   - the array is shared by all calls on a device and keeps the previous call's contents; the
+ *     part a call uses is cleared first.  Calls whose GPU work overlaps (other streams or
+ *     threads) race on it: serialise them;
+ *   - the first call on each device looks up the array's device address; make that first call
+ *     outside any stream capture.
+ * Calls no cudaMalloc/cudaFree or other allocating routine.
+ * Errors: JAC_EINVAL (null u or out, ndim not 2 or 3, a size < 1), JAC_ELIMIT, JAC_ECUDA. */
+int jac_residual_dense_static(int ndim, const int64_t *n, const double *dev_u,
+                              const double *dev_f, const double *host_bvals, void *stream,
+                              double *host_out_l2);
 
 /* Number of kernel launches this context has issued so far (HOST output). */
 int jac_launch_count(const jac_ctx *ctx, int64_t *host_out);

@@ -13,7 +13,7 @@ PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libjac.so"
-SOURCES = [CSRC / "jac.cu"]
+SOURCES = [CSRC / "jac.cu", CSRC / "jac_static.cu"]
 HEADERS = [ROOT / "include" / "jac.h", *sorted(CSRC.glob("*.h")), *sorted(CSRC.glob("*.cuh"))]
 
 NVCC_FLAGS = [

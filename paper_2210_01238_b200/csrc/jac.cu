@@ -637,6 +637,7 @@ const char* jac_strerror(int code)
         case JAC_ENOMEM: return "workspace missing, too small or misaligned";
         case JAC_ECUDA: return "CUDA runtime error";
         case JAC_ENODEV: return "no usable CUDA device";
+        case JAC_ELIMIT: return "problem exceeds the fixed scratch of the no-allocation entry point";
         default: return "unknown error code";
     }
 }

@@ -25,14 +25,14 @@ MODE_FUSED, MODE_PERTASK, MODE_TEMPORAL, MODE_EXCHANGE = 0, 1, 2, 3
 MODES = {"fused": MODE_FUSED, "pertask": MODE_PERTASK, "temporal": MODE_TEMPORAL,
          "exchange": MODE_EXCHANGE}
 
-OK, EINVAL, ENOMEM, ECUDA, ENODEV = 0, -1, -2, -3, -4
+OK, EINVAL, ENOMEM, ECUDA, ENODEV, ELIMIT = 0, -1, -2, -3, -4, -5
 
 EXPORTS = [
     "jac_workspace_bytes", "jac_get_layout", "jac_create", "jac_destroy",
     "jac_set_u", "jac_set_f", "jac_get_u", "jac_set_u_device", "jac_set_f_device",
     "jac_get_u_device", "jac_set_boundary", "jac_get_block_padded", "jac_get_halo_buffer",
     "jac_pack_halos", "jac_unpack_halos", "jac_sweep", "jac_residual", "jac_launch_count",
-    "jac_last_cuda_error", "jac_strerror",
+    "jac_last_cuda_error", "jac_strerror", "jac_residual_dense_static",
 ]
 
 
@@ -85,6 +85,8 @@ def lib() -> C.CDLL:
         L.jac_launch_count.argtypes = [vp, C.POINTER(C.c_int64)]
         L.jac_last_cuda_error.argtypes = [vp]
         L.jac_strerror.argtypes = [C.c_int]
+        L.jac_residual_dense_static.argtypes = [C.c_int, C.POINTER(C.c_int64), vp, vp,
+                                                C.POINTER(C.c_double), vp, dp]
         L.jac_strerror.restype = C.c_char_p
         for name in EXPORTS:
             if name != "jac_strerror":
@@ -124,6 +126,33 @@ def get_layout(desc: Desc) -> Layout:
     if rc:
         raise JacError(rc, "jac_get_layout")
     return out
+
+
+def residual_dense_static(u, f=None, bvals=None, stream=None) -> float:
+    """Residual norm of dense CUDA tensors ``u`` (and ``f``) of shape (ny, nx) / (nz, ny, nx)
+    through the entry point that allocates nothing (no context, no workspace).
+
+    For callers that may not allocate device memory; see ``jac_residual_dense_static`` in
+    ``include/jac.h`` for the size limit (2^29 points) and the rule that calls on one device
+    must not overlap.  The first call on a device should be made outside stream capture.
+    """
+    import torch
+    assert u.is_cuda and u.dtype == torch.float64 and u.is_contiguous() and u.dim() in (2, 3)
+    if f is not None:
+        assert f.is_cuda and f.dtype == torch.float64 and f.is_contiguous() and f.shape == u.shape
+    ndim = u.dim()
+    n = (C.c_int64 * 3)(*(list(reversed(u.shape)) + [1] * (3 - ndim)))
+    bv = None
+    if bvals is not None:
+        assert len(bvals) == 2 * ndim
+        bv = (C.c_double * 6)(*([float(x) for x in bvals] + [0.0] * (6 - 2 * ndim)))
+    st = stream if stream is not None else torch.cuda.current_stream()
+    out = C.c_double(0.0)
+    rc = lib().jac_residual_dense_static(ndim, n, u.data_ptr(), f.data_ptr() if f is not None else None,
+                                         bv, st.cuda_stream or None, C.byref(out))
+    if rc:
+        raise JacError(rc, "jac_residual_dense_static")
+    return out.value
 
 
 def _host_ptr(a: np.ndarray):

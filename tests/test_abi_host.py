@@ -36,7 +36,7 @@ def test_library_exports_every_declared_symbol(jac):
 
 def test_strerror(jac):
     assert jac.strerror(0) == "ok"
-    for code in (-1, -2, -3, -4):
+    for code in (-1, -2, -3, -4, -5):
         assert jac.strerror(code) not in ("ok", "unknown error code")
     assert jac.strerror(-99) == "unknown error code"
 
