@@ -2,7 +2,7 @@
 """Benchmark of the Jacobi hot path on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload c3_eigenmode_16384] [--mode fused] [--tsteps T]
+                    [--workload c3_eigenmode_16384] [--mode auto] [--tsteps T]
 
 One *step* is one whole job of the workload: its sweeps (every sweep with its halo exchange:
 pack, unpack, update) followed by the residual reduction.  The metric is Jacobi GLUP/s
@@ -41,9 +41,13 @@ L2_BYTES = 126e6
 
 # DRAM bytes per launch of the dominant kernel from an ncu capture (profiles/), and the hash of
 # the kernel sources the capture was taken with; reported as null once the sources changed.
+# key: (schedule, tsteps, ndim, has_f)
 NCU_TRAFFIC = {
-    "fused": {"kernel": "sweep2d_kernel", "bytes_per_launch": None, "src_sha": None},
 }
+KERNEL_NAMES = {("temporal", 2): "temporal2d_kernel", ("fused", 2): "sweep2d_kernel (update + ghost push)",
+                ("exchange", 2): "sweep2d_kernel", ("pertask", 2): "sweep2d_kernel (one launch per block)",
+                ("fused", 3): "sweep3d_kernel (update + ghost push)", ("exchange", 3): "sweep3d_kernel",
+                ("pertask", 3): "sweep3d_kernel (one launch per block)"}
 
 
 def log(*a):
@@ -182,6 +186,27 @@ def run_reference(args, w: inputs.Workload):
 
 
 # ----------------------------------------------------------------------------- our arm
+def reduce_max_over_ranks(ms: float, device: str) -> float:
+    """The slowest rank's time: what a job of independent replicas takes as a whole."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replicated_glups(updates_per_rank: float, world: int, ms: float) -> float:
+    """Whole-job throughput of `world` independent replicas that all finish within `ms`."""
+    return updates_per_rank * world / (ms * 1e-3) / 1e9
+
+
+def default_schedule(w: inputs.Workload):
+    """Fastest schedule the library has for the workload (all schedules give identical bits)."""
+    if w.ndim == 2 and w.b[0] % 4 == 0:
+        return "temporal", 4
+    return "exchange", 1
+
+
 def run_ours(args, w: inputs.Workload):
     import torch
     import torch.distributed as dist
@@ -202,77 +227,94 @@ def run_ours(args, w: inputs.Workload):
             dist.barrier()
         torch.cuda.synchronize()
 
+    def max_over_ranks(ms: float) -> float:
+        return reduce_max_over_ranks(ms, "cuda") if distributed else ms
+
     stream = torch.cuda.current_stream()
     u0, f = make_inputs(w)
     sweeps = args.sweeps if args.sweeps > 0 else w.sweeps
-    J = jac.Jacobi(w.n, w.b, w.halo, w.has_f, args.mode, args.tsteps)
-    for face, v in enumerate(w.boundary()):
-        J.set_boundary(face, v)
     u0_dev = torch.from_numpy(u0).cuda()
-    if f is not None:
-        J.set_f(f)
-    del f
+    props = torch.cuda.get_device_properties(local)
+    uuid = str(props.uuid) if hasattr(props, "uuid") else None
+    if uuid and not uuid.startswith("GPU-"):
+        uuid = "GPU-" + uuid
+    peak, peak_kind = measured_peak_gbs()
 
-    def job():
-        J.set_u_device(u0_dev)      # device-resident input -> blocks (inside the timed job)
-        J.sweep(sweeps)
-        return J.residual()
+    def make_ctx(mode, tsteps):
+        J = jac.Jacobi(w.n, w.b, w.halo, w.has_f, mode, tsteps)
+        for face, v in enumerate(w.boundary()):
+            J.set_boundary(face, v)
+        if f is not None:
+            J.set_f(f)
+        return J
 
-    # ---- device-resident timing: K steps between two barriers, CUDA events on the launch stream
-    for _ in range(args.warmup):
-        res = job()
-    barrier()
-    sampler = ClockSampler(str(torch.cuda.get_device_properties(local).uuid)
-                           if hasattr(torch.cuda.get_device_properties(local), "uuid") else None)
-    if sampler.uuid and not sampler.uuid.startswith("GPU-"):
-        sampler.uuid = "GPU-" + sampler.uuid
-    sampler.start()
-    l0 = J.launch_count()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sweep_ms = []
-    ev0.record(stream)
-    for _ in range(args.steps):
-        J.set_u_device(u0_dev)
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(stream)
-        J.sweep(sweeps)
-        b.record(stream)
-        res = J.residual()
-        sweep_ms.append((a, b))
-    ev1.record(stream)
-    barrier()
-    launches = J.launch_count() - l0
-    clocks = sampler.stop()
-    ms_total = ev0.elapsed_time(ev1)
-    sweep_only_ms = sum(a.elapsed_time(b) for a, b in sweep_ms)
-    if distributed:
-        t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
-    value = job_updates(w, sweeps) * args.steps * world / (ms_total * 1e-3) / 1e9
+    def time_schedule(J, mode, tsteps, steps, warmup, sample_clocks):
+        """K steps (each: input -> blocks, the sweeps, the residual) between two barriers, timed
+        with CUDA events on the launch stream; the sweep calls are also timed on their own."""
+        res = None
+        for _ in range(warmup):
+            J.set_u_device(u0_dev)
+            J.sweep(sweeps)
+            res = J.residual()
+        barrier()
+        sampler = ClockSampler(uuid) if sample_clocks else None
+        if sampler:
+            sampler.start()
+        l0 = J.launch_count()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        pairs = []
+        ev0.record(stream)
+        for _ in range(steps):
+            J.set_u_device(u0_dev)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            J.sweep(sweeps)
+            b.record(stream)
+            res = J.residual()
+            pairs.append((a, b))
+        ev1.record(stream)
+        barrier()
+        launches = J.launch_count() - l0
+        clocks = sampler.stop() if sampler else None
+        ms_total = max_over_ranks(ev0.elapsed_time(ev1))
+        sweep_ms = sum(a.elapsed_time(b) for a, b in pairs)
+        n_launch = -(-sweeps // tsteps) if mode == "temporal" else sweeps
+        glups = replicated_glups(job_updates(w, sweeps) * steps, world, ms_total)
+        return {"glups": glups, "ms_total": ms_total, "launch_ms": sweep_ms / (steps * n_launch),
+                "sweeps_per_launch": sweeps / n_launch, "launches": int(launches), "residual": res,
+                "clocks": clocks}
+
+    mode, tsteps = args.mode, args.tsteps
+    if mode == "auto":
+        mode, tsteps = default_schedule(w)
+    if mode == "temporal" and not tsteps:
+        tsteps = 4
+    if mode != "temporal":
+        tsteps = 1
+    J = make_ctx(mode, tsteps)
+    main_run = time_schedule(J, mode, tsteps, args.steps, args.warmup, True)
+    value = main_run["glups"]
 
     # ---- roofline of the dominant kernel (the sweep): algorithmic bytes per launch / mean launch time
-    peak, peak_kind = measured_peak_gbs()
-    tsteps = 1
-    if args.mode == "temporal":
-        tsteps = args.tsteps or 4
-        n_launch = -(-sweeps // tsteps)
-    else:
-        n_launch = sweeps
-    sweeps_per_launch = sweeps / n_launch
-    alg_bytes_per_launch = w.points * w.bytes_per_point * sweeps_per_launch
-    launch_ms = sweep_only_ms / (args.steps * n_launch)
-    achieved = alg_bytes_per_launch / (launch_ms * 1e-3) / 1e9
+    alg_bytes_per_launch = w.points * w.bytes_per_point * main_run["sweeps_per_launch"]
+    achieved = alg_bytes_per_launch / (main_run["launch_ms"] * 1e-3) / 1e9
     traffic = None
-    rec = NCU_TRAFFIC.get(args.mode)
-    if rec and rec["bytes_per_launch"] and rec["src_sha"] == kernel_src_sha():
-        traffic = rec["bytes_per_launch"]
+    rec = NCU_TRAFFIC.get((mode, tsteps, w.ndim, w.has_f))
+    if rec and rec["src_sha"] == kernel_src_sha():
+        traffic = rec["bytes_per_point_per_launch"] * w.points
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
-                "kernel": "sweep (one launch covers all blocks)",
-                "launch_ms": launch_ms, "sweeps_per_launch": sweeps_per_launch,
+                "kernel": KERNEL_NAMES.get((mode, w.ndim), "sweep"),
+                "launch_ms": main_run["launch_ms"], "sweeps_per_launch": main_run["sweeps_per_launch"],
+                "algorithmic_bytes_per_launch": alg_bytes_per_launch,
                 "frac_of_nominal_8TBs": achieved / 8000.0,
-                "note": "time per launch includes the pack/unpack launches in the exchange schedule"}
+                "dram_gbs": traffic / (main_run["launch_ms"] * 1e-3) / 1e9 if traffic else None,
+                "note": ("one launch performs sweeps_per_launch sweeps: bytes are counted per sweep "
+                         "(16 or 24 B/point), so frac > 1 means DRAM traffic per sweep is below the "
+                         "compulsory bytes of a one-sweep-per-pass kernel; dram_gbs is the measured traffic rate"
+                         if main_run["sweeps_per_launch"] > 1 else
+                         "launch time is the mean over the timed jac_sweep calls"
+                         + (" and includes the pack and unpack launches" if mode == "exchange" else ""))}
 
     # ---- end to end through the C ABI with host buffers: H2D of u0, the job, D2H of the solution
     e2e = None
@@ -288,30 +330,42 @@ def run_ours(args, w: inputs.Workload):
         for _ in range(e2e_steps):
             J.set_u_pinned(host_in)
             J.sweep(sweeps)
-            res_e2e = J.residual()
+            J.residual()
             J.get_u_pinned(host_out)
         e1.record(stream)
         barrier()
         wall = time.perf_counter() - t0
-        ms_e2e = max(e0.elapsed_time(e1), wall * 1e3)  # the copies run on the stream; host gaps count too
-        if distributed:
-            t = torch.tensor([ms_e2e], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
+        # the copies run on the stream, so the events see them; host-side gaps count too
+        ms_e2e = max_over_ranks(max(e0.elapsed_time(e1), wall * 1e3))
         e2e = {"value": job_updates(w, sweeps) * e2e_steps * world / (ms_e2e * 1e-3) / 1e9, "unit": UNIT,
                "h2d_bytes_per_step": int(u0.nbytes), "d2h_bytes_per_step": int(u0.nbytes) + 8,
                "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps,
                "what": "jac_set_u(pinned host) + jac_sweep + jac_residual + jac_get_u(pinned host)"}
         del host_in, host_out
     J.close()
+
+    # ---- the other schedules, briefly, for context (same job, fewer steps)
+    others = {}
+    if not args.no_others and world == 1:
+        alts = [("exchange", 1), ("fused", 1)]
+        if w.ndim == 2 and w.b[0] % 4 == 0:
+            alts += [("temporal", 1), ("temporal", 2), ("temporal", 4)]
+        for m, t in alts:
+            if (m, t) == (mode, tsteps):
+                continue
+            Jo = make_ctx(m, t)
+            r = time_schedule(Jo, m, t, 2, 1, False)
+            Jo.close()
+            others[f"{m}{t if m == 'temporal' else ''}"] = {
+                "glups": r["glups"], "effective_gbs": r["glups"] * w.bytes_per_point,
+                "launch_ms": r["launch_ms"], "launches": r["launches"]}
     del u0_dev
     torch.cuda.empty_cache()
 
     # ---- the oracle on the host cores, bounded sample (rank 0, single-GPU runs only)
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        fcpu = inputs.rhs(w)
-        g, osw, dt, threads = oracle_time_job(w, u0, fcpu, 12.0, w.sweeps)
+        g, osw, dt, threads = oracle_time_job(w, u0, f, 12.0, w.sweeps)
         cpu_baseline = {"value": g, "unit": UNIT, "cores": threads, "kind": "oracle",
                         "sample": f"{osw} of {w.sweeps} sweeps (+1 residual) of the full "
                                   f"{'x'.join(map(str, w.n))} grid, {dt:.1f} s"}
@@ -319,19 +373,20 @@ def run_ours(args, w: inputs.Workload):
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
+            "warmup": args.warmup, "ms_per_step": main_run["ms_total"] / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": w.name, "grid": list(w.n), "block": list(w.b), "halo": w.halo,
                        "has_f": w.has_f, "sweeps_per_step": sweeps, "residuals_per_step": 1,
-                       "schedule": args.mode, "tsteps": tsteps,
+                       "schedule": mode, "tsteps": tsteps,
                        "l2": f"arrays of {w.points * 8 / 1e6:.0f} MB each exceed the {L2_BYTES / 1e6:.0f} MB L2"
                              if w.points * 8 > L2_BYTES else "arrays fit in L2 (no flush; latency-bound case)",
                        "replicas": world},
-            "effective_gbs": value * w.bytes_per_point,
+            "effective_gbs": value * w.bytes_per_point / world,
             "frac_of_8TBs": value * w.bytes_per_point / 8000.0 / world,
-            "residual": res,
+            "residual": main_run["residual"],
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e,
-            "gpu_launches": int(launches), "clocks": clocks,
+            "gpu_launches": main_run["launches"], "clocks": main_run["clocks"],
+            "other_schedules": others,
         }
         print(json.dumps(line), flush=True)
     if distributed:
@@ -341,15 +396,17 @@ def run_ours(args, w: inputs.Workload):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3_eigenmode_16384", choices=sorted(inputs.CONFIGS))
-    ap.add_argument("--mode", default="fused", choices=["fused", "exchange", "pertask", "temporal"])
+    ap.add_argument("--mode", default="auto", choices=["auto", "fused", "exchange", "pertask", "temporal"],
+                    help="schedule of jac_sweep; auto = the fastest one the library has for the workload")
     ap.add_argument("--tsteps", type=int, default=0)
     ap.add_argument("--sweeps", type=int, default=0, help="sweeps per step (default: the workload's)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-others", action="store_true", help="skip the brief runs of the other schedules")
     ap.add_argument("--n", type=int, default=0,
                     help="profiling aid: same recipe on an n^d grid (block size unchanged)")
     args = ap.parse_args()
