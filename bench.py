@@ -42,7 +42,12 @@ L2_BYTES = 126e6
 # DRAM bytes per launch of the dominant kernel from an ncu capture (profiles/), and the hash of
 # the kernel sources the capture was taken with; reported as null once the sources changed.
 # key: (schedule, tsteps, ndim, has_f)
+# bytes_per_point_per_launch: (dram__bytes_read.sum + dram__bytes_write.sum) / points of the captured
+# launch (profiles/temporal2d_t4_eigenmode_8192.md: 8192^2, scaled to the workload by its points --
+# traffic is proportional to the points: every strip reads and writes its own columns once).
 NCU_TRAFFIC = {
+    ("temporal", 4, 2, False): {"bytes_per_point_per_launch": (606.650368e6 + 490.201856e6) / 8192 ** 2,
+                                "src_sha": "46c902c3cd6527b9"},
 }
 KERNEL_NAMES = {("temporal", 2): "temporal2d_kernel", ("fused", 2): "sweep2d_kernel (update + ghost push)",
                 ("exchange", 2): "sweep2d_kernel", ("pertask", 2): "sweep2d_kernel (one launch per block)",
