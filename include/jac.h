@@ -147,6 +147,14 @@ int jac_pack_halos(jac_ctx *ctx);
  * unpack is the neighbour reading the send buffer in place. */
 int jac_unpack_halos(jac_ctx *ctx);
 
+/* Pack / unpack only the faces whose bit is set in face_mask (bit i = face i).  Same kernels
+ * and buffers as jac_pack_halos / jac_unpack_halos, one launch over all blocks; a mask with all
+ * 2*ndim bits set is exactly those calls.  A partial exchange never marks the ghosts as current.
+ * Lets a caller exchange one axis at a time, and lets the strided (x) and contiguous (y, z) faces
+ * be timed apart.  Errors: JAC_EINVAL for bits beyond 2*ndim. */
+int jac_pack_faces(jac_ctx *ctx, unsigned face_mask);
+int jac_unpack_faces(jac_ctx *ctx, unsigned face_mask);
+
 /* nsweeps Jacobi iterations, each "exchange halos, then update every block" (paper Section
  * V-C), scheduled as desc.mode says.  Afterwards the interiors hold the new state; the
  * inter-block ghost cells are only guaranteed current after the next jac_pack_halos +

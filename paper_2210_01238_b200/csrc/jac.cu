@@ -216,11 +216,11 @@ int halo_chunks(const jac_ctx* c, int face_lo, int face_hi)
 
 // pack or unpack all faces of all blocks in one launch
 template <bool UNPACK>
-int launch_halo_all(jac_ctx* c)
+int launch_halo_all(jac_ctx* c, unsigned face_mask = 0x3fu)
 {
     const int chunks = halo_chunks(c, 0, c->g.nfaces);
     const unsigned grid = (unsigned)(c->g.nblocks * c->g.nfaces * chunks);
-    jac::halo_kernel<UNPACK><<<grid, 256, 0, c->stream>>>(c->u[c->cur], c->send, c->g, 0, chunks);
+    jac::halo_kernel<UNPACK><<<grid, 256, 0, c->stream>>>(c->u[c->cur], c->send, c->g, 0, chunks, face_mask);
     return check_launch(c);
 }
 
@@ -241,7 +241,7 @@ int launch_halo_pertask(jac_ctx* c)
             if (!has_neighbour(c->g, blk, face)) continue;
             const int chunks = halo_chunks(c, face, face + 1);
             jac::halo_kernel<UNPACK><<<(unsigned)chunks, 256, 0, c->stream>>>(
-                c->u[c->cur], c->send, c->g, blk * c->g.nfaces + face, chunks);
+                c->u[c->cur], c->send, c->g, blk * c->g.nfaces + face, chunks, 0x3fu);
             const int rc = check_launch(c);
             if (rc) return rc;
         }
@@ -544,6 +544,28 @@ int jac_unpack_halos(jac_ctx* c)
     // ghosts are current only if the buffers were packed from the current state
     c->ghosts_fresh = c->packed_current;
     return JAC_OK;
+}
+
+int jac_pack_faces(jac_ctx* c, unsigned face_mask)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    const unsigned all = (1u << c->g.nfaces) - 1u;
+    if (face_mask & ~all) return JAC_EINVAL;
+    if (face_mask == all) return jac_pack_halos(c);
+    if (!face_mask) return JAC_OK;
+    return launch_halo_all<false>(c, face_mask);
+}
+
+int jac_unpack_faces(jac_ctx* c, unsigned face_mask)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    const unsigned all = (1u << c->g.nfaces) - 1u;
+    if (face_mask & ~all) return JAC_EINVAL;
+    if (face_mask == all) return jac_unpack_halos(c);
+    if (!face_mask) return JAC_OK;
+    return launch_halo_all<true>(c, face_mask);
 }
 
 int jac_sweep(jac_ctx* c, int nsweeps)

@@ -246,7 +246,7 @@ reduce_partials_kernel(const double* __restrict__ partials, const long long n, d
 // ---------------------------------------------------------------------------------------
 // Halo pack / unpack.  One launch covers `npairs` consecutive (block, face) pairs starting at
 // pair0 (pair = block * nfaces + face); each pair is cut into chunks of blockDim.x * EPT
-// elements.  Pairs whose face lies on the domain boundary do nothing.
+// elements.  Pairs whose face lies on the domain boundary, or is not in face_mask, do nothing.
 //
 // Element e of a packed face (source memory order):
 //   x face: e = (k*by + j)*h + c      y face: e = (k*h + r)*bx + i      z face: e = (p*by + j)*bx + i
@@ -287,13 +287,14 @@ __device__ __forceinline__ long long strip_offset(const JacGeom& g, int face, lo
 template <bool UNPACK>
 __global__ void __launch_bounds__(256)
 halo_kernel(double* __restrict__ u, double* __restrict__ send, const JacGeom g,
-            const long long pair0, const int chunks)
+            const long long pair0, const int chunks, const unsigned face_mask)
 {
     const long long t = blockIdx.x;
     const long long pair = pair0 + t / chunks;
     const int chunk = (int)(t % chunks);
     const long long blk = pair / g.nfaces;
     const int face = (int)(pair % g.nfaces);
+    if (!((face_mask >> face) & 1u)) return;
     const long long nb = neighbour_block(g, blk, face);
     if (nb < 0) return;
     const long long n = g.face_elems[face];

@@ -31,7 +31,7 @@ EXPORTS = [
     "jac_workspace_bytes", "jac_get_layout", "jac_create", "jac_destroy",
     "jac_set_u", "jac_set_f", "jac_get_u", "jac_set_u_device", "jac_set_f_device",
     "jac_get_u_device", "jac_set_boundary", "jac_get_block_padded", "jac_get_halo_buffer",
-    "jac_pack_halos", "jac_unpack_halos", "jac_sweep", "jac_residual", "jac_launch_count",
+    "jac_pack_halos", "jac_unpack_halos", "jac_pack_faces", "jac_unpack_faces", "jac_sweep", "jac_residual", "jac_launch_count",
     "jac_last_cuda_error", "jac_strerror", "jac_residual_dense_static",
 ]
 
@@ -80,6 +80,8 @@ def lib() -> C.CDLL:
         L.jac_get_halo_buffer.argtypes = [vp, C.c_int64, C.c_int, vp]
         L.jac_pack_halos.argtypes = [vp]
         L.jac_unpack_halos.argtypes = [vp]
+        L.jac_pack_faces.argtypes = [vp, C.c_uint]
+        L.jac_unpack_faces.argtypes = [vp, C.c_uint]
         L.jac_sweep.argtypes = [vp, C.c_int]
         L.jac_residual.argtypes = [vp, dp]
         L.jac_launch_count.argtypes = [vp, C.POINTER(C.c_int64)]
@@ -289,6 +291,12 @@ class Jacobi:
 
     def unpack_halos(self):
         self._call("jac_unpack_halos", lib().jac_unpack_halos(self._ctx))
+
+    def pack_faces(self, face_mask: int):
+        self._call("jac_pack_faces", lib().jac_pack_faces(self._ctx, int(face_mask)))
+
+    def unpack_faces(self, face_mask: int):
+        self._call("jac_unpack_faces", lib().jac_unpack_faces(self._ctx, int(face_mask)))
 
     def sweep(self, nsweeps: int = 1):
         self._call("jac_sweep", lib().jac_sweep(self._ctx, int(nsweeps)))

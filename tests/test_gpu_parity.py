@@ -223,3 +223,34 @@ def test_temporal_mode_rejects_unsupported_shapes(jac):
         jac.Jacobi((12, 8), (6, 4), mode="temporal")          # bx % 4 != 0
     with pytest.raises(jac.JacError):
         jac.Jacobi((8, 8, 8), (4, 4, 4), mode="temporal")     # 3D
+
+
+def test_partial_exchange_by_face_mask(jac, orc):
+    """x faces first, then y (and z): the result equals one full exchange; bad masks are refused."""
+    for n, b, h in [((36, 24), (12, 8), 2), ((24, 18, 12), (8, 6, 4), 1)]:
+        ndim = len(n)
+        dense = inputs.uniform_field(n, 4)
+        J = jac.Jacobi(n, b, h, False, "exchange")
+        B = orc.Blocked(n, b, h, False)
+        J.set_u(dense)
+        B.set_u(dense)
+        B.pack()
+        B.unpack()
+        J.pack_faces(0b11)
+        J.unpack_faces(0b11)
+        # only x ghosts are filled so far
+        for blk in range(B.nblocks):
+            got, want = J.get_block_padded(blk), B.get_block_padded(blk)
+            sl = [slice(h, -h)] * ndim
+            assert np.array_equal(got[tuple(sl)][..., :], want[tuple(sl)][..., :])
+            ysl = list(sl); ysl[ndim - 2] = slice(0, h)
+            assert np.all(got[tuple(ysl)] == 0.0)
+        rest = (1 << (2 * ndim)) - 1 - 0b11
+        J.pack_faces(rest)
+        J.unpack_faces(rest)
+        for blk in range(B.nblocks):
+            assert np.array_equal(J.get_block_padded(blk), B.get_block_padded(blk))
+        with pytest.raises(jac.JacError):
+            J.pack_faces(1 << (2 * ndim))
+        J.close()
+        B.close()
