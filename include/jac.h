@@ -50,9 +50,10 @@ extern "C" {
 #define JAC_ELIMIT   (-5)  /* problem larger than the fixed scratch of jac_residual_dense_static */
 
 /* How jac_sweep schedules one iteration.  All modes leave bit-identical interiors. */
-#define JAC_MODE_FUSED    0 /* one launch per sweep over all blocks; the update also writes each
-                               new face value straight into the neighbour's ghost cells, so the
-                               exchange for the next sweep is already done                       */
+#define JAC_MODE_FUSED    0 /* one launch per sweep over all blocks; across a face with a neighbour
+                               block the update reads the neighbour's interior cell directly (the
+                               value its packed face would carry): the exchange is fused into
+                               the sweep and the inter-block ghost cells are not touched         */
 #define JAC_MODE_PERTASK  1 /* the task-per-block schedule: per sweep one pack launch per
                                (block, face), one unpack launch per (block, face), one update
                                launch per block                                                  */

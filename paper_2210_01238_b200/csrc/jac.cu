@@ -307,9 +307,15 @@ int copy_dense_host(jac_ctx* c, double* arr, double* host, bool to_device)
 template <bool TO_BLOCKS>
 int copy_dense_device(jac_ctx* c, double* arr, double* dense)
 {
-    const long long total = c->g.nx * c->g.ny * c->g.nz;
-    const unsigned grid = (unsigned)std::min<long long>(ceil_div(total, 256), (long long)kNumSMs * 32);
-    jac::dense_copy_kernel<TO_BLOCKS><<<grid, 256, 0, c->stream>>>(arr, dense, c->g);
+    const JacGeom& g = c->g;
+    const int nv = ((g.bx % 2 == 0) && (((uintptr_t)dense & 15u) == 0)) ? 2 : 1;
+    const int segs = (int)ceil_div(ceil_div(g.nx, nv), 256);
+    const long long ctas = g.ny * g.nz * segs;
+    if (ctas > kMaxGrid) return JAC_EINVAL;
+    if (nv == 2)
+        jac::dense_copy_kernel<TO_BLOCKS, 2><<<(unsigned)ctas, 256, 0, c->stream>>>(arr, dense, g, segs);
+    else
+        jac::dense_copy_kernel<TO_BLOCKS, 1><<<(unsigned)ctas, 256, 0, c->stream>>>(arr, dense, g, segs);
     return check_launch(c);
 }
 
@@ -577,14 +583,13 @@ int jac_sweep(jac_ctx* c, int nsweeps)
     const JacGeom& g = c->g;
     switch (c->desc.mode) {
         case JAC_MODE_FUSED:
-            if (!c->ghosts_fresh && (rc = do_exchange(c))) return rc;
             for (int s = 0; s < nsweeps; ++s) {
-                if ((rc = launch_sweep<jac::OP_UPDATE_PUSH>(c, c->u[c->cur], c->u[c->cur ^ 1], 0, g.nblocks)))
+                if ((rc = launch_sweep<jac::OP_UPDATE_PULL>(c, c->u[c->cur], c->u[c->cur ^ 1], 0, g.nblocks)))
                     return rc;
                 c->cur ^= 1;
-                c->packed_current = false;
             }
-            c->ghosts_fresh = true;
+            c->ghosts_fresh = false;
+            c->packed_current = false;
             break;
         case JAC_MODE_EXCHANGE:
             for (int s = 0; s < nsweeps; ++s) {

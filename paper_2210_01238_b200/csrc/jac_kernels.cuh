@@ -13,7 +13,7 @@
 
 namespace jac {
 
-enum : int { OP_UPDATE = 0, OP_UPDATE_PUSH = 1, OP_RESIDUAL = 2 };
+enum : int { OP_UPDATE = 0, OP_UPDATE_PULL = 1, OP_RESIDUAL = 2 };
 
 __device__ __forceinline__ double add_rn(double a, double b) { return __dadd_rn(a, b); }
 __device__ __forceinline__ double sub_rn(double a, double b) { return __dsub_rn(a, b); }
@@ -61,11 +61,11 @@ __device__ __forceinline__ double block_sum(double v) {
 // west/east neighbours of the strip are read through L1 (those sectors were just fetched by
 // the neighbouring lanes' vector loads).  DRAM sees each interior point once.
 //
-// OP_UPDATE       u' <- update(u)
-// OP_UPDATE_PUSH  same, and every new value within h of a block face that has a neighbour is
-//                 also stored into that neighbour's ghost cell of u' (the exchange for the
-//                 next sweep, done while the value is in a register)
-// OP_RESIDUAL     per-CTA partial of sum r^2, r = s - 4u
+// OP_UPDATE       u' <- update(u), every out-of-block neighbour read from the block's ghosts
+// OP_UPDATE_PULL  same arithmetic, but across a face that has a neighbour block the value is
+//                 read from that block's interior (the cell its packed face would carry), so
+//                 no exchange has to run before the sweep; Dirichlet ghosts are still read
+// OP_RESIDUAL     per-CTA partial of sum r^2, r = s - 4u (ghost-reading)
 // ---------------------------------------------------------------------------------------
 template <int NV, bool HAS_F, int OP>
 __global__ void __launch_bounds__(256)
@@ -89,19 +89,26 @@ sweep2d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
         const double* fb = HAS_F ? f + base : nullptr;
         double* ob = (OP == OP_RESIDUAL) ? nullptr : un + base;
 
-        const int bxi = (int)(blk % g.gx), byi = (int)(blk / g.gx);
-        const bool nb_mx = bxi > 0, nb_px = bxi + 1 < g.gx;
-        const bool nb_my = byi > 0, nb_py = byi + 1 < g.gy;
-        const long long bs = g.block_stride;
+        // where the neighbours outside the block are found, relative to the row's own address
+        long long off_w = -1, off_e = NV;             // ghost columns
+        long long off_s0 = -PX, off_n1 = PX;          // ghost rows below row 0 / above row by-1
+        if (OP == OP_UPDATE_PULL) {
+            const int bxi = (int)(blk % g.gx), byi = (int)(blk / g.gx);
+            const long long bs = g.block_stride;
+            if (x == 0 && bxi > 0) off_w = -bs + g.bx - 1;                     // left block, last column
+            if (x + NV == g.bx && bxi + 1 < g.gx) off_e = bs - g.bx + NV;      // right block, column 0
+            if (byi > 0) off_s0 = -bs * g.gx + (long long)(g.by - 1) * PX;     // block below, last row
+            if (byi + 1 < g.gy) off_n1 = bs * g.gx - (long long)(g.by - 1) * PX;  // block above, row 0
+        }
 
-        Vec<NV> S = load_vec<NV>(ub + (long long)(j0 - 1) * PX);
+        Vec<NV> S = load_vec<NV>(ub + (j0 == 0 ? off_s0 : (long long)(j0 - 1) * PX));
         Vec<NV> Cc = load_vec<NV>(ub + (long long)j0 * PX);
 #pragma unroll 4
         for (int j = j0; j < j1; ++j) {
             const long long ro = (long long)j * PX;
-            const Vec<NV> N = load_vec<NV>(ub + ro + PX);
-            const double w = ub[ro - 1];
-            const double e = ub[ro + NV];
+            const Vec<NV> N = load_vec<NV>(ub + ro + ((OP == OP_UPDATE_PULL && j + 1 == g.by) ? off_n1 : PX));
+            const double w = ub[ro + off_w];
+            const double e = ub[ro + off_e];
             Vec<NV> ff;
             if (HAS_F) ff = load_vec<NV>(fb + ro);
             Vec<NV> o;
@@ -119,20 +126,6 @@ sweep2d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
                 }
             }
             if (OP != OP_RESIDUAL) store_vec<NV>(ob + ro, o);
-            if (OP == OP_UPDATE_PUSH) {
-                // my interior column c < h is the left neighbour's ghost column bx + c;
-                // my column c >= bx - h is the right neighbour's ghost column c - bx
-#pragma unroll
-                for (int q = 0; q < NV; ++q) {
-                    const int c = x + q;
-                    if (nb_mx && c < g.h) ob[ro + q - bs + g.bx] = o.v[q];
-                    if (nb_px && c >= g.bx - g.h) ob[ro + q + bs - g.bx] = o.v[q];
-                }
-                if (nb_my && j < g.h)
-                    store_vec<NV>(ob - bs * g.gx + (long long)(g.by + j) * PX, o);
-                if (nb_py && j >= g.by - g.h)
-                    store_vec<NV>(ob + bs * g.gx + (long long)(j - g.by) * PX, o);
-            }
             S = Cc;
             Cc = N;
         }
@@ -148,6 +141,7 @@ sweep2d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
 // `planes` z-planes and marches along z.  Planes k-1, k, k+1 of a thread's own column are
 // in registers (DRAM traffic: one load per point); the y and x neighbours of plane k come
 // through L1, which holds the plane since it was fetched as "k+1" one step earlier.
+// OP as for the 2D kernel.
 // ---------------------------------------------------------------------------------------
 template <int NV, bool HAS_F, int OP>
 __global__ void __launch_bounds__(512)
@@ -174,25 +168,32 @@ sweep3d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
         const double* fb = HAS_F ? f + base : nullptr;
         double* ob = (OP == OP_RESIDUAL) ? nullptr : un + base;
 
-        const int bxi = (int)(blk % g.gx);
-        const int byi = (int)((blk / g.gx) % g.gy);
-        const int bzi = (int)(blk / ((long long)g.gx * g.gy));
-        const bool nb_mx = bxi > 0, nb_px = bxi + 1 < g.gx;
-        const bool nb_my = byi > 0, nb_py = byi + 1 < g.gy;
-        const bool nb_mz = bzi > 0, nb_pz = bzi + 1 < g.gz;
-        const long long bs = g.block_stride;
-        const long long bsy = bs * g.gx, bsz = bs * g.gx * g.gy;
+        long long off_w = -1, off_e = NV, off_s = -PX, off_n = PX;   // within the plane
+        long long off_d0 = -PXY, off_u1 = PXY;                        // below plane 0 / above plane bz-1
+        if (OP == OP_UPDATE_PULL) {
+            const int bxi = (int)(blk % g.gx);
+            const int byi = (int)((blk / g.gx) % g.gy);
+            const int bzi = (int)(blk / ((long long)g.gx * g.gy));
+            const long long bs = g.block_stride;
+            const long long bsy = bs * g.gx, bsz = bs * g.gx * g.gy;
+            if (x == 0 && bxi > 0) off_w = -bs + g.bx - 1;
+            if (x + NV == g.bx && bxi + 1 < g.gx) off_e = bs - g.bx + NV;
+            if (y == 0 && byi > 0) off_s = -bsy + (long long)(g.by - 1) * PX;
+            if (y + 1 == g.by && byi + 1 < g.gy) off_n = bsy - (long long)(g.by - 1) * PX;
+            if (bzi > 0) off_d0 = -bsz + (long long)(g.bz - 1) * PXY;
+            if (bzi + 1 < g.gz) off_u1 = bsz - (long long)(g.bz - 1) * PXY;
+        }
 
-        Vec<NV> D = load_vec<NV>(ub + (long long)(k0 - 1) * PXY);
+        Vec<NV> D = load_vec<NV>(ub + (k0 == 0 ? off_d0 : (long long)(k0 - 1) * PXY));
         Vec<NV> Cc = load_vec<NV>(ub + (long long)k0 * PXY);
 #pragma unroll 2
         for (int k = k0; k < k1; ++k) {
             const long long po = (long long)k * PXY;
-            const Vec<NV> U = load_vec<NV>(ub + po + PXY);
-            const Vec<NV> S = load_vec<NV>(ub + po - PX);
-            const Vec<NV> N = load_vec<NV>(ub + po + PX);
-            const double w = ub[po - 1];
-            const double e = ub[po + NV];
+            const Vec<NV> U = load_vec<NV>(ub + po + ((OP == OP_UPDATE_PULL && k + 1 == g.bz) ? off_u1 : PXY));
+            const Vec<NV> S = load_vec<NV>(ub + po + off_s);
+            const Vec<NV> N = load_vec<NV>(ub + po + off_n);
+            const double w = ub[po + off_w];
+            const double e = ub[po + off_e];
             Vec<NV> ff;
             if (HAS_F) ff = load_vec<NV>(fb + po);
             Vec<NV> o;
@@ -211,18 +212,6 @@ sweep3d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
                 }
             }
             if (OP != OP_RESIDUAL) store_vec<NV>(ob + po, o);
-            if (OP == OP_UPDATE_PUSH) {
-#pragma unroll
-                for (int q = 0; q < NV; ++q) {
-                    const int c = x + q;
-                    if (nb_mx && c < g.h) ob[po + q - bs + g.bx] = o.v[q];
-                    if (nb_px && c >= g.bx - g.h) ob[po + q + bs - g.bx] = o.v[q];
-                }
-                if (nb_my && y < g.h) store_vec<NV>(ob + po - bsy + (long long)g.by * PX, o);
-                if (nb_py && y >= g.by - g.h) store_vec<NV>(ob + po + bsy - (long long)g.by * PX, o);
-                if (nb_mz && k < g.h) store_vec<NV>(ob + po - bsz + (long long)g.bz * PXY, o);
-                if (nb_pz && k >= g.bz - g.h) store_vec<NV>(ob + po + bsz - (long long)g.bz * PXY, o);
-            }
             D = Cc;
             Cc = U;
         }
@@ -354,25 +343,27 @@ fill_boundary_kernel(double* __restrict__ u0, double* __restrict__ u1, const Jac
     }
 }
 
-// Dense array (x fastest over the global interior) <-> block interiors.
-template <bool TO_BLOCKS>
+// Dense array (x fastest over the global interior) <-> block interiors.  One CTA copies a
+// segment of one dense row: the row decomposition is done once per CTA, threads move NV
+// consecutive doubles each (NV = 2 when bx is even: both sides are 16-byte aligned).
+template <bool TO_BLOCKS, int NV>
 __global__ void __launch_bounds__(256)
-dense_copy_kernel(double* __restrict__ blocks, double* __restrict__ dense, const JacGeom g)
+dense_copy_kernel(double* __restrict__ blocks, double* __restrict__ dense, const JacGeom g,
+                  const int segs_per_row)
 {
-    const long long total = g.nx * g.ny * g.nz;
-    for (long long p = (long long)blockIdx.x * blockDim.x + threadIdx.x; p < total;
-         p += (long long)gridDim.x * blockDim.x) {
-        const long long gi = p % g.nx;
-        const long long t = p / g.nx;
-        const long long gj = t % g.ny;
-        const long long gk = t / g.ny;
-        const long long bxi = gi / g.bx, byi = gj / g.by, bzi = gk / g.bz;
-        const long long blk = (bzi * g.gy + byi) * g.gx + bxi;
-        const long long off = blk * g.block_stride + g.origin + (gk - bzi * g.bz) * g.PXY +
-                              (gj - byi * g.by) * g.PX + (gi - bxi * g.bx);
-        if (TO_BLOCKS) blocks[off] = dense[p];
-        else dense[p] = blocks[off];
-    }
+    const long long row = blockIdx.x / segs_per_row;          // gj + ny * gk
+    const int seg = (int)(blockIdx.x % segs_per_row);
+    const long long gj = row % g.ny, gk = row / g.ny;
+    const long long byi = gj / g.by, bzi = gk / g.bz;
+    const long long row_off = ((bzi * g.gy + byi) * g.gx) * g.block_stride + g.origin +
+                              (gk - bzi * g.bz) * g.PXY + (gj - byi * g.by) * g.PX;
+    const long long gi = ((long long)seg * blockDim.x + threadIdx.x) * NV;
+    if (gi >= g.nx) return;
+    const long long bxi = gi / g.bx;
+    double* bp = blocks + row_off + bxi * g.block_stride + (gi - bxi * g.bx);
+    double* dp = dense + row * g.nx + gi;
+    if (TO_BLOCKS) store_vec<NV>(bp, load_vec<NV>(dp));
+    else store_vec<NV>(dp, load_vec<NV>(bp));
 }
 
 // ---------------------------------------------------------------------------------------

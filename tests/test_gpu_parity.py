@@ -107,17 +107,14 @@ def test_pack_and_unpack_are_bit_exact(jac, orc, n, b, h, mode):
     B.close()
 
 
-def test_ghosts_after_a_fused_sweep_are_current(jac, orc):
-    """The fused schedule writes new face values straight into the neighbours' ghosts: after the
-    sweep the padded blocks must equal the oracle's after sweep + pack + unpack."""
+def test_fused_sweep_needs_no_exchange_and_leaves_ghosts_alone(jac, orc):
+    """The fused schedule reads neighbour interiors directly.  No exchange ever runs here, so the
+    inter-block ghosts stay at their initial zeros: a kernel that read them would get wrong values."""
     for n, b, h in [((36, 24), (12, 8), 2), ((24, 18, 12), (8, 6, 4), 3), ((15, 9), (5, 3), 1)]:
         J, B = _setup_pair(jac, orc, n, b, h, True, "fused", seed=3)
         J.sweep(3)
         B.sweep(3)
-        B.pack()
-        B.unpack()
-        for blk in range(B.nblocks):
-            assert np.array_equal(J.get_block_padded(blk), B.get_block_padded(blk)), (n, blk)
+        assert np.array_equal(J.get_u(), B.get_u()), n
         J.close()
         B.close()
 
@@ -177,7 +174,7 @@ def test_empty_and_error_paths(jac):
 
 
 def test_launch_counts_per_schedule(jac):
-    """fused: one launch per sweep (after one initial exchange); exchange: three; per-task: one per
+    """fused: one launch per sweep; exchange: three; per-task: one per
     block face with a neighbour, twice, plus one per block."""
     n, b = (32, 24), (8, 8)   # 4 x 3 blocks, interior faces: 2*(3*3 + 4*2) = 34
     counts = {}
@@ -188,7 +185,7 @@ def test_launch_counts_per_schedule(jac):
         J.sweep(5)
         counts[mode] = J.launch_count() - c0
         J.close()
-    assert counts["fused"] == 2 + 5
+    assert counts["fused"] == 5
     assert counts["exchange"] == 3 * 5
     assert counts["pertask"] == 5 * (2 * 34 + 12)
 
