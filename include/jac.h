@@ -59,7 +59,8 @@ extern "C" {
                                launch per block                                                  */
 #define JAC_MODE_TEMPORAL 2 /* `tsteps` sweeps per launch; tiles read across block borders
                                directly (equivalent to an exchange before every sweep).
-                               2D only, b[0] % 4 == 0; jac_create returns JAC_EINVAL otherwise   */
+                               2D: b[0] % 4 == 0, tsteps <= 4; 3D: b[0] % 2 == 0, tsteps <= 2;
+                               jac_create returns JAC_EINVAL otherwise                           */
 #define JAC_MODE_EXCHANGE 3 /* per sweep three launches over all blocks: pack, unpack, update    */
 
 typedef struct jac_ctx jac_ctx; /* opaque, host memory, owned by the library */
@@ -69,7 +70,7 @@ typedef struct jac_desc {
     int32_t halo;    /* ghost width h, 1 <= h <= min(b[a]) and h <= 8                            */
     int32_t has_f;   /* 0: f == 0 and is never read (16 B/point/sweep); 1: f present (24 B)      */
     int32_t mode;    /* JAC_MODE_*                                                               */
-    int32_t tsteps;  /* JAC_MODE_TEMPORAL: sweeps per launch, 1..4; 0 = library default (4)      */
+    int32_t tsteps;  /* JAC_MODE_TEMPORAL: sweeps per launch; 0 = library default (2D 4, 3D 2)   */
     int32_t reserved;/* must be 0                                                                */
     int64_t n[3];    /* global interior points; n[2] ignored (taken as 1) when ndim == 2         */
     int64_t b[3];    /* block interior points; n[a] % b[a] == 0                                  */

@@ -326,7 +326,33 @@ int usable(jac_ctx* c)
     return JAC_OK;
 }
 
-int default_tsteps(const jac_desc& d) { return d.tsteps > 0 ? d.tsteps : 4; }
+int default_tsteps(const jac_desc& d) { return d.tsteps > 0 ? d.tsteps : (d.ndim == 2 ? 4 : 2); }
+
+// T sweeps in one launch (3D, tiles of 64 x 48 streamed along z)
+template <int T, bool HAS_F>
+int launch_temporal3d_t(jac_ctx* c, const double* u, double* un)
+{
+    const JacGeom& g = c->g;
+    const int tiles_x = (int)ceil_div(g.nx, 60);
+    const int tiles_y = (int)ceil_div(g.ny, jac::k3dTileRows - 2 * T);
+    int zchunk = 128;
+    while (zchunk > 16 && (long long)tiles_x * tiles_y * ceil_div(g.nz, zchunk) < (long long)kNumSMs * 4) zchunk /= 2;
+    const int tiles_z = (int)ceil_div(g.nz, zchunk);
+    const long long ctas = (long long)tiles_x * tiles_y * tiles_z;
+    if (ctas > kMaxGrid) return JAC_EINVAL;
+    auto kern = jac::temporal3d_kernel<T, HAS_F>;
+    JAC_CK(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)jac::k3dSmemBytes));
+    kern<<<(unsigned)ctas, jac::k3dWarps * 32, jac::k3dSmemBytes, c->stream>>>(u, un, c->f, g, tiles_x, tiles_y,
+                                                                             tiles_z, zchunk);
+    return check_launch(c);
+}
+
+int launch_temporal3d_n(jac_ctx* c, int t, const double* u, double* un)
+{
+    const bool f = c->desc.has_f != 0;
+    if (t == 1) return f ? launch_temporal3d_t<1, true>(c, u, un) : launch_temporal3d_t<1, false>(c, u, un);
+    return f ? launch_temporal3d_t<2, true>(c, u, un) : launch_temporal3d_t<2, false>(c, u, un);
+}
 
 // T sweeps in one launch (2D, register-streaming temporal blocking)
 template <int T>
@@ -392,9 +418,12 @@ int jac_create(const jac_desc* desc, void* dev_workspace, size_t bytes, jac_ctx*
     jac_layout L;
     int rc = build_geometry(desc, &g, &L);
     if (rc) return rc;
-    if (desc->mode == JAC_MODE_TEMPORAL &&
-        (desc->ndim != 2 || desc->b[0] % 4 != 0 || desc->n[1] >= (1LL << 30)))
-        return JAC_EINVAL;
+    if (desc->mode == JAC_MODE_TEMPORAL) {
+        if (desc->n[1] >= (1LL << 30)) return JAC_EINVAL;
+        if (desc->ndim == 2 && desc->b[0] % 4 != 0) return JAC_EINVAL;
+        if (desc->ndim == 3 && (desc->b[0] % 2 != 0 || desc->tsteps > 2 || desc->n[2] >= (1LL << 30)))
+            return JAC_EINVAL;
+    }
     if (!dev_workspace || bytes < (size_t)L.total_bytes || ((uintptr_t)dev_workspace & 255u))
         return JAC_ENOMEM;
     int dev = -1;
@@ -616,7 +645,9 @@ int jac_sweep(jac_ctx* c, int nsweeps)
             const int T = default_tsteps(c->desc);
             for (int left = nsweeps; left > 0;) {
                 const int t = std::min(T, left);
-                if ((rc = launch_temporal_n(c, t, c->u[c->cur], c->u[c->cur ^ 1]))) return rc;
+                rc = (g.ndim == 2) ? launch_temporal_n(c, t, c->u[c->cur], c->u[c->cur ^ 1])
+                                   : launch_temporal3d_n(c, t, c->u[c->cur], c->u[c->cur ^ 1]);
+                if (rc) return rc;
                 c->cur ^= 1;
                 left -= t;
             }

@@ -628,4 +628,299 @@ temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
     cp_async_wait<0>();
 }
 
+// ---------------------------------------------------------------------------------------
+// 3D temporal blocking: T (1 or 2) sweeps per launch.
+//
+// A CTA of 8 warps owns a tile of 64 columns x 48 rows and streams it along z.  A lane holds 2
+// consecutive points of each of its warp's 6 rows, so a warp covers 64 x 6 points of a plane.
+// Input plane p enters at level 0; level s produces plane p - 2s + 1 (two planes behind the level
+// below, so the levels of one step are independent).  Each level keeps a 3-plane window of its
+// own rows in registers (3 * 6 * 2 doubles per lane and level).  West/east neighbours come by
+// shuffle, north/south neighbours inside a warp from registers, and across warps from shared
+// memory: level-0 planes sit in the cp.async ring anyway, and every warp publishes the first and
+// last row of its level-1 plane in a small exchange buffer.  One __syncthreads per step.
+// Two columns / two rows at every tile side lose validity (one per level): 60 x (48 - 2T) points
+// per plane are stored.  Tiles read across block borders directly; Dirichlet values are
+// injected outside the domain at every level (EDGE variant only).  Requires bx % 2 == 0.
+// ---------------------------------------------------------------------------------------
+constexpr int k3dWarps = 8;          // warps per CTA, stacked along y
+constexpr int k3dRows = 6;           // rows per warp
+constexpr int k3dTileRows = k3dWarps * k3dRows;   // 48
+constexpr int k3dStages = 5;         // level-0 planes resident in shared memory (3 of them in flight)
+constexpr int k3dPlaneElems = k3dTileRows * 64;   // doubles per ring stage
+constexpr size_t k3dSmemBytes = (size_t)(k3dStages * k3dPlaneElems + 3 * k3dWarps * 2 * 64) * sizeof(double);
+
+struct Row2 { double v[2]; };
+__device__ __forceinline__ Row2 fill_row2(double c) { Row2 r; r.v[0] = r.v[1] = c; return r; }
+__device__ __forceinline__ Row2 lds_row2(const double* p) {
+    const double2 a = *reinterpret_cast<const double2*>(p);
+    Row2 r; r.v[0] = a.x; r.v[1] = a.y; return r;
+}
+__device__ __forceinline__ Row2 ldg_row2(const double* p) {
+    const double2 a = *reinterpret_cast<const double2*>(p);
+    Row2 r; r.v[0] = a.x; r.v[1] = a.y; return r;
+}
+
+struct Plane6 { Row2 row[k3dRows]; };
+
+struct T3Ctx {
+    const double* ub;        // u + lane column base
+    const double* fb;
+    double* ob;
+    long long row_off[k3dRows];   // element offset of each of the warp's rows (valid rows only)
+    long long bsz;           // elements between blocks adjacent in z
+    double* ring;            // shared: [stage][tile row][64]
+    double* exch;            // shared: [slot][warp][first/last][64]
+    int nz, p0, in_end, Z0, Z1;
+    int warp, lane;
+    unsigned row_out_lo, row_out_hi;   // bit r: the warp's row r lies below / above the domain
+    bool nb_lo_out_lo, nb_lo_out_hi, nb_hi_out_lo, nb_hi_out_hi;  // same for the rows just outside the warp
+    unsigned row_store;      // bit r: row r is an output row of the tile and inside the domain
+    double cx, c_my, c_py, c_mz, c_pz;
+    bool xout, store_lane;
+};
+
+// plane cursor: element offset of global plane gz, block-aware
+struct PlaneCursor {
+    long long off;
+    int k;
+    __device__ __forceinline__ void init(int gz, const JacGeom& g, long long bsz) {
+        if (gz < 0) { k = gz; off = (long long)gz * g.PXY; }
+        else {
+            const int bzi = gz / g.bz;
+            k = gz - bzi * g.bz;
+            off = bzi * bsz + (long long)k * g.PXY;
+        }
+    }
+    __device__ __forceinline__ void advance(const JacGeom& g, long long bsz) {
+        ++k;
+        off += g.PXY;
+        if (k == g.bz) { k = 0; off += bsz - (long long)g.bz * g.PXY; }
+    }
+};
+
+__device__ __forceinline__ void t3_issue_plane(const T3Ctx& c, int p, const PlaneCursor& cur) {
+    if (p >= 0 && p < c.nz && p < c.in_end && !c.xout) {
+        double* st = c.ring + ((p - c.p0) % k3dStages) * k3dPlaneElems + (c.warp * k3dRows) * 64 + 2 * c.lane;
+#pragma unroll
+        for (int r = 0; r < k3dRows; ++r)
+            if (!(((c.row_out_lo | c.row_out_hi) >> r) & 1u))
+                cp_async16(st + r * 64, c.ub + cur.off + c.row_off[r]);
+    }
+    cp_async_commit();
+}
+
+// Dirichlet value of a point that lies outside the domain (plane, then row, then column decide)
+template <bool EDGE>
+__device__ __forceinline__ bool t3_outside(const T3Ctx& c, int plane, bool row_lo, bool row_hi, double* val) {
+    if (!EDGE) return false;
+    if (plane < 0) { *val = c.c_mz; return true; }
+    if (plane >= c.nz) { *val = c.c_pz; return true; }
+    if (row_lo) { *val = c.c_my; return true; }
+    if (row_hi) { *val = c.c_py; return true; }
+    if (c.xout) { *val = c.cx; return true; }
+    return false;
+}
+
+// one level: plane `q` of the level from the window (D, M, U) of the level below
+template <bool HAS_F, bool EDGE>
+__device__ __forceinline__ void t3_level(const T3Ctx& c, const Plane6& D, const Plane6& M, const Plane6& U,
+                                         const Row2& below, const Row2& above, int q,
+                                         const double* fplane, Plane6& out)
+{
+    const double c6 = 1.0 / 6.0;
+#pragma unroll
+    for (int r = 0; r < k3dRows; ++r) {
+        const Row2& S = (r == 0) ? below : M.row[r - 1];
+        const Row2& N = (r == k3dRows - 1) ? above : M.row[r + 1];
+        const double w = __shfl_up_sync(0xffffffffu, M.row[r].v[1], 1);
+        const double e = __shfl_down_sync(0xffffffffu, M.row[r].v[0], 1);
+        const bool rlo = (c.row_out_lo >> r) & 1u, rhi = (c.row_out_hi >> r) & 1u;
+        double cval = 0.0;
+        const bool outside = t3_outside<EDGE>(c, q, rlo, rhi, &cval);
+        Row2 ff = fill_row2(0.0);
+        if (HAS_F && !outside) ff = ldg_row2(fplane + c.row_off[r]);
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const double W = (i == 0) ? w : M.row[r].v[0];
+            const double E = (i == 1) ? e : M.row[r].v[1];
+            double s = add_rn(add_rn(W, E), add_rn(S.v[i], N.v[i]));
+            s = add_rn(s, add_rn(D.row[r].v[i], U.row[r].v[i]));
+            if (HAS_F) s = add_rn(s, ff.v[i]);
+            out.row[r].v[i] = mul_rn(s, c6);
+        }
+        if (EDGE && outside) out.row[r] = fill_row2(cval);
+    }
+}
+
+template <int T, bool HAS_F, int PH, bool EDGE>
+__device__ __forceinline__ void t3_step(Plane6 (&L0)[3], Plane6 (&L1)[3], const T3Ctx& c, const JacGeom& g,
+                                        int p, PlaneCursor& load_cur, PlaneCursor& l1_cur, PlaneCursor& l2_cur)
+{
+    const int wlo = c.warp > 0 ? c.warp - 1 : 0;
+    const int whi = c.warp + 1 < k3dWarps ? c.warp + 1 : c.warp;
+
+    // ---- top level first: it only needs planes finished in earlier steps
+    if (T == 2) {
+        const int q = p - 3;
+        const double* ex = c.exch + slot3(PH, -2) * (k3dWarps * 2 * 64) + 2 * c.lane;
+        Row2 below = lds_row2(ex + (wlo * 2 + 1) * 64);   // last row of the warp below
+        Row2 above = lds_row2(ex + (whi * 2 + 0) * 64);   // first row of the warp above
+        Plane6 o;
+        t3_level<HAS_F, EDGE>(c, L1[slot3(PH, -4)], L1[slot3(PH, -3)], L1[slot3(PH, -2)], below, above, q,
+                              HAS_F ? c.fb + l2_cur.off : nullptr, o);
+        if (c.store_lane && q >= c.Z0 && q < c.Z1) {
+#pragma unroll
+            for (int r = 0; r < k3dRows; ++r)
+                if ((c.row_store >> r) & 1u)
+                    *reinterpret_cast<double2*>(c.ob + l2_cur.off + c.row_off[r]) = make_double2(o.row[r].v[0], o.row[r].v[1]);
+        }
+        l2_cur.advance(g, c.bsz);
+    }
+
+    // ---- input plane p: wait for this warp's rows, take them into registers
+    cp_async_wait<k3dStages - 3>();
+    {
+        const double* st = c.ring + ((p - c.p0) % k3dStages) * k3dPlaneElems + (c.warp * k3dRows) * 64 + 2 * c.lane;
+#pragma unroll
+        for (int r = 0; r < k3dRows; ++r) {
+            double cval = 0.0;
+            if (t3_outside<EDGE>(c, p, (c.row_out_lo >> r) & 1u, (c.row_out_hi >> r) & 1u, &cval))
+                L0[PH].row[r] = fill_row2(cval);
+            else
+                L0[PH].row[r] = lds_row2(st + r * 64);
+        }
+    }
+    // stage of plane p - 2 is no longer read by anyone (barrier of the previous step): refill it
+    t3_issue_plane(c, p - 2 + k3dStages, load_cur);
+    load_cur.advance(g, c.bsz);
+
+    // ---- level 1: plane p - 1 from level-0 planes p-2, p-1, p
+    {
+        const int q = p - 1;
+        const double* st = c.ring + ((q - c.p0 + k3dStages) % k3dStages) * k3dPlaneElems + 2 * c.lane;
+        Row2 below, above;
+        double cval = 0.0;
+        if (t3_outside<EDGE>(c, q, c.nb_lo_out_lo, c.nb_lo_out_hi, &cval)) below = fill_row2(cval);
+        else below = lds_row2(st + max(c.warp * k3dRows - 1, 0) * 64);
+        if (t3_outside<EDGE>(c, q, c.nb_hi_out_lo, c.nb_hi_out_hi, &cval)) above = fill_row2(cval);
+        else above = lds_row2(st + min(c.warp * k3dRows + k3dRows, k3dTileRows - 1) * 64);
+        if (T == 1) {
+            Plane6 o;
+            t3_level<HAS_F, EDGE>(c, L0[slot3(PH, -2)], L0[slot3(PH, -1)], L0[PH], below, above, q,
+                                  HAS_F ? c.fb + l1_cur.off : nullptr, o);
+            if (c.store_lane && q >= c.Z0 && q < c.Z1) {
+#pragma unroll
+                for (int r = 0; r < k3dRows; ++r)
+                    if ((c.row_store >> r) & 1u)
+                        *reinterpret_cast<double2*>(c.ob + l1_cur.off + c.row_off[r]) = make_double2(o.row[r].v[0], o.row[r].v[1]);
+            }
+        } else {
+            Plane6& o = L1[slot3(PH, -1)];
+            t3_level<HAS_F, EDGE>(c, L0[slot3(PH, -2)], L0[slot3(PH, -1)], L0[PH], below, above, q,
+                                  HAS_F ? c.fb + l1_cur.off : nullptr, o);
+            double* ex = c.exch + PH * (k3dWarps * 2 * 64) + (c.warp * 2) * 64 + 2 * c.lane;
+            *reinterpret_cast<double2*>(ex) = make_double2(o.row[0].v[0], o.row[0].v[1]);
+            *reinterpret_cast<double2*>(ex + 64) = make_double2(o.row[k3dRows - 1].v[0], o.row[k3dRows - 1].v[1]);
+        }
+        l1_cur.advance(g, c.bsz);
+    }
+    __syncthreads();
+}
+
+template <int T, bool HAS_F>
+__global__ void __launch_bounds__(k3dWarps * 32, 1)
+temporal3d_kernel(const double* __restrict__ u, double* __restrict__ un, const double* __restrict__ f,
+                  const JacGeom g, const int tiles_x, const int tiles_y, const int tiles_z, const int zchunk)
+{
+    extern __shared__ __align__(16) double t3_smem[];
+    T3Ctx c;
+    c.ring = t3_smem;
+    c.exch = t3_smem + k3dStages * k3dPlaneElems;
+    c.lane = threadIdx.x & 31;
+    c.warp = threadIdx.x >> 5;
+    const long long tix = blockIdx.x;
+    const int sx = (int)(tix % tiles_x);
+    const int sy = (int)((tix / tiles_x) % tiles_y);
+    const int sz = (int)(tix / ((long long)tiles_x * tiles_y));
+
+    const long long X0 = (long long)sx * 60 - 2;
+    const long long gx = X0 + 2 * c.lane;
+    c.xout = gx < 0 || gx >= g.nx;
+    c.cx = gx < 0 ? g.bval[0] : g.bval[1];
+    c.c_my = g.bval[2]; c.c_py = g.bval[3]; c.c_mz = g.bval[4]; c.c_pz = g.bval[5];
+    c.store_lane = c.lane >= 1 && c.lane <= 30 && !c.xout;
+    const long long col = c.xout ? g.origin : column_base(g, gx);
+    c.ub = u + col;
+    c.fb = HAS_F ? f + col : nullptr;
+    c.ob = un + col;
+
+    const int out_rows = k3dTileRows - 2 * T;
+    const int Yt0 = sy * out_rows - T;                       // global row of tile row 0
+    const long long bsy = g.block_stride * g.gx;
+    c.bsz = bsy * g.gy;
+    c.row_out_lo = c.row_out_hi = c.row_store = 0u;
+#pragma unroll
+    for (int r = 0; r < k3dRows; ++r) {
+        const int trow = c.warp * k3dRows + r;
+        const long long gy = (long long)Yt0 + trow;
+        c.row_off[r] = 0;
+        if (gy < 0) c.row_out_lo |= 1u << r;
+        else if (gy >= g.ny) c.row_out_hi |= 1u << r;
+        else {
+            const long long byi = gy / g.by;
+            c.row_off[r] = byi * bsy + (gy - byi * g.by) * g.PX;
+            if (trow >= T && trow < k3dTileRows - T) c.row_store |= 1u << r;
+        }
+    }
+    {
+        const long long glo = (long long)Yt0 + c.warp * k3dRows - 1, ghi = (long long)Yt0 + c.warp * k3dRows + k3dRows;
+        c.nb_lo_out_lo = glo < 0; c.nb_lo_out_hi = glo >= g.ny;
+        c.nb_hi_out_lo = ghi < 0; c.nb_hi_out_hi = ghi >= g.ny;
+    }
+    c.nz = (int)g.nz;
+    c.Z0 = sz * zchunk;
+    c.Z1 = min(c.nz, c.Z0 + zchunk);
+    c.p0 = c.Z0 - T;
+    c.in_end = c.Z1 + T;
+    const int p_end = c.Z1 + 2 * T - 1;
+
+    // does this tile ever see a point outside the domain in x or y?  (z is checked per step)
+    const bool edge_xy = (sx == 0) || (X0 + 64 > g.nx) || (Yt0 < 0) || ((long long)Yt0 + k3dTileRows > g.ny);
+
+    Plane6 L0[3], L1[3];
+#pragma unroll
+    for (int k = 0; k < 3; ++k)
+#pragma unroll
+        for (int r = 0; r < k3dRows; ++r) { L0[k].row[r] = fill_row2(0.0); L1[k].row[r] = fill_row2(0.0); }
+    // the exchange buffer is read before it is first written: give it defined contents
+    for (int i = threadIdx.x; i < 3 * k3dWarps * 2 * 64; i += blockDim.x) c.exch[i] = 0.0;
+
+    PlaneCursor load_cur, l1_cur, l2_cur;
+    load_cur.init(c.p0, g, c.bsz);
+    l1_cur.init(c.p0 - 1, g, c.bsz);
+    l2_cur.init(c.p0 - 3, g, c.bsz);
+#pragma unroll 1
+    for (int k = 0; k < k3dStages - 2; ++k) {
+        t3_issue_plane(c, c.p0 + k, load_cur);
+        load_cur.advance(g, c.bsz);
+    }
+    __syncthreads();
+
+#define JAC_T3_STEP(PHASE, PL)                                                                   \
+    do {                                                                                         \
+        const bool edge = edge_xy || ((PL) - 2 * T - 1 < 0) || ((PL) >= c.nz);                   \
+        if (edge) t3_step<T, HAS_F, PHASE, true>(L0, L1, c, g, (PL), load_cur, l1_cur, l2_cur);  \
+        else t3_step<T, HAS_F, PHASE, false>(L0, L1, c, g, (PL), load_cur, l1_cur, l2_cur);      \
+    } while (0)
+
+    for (int p = c.p0; p < p_end; p += 3) {
+        JAC_T3_STEP(0, p);
+        if (p + 1 < p_end) JAC_T3_STEP(1, p + 1);
+        if (p + 2 < p_end) JAC_T3_STEP(2, p + 2);
+    }
+#undef JAC_T3_STEP
+    cp_async_wait<0>();
+}
+
 }  // namespace jac

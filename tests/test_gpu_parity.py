@@ -215,11 +215,38 @@ def test_temporal_blocking_matches_oracle(jac, orc, n, b, tsteps, has_f):
     B.close()
 
 
+# 3D: tiles are 60 x (48 - 2T) outputs wide and stream z in chunks: shapes with ragged tiles in
+# x and y, several z chunks, blocks smaller and larger than a tile
+TEMPORAL_SHAPES_3D = [((8, 8, 8), (4, 4, 4)), ((24, 18, 12), (8, 6, 4)), ((64, 48, 40), (32, 24, 20)),
+                      ((130, 100, 36), (130, 50, 18)), ((132, 20, 70), (66, 10, 35)),
+                      ((256, 128, 24), (128, 128, 8)), ((62, 46, 20), (2, 2, 2))]
+
+
+@pytest.mark.parametrize("n,b", TEMPORAL_SHAPES_3D)
+@pytest.mark.parametrize("tsteps", [1, 2])
+@pytest.mark.parametrize("has_f", [False, True])
+def test_temporal_blocking_3d_matches_oracle(jac, orc, n, b, tsteps, has_f):
+    J, B = _setup_pair(jac, orc, n, b, 1, has_f, "temporal", seed=4, tsteps=tsteps)
+    for nsw in (1, 2, 5):
+        J.sweep(nsw)
+        B.sweep(nsw)
+        _assert_sweep_close(J.get_u(), B.get_u())
+    r_gpu, r_cpu = J.residual(), B.residual()
+    assert abs(r_gpu - r_cpu) <= RESID_TOL * r_cpu
+    J.sweep(4)
+    B.sweep(4)
+    _assert_sweep_close(J.get_u(), B.get_u())
+    J.close()
+    B.close()
+
+
 def test_temporal_mode_rejects_unsupported_shapes(jac):
     with pytest.raises(jac.JacError):
-        jac.Jacobi((12, 8), (6, 4), mode="temporal")          # bx % 4 != 0
+        jac.Jacobi((12, 8), (6, 4), mode="temporal")          # 2D: bx % 4 != 0
     with pytest.raises(jac.JacError):
-        jac.Jacobi((8, 8, 8), (4, 4, 4), mode="temporal")     # 3D
+        jac.Jacobi((9, 8, 8), (3, 4, 4), mode="temporal")     # 3D: bx % 2 != 0
+    with pytest.raises(jac.JacError):
+        jac.Jacobi((8, 8, 8), (4, 4, 4), mode="temporal", tsteps=3)   # 3D: at most 2 sweeps per launch
 
 
 def test_partial_exchange_by_face_mask(jac, orc):
