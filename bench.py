@@ -49,9 +49,9 @@ NCU_TRAFFIC = {
     ("temporal", 4, 2, False): {"bytes_per_point_per_launch": (606.650368e6 + 490.201856e6) / 8192 ** 2,
                                 "src_sha": "46c902c3cd6527b9"},
 }
-KERNEL_NAMES = {("temporal", 2): "temporal2d_kernel", ("fused", 2): "sweep2d_kernel (update + ghost push)",
+KERNEL_NAMES = {("temporal", 2): "temporal2d_kernel", ("temporal", 3): "temporal3d_kernel", ("fused", 2): "sweep2d_kernel (update pulling neighbour interiors)",
                 ("exchange", 2): "sweep2d_kernel", ("pertask", 2): "sweep2d_kernel (one launch per block)",
-                ("fused", 3): "sweep3d_kernel (update + ghost push)", ("exchange", 3): "sweep3d_kernel",
+                ("fused", 3): "sweep3d_kernel (update pulling neighbour interiors)", ("exchange", 3): "sweep3d_kernel",
                 ("pertask", 3): "sweep3d_kernel (one launch per block)"}
 
 
@@ -209,6 +209,8 @@ def default_schedule(w: inputs.Workload):
     """Fastest schedule the library has for the workload (all schedules give identical bits)."""
     if w.ndim == 2 and w.b[0] % 4 == 0:
         return "temporal", 4
+    if w.ndim == 3 and w.b[0] % 2 == 0:
+        return "temporal", 2
     return "exchange", 1
 
 
@@ -293,7 +295,7 @@ def run_ours(args, w: inputs.Workload):
     if mode == "auto":
         mode, tsteps = default_schedule(w)
     if mode == "temporal" and not tsteps:
-        tsteps = 4
+        tsteps = 4 if w.ndim == 2 else 2
     if mode != "temporal":
         tsteps = 1
     J = make_ctx(mode, tsteps)
@@ -355,6 +357,8 @@ def run_ours(args, w: inputs.Workload):
         alts = [("exchange", 1), ("fused", 1)]
         if w.ndim == 2 and w.b[0] % 4 == 0:
             alts += [("temporal", 1), ("temporal", 2), ("temporal", 4)]
+        if w.ndim == 3 and w.b[0] % 2 == 0:
+            alts += [("temporal", 1), ("temporal", 2)]
         for m, t in alts:
             if (m, t) == (mode, tsteps):
                 continue

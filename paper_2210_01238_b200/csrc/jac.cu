@@ -341,8 +341,9 @@ int launch_temporal3d_t(jac_ctx* c, const double* u, double* un)
     const long long ctas = (long long)tiles_x * tiles_y * tiles_z;
     if (ctas > kMaxGrid) return JAC_EINVAL;
     auto kern = jac::temporal3d_kernel<T, HAS_F>;
-    JAC_CK(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)jac::k3dSmemBytes));
-    kern<<<(unsigned)ctas, jac::k3dWarps * 32, jac::k3dSmemBytes, c->stream>>>(u, un, c->f, g, tiles_x, tiles_y,
+    const size_t smem = jac::k3d_smem_bytes(HAS_F);
+    JAC_CK(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kern<<<(unsigned)ctas, jac::k3dWarps * 32, smem, c->stream>>>(u, un, c->f, g, tiles_x, tiles_y,
                                                                              tiles_z, zchunk);
     return check_launch(c);
 }

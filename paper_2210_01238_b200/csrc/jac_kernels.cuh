@@ -646,17 +646,19 @@ temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
 constexpr int k3dWarps = 8;          // warps per CTA, stacked along y
 constexpr int k3dRows = 6;           // rows per warp
 constexpr int k3dTileRows = k3dWarps * k3dRows;   // 48
-constexpr int k3dStages = 5;         // level-0 planes resident in shared memory (3 of them in flight)
 constexpr int k3dPlaneElems = k3dTileRows * 64;   // doubles per ring stage
-constexpr size_t k3dSmemBytes = (size_t)(k3dStages * k3dPlaneElems + 3 * k3dWarps * 2 * 64) * sizeof(double);
+constexpr int k3dFStages = 4;        // f planes resident (levels 1 and 2 read planes p-1 and p-3)
+// u planes resident: p-1 and p are read, the others are in flight.  With f the shared memory
+// is split between the two rings.
+__host__ __device__ constexpr int k3d_stages(bool has_f) { return has_f ? 4 : 5; }
+__host__ __device__ constexpr size_t k3d_smem_bytes(bool has_f) {
+    return (size_t)((k3d_stages(has_f) + (has_f ? k3dFStages : 0)) * k3dPlaneElems + 3 * k3dWarps * 2 * 64) *
+           sizeof(double);
+}
 
 struct Row2 { double v[2]; };
 __device__ __forceinline__ Row2 fill_row2(double c) { Row2 r; r.v[0] = r.v[1] = c; return r; }
 __device__ __forceinline__ Row2 lds_row2(const double* p) {
-    const double2 a = *reinterpret_cast<const double2*>(p);
-    Row2 r; r.v[0] = a.x; r.v[1] = a.y; return r;
-}
-__device__ __forceinline__ Row2 ldg_row2(const double* p) {
     const double2 a = *reinterpret_cast<const double2*>(p);
     Row2 r; r.v[0] = a.x; r.v[1] = a.y; return r;
 }
@@ -670,6 +672,7 @@ struct T3Ctx {
     long long row_off[k3dRows];   // element offset of each of the warp's rows (valid rows only)
     long long bsz;           // elements between blocks adjacent in z
     double* ring;            // shared: [stage][tile row][64]
+    double* fring;           // shared: [stage][tile row][64], right-hand side
     double* exch;            // shared: [slot][warp][first/last][64]
     int nz, p0, in_end, Z0, Z1;
     int warp, lane;
@@ -699,13 +702,26 @@ struct PlaneCursor {
     }
 };
 
-__device__ __forceinline__ void t3_issue_plane(const T3Ctx& c, int p, const PlaneCursor& cur) {
+// start the copies of u plane p (and, with f, of f plane p - 1) into their ring stages; one group
+template <bool HAS_F>
+__device__ __forceinline__ void t3_issue_plane(const T3Ctx& c, int p, const PlaneCursor& cur, const PlaneCursor& fcur) {
+    constexpr int NST = k3d_stages(HAS_F);
+    const unsigned rows_out = c.row_out_lo | c.row_out_hi;
     if (p >= 0 && p < c.nz && p < c.in_end && !c.xout) {
-        double* st = c.ring + ((p - c.p0) % k3dStages) * k3dPlaneElems + (c.warp * k3dRows) * 64 + 2 * c.lane;
+        double* st = c.ring + ((p - c.p0) % NST) * k3dPlaneElems + (c.warp * k3dRows) * 64 + 2 * c.lane;
 #pragma unroll
         for (int r = 0; r < k3dRows; ++r)
-            if (!(((c.row_out_lo | c.row_out_hi) >> r) & 1u))
-                cp_async16(st + r * 64, c.ub + cur.off + c.row_off[r]);
+            if (!((rows_out >> r) & 1u)) cp_async16(st + r * 64, c.ub + cur.off + c.row_off[r]);
+    }
+    if (HAS_F) {
+        const int q = p - 1;
+        if (q >= 0 && q < c.nz && q < c.in_end && !c.xout) {
+            double* st = c.fring + ((q - c.p0 + 2 * k3dFStages) % k3dFStages) * k3dPlaneElems +
+                         (c.warp * k3dRows) * 64 + 2 * c.lane;
+#pragma unroll
+            for (int r = 0; r < k3dRows; ++r)
+                if (!((rows_out >> r) & 1u)) cp_async16(st + r * 64, c.fb + fcur.off + c.row_off[r]);
+        }
     }
     cp_async_commit();
 }
@@ -726,7 +742,8 @@ __device__ __forceinline__ bool t3_outside(const T3Ctx& c, int plane, bool row_l
 template <bool HAS_F, bool EDGE>
 __device__ __forceinline__ void t3_level(const T3Ctx& c, const Plane6& D, const Plane6& M, const Plane6& U,
                                          const Row2& below, const Row2& above, int q,
-                                         const double* fplane, Plane6& out)
+                                         const double* fplane /* ring stage of f plane q, this warp's rows */,
+                                         Plane6& out)
 {
     const double c6 = 1.0 / 6.0;
 #pragma unroll
@@ -739,7 +756,7 @@ __device__ __forceinline__ void t3_level(const T3Ctx& c, const Plane6& D, const 
         double cval = 0.0;
         const bool outside = t3_outside<EDGE>(c, q, rlo, rhi, &cval);
         Row2 ff = fill_row2(0.0);
-        if (HAS_F && !outside) ff = ldg_row2(fplane + c.row_off[r]);
+        if (HAS_F && !outside) ff = lds_row2(fplane + r * 64);   // this lane copied it itself
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
             const double W = (i == 0) ? w : M.row[r].v[0];
@@ -755,8 +772,12 @@ __device__ __forceinline__ void t3_level(const T3Ctx& c, const Plane6& D, const 
 
 template <int T, bool HAS_F, int PH, bool EDGE>
 __device__ __forceinline__ void t3_step(Plane6 (&L0)[3], Plane6 (&L1)[3], const T3Ctx& c, const JacGeom& g,
-                                        int p, PlaneCursor& load_cur, PlaneCursor& l1_cur, PlaneCursor& l2_cur)
+                                        int p, PlaneCursor& load_cur, PlaneCursor& fload_cur,
+                                        PlaneCursor& l1_cur, PlaneCursor& l2_cur)
 {
+    constexpr int NST = k3d_stages(HAS_F);
+    constexpr int LEAD = NST - 2;          // u planes issued ahead of the one being consumed
+    const double* fmine = HAS_F ? c.fring + (c.warp * k3dRows) * 64 + 2 * c.lane : nullptr;
     const int wlo = c.warp > 0 ? c.warp - 1 : 0;
     const int whi = c.warp + 1 < k3dWarps ? c.warp + 1 : c.warp;
 
@@ -768,7 +789,7 @@ __device__ __forceinline__ void t3_step(Plane6 (&L0)[3], Plane6 (&L1)[3], const 
         Row2 above = lds_row2(ex + (whi * 2 + 0) * 64);   // first row of the warp above
         Plane6 o;
         t3_level<HAS_F, EDGE>(c, L1[slot3(PH, -4)], L1[slot3(PH, -3)], L1[slot3(PH, -2)], below, above, q,
-                              HAS_F ? c.fb + l2_cur.off : nullptr, o);
+                              HAS_F ? fmine + ((q - c.p0 + 2 * k3dFStages) % k3dFStages) * k3dPlaneElems : nullptr, o);
         if (c.store_lane && q >= c.Z0 && q < c.Z1) {
 #pragma unroll
             for (int r = 0; r < k3dRows; ++r)
@@ -779,9 +800,9 @@ __device__ __forceinline__ void t3_step(Plane6 (&L0)[3], Plane6 (&L1)[3], const 
     }
 
     // ---- input plane p: wait for this warp's rows, take them into registers
-    cp_async_wait<k3dStages - 3>();
+    cp_async_wait<LEAD - 1>();
     {
-        const double* st = c.ring + ((p - c.p0) % k3dStages) * k3dPlaneElems + (c.warp * k3dRows) * 64 + 2 * c.lane;
+        const double* st = c.ring + ((p - c.p0) % NST) * k3dPlaneElems + (c.warp * k3dRows) * 64 + 2 * c.lane;
 #pragma unroll
         for (int r = 0; r < k3dRows; ++r) {
             double cval = 0.0;
@@ -791,14 +812,17 @@ __device__ __forceinline__ void t3_step(Plane6 (&L0)[3], Plane6 (&L1)[3], const 
                 L0[PH].row[r] = lds_row2(st + r * 64);
         }
     }
-    // stage of plane p - 2 is no longer read by anyone (barrier of the previous step): refill it
-    t3_issue_plane(c, p - 2 + k3dStages, load_cur);
+    // the stage of u plane p - 2 is no longer read by anyone (barrier of the previous step), and this
+    // thread has just read its part of f plane p - 3: refill both
+    t3_issue_plane<HAS_F>(c, p + LEAD, load_cur, fload_cur);
     load_cur.advance(g, c.bsz);
+    if (HAS_F) fload_cur.advance(g, c.bsz);
 
     // ---- level 1: plane p - 1 from level-0 planes p-2, p-1, p
     {
         const int q = p - 1;
-        const double* st = c.ring + ((q - c.p0 + k3dStages) % k3dStages) * k3dPlaneElems + 2 * c.lane;
+        const double* st = c.ring + ((q - c.p0 + NST) % NST) * k3dPlaneElems + 2 * c.lane;
+        const double* f1 = HAS_F ? fmine + ((q - c.p0 + 2 * k3dFStages) % k3dFStages) * k3dPlaneElems : nullptr;
         Row2 below, above;
         double cval = 0.0;
         if (t3_outside<EDGE>(c, q, c.nb_lo_out_lo, c.nb_lo_out_hi, &cval)) below = fill_row2(cval);
@@ -807,8 +831,7 @@ __device__ __forceinline__ void t3_step(Plane6 (&L0)[3], Plane6 (&L1)[3], const 
         else above = lds_row2(st + min(c.warp * k3dRows + k3dRows, k3dTileRows - 1) * 64);
         if (T == 1) {
             Plane6 o;
-            t3_level<HAS_F, EDGE>(c, L0[slot3(PH, -2)], L0[slot3(PH, -1)], L0[PH], below, above, q,
-                                  HAS_F ? c.fb + l1_cur.off : nullptr, o);
+            t3_level<HAS_F, EDGE>(c, L0[slot3(PH, -2)], L0[slot3(PH, -1)], L0[PH], below, above, q, f1, o);
             if (c.store_lane && q >= c.Z0 && q < c.Z1) {
 #pragma unroll
                 for (int r = 0; r < k3dRows; ++r)
@@ -817,8 +840,7 @@ __device__ __forceinline__ void t3_step(Plane6 (&L0)[3], Plane6 (&L1)[3], const 
             }
         } else {
             Plane6& o = L1[slot3(PH, -1)];
-            t3_level<HAS_F, EDGE>(c, L0[slot3(PH, -2)], L0[slot3(PH, -1)], L0[PH], below, above, q,
-                                  HAS_F ? c.fb + l1_cur.off : nullptr, o);
+            t3_level<HAS_F, EDGE>(c, L0[slot3(PH, -2)], L0[slot3(PH, -1)], L0[PH], below, above, q, f1, o);
             double* ex = c.exch + PH * (k3dWarps * 2 * 64) + (c.warp * 2) * 64 + 2 * c.lane;
             *reinterpret_cast<double2*>(ex) = make_double2(o.row[0].v[0], o.row[0].v[1]);
             *reinterpret_cast<double2*>(ex + 64) = make_double2(o.row[k3dRows - 1].v[0], o.row[k3dRows - 1].v[1]);
@@ -835,8 +857,10 @@ temporal3d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
 {
     extern __shared__ __align__(16) double t3_smem[];
     T3Ctx c;
+    constexpr int NST = k3d_stages(HAS_F);
     c.ring = t3_smem;
-    c.exch = t3_smem + k3dStages * k3dPlaneElems;
+    c.fring = t3_smem + NST * k3dPlaneElems;
+    c.exch = c.fring + (HAS_F ? k3dFStages : 0) * k3dPlaneElems;
     c.lane = threadIdx.x & 31;
     c.warp = threadIdx.x >> 5;
     const long long tix = blockIdx.x;
@@ -896,22 +920,24 @@ temporal3d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
     // the exchange buffer is read before it is first written: give it defined contents
     for (int i = threadIdx.x; i < 3 * k3dWarps * 2 * 64; i += blockDim.x) c.exch[i] = 0.0;
 
-    PlaneCursor load_cur, l1_cur, l2_cur;
+    PlaneCursor load_cur, fload_cur, l1_cur, l2_cur;
     load_cur.init(c.p0, g, c.bsz);
-    l1_cur.init(c.p0 - 1, g, c.bsz);
-    l2_cur.init(c.p0 - 3, g, c.bsz);
+    fload_cur.init(c.p0 - 1, g, c.bsz);    // the f plane that travels with u plane p is p - 1
+    l1_cur.init(c.p0 - 1, g, c.bsz);       // output plane of level 1 (stores when T == 1)
+    l2_cur.init(c.p0 - 3, g, c.bsz);       // output plane of level 2
 #pragma unroll 1
-    for (int k = 0; k < k3dStages - 2; ++k) {
-        t3_issue_plane(c, c.p0 + k, load_cur);
+    for (int k = 0; k < NST - 2; ++k) {
+        t3_issue_plane<HAS_F>(c, c.p0 + k, load_cur, fload_cur);
         load_cur.advance(g, c.bsz);
+        if (HAS_F) fload_cur.advance(g, c.bsz);
     }
     __syncthreads();
 
 #define JAC_T3_STEP(PHASE, PL)                                                                   \
     do {                                                                                         \
         const bool edge = edge_xy || ((PL) - 2 * T - 1 < 0) || ((PL) >= c.nz);                   \
-        if (edge) t3_step<T, HAS_F, PHASE, true>(L0, L1, c, g, (PL), load_cur, l1_cur, l2_cur);  \
-        else t3_step<T, HAS_F, PHASE, false>(L0, L1, c, g, (PL), load_cur, l1_cur, l2_cur);      \
+        if (edge) t3_step<T, HAS_F, PHASE, true>(L0, L1, c, g, (PL), load_cur, fload_cur, l1_cur, l2_cur);  \
+        else t3_step<T, HAS_F, PHASE, false>(L0, L1, c, g, (PL), load_cur, fload_cur, l1_cur, l2_cur);      \
     } while (0)
 
     for (int p = c.p0; p < p_end; p += 3) {

@@ -170,7 +170,7 @@ def test_c5_poisson3d_1024(jac, orc):
     w = inputs.POISSON3D_1024
     f = inputs.rhs(w)
     norm_f = float(np.sqrt(np.sum(np.square(f, dtype=np.float64))))
-    with _make(jac, w, "fused") as J:
+    with _make(jac, w, "temporal", 2) as J:     # the schedule the benchmark times
         J.set_f(f)
         r0 = J.residual()
         got_r = []
@@ -216,7 +216,7 @@ def test_c5_scaled_256_whole_field_and_residuals(jac, orc):
         want_r.append(B.residual())
     want = B.get_u()
     B.close()
-    for mode in ("fused", "exchange"):
+    for mode in ("fused", "exchange", "temporal"):
         with _make(jac, w, mode) as J:
             J.set_f(f)
             got_r = []
@@ -232,7 +232,7 @@ def test_paper_strong_scaling_shape_1024x1024x768(jac, orc):
     n, b = (1024, 1024, 768), (128, 128, 128)
     rng = np.random.default_rng(3)
     f = rng.standard_normal(int(np.prod(n))).reshape(tuple(reversed(n)))
-    with jac.Jacobi(n, b, 1, True, "fused") as J:
+    with jac.Jacobi(n, b, 1, True, "temporal") as J:
         J.set_f(f)
         J.sweep(20)
         got = J.get_u()
