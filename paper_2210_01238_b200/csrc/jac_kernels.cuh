@@ -437,6 +437,16 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N> __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
 }
+#ifndef JAC_FPREFETCH
+#define JAC_FPREFETCH 2   // 0: none, 1: into L1, 2: into L2
+#endif
+__device__ __forceinline__ void prefetch_line(const void* p) {
+#if JAC_FPREFETCH == 1
+    asm volatile("prefetch.global.L1 [%0];\n" ::"l"(p));
+#elif JAC_FPREFETCH == 2
+    asm volatile("prefetch.global.L2 [%0];\n" ::"l"(p));
+#endif
+}
 
 // Per-lane constants of a strip.  A ring stage holds one row as 64 chunks of 16 bytes in
 // natural order (chunk k = columns 2k, 2k+1 of the strip).  One copy instruction of the warp
@@ -463,12 +473,15 @@ struct TemporalCtx {
     bool xout, edge_x, store_lane;
 };
 
-// start the copy of input row r into its ring stage (nothing to copy outside the domain)
+// start the copy of input row r into its ring stage (nothing to copy outside the domain); with a
+// right-hand side, also ask for the lane's part of f row r, which the levels read DEPTH steps later
+template <bool HAS_F>
 __device__ __forceinline__ void issue_row(const TemporalCtx& c, int r, const RowCursor& cur) {
     if (r >= 0 && r < c.ny && r < c.in_end) {
         const int st = ((r - c.r0) % kTemporalDepth) * 64;
         if (c.copy_a) cp_async16(c.dst_a + st, c.src_a + cur.off);
         if (c.copy_b) cp_async16(c.dst_b + st, c.src_b + cur.off);
+        if (HAS_F && !c.xout) prefetch_line(c.fb + cur.off);
     }
     cp_async_commit();
 }
@@ -500,7 +513,7 @@ __device__ __forceinline__ void temporal_step(Row4 (&win)[T][3], const TemporalC
     __syncwarp();                                    // the other lanes' chunks of row r have landed too
     win[0][PH] = take_row<EDGE>(c, r);
     __syncwarp();                                    // everyone has read the stage before it is refilled
-    issue_row(c, r + kTemporalDepth, load_cur);
+    issue_row<HAS_F>(c, r + kTemporalDepth, load_cur);
     load_cur.advance(g, c.brs);
 #pragma unroll
     for (int s = T; s >= 1; --s) {
@@ -616,7 +629,7 @@ temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
     // fill the ring with the first DEPTH rows
 #pragma unroll 1
     for (int k = 0; k < kTemporalDepth; ++k) {
-        issue_row(c, c.r0 + k, load_cur);
+        issue_row<HAS_F>(c, c.r0 + k, load_cur);
         load_cur.advance(g, c.brs);
     }
 
