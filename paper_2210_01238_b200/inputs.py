@@ -57,7 +57,12 @@ EIGENMODE_16384 = Workload("c3_eigenmode_16384", (16384, 16384), (1024, 1024), 1
                            "sine", "none", 0)
 POISSON3D_1024 = Workload("c5_poisson3d_1024", (1024, 1024, 1024), (128, 128, 128), 1, 50, 10,
                           "zero", "normal", 3)
-CONFIGS = {w.name: w for w in (HEATED_EDGE_256, POISSON_4096, EIGENMODE_16384, POISSON3D_1024)}
+# The one domain shape the paper states (Section V-C, strong scaling): 1024 x 1024 x 768, here in
+# 128^3 blocks with the recipe of POISSON3D_1024.  Context, not one of the five configurations.
+PAPER_DOMAIN_1024x1024x768 = Workload("paper_domain_1024x1024x768", (1024, 1024, 768), (128, 128, 128), 1,
+                                      50, 10, "zero", "normal", 3)
+CONFIGS = {w.name: w for w in (HEATED_EDGE_256, POISSON_4096, EIGENMODE_16384, POISSON3D_1024,
+                               PAPER_DOMAIN_1024x1024x768)}
 
 # Halo pack/unpack microbenchmark: block edge B -> block grid G x G, so that every kind
 # of face has interior instances; halo widths 1 and 4; data Uniform[-1,1], seed 2.
