@@ -111,7 +111,8 @@ int build_geometry(const jac_desc* d, JacGeom* g, jac_layout* L)
     if (ctas > kMaxGrid) return JAC_EINVAL;
     long long max_face = 0;
     for (int fc = 0; fc < 6; ++fc) max_face = std::max(max_face, g->face_elems[fc]);
-    if (g->nblocks * g->nfaces * ceil_div(max_face, 1024) > kMaxGrid) return JAC_EINVAL;
+    if (max_face >= (1LL << 31)) return JAC_EINVAL;
+    if (g->nblocks * g->nfaces * ceil_div(round_up(ceil_div(max_face, 2), 32), 256) > kMaxGrid) return JAC_EINVAL;
 
     if (L) {
         std::memset(L, 0, sizeof(*L));
@@ -207,21 +208,31 @@ int launch_sweep(jac_ctx* c, const double* u, double* un, long long blk0, long l
     return check_launch(c);
 }
 
-int halo_chunks(const jac_ctx* c, int face_lo, int face_hi)
+// threads reserved per (block, face) pair: one per two elements of the largest face, whole warps
+int halo_slots(const jac_ctx* c, unsigned face_mask)
 {
-    long long m = 1;
-    for (int fc = face_lo; fc < face_hi; ++fc) m = std::max(m, c->g.face_elems[fc]);
-    return (int)ceil_div(m, 256 * 4);
+    long long m = 2;
+    for (int fc = 0; fc < c->g.nfaces; ++fc)
+        if ((face_mask >> fc) & 1u) m = std::max(m, c->g.face_elems[fc]);
+    return (int)round_up(ceil_div(m, 2), 32);
 }
 
-// pack or unpack all faces of all blocks in one launch
+template <bool UNPACK>
+int launch_halo(jac_ctx* c, long long pair0, long long npairs, unsigned face_mask)
+{
+    const int slots = halo_slots(c, face_mask);
+    const long long ctas = ceil_div(npairs * slots, 256);
+    if (ctas > kMaxGrid) return JAC_EINVAL;
+    jac::halo_kernel<UNPACK><<<(unsigned)ctas, 256, 0, c->stream>>>(c->u[c->cur], c->send, c->g, pair0, npairs,
+                                                                  slots, face_mask);
+    return check_launch(c);
+}
+
+// pack or unpack the faces in face_mask of all blocks in one launch
 template <bool UNPACK>
 int launch_halo_all(jac_ctx* c, unsigned face_mask = 0x3fu)
 {
-    const int chunks = halo_chunks(c, 0, c->g.nfaces);
-    const unsigned grid = (unsigned)(c->g.nblocks * c->g.nfaces * chunks);
-    jac::halo_kernel<UNPACK><<<grid, 256, 0, c->stream>>>(c->u[c->cur], c->send, c->g, 0, chunks, face_mask);
-    return check_launch(c);
+    return launch_halo<UNPACK>(c, 0, c->g.nblocks * c->g.nfaces, face_mask);
 }
 
 bool has_neighbour(const JacGeom& g, long long blk, int face)
@@ -239,10 +250,7 @@ int launch_halo_pertask(jac_ctx* c)
     for (long long blk = 0; blk < c->g.nblocks; ++blk)
         for (int face = 0; face < c->g.nfaces; ++face) {
             if (!has_neighbour(c->g, blk, face)) continue;
-            const int chunks = halo_chunks(c, face, face + 1);
-            jac::halo_kernel<UNPACK><<<(unsigned)chunks, 256, 0, c->stream>>>(
-                c->u[c->cur], c->send, c->g, blk * c->g.nfaces + face, chunks, 0x3fu);
-            const int rc = check_launch(c);
+            const int rc = launch_halo<UNPACK>(c, blk * c->g.nfaces + face, 1, 1u << face);
             if (rc) return rc;
         }
     return JAC_OK;

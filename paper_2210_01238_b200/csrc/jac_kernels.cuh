@@ -234,8 +234,8 @@ reduce_partials_kernel(const double* __restrict__ partials, const long long n, d
 
 // ---------------------------------------------------------------------------------------
 // Halo pack / unpack.  One launch covers `npairs` consecutive (block, face) pairs starting at
-// pair0 (pair = block * nfaces + face); each pair is cut into chunks of blockDim.x * EPT
-// elements.  Pairs whose face lies on the domain boundary, or is not in face_mask, do nothing.
+// pair0 (pair = block * nfaces + face).  Pairs whose face lies on the domain boundary, or is
+// not in face_mask, do nothing.
 //
 // Element e of a packed face (source memory order):
 //   x face: e = (k*by + j)*h + c      y face: e = (k*h + r)*bx + i      z face: e = (p*by + j)*bx + i
@@ -273,40 +273,46 @@ __device__ __forceinline__ long long strip_offset(const JacGeom& g, int face, lo
     return z * g.PXY + y * g.PX + x;
 }
 
+// A thread moves two consecutive elements of one face; `slots` threads (a multiple of 32, so a
+// warp never straddles faces) are reserved per (block, face) pair, and the grid is packed over
+// threads, not faces: small faces do not leave CTAs mostly idle.  On y and z faces with an even
+// block width the two elements are adjacent in memory on both sides and move as one 128-bit
+// access; on x faces they are two strided cells.
 template <bool UNPACK>
 __global__ void __launch_bounds__(256)
 halo_kernel(double* __restrict__ u, double* __restrict__ send, const JacGeom g,
-            const long long pair0, const int chunks, const unsigned face_mask)
+            const long long pair0, const long long npairs, const int slots, const unsigned face_mask)
 {
-    const long long t = blockIdx.x;
-    const long long pair = pair0 + t / chunks;
-    const int chunk = (int)(t % chunks);
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long pr = t / slots;
+    if (pr >= npairs) return;
+    const long long e = 2 * (t - pr * slots);
+    const long long pair = pair0 + pr;
     const long long blk = pair / g.nfaces;
-    const int face = (int)(pair % g.nfaces);
+    const int face = (int)(pair - blk * g.nfaces);
     if (!((face_mask >> face) & 1u)) return;
+    const long long n = g.face_elems[face];
+    if (e >= n) return;
     const long long nb = neighbour_block(g, blk, face);
     if (nb < 0) return;
-    const long long n = g.face_elems[face];
     const int axis = face >> 1;
     const int ext = axis == 0 ? g.bx : (axis == 1 ? g.by : g.bz);
     double* ub = u + blk * g.block_stride + g.origin;
-    constexpr int EPT = 4;
-    const long long e0 = (long long)chunk * blockDim.x * EPT + threadIdx.x;
-    if (!UNPACK) {
-        double* buf = send + blk * g.send_stride + g.face_off[face];
-        const int lo = (face & 1) ? ext - g.h : 0;
-#pragma unroll
-        for (int q = 0; q < EPT; ++q) {
-            const long long e = e0 + (long long)q * blockDim.x;
-            if (e < n) buf[e] = ub[strip_offset(g, face, e, lo)];
-        }
+    // pack reads the interior strip next to the face; unpack writes the ghost strip
+    const int lo = UNPACK ? ((face & 1) ? ext : -g.h) : ((face & 1) ? ext - g.h : 0);
+    double* buf = UNPACK ? send + nb * g.send_stride + g.face_off[face ^ 1]
+                         : send + blk * g.send_stride + g.face_off[face];
+    const bool pair_ok = e + 1 < n;
+    if (axis != 0 && (g.bx & 1) == 0) {
+        double2* cell = reinterpret_cast<double2*>(ub + strip_offset(g, face, e, lo));
+        double2* slot = reinterpret_cast<double2*>(buf + e);
+        if (UNPACK) *cell = *slot; else *slot = *cell;
     } else {
-        const double* buf = send + nb * g.send_stride + g.face_off[face ^ 1];
-        const int lo = (face & 1) ? ext : -g.h;
-#pragma unroll
-        for (int q = 0; q < EPT; ++q) {
-            const long long e = e0 + (long long)q * blockDim.x;
-            if (e < n) ub[strip_offset(g, face, e, lo)] = buf[e];
+        double* c0 = ub + strip_offset(g, face, e, lo);
+        if (UNPACK) *c0 = buf[e]; else buf[e] = *c0;
+        if (pair_ok) {
+            double* c1 = ub + strip_offset(g, face, e + 1, lo);
+            if (UNPACK) *c1 = buf[e + 1]; else buf[e + 1] = *c1;
         }
     }
 }
