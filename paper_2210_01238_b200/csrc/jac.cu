@@ -371,6 +371,8 @@ int launch_temporal(jac_ctx* c, const double* u, double* un)
     const int strips_x = (int)ceil_div(g.nx, 120);
     int rows = 256;
     while (rows > 32 && (long long)strips_x * ceil_div(g.ny, rows) < (long long)kNumSMs * 48) rows /= 2;
+    // tiny grids: not even one warp per scheduler; shorter strips cut the serial length of a launch
+    while (rows > 8 && (long long)strips_x * ceil_div(g.ny, rows) < (long long)kNumSMs * 4) rows /= 2;
     const int strips_y = (int)ceil_div(g.ny, rows);
     const unsigned grid = (unsigned)ceil_div((long long)strips_x * strips_y, jac::kTemporalWarps);
     const int threads = jac::kTemporalWarps * 32;
