@@ -207,10 +207,8 @@ def replicated_glups(updates_per_rank: float, world: int, ms: float) -> float:
 
 def default_schedule(w: inputs.Workload):
     """Fastest schedule the library has for the workload (all schedules give identical bits)."""
-    if w.ndim == 2 and w.b[0] % 4 == 0:
-        return "temporal", 4
-    if w.ndim == 3 and w.b[0] % 2 == 0:
-        return "temporal", 2
+    if (w.ndim == 2 and w.b[0] % 4 == 0) or (w.ndim == 3 and w.b[0] % 2 == 0):
+        return "temporal", 0          # 0: the library picks the sweeps per launch
     return "exchange", 1
 
 
@@ -294,11 +292,10 @@ def run_ours(args, w: inputs.Workload):
     mode, tsteps = args.mode, args.tsteps
     if mode == "auto":
         mode, tsteps = default_schedule(w)
-    if mode == "temporal" and not tsteps:
-        tsteps = 4 if w.ndim == 2 else 2
     if mode != "temporal":
         tsteps = 1
     J = make_ctx(mode, tsteps)
+    tsteps = J.sweeps_per_launch()
     main_run = time_schedule(J, mode, tsteps, args.steps, args.warmup, True)
     value = main_run["glups"]
 
@@ -356,7 +353,7 @@ def run_ours(args, w: inputs.Workload):
     if not args.no_others and world == 1:
         alts = [("exchange", 1), ("fused", 1)]
         if w.ndim == 2 and w.b[0] % 4 == 0:
-            alts += [("temporal", 1), ("temporal", 2), ("temporal", 4)]
+            alts += [("temporal", 1), ("temporal", 2), ("temporal", 4), ("temporal", 8)]
         if w.ndim == 3 and w.b[0] % 2 == 0:
             alts += [("temporal", 1), ("temporal", 2)]
         for m, t in alts:

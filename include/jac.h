@@ -59,7 +59,7 @@ extern "C" {
                                launch per block                                                  */
 #define JAC_MODE_TEMPORAL 2 /* `tsteps` sweeps per launch; tiles read across block borders
                                directly (equivalent to an exchange before every sweep).
-                               2D: b[0] % 4 == 0, tsteps <= 4; 3D: b[0] % 2 == 0, tsteps <= 2;
+                               2D: b[0] % 4 == 0, tsteps <= 8; 3D: b[0] % 2 == 0, tsteps <= 2;
                                jac_create returns JAC_EINVAL otherwise                           */
 #define JAC_MODE_EXCHANGE 3 /* per sweep three launches over all blocks: pack, unpack, update    */
 
@@ -70,7 +70,7 @@ typedef struct jac_desc {
     int32_t halo;    /* ghost width h, 1 <= h <= min(b[a]) and h <= 8                            */
     int32_t has_f;   /* 0: f == 0 and is never read (16 B/point/sweep); 1: f present (24 B)      */
     int32_t mode;    /* JAC_MODE_*                                                               */
-    int32_t tsteps;  /* JAC_MODE_TEMPORAL: sweeps per launch; 0 = library default (2D 4, 3D 2)   */
+    int32_t tsteps;  /* JAC_MODE_TEMPORAL: sweeps per launch; 0 = the library chooses             */
     int32_t reserved;/* must be 0                                                                */
     int64_t n[3];    /* global interior points; n[2] ignored (taken as 1) when ndim == 2         */
     int64_t b[3];    /* block interior points; n[a] % b[a] == 0                                  */
@@ -197,6 +197,10 @@ int jac_residual(jac_ctx *ctx, double *host_out_l2);
 int jac_residual_dense_static(int ndim, const int64_t *n, const double *dev_u,
                               const double *dev_f, const double *host_bvals, void *stream,
                               double *host_out_l2);
+
+/* Sweeps one launch of jac_sweep performs for this context (HOST output): desc.tsteps, or the
+ * library's choice when that was 0, in JAC_MODE_TEMPORAL; 1 in every other mode. */
+int jac_sweeps_per_launch(const jac_ctx *ctx, int *host_out);
 
 /* Number of kernel launches this context has issued so far (HOST output). */
 int jac_launch_count(const jac_ctx *ctx, int64_t *host_out);

@@ -403,6 +403,9 @@ dense_copy_kernel(double* __restrict__ blocks, double* __restrict__ dense, const
 #endif
 constexpr int kTemporalWarps = JAC_TW;
 constexpr int kTemporalDepth = JAC_TD;
+// lanes at each end of a warp whose points are no longer exact after T levels (4 points per lane)
+__host__ __device__ constexpr int temporal_halo_lanes(int T) { return (T + 3) / 4; }
+__host__ __device__ constexpr int temporal_strip_cols(int T) { return 128 - 8 * temporal_halo_lanes(T); }
 
 struct RowCursor {
     long long off;  // element offset of the row within the array, relative to a lane's column base
@@ -583,7 +586,7 @@ __device__ __forceinline__ void temporal_step_any(Row4 (&win)[T][3], const Tempo
 }
 
 template <int T, bool HAS_F>
-__global__ void __launch_bounds__(kTemporalWarps * 32, JAC_TOCC)
+__global__ void __launch_bounds__(kTemporalWarps * 32, (T > 4 ? 2 : JAC_TOCC))
 temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const double* __restrict__ f,
                   const JacGeom g, const int strips_x, const int strips_y, const int rows_per_strip)
 {
@@ -594,14 +597,15 @@ temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
     const int sx = (int)(wid % strips_x), sy = (int)(wid / strips_x);
 
     TemporalCtx c;
-    const long long X0 = (long long)sx * 120 - 4;
+    constexpr int HL = temporal_halo_lanes(T);
+    const long long X0 = (long long)sx * temporal_strip_cols(T) - 4 * HL;
     const long long gx = X0 + 4 * lane;
     c.xout = gx < 0 || gx >= g.nx;
     c.cx = gx < 0 ? g.bval[0] : g.bval[1];
     c.c_my = g.bval[2];
     c.c_py = g.bval[3];
     c.edge_x = (sx == 0) || (X0 + 128 > g.nx);
-    c.store_lane = lane >= 1 && lane <= 30 && !c.xout;
+    c.store_lane = lane >= HL && lane <= 31 - HL && !c.xout;
     const long long col = c.xout ? g.origin : column_base(g, gx);
     c.fb = HAS_F ? f + col : nullptr;
     c.ob = un + col;

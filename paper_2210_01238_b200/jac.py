@@ -32,7 +32,7 @@ EXPORTS = [
     "jac_set_u", "jac_set_f", "jac_get_u", "jac_set_u_device", "jac_set_f_device",
     "jac_get_u_device", "jac_set_boundary", "jac_get_block_padded", "jac_get_halo_buffer",
     "jac_pack_halos", "jac_unpack_halos", "jac_pack_faces", "jac_unpack_faces", "jac_sweep", "jac_residual", "jac_launch_count",
-    "jac_last_cuda_error", "jac_strerror", "jac_residual_dense_static",
+    "jac_last_cuda_error", "jac_strerror", "jac_residual_dense_static", "jac_sweeps_per_launch",
 ]
 
 
@@ -85,6 +85,7 @@ def lib() -> C.CDLL:
         L.jac_sweep.argtypes = [vp, C.c_int]
         L.jac_residual.argtypes = [vp, dp]
         L.jac_launch_count.argtypes = [vp, C.POINTER(C.c_int64)]
+        L.jac_sweeps_per_launch.argtypes = [vp, C.POINTER(C.c_int)]
         L.jac_last_cuda_error.argtypes = [vp]
         L.jac_strerror.argtypes = [C.c_int]
         L.jac_residual_dense_static.argtypes = [C.c_int, C.POINTER(C.c_int64), vp, vp,
@@ -304,6 +305,11 @@ class Jacobi:
     def residual(self) -> float:
         out = C.c_double(0.0)
         self._call("jac_residual", lib().jac_residual(self._ctx, C.byref(out)))
+        return out.value
+
+    def sweeps_per_launch(self) -> int:
+        out = C.c_int(0)
+        self._call("jac_sweeps_per_launch", lib().jac_sweeps_per_launch(self._ctx, C.byref(out)))
         return out.value
 
     def launch_count(self) -> int:

@@ -49,7 +49,7 @@ def test_strerror(jac):
     dict(n=(12, 8), b=(0, 4)),
     dict(n=(12, 8), b=(24, 8)),
     dict(n=(12, 8), b=(4, 4), mode=7),
-    dict(n=(12, 8), b=(4, 4), tsteps=5),
+    dict(n=(12, 8), b=(4, 4), tsteps=9),
     dict(n=(12,), b=(4,)),                # ndim 1
 ])
 def test_invalid_descriptors_are_rejected(jac, kw):

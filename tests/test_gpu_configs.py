@@ -121,8 +121,10 @@ def test_c3_eigenmode_16384(jac, orc):
     lam = (math.cos(math.pi / (w.n[0] + 1)) + math.cos(math.pi / (w.n[1] + 1))) / 2.0
     closed_r = 4.0 * (1.0 - lam) * lam ** w.sweeps * (w.n[0] + 1) / 2.0
     assert np.max(np.abs(want - lam ** w.sweeps * u0)) < 2e-13      # the oracle itself, closed form
-    for mode, ts in (("temporal", 4), ("fused", 0), ("exchange", 0)):
+    for mode, ts in (("temporal", 0), ("temporal", 4), ("fused", 0), ("exchange", 0)):
         with _make(jac, w, mode, ts) as J:
+            if (mode, ts) == ("temporal", 0):
+                assert J.sweeps_per_launch() == 8     # the configuration the benchmark times
             J.set_u(u0)
             J.sweep(w.sweeps)
             got, got_r = J.get_u(), J.residual()

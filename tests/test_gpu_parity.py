@@ -198,11 +198,11 @@ TEMPORAL_SHAPES = [((8, 8), (4, 4)), ((120, 40), (60, 20)), ((124, 33), (124, 33
 
 
 @pytest.mark.parametrize("n,b", TEMPORAL_SHAPES)
-@pytest.mark.parametrize("tsteps", [1, 2, 3, 4])
+@pytest.mark.parametrize("tsteps", [1, 2, 3, 4, 5, 6, 7, 8])
 @pytest.mark.parametrize("has_f", [False, True])
 def test_temporal_blocking_matches_oracle(jac, orc, n, b, tsteps, has_f):
     J, B = _setup_pair(jac, orc, n, b, 1, has_f, "temporal", seed=2, tsteps=tsteps)
-    for nsw in (1, 4, 7):
+    for nsw in (1, 4, 17):
         J.sweep(nsw)
         B.sweep(nsw)
         _assert_sweep_close(J.get_u(), B.get_u())
