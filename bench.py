@@ -43,11 +43,19 @@ L2_BYTES = 126e6
 # the kernel sources the capture was taken with; reported as null once the sources changed.
 # key: (schedule, tsteps, ndim, has_f)
 # bytes_per_point_per_launch: (dram__bytes_read.sum + dram__bytes_write.sum) / points of the captured
-# launch (profiles/temporal2d_t4_eigenmode_8192.md: 8192^2, scaled to the workload by its points --
-# traffic is proportional to the points: every strip reads and writes its own columns once).
+# launch (a smaller case of the same workload, named beside each entry), scaled to the workload by
+# its points -- traffic is proportional to the points: every strip or tile reads and writes its own
+# part of the grid once per launch.
 NCU_TRAFFIC = {
-    ("temporal", 4, 2, False): {"bytes_per_point_per_launch": (606.650368e6 + 490.201856e6) / 8192 ** 2,
-                                "src_sha": "46c902c3cd6527b9"},
+    # profiles/temporal2d_eigenmode_8192.md
+    ("temporal", 8, 2, False): {"bytes_per_point_per_launch": (625.100032e6 + 490.793728e6) / 8192 ** 2,
+                                "src_sha": "a067f0d0087e06c8"},
+    # profiles/temporal3d_poisson_512.md
+    ("temporal", 2, 3, True): {"bytes_per_point_per_launch": (2.497591e9 + 1.047600e9) / 512 ** 3,
+                               "src_sha": "a067f0d0087e06c8"},
+    # profiles/exchange_schedule_eigenmode_8192.md (the update launch alone)
+    ("exchange", 1, 2, False): {"bytes_per_point_per_launch": (574.281984e6 + 494.291200e6) / 8192 ** 2,
+                                "src_sha": "a067f0d0087e06c8"},
 }
 KERNEL_NAMES = {("temporal", 2): "temporal2d_kernel", ("temporal", 3): "temporal3d_kernel", ("fused", 2): "sweep2d_kernel (update pulling neighbour interiors)",
                 ("exchange", 2): "sweep2d_kernel", ("pertask", 2): "sweep2d_kernel (one launch per block)",
