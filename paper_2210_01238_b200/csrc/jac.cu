@@ -388,10 +388,16 @@ int launch_temporal(jac_ctx* c, const double* u, double* un)
     const int strips_y = (int)ceil_div(g.ny, rows);
     const unsigned grid = (unsigned)ceil_div((long long)strips_x * strips_y, jac::kTemporalWarps);
     const int threads = jac::kTemporalWarps * 32;
-    if (c->desc.has_f)
-        jac::temporal2d_kernel<T, true><<<grid, threads, 0, c->stream>>>(u, un, c->f, g, strips_x, strips_y, rows);
-    else
-        jac::temporal2d_kernel<T, false><<<grid, threads, 0, c->stream>>>(u, un, c->f, g, strips_x, strips_y, rows);
+    if (c->desc.has_f) {
+        auto kern = jac::temporal2d_kernel<T, true>;
+        const size_t smem = jac::temporal_smem_bytes(T, true);
+        JAC_CK(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        kern<<<grid, threads, smem, c->stream>>>(u, un, c->f, g, strips_x, strips_y, rows);
+    } else {
+        auto kern = jac::temporal2d_kernel<T, false>;
+        const size_t smem = jac::temporal_smem_bytes(T, false);
+        kern<<<grid, threads, smem, c->stream>>>(u, un, c->f, g, strips_x, strips_y, rows);
+    }
     return check_launch(c);
 }
 

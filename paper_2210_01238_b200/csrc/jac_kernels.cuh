@@ -403,6 +403,17 @@ dense_copy_kernel(double* __restrict__ blocks, double* __restrict__ dense, const
 #endif
 constexpr int kTemporalWarps = JAC_TW;
 constexpr int kTemporalDepth = JAC_TD;
+// Right-hand side rows of the 2D temporal kernel: up to T = 4 they travel through a second
+// cp.async ring (a row is copied together with the u row of the same index and stays until the
+// top level has used it, DEPTH + 2T steps later); deeper pipelines read f through L1 instead.
+constexpr int kTemporalFDepth = 16;
+__host__ __device__ constexpr bool temporal_f_ring(int T, bool has_f) { return has_f && T <= 4; }
+__host__ __device__ constexpr int temporal_stages_per_warp(int T, bool has_f) {
+    return kTemporalDepth + (temporal_f_ring(T, has_f) ? kTemporalFDepth : 0);
+}
+__host__ __device__ constexpr size_t temporal_smem_bytes(int T, bool has_f) {
+    return (size_t)kTemporalWarps * temporal_stages_per_warp(T, has_f) * 64 * sizeof(double2);
+}
 // lanes at each end of a warp whose points are no longer exact after T levels (4 points per lane)
 __host__ __device__ constexpr int temporal_halo_lanes(int T) { return (T + 3) / 4; }
 __host__ __device__ constexpr int temporal_strip_cols(int T) { return 128 - 8 * temporal_halo_lanes(T); }
@@ -471,6 +482,7 @@ struct TemporalCtx {
     double2* dst_a;       // ring positions (stage 0) of the two chunks this lane copies
     double2* dst_b;
     const double2* mine;  // ring position (stage 0) of this lane's first chunk
+    long long fdelta;     // f - u in elements: the same copy sources serve the f ring
     long long brs;        // elements between vertically adjacent blocks
     int ny;
     int r0;               // first input row of the strip
@@ -482,15 +494,22 @@ struct TemporalCtx {
     bool xout, edge_x, store_lane;
 };
 
-// start the copy of input row r into its ring stage (nothing to copy outside the domain); with a
-// right-hand side, also ask for the lane's part of f row r, which the levels read DEPTH steps later
-template <bool HAS_F>
+// start the copy of input row r into its ring stage (nothing to copy outside the domain).  With a
+// right-hand side, f row r goes into the f ring (F_RING: stages follow the u stages of the warp),
+// or is at least requested into L2 for the loads that follow DEPTH steps later.
+template <bool HAS_F, bool F_RING>
 __device__ __forceinline__ void issue_row(const TemporalCtx& c, int r, const RowCursor& cur) {
     if (r >= 0 && r < c.ny && r < c.in_end) {
         const int st = ((r - c.r0) % kTemporalDepth) * 64;
         if (c.copy_a) cp_async16(c.dst_a + st, c.src_a + cur.off);
         if (c.copy_b) cp_async16(c.dst_b + st, c.src_b + cur.off);
-        if (HAS_F && !c.xout) prefetch_line(c.fb + cur.off);
+        if (F_RING) {
+            const int fs = (kTemporalDepth + ((r - c.r0) % kTemporalFDepth)) * 64;
+            if (c.copy_a) cp_async16(c.dst_a + fs, c.src_a + c.fdelta + cur.off);
+            if (c.copy_b) cp_async16(c.dst_b + fs, c.src_b + c.fdelta + cur.off);
+        } else if (HAS_F && !c.xout) {
+            prefetch_line(c.fb + cur.off);
+        }
     }
     cp_async_commit();
 }
@@ -522,7 +541,8 @@ __device__ __forceinline__ void temporal_step(Row4 (&win)[T][3], const TemporalC
     __syncwarp();                                    // the other lanes' chunks of row r have landed too
     win[0][PH] = take_row<EDGE>(c, r);
     __syncwarp();                                    // everyone has read the stage before it is refilled
-    issue_row<HAS_F>(c, r + kTemporalDepth, load_cur);
+    constexpr bool F_RING = temporal_f_ring(T, HAS_F);
+    issue_row<HAS_F, F_RING>(c, r + kTemporalDepth, load_cur);
     load_cur.advance(g, c.brs);
 #pragma unroll
     for (int s = T; s >= 1; --s) {
@@ -537,7 +557,13 @@ __device__ __forceinline__ void temporal_step(Row4 (&win)[T][3], const TemporalC
         if (HAS_F) {
             // f of row rs: the output cursor points at row r - 2T + 1, i.e. (T - s) * 2 rows below rs
             const bool ok = EDGE ? (rs >= 0 && rs < c.ny && !c.xout) : true;
-            if (ok) {
+            if (ok && F_RING) {
+                // copied DEPTH + 2s - 1 steps ago; the warp-wide barriers of the steps in between
+                // made the other lanes' chunks visible
+                const double2* fr = c.mine + (kTemporalDepth + ((rs - c.r0) & (kTemporalFDepth - 1))) * 64;
+                const double2 a = fr[0], b = fr[1];
+                ff.v[0] = a.x; ff.v[1] = a.y; ff.v[2] = b.x; ff.v[3] = b.y;
+            } else if (ok) {
                 RowCursor fc = out_cur;
 #pragma unroll
                 for (int k = 0; k < 2 * (T - s); ++k) fc.advance(g, c.brs);
@@ -586,11 +612,12 @@ __device__ __forceinline__ void temporal_step_any(Row4 (&win)[T][3], const Tempo
 }
 
 template <int T, bool HAS_F>
-__global__ void __launch_bounds__(kTemporalWarps * 32, (T > 4 ? 2 : JAC_TOCC))
+__global__ void __launch_bounds__(kTemporalWarps * 32, ((T > 4 || temporal_f_ring(T, HAS_F)) ? 2 : JAC_TOCC))
 temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const double* __restrict__ f,
                   const JacGeom g, const int strips_x, const int strips_y, const int rows_per_strip)
 {
-    __shared__ double2 ring_mem[kTemporalWarps][kTemporalDepth][64];
+    extern __shared__ __align__(16) double2 t2_ring_mem[];   // [warp][u stages, then f stages][64]
+    constexpr bool F_RING = temporal_f_ring(T, HAS_F);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const long long wid = (long long)blockIdx.x * kTemporalWarps + warp;
     if (wid >= (long long)strips_x * strips_y) return;   // whole warps only; warps never meet at a barrier
@@ -614,7 +641,8 @@ temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
     c.copy_b = xb >= 0 && xb < g.nx;
     c.src_a = u + (c.copy_a ? column_base(g, xa) : g.origin);
     c.src_b = u + (c.copy_b ? column_base(g, xb) : g.origin);
-    double2* ring = &ring_mem[warp][0][0];
+    double2* ring = t2_ring_mem + warp * temporal_stages_per_warp(T, HAS_F) * 64;
+    c.fdelta = HAS_F ? (long long)(f - u) : 0;
     c.dst_a = ring + lane;        // chunk k = lane
     c.dst_b = ring + 32 + lane;   // chunk k = 32 + lane
     c.mine = ring + 2 * lane;     // chunks 2*lane and 2*lane + 1
@@ -639,7 +667,7 @@ temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
     // fill the ring with the first DEPTH rows
 #pragma unroll 1
     for (int k = 0; k < kTemporalDepth; ++k) {
-        issue_row<HAS_F>(c, c.r0 + k, load_cur);
+        issue_row<HAS_F, F_RING>(c, c.r0 + k, load_cur);
         load_cur.advance(g, c.brs);
     }
 
