@@ -114,3 +114,16 @@ def test_binding_refuses_to_run_without_a_gpu(jac):
         pytest.skip("a GPU is present")
     with pytest.raises(RuntimeError):
         jac.Jacobi((8, 8), (4, 4))
+
+
+def test_product_code_never_touches_the_oracle():
+    """The oracle is test infrastructure: nothing in the package (binding, build, inputs, kernels)
+    may import, load or name it, and the oracle may not reach into the package's CUDA side."""
+    pkg = ROOT / "paper_2210_01238_b200"
+    for path in list(pkg.rglob("*.py")) + list(pkg.rglob("*.cu*")) + list(pkg.rglob("*.h")):
+        text = path.read_text()
+        assert "oracle" not in text.lower() and "liborc" not in text, path
+    for path in (ROOT / "oracle").glob("*"):
+        if path.suffix in (".py", ".c"):
+            text = path.read_text()
+            assert "libjac" not in text and "import jac" not in text and "csrc" not in text, path

@@ -278,3 +278,14 @@ def test_partial_exchange_by_face_mask(jac, orc):
             J.pack_faces(1 << (2 * ndim))
         J.close()
         B.close()
+
+
+def test_sweeps_per_launch_query(jac):
+    cases = [(dict(n=(64, 64), b=(32, 32), mode="exchange"), 1),
+             (dict(n=(64, 64), b=(32, 32), mode="temporal", tsteps=3), 3),
+             (dict(n=(64, 64), b=(32, 32), mode="temporal"), 4),            # small grid: 4
+             (dict(n=(64, 64), b=(32, 32), mode="temporal", has_f=True), 4),
+             (dict(n=(16, 16, 16), b=(8, 8, 8), mode="temporal"), 2)]
+    for kw, want in cases:
+        with jac.Jacobi(**kw) as J:
+            assert J.sweeps_per_launch() == want, kw
