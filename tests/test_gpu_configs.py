@@ -243,3 +243,33 @@ def test_paper_strong_scaling_shape_1024x1024x768(jac, orc):
     want = orc.sample_points(n, 20, pts, zeros, _box(f))
     for p, v in zip(pts, want):
         assert got[p[2], p[1], p[0]] == v, p
+
+
+def test_offsets_beyond_2_to_31_elements(jac, orc):
+    """A 49152 x 45056 grid (2.2e9 points, 17.7 GB per array): element offsets exceed 2^31, so any
+    32-bit index arithmetic in a kernel or in the host code would show.  Inputs are drawn on the
+    device (seeded), the oracle evaluates sampled outputs from the windows it is handed."""
+    import torch
+    free, _ = torch.cuda.mem_get_info()
+    if free < 100 * 2 ** 30:
+        pytest.skip("needs about 100 GB of free device memory")
+    n, b = (49152, 45056), (1024, 1024)
+    gen = torch.Generator(device="cuda").manual_seed(7)
+    u0 = torch.rand((n[1], n[0]), dtype=torch.float64, device="cuda", generator=gen)
+    pts = [(0, 0), (49151, 45055), (49151, 0), (0, 45055), (1023, 1024), (24576, 22528),
+           (48127, 44031), (48128, 44032), (33333, 40000)]
+
+    def window(lo, hi):
+        return u0[lo[1]:hi[1], lo[0]:hi[0]].cpu().numpy()
+
+    for mode, sweeps in (("temporal", 8), ("fused", 2), ("exchange", 2)):
+        with jac.Jacobi(n, b, 1, False, mode) as J:
+            J.set_boundary(1, 0.5)
+            J.set_boundary(3, -0.25)
+            J.set_u_device(u0)
+            J.sweep(sweeps)
+            out = J.get_u_device()
+        want = orc.sample_points(n, sweeps, pts, window, None, [0.0, 0.5, 0.0, -0.25])
+        got = np.array([float(out[p[1], p[0]]) for p in pts])
+        assert np.array_equal(got, want), (mode, got - want)
+        del out
