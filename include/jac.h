@@ -164,6 +164,23 @@ int jac_unpack_faces(jac_ctx *ctx, unsigned face_mask);
  * nsweeps < 0 is JAC_EINVAL. */
 int jac_sweep(jac_ctx *ctx, int nsweeps);
 
+/* jac_sweep(nsweeps) and, from the same pass over memory, the L2 residual norm of the state
+ * BEFORE the last of those sweeps: the last sweep has s(p) of that state in a register anyway and
+ * also accumulates ( s(p) - c*u(p) )^2, so the norm costs no extra memory traffic (jac_residual
+ * reads u, and f, once more).  The value equals what jac_residual would return after
+ * nsweeps - 1 sweeps, up to summation order (<= 1e-10 relative).  nsweeps >= 1.  Synchronises the
+ * stream and writes one HOST double.  (The paper runs a fixed iteration count; this is the usual
+ * one-iteration-lagged convergence monitor of a Jacobi solver.) */
+int jac_sweep_residual(jac_ctx *ctx, int nsweeps, double *host_out_l2);
+
+/* Iterate until converged: runs sweeps in groups of check_every (each group through
+ * jac_sweep_residual) until the lagged residual norm is <= tol or max_sweeps sweeps have run.
+ * HOST outputs: the sweeps actually done and the last norm measured (the residual of the state one
+ * sweep before the final one).  Errors: JAC_EINVAL for max_sweeps < 1, check_every < 1, tol < 0 or
+ * NaN, null outputs. */
+int jac_solve(jac_ctx *ctx, int max_sweeps, int check_every, double tol, int *host_sweeps_done,
+              double *host_residual);
+
 /* L2 norm of the residual of the current state, sqrt( sum_p ( s(p) - c*u(p) )^2 ) with s as in
  * the update (including + f), over all interior points, not normalised.  (The paper runs a
  * fixed iteration count and has no residual; this is the convergence measure of the same

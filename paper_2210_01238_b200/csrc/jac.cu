@@ -61,6 +61,55 @@ Tiling make_tiling(const JacGeom& g)
     return t;
 }
 
+// Geometry of the temporal launches (also bounds the reduction scratch they may fill).
+struct TemporalGrid {
+    int a, b, c, chunk;   // 2D: strips_x, strips_y, -, rows per strip; 3D: tiles x, y, z, planes per chunk
+    long long warps;      // partial sums a residual-carrying launch writes
+    long long ctas;
+};
+
+TemporalGrid temporal_grid_2d(const JacGeom& g, int T)
+{
+    TemporalGrid t{};
+    t.a = (int)ceil_div(g.nx, jac::temporal_strip_cols(T));
+    // strips of 256 rows amortise the 4T - 1 steps of pipeline fill; shorter ones when the grid
+    // would otherwise give fewer than four rounds of resident warps (longer strips were measured
+    // slower at 16384^2: 512 rows lose 8 % at T = 8)
+    int rows = 256;
+    while (rows > 32 && (long long)t.a * ceil_div(g.ny, rows) < (long long)kNumSMs * 48) rows /= 2;
+    // tiny grids: not even one warp per scheduler; shorter strips cut the serial length of a launch
+    while (rows > 8 && (long long)t.a * ceil_div(g.ny, rows) < (long long)kNumSMs * 4) rows /= 2;
+    t.chunk = rows;
+    t.b = (int)ceil_div(g.ny, rows);
+    t.c = 1;
+    t.warps = (long long)t.a * t.b;
+    t.ctas = ceil_div(t.warps, jac::kTemporalWarps);
+    return t;
+}
+
+TemporalGrid temporal_grid_3d(const JacGeom& g, int T)
+{
+    TemporalGrid t{};
+    t.a = (int)ceil_div(g.nx, 60);
+    t.b = (int)ceil_div(g.ny, jac::k3dTileRows - 2 * T);
+    int zchunk = 128;
+    while (zchunk > 16 && (long long)t.a * t.b * ceil_div(g.nz, zchunk) < (long long)kNumSMs * 4) zchunk /= 2;
+    t.chunk = zchunk;
+    t.c = (int)ceil_div(g.nz, zchunk);
+    t.ctas = (long long)t.a * t.b * t.c;
+    t.warps = t.ctas * jac::k3dWarps;
+    return t;
+}
+
+// largest number of partial sums any launch of this geometry can write
+long long max_partials(const JacGeom& g, long long sweep_ctas)
+{
+    long long m = sweep_ctas;
+    if (g.ndim == 2) for (int T = 1; T <= 8; ++T) m = std::max(m, temporal_grid_2d(g, T).warps);
+    else for (int T = 1; T <= 2; ++T) m = std::max(m, temporal_grid_3d(g, T).warps);
+    return m;
+}
+
 int build_geometry(const jac_desc* d, JacGeom* g, jac_layout* L)
 {
     if (!d) return JAC_EINVAL;
@@ -127,7 +176,7 @@ int build_geometry(const jac_desc* d, JacGeom* g, jac_layout* L)
             L->face_offset[fc] = g->face_off[fc];
         }
         L->send_stride = g->send_stride;
-        L->partials = round_up(ctas, 32);
+        L->partials = round_up(max_partials(*g, ctas), 32);
         const long long arr_bytes = round_up(g->nblocks * g->block_stride * 8, 256);
         long long o = 0;
         L->off_u[0] = o; o += arr_bytes;
@@ -186,12 +235,14 @@ void launch_sweep_t(jac_ctx* c, const double* u, double* un, long long blk0, lon
 {
     const Tiling& t = c->tile;
     const unsigned grid = (unsigned)(nblk * t.ctas_per_block);
+    // a launch over a sub-range of blocks writes its partial sums where a full launch would
+    double* parts = c->partials + blk0 * t.ctas_per_block;
     if (c->g.ndim == 2)
         jac::sweep2d_kernel<NV, HAS_F, OP><<<grid, t.block, 0, c->stream>>>(
-            u, un, c->f, c->partials, c->g, blk0, t.tiles_x, t.tiles_y, t.march);
+            u, un, c->f, parts, c->g, blk0, t.tiles_x, t.tiles_y, t.march);
     else
         jac::sweep3d_kernel<NV, HAS_F, OP><<<grid, t.block, 0, c->stream>>>(
-            u, un, c->f, c->partials, c->g, blk0, t.tiles_x, t.tiles_y, t.tiles_z, t.march);
+            u, un, c->f, parts, c->g, blk0, t.tiles_x, t.tiles_y, t.tiles_z, t.march);
 }
 
 template <int OP>
@@ -345,74 +396,156 @@ int default_tsteps(const jac_desc& d)
     return (!d.has_f && large) ? 8 : 4;
 }
 
-// T sweeps in one launch (3D, tiles of 64 x 48 streamed along z)
-template <int T, bool HAS_F>
-int launch_temporal3d_t(jac_ctx* c, const double* u, double* un)
+// T sweeps in one launch (3D, tiles of 64 x 48 streamed along z).  RES: the launch also leaves
+// per-warp partial sums of the squared residual of the state before its last sweep.
+template <int T, bool HAS_F, bool RES>
+int launch_temporal3d_t(jac_ctx* c, const double* u, double* un, long long* nparts)
 {
-    const JacGeom& g = c->g;
-    const int tiles_x = (int)ceil_div(g.nx, 60);
-    const int tiles_y = (int)ceil_div(g.ny, jac::k3dTileRows - 2 * T);
-    int zchunk = 128;
-    while (zchunk > 16 && (long long)tiles_x * tiles_y * ceil_div(g.nz, zchunk) < (long long)kNumSMs * 4) zchunk /= 2;
-    const int tiles_z = (int)ceil_div(g.nz, zchunk);
-    const long long ctas = (long long)tiles_x * tiles_y * tiles_z;
-    if (ctas > kMaxGrid) return JAC_EINVAL;
-    auto kern = jac::temporal3d_kernel<T, HAS_F>;
+    const TemporalGrid t = temporal_grid_3d(c->g, T);
+    if (t.ctas > kMaxGrid) return JAC_EINVAL;
+    auto kern = jac::temporal3d_kernel<T, HAS_F, RES>;
     const size_t smem = jac::k3d_smem_bytes(HAS_F);
     JAC_CK(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    kern<<<(unsigned)ctas, jac::k3dWarps * 32, smem, c->stream>>>(u, un, c->f, g, tiles_x, tiles_y,
-                                                                             tiles_z, zchunk);
+    kern<<<(unsigned)t.ctas, jac::k3dWarps * 32, smem, c->stream>>>(u, un, c->f, c->partials, c->g, t.a, t.b, t.c,
+                                                                   t.chunk);
+    if (RES) *nparts = t.warps;
     return check_launch(c);
 }
 
-int launch_temporal3d_n(jac_ctx* c, int t, const double* u, double* un)
+int launch_temporal3d_n(jac_ctx* c, int t, const double* u, double* un, bool res, long long* nparts)
 {
     const bool f = c->desc.has_f != 0;
-    if (t == 1) return f ? launch_temporal3d_t<1, true>(c, u, un) : launch_temporal3d_t<1, false>(c, u, un);
-    return f ? launch_temporal3d_t<2, true>(c, u, un) : launch_temporal3d_t<2, false>(c, u, un);
+    if (res) {
+        if (t == 1) return f ? launch_temporal3d_t<1, true, true>(c, u, un, nparts)
+                             : launch_temporal3d_t<1, false, true>(c, u, un, nparts);
+        return f ? launch_temporal3d_t<2, true, true>(c, u, un, nparts)
+                 : launch_temporal3d_t<2, false, true>(c, u, un, nparts);
+    }
+    if (t == 1) return f ? launch_temporal3d_t<1, true, false>(c, u, un, nparts)
+                         : launch_temporal3d_t<1, false, false>(c, u, un, nparts);
+    return f ? launch_temporal3d_t<2, true, false>(c, u, un, nparts)
+             : launch_temporal3d_t<2, false, false>(c, u, un, nparts);
 }
 
 // T sweeps in one launch (2D, register-streaming temporal blocking)
-template <int T>
-int launch_temporal(jac_ctx* c, const double* u, double* un)
+template <int T, bool HAS_F, bool RES>
+int launch_temporal_t(jac_ctx* c, const double* u, double* un, long long* nparts)
 {
-    const JacGeom& g = c->g;
-    const int strips_x = (int)ceil_div(g.nx, jac::temporal_strip_cols(T));
-    // strips of 256 rows amortise the 4T - 1 steps of pipeline fill; shorter ones when the grid
-    // would otherwise give fewer than four rounds of resident warps (longer strips were measured
-    // slower at 16384^2: 512 rows lose 8 % at T = 8)
-    int rows = 256;
-    while (rows > 32 && (long long)strips_x * ceil_div(g.ny, rows) < (long long)kNumSMs * 48) rows /= 2;
-    // tiny grids: not even one warp per scheduler; shorter strips cut the serial length of a launch
-    while (rows > 8 && (long long)strips_x * ceil_div(g.ny, rows) < (long long)kNumSMs * 4) rows /= 2;
-    const int strips_y = (int)ceil_div(g.ny, rows);
-    const unsigned grid = (unsigned)ceil_div((long long)strips_x * strips_y, jac::kTemporalWarps);
-    const int threads = jac::kTemporalWarps * 32;
-    if (c->desc.has_f) {
-        auto kern = jac::temporal2d_kernel<T, true>;
-        const size_t smem = jac::temporal_smem_bytes(T, true);
+    const TemporalGrid t = temporal_grid_2d(c->g, T);
+    auto kern = jac::temporal2d_kernel<T, HAS_F, RES>;
+    const size_t smem = jac::temporal_smem_bytes(T, HAS_F);
+    if (smem > 48 * 1024)
         JAC_CK(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        kern<<<grid, threads, smem, c->stream>>>(u, un, c->f, g, strips_x, strips_y, rows);
-    } else {
-        auto kern = jac::temporal2d_kernel<T, false>;
-        const size_t smem = jac::temporal_smem_bytes(T, false);
-        kern<<<grid, threads, smem, c->stream>>>(u, un, c->f, g, strips_x, strips_y, rows);
-    }
+    kern<<<(unsigned)t.ctas, jac::kTemporalWarps * 32, smem, c->stream>>>(u, un, c->f, c->partials, c->g, t.a, t.b,
+                                                                         t.chunk);
+    if (RES) *nparts = t.warps;
     return check_launch(c);
 }
 
-int launch_temporal_n(jac_ctx* c, int t, const double* u, double* un)
+template <int T>
+int launch_temporal(jac_ctx* c, const double* u, double* un, bool res, long long* nparts)
+{
+    const bool f = c->desc.has_f != 0;
+    if (res) return f ? launch_temporal_t<T, true, true>(c, u, un, nparts)
+                      : launch_temporal_t<T, false, true>(c, u, un, nparts);
+    return f ? launch_temporal_t<T, true, false>(c, u, un, nparts)
+             : launch_temporal_t<T, false, false>(c, u, un, nparts);
+}
+
+int launch_temporal_n(jac_ctx* c, int t, const double* u, double* un, bool res, long long* nparts)
 {
     switch (t) {
-        case 1: return launch_temporal<1>(c, u, un);
-        case 2: return launch_temporal<2>(c, u, un);
-        case 3: return launch_temporal<3>(c, u, un);
-        case 4: return launch_temporal<4>(c, u, un);
-        case 5: return launch_temporal<5>(c, u, un);
-        case 6: return launch_temporal<6>(c, u, un);
-        case 7: return launch_temporal<7>(c, u, un);
-        default: return launch_temporal<8>(c, u, un);
+        case 1: return launch_temporal<1>(c, u, un, res, nparts);
+        case 2: return launch_temporal<2>(c, u, un, res, nparts);
+        case 3: return launch_temporal<3>(c, u, un, res, nparts);
+        case 4: return launch_temporal<4>(c, u, un, res, nparts);
+        case 5: return launch_temporal<5>(c, u, un, res, nparts);
+        case 6: return launch_temporal<6>(c, u, un, res, nparts);
+        case 7: return launch_temporal<7>(c, u, un, res, nparts);
+        default: return launch_temporal<8>(c, u, un, res, nparts);
     }
+}
+
+// nsweeps iterations in the context's schedule.  With `res`, the last sweep also leaves partial
+// sums of the squared residual of the state it reads in the scratch (*nparts of them).
+int run_sweeps(jac_ctx* c, int nsweeps, bool res, long long* nparts)
+{
+    int rc = JAC_OK;
+    const JacGeom& g = c->g;
+    const long long sweep_parts = g.nblocks * c->tile.ctas_per_block;
+    switch (c->desc.mode) {
+        case JAC_MODE_FUSED:
+            for (int s = 0; s < nsweeps; ++s) {
+                const bool last = res && s + 1 == nsweeps;
+                rc = last ? launch_sweep<jac::OP_UPDATE_PULL_RES>(c, c->u[c->cur], c->u[c->cur ^ 1], 0, g.nblocks)
+                          : launch_sweep<jac::OP_UPDATE_PULL>(c, c->u[c->cur], c->u[c->cur ^ 1], 0, g.nblocks);
+                if (rc) return rc;
+                c->cur ^= 1;
+            }
+            if (res) *nparts = sweep_parts;
+            c->ghosts_fresh = false;
+            c->packed_current = false;
+            break;
+        case JAC_MODE_EXCHANGE:
+            for (int s = 0; s < nsweeps; ++s) {
+                const bool last = res && s + 1 == nsweeps;
+                if ((rc = do_exchange(c))) return rc;
+                rc = last ? launch_sweep<jac::OP_UPDATE_RES>(c, c->u[c->cur], c->u[c->cur ^ 1], 0, g.nblocks)
+                          : launch_sweep<jac::OP_UPDATE>(c, c->u[c->cur], c->u[c->cur ^ 1], 0, g.nblocks);
+                if (rc) return rc;
+                c->cur ^= 1;
+                c->ghosts_fresh = false;
+                c->packed_current = false;
+            }
+            if (res) *nparts = sweep_parts;
+            break;
+        case JAC_MODE_PERTASK:
+            for (int s = 0; s < nsweeps; ++s) {
+                const bool last = res && s + 1 == nsweeps;
+                if ((rc = do_exchange(c))) return rc;
+                for (long long blk = 0; blk < g.nblocks; ++blk) {
+                    rc = last ? launch_sweep<jac::OP_UPDATE_RES>(c, c->u[c->cur], c->u[c->cur ^ 1], blk, 1)
+                              : launch_sweep<jac::OP_UPDATE>(c, c->u[c->cur], c->u[c->cur ^ 1], blk, 1);
+                    if (rc) return rc;
+                }
+                c->cur ^= 1;
+                c->ghosts_fresh = false;
+                c->packed_current = false;
+            }
+            if (res) *nparts = sweep_parts;
+            break;
+        case JAC_MODE_TEMPORAL: {
+            const int T = default_tsteps(c->desc);
+            for (int left = nsweeps; left > 0;) {
+                const int t = std::min(T, left);
+                const bool last = res && left == t;
+                rc = (g.ndim == 2) ? launch_temporal_n(c, t, c->u[c->cur], c->u[c->cur ^ 1], last, nparts)
+                                   : launch_temporal3d_n(c, t, c->u[c->cur], c->u[c->cur ^ 1], last, nparts);
+                if (rc) return rc;
+                c->cur ^= 1;
+                left -= t;
+            }
+            c->ghosts_fresh = false;
+            c->packed_current = false;
+            break;
+        }
+        default:
+            return JAC_EINVAL;
+    }
+    return JAC_OK;
+}
+
+// fixed-order sum of the first nparts partial sums -> host, as a norm
+int finish_norm(jac_ctx* c, long long nparts, double* host_out_l2)
+{
+    jac::reduce_partials_kernel<<<1, 1024, 0, c->stream>>>(c->partials, nparts, c->result);
+    int rc = check_launch(c);
+    if (rc) return rc;
+    double sum = 0.0;
+    JAC_CK(c, cudaMemcpyAsync(&sum, c->result, sizeof(double), cudaMemcpyDeviceToHost, c->stream));
+    JAC_CK(c, cudaStreamSynchronize(c->stream));
+    *host_out_l2 = std::sqrt(sum);
+    return JAC_OK;
 }
 
 }  // namespace
@@ -642,55 +775,38 @@ int jac_sweep(jac_ctx* c, int nsweeps)
     if (rc) return rc;
     if (nsweeps < 0) return JAC_EINVAL;
     if (nsweeps == 0) return JAC_OK;
-    const JacGeom& g = c->g;
-    switch (c->desc.mode) {
-        case JAC_MODE_FUSED:
-            for (int s = 0; s < nsweeps; ++s) {
-                if ((rc = launch_sweep<jac::OP_UPDATE_PULL>(c, c->u[c->cur], c->u[c->cur ^ 1], 0, g.nblocks)))
-                    return rc;
-                c->cur ^= 1;
-            }
-            c->ghosts_fresh = false;
-            c->packed_current = false;
-            break;
-        case JAC_MODE_EXCHANGE:
-            for (int s = 0; s < nsweeps; ++s) {
-                if ((rc = do_exchange(c))) return rc;
-                if ((rc = launch_sweep<jac::OP_UPDATE>(c, c->u[c->cur], c->u[c->cur ^ 1], 0, g.nblocks)))
-                    return rc;
-                c->cur ^= 1;
-                c->ghosts_fresh = false;
-                c->packed_current = false;
-            }
-            break;
-        case JAC_MODE_PERTASK:
-            for (int s = 0; s < nsweeps; ++s) {
-                if ((rc = do_exchange(c))) return rc;
-                for (long long blk = 0; blk < g.nblocks; ++blk)
-                    if ((rc = launch_sweep<jac::OP_UPDATE>(c, c->u[c->cur], c->u[c->cur ^ 1], blk, 1)))
-                        return rc;
-                c->cur ^= 1;
-                c->ghosts_fresh = false;
-                c->packed_current = false;
-            }
-            break;
-        case JAC_MODE_TEMPORAL: {
-            const int T = default_tsteps(c->desc);
-            for (int left = nsweeps; left > 0;) {
-                const int t = std::min(T, left);
-                rc = (g.ndim == 2) ? launch_temporal_n(c, t, c->u[c->cur], c->u[c->cur ^ 1])
-                                   : launch_temporal3d_n(c, t, c->u[c->cur], c->u[c->cur ^ 1]);
-                if (rc) return rc;
-                c->cur ^= 1;
-                left -= t;
-            }
-            c->ghosts_fresh = false;
-            c->packed_current = false;
-            break;
-        }
-        default:
-            return JAC_EINVAL;
+    return run_sweeps(c, nsweeps, false, nullptr);
+}
+
+int jac_sweep_residual(jac_ctx* c, int nsweeps, double* host_out_l2)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    if (nsweeps < 1 || !host_out_l2) return JAC_EINVAL;
+    long long nparts = 0;
+    if ((rc = run_sweeps(c, nsweeps, true, &nparts))) return rc;
+    return finish_norm(c, nparts, host_out_l2);
+}
+
+int jac_solve(jac_ctx* c, int max_sweeps, int check_every, double tol, int* host_sweeps_done,
+              double* host_residual)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    if (max_sweeps < 1 || check_every < 1 || !(tol >= 0.0) || !host_sweeps_done || !host_residual)
+        return JAC_EINVAL;
+    int done = 0;
+    double res = 0.0;
+    while (done < max_sweeps) {
+        const int n = std::min(check_every, max_sweeps - done);
+        long long nparts = 0;
+        if ((rc = run_sweeps(c, n, true, &nparts))) return rc;
+        if ((rc = finish_norm(c, nparts, &res))) return rc;
+        done += n;
+        if (res <= tol) break;
     }
+    *host_sweeps_done = done;
+    *host_residual = res;
     return JAC_OK;
 }
 
@@ -701,14 +817,7 @@ int jac_residual(jac_ctx* c, double* host_out_l2)
     if (!host_out_l2) return JAC_EINVAL;
     if (!c->ghosts_fresh && (rc = do_exchange(c))) return rc;
     if ((rc = launch_sweep<jac::OP_RESIDUAL>(c, c->u[c->cur], nullptr, 0, c->g.nblocks))) return rc;
-    const long long nparts = c->g.nblocks * c->tile.ctas_per_block;
-    jac::reduce_partials_kernel<<<1, 1024, 0, c->stream>>>(c->partials, nparts, c->result);
-    if ((rc = check_launch(c))) return rc;
-    double sum = 0.0;
-    JAC_CK(c, cudaMemcpyAsync(&sum, c->result, sizeof(double), cudaMemcpyDeviceToHost, c->stream));
-    JAC_CK(c, cudaStreamSynchronize(c->stream));
-    *host_out_l2 = std::sqrt(sum);
-    return JAC_OK;
+    return finish_norm(c, c->g.nblocks * c->tile.ctas_per_block, host_out_l2);
 }
 
 int jac_sweeps_per_launch(const jac_ctx* c, int* host_out)

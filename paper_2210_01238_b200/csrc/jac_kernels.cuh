@@ -13,7 +13,10 @@
 
 namespace jac {
 
-enum : int { OP_UPDATE = 0, OP_UPDATE_PULL = 1, OP_RESIDUAL = 2 };
+enum : int { OP_UPDATE = 0, OP_UPDATE_PULL = 1, OP_RESIDUAL = 2, OP_UPDATE_RES = 3, OP_UPDATE_PULL_RES = 4 };
+__host__ __device__ constexpr bool op_stores(int op) { return op != OP_RESIDUAL; }
+__host__ __device__ constexpr bool op_pulls(int op) { return op == OP_UPDATE_PULL || op == OP_UPDATE_PULL_RES; }
+__host__ __device__ constexpr bool op_sums(int op) { return op == OP_RESIDUAL || op == OP_UPDATE_RES || op == OP_UPDATE_PULL_RES; }
 
 __device__ __forceinline__ double add_rn(double a, double b) { return __dadd_rn(a, b); }
 __device__ __forceinline__ double sub_rn(double a, double b) { return __dsub_rn(a, b); }
@@ -66,6 +69,8 @@ __device__ __forceinline__ double block_sum(double v) {
 //                 read from that block's interior (the cell its packed face would carry), so
 //                 no exchange has to run before the sweep; Dirichlet ghosts are still read
 // OP_RESIDUAL     per-CTA partial of sum r^2, r = s - 4u (ghost-reading)
+// OP_UPDATE_RES, OP_UPDATE_PULL_RES  the update, and in the same pass the partial of sum r^2 of the
+//                 state being read (s is in a register anyway): the residual at no extra traffic
 // ---------------------------------------------------------------------------------------
 template <int NV, bool HAS_F, int OP>
 __global__ void __launch_bounds__(256)
@@ -87,12 +92,12 @@ sweep2d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
         const long long base = blk * g.block_stride + g.origin + x;
         const double* ub = u + base;
         const double* fb = HAS_F ? f + base : nullptr;
-        double* ob = (OP == OP_RESIDUAL) ? nullptr : un + base;
+        double* ob = op_stores(OP) ? un + base : nullptr;
 
         // where the neighbours outside the block are found, relative to the row's own address
         long long off_w = -1, off_e = NV;             // ghost columns
         long long off_s0 = -PX, off_n1 = PX;          // ghost rows below row 0 / above row by-1
-        if (OP == OP_UPDATE_PULL) {
+        if (op_pulls(OP)) {
             const int bxi = (int)(blk % g.gx), byi = (int)(blk / g.gx);
             const long long bs = g.block_stride;
             if (x == 0 && bxi > 0) off_w = -bs + g.bx - 1;                     // left block, last column
@@ -106,7 +111,7 @@ sweep2d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
 #pragma unroll 4
         for (int j = j0; j < j1; ++j) {
             const long long ro = (long long)j * PX;
-            const Vec<NV> N = load_vec<NV>(ub + ro + ((OP == OP_UPDATE_PULL && j + 1 == g.by) ? off_n1 : PX));
+            const Vec<NV> N = load_vec<NV>(ub + ro + ((op_pulls(OP) && j + 1 == g.by) ? off_n1 : PX));
             const double w = ub[ro + off_w];
             const double e = ub[ro + off_e];
             Vec<NV> ff;
@@ -118,19 +123,18 @@ sweep2d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
                 const double E = (q == NV - 1) ? e : Cc.v[q + 1];
                 double s = add_rn(add_rn(W, E), add_rn(S.v[q], N.v[q]));
                 if (HAS_F) s = add_rn(s, ff.v[q]);
-                if (OP == OP_RESIDUAL) {
+                if (op_sums(OP)) {
                     const double r = sub_rn(s, mul_rn(4.0, Cc.v[q]));
                     acc = add_rn(acc, mul_rn(r, r));
-                } else {
-                    o.v[q] = mul_rn(s, 0.25);
                 }
+                if (op_stores(OP)) o.v[q] = mul_rn(s, 0.25);
             }
-            if (OP != OP_RESIDUAL) store_vec<NV>(ob + ro, o);
+            if (op_stores(OP)) store_vec<NV>(ob + ro, o);
             S = Cc;
             Cc = N;
         }
     }
-    if (OP == OP_RESIDUAL) {
+    if (op_sums(OP)) {
         const double total = block_sum(acc);
         if (threadIdx.x == 0) partials[blockIdx.x] = total;
     }
@@ -166,11 +170,11 @@ sweep3d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
         const long long base = blk * g.block_stride + g.origin + (long long)y * PX + x;
         const double* ub = u + base;
         const double* fb = HAS_F ? f + base : nullptr;
-        double* ob = (OP == OP_RESIDUAL) ? nullptr : un + base;
+        double* ob = op_stores(OP) ? un + base : nullptr;
 
         long long off_w = -1, off_e = NV, off_s = -PX, off_n = PX;   // within the plane
         long long off_d0 = -PXY, off_u1 = PXY;                        // below plane 0 / above plane bz-1
-        if (OP == OP_UPDATE_PULL) {
+        if (op_pulls(OP)) {
             const int bxi = (int)(blk % g.gx);
             const int byi = (int)((blk / g.gx) % g.gy);
             const int bzi = (int)(blk / ((long long)g.gx * g.gy));
@@ -189,7 +193,7 @@ sweep3d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
 #pragma unroll 2
         for (int k = k0; k < k1; ++k) {
             const long long po = (long long)k * PXY;
-            const Vec<NV> U = load_vec<NV>(ub + po + ((OP == OP_UPDATE_PULL && k + 1 == g.bz) ? off_u1 : PXY));
+            const Vec<NV> U = load_vec<NV>(ub + po + ((op_pulls(OP) && k + 1 == g.bz) ? off_u1 : PXY));
             const Vec<NV> S = load_vec<NV>(ub + po + off_s);
             const Vec<NV> N = load_vec<NV>(ub + po + off_n);
             const double w = ub[po + off_w];
@@ -204,19 +208,18 @@ sweep3d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
                 double s = add_rn(add_rn(W, E), add_rn(S.v[q], N.v[q]));
                 s = add_rn(s, add_rn(D.v[q], U.v[q]));
                 if (HAS_F) s = add_rn(s, ff.v[q]);
-                if (OP == OP_RESIDUAL) {
+                if (op_sums(OP)) {
                     const double r = sub_rn(s, mul_rn(6.0, Cc.v[q]));
                     acc = add_rn(acc, mul_rn(r, r));
-                } else {
-                    o.v[q] = mul_rn(s, c6);
                 }
+                if (op_stores(OP)) o.v[q] = mul_rn(s, c6);
             }
-            if (OP != OP_RESIDUAL) store_vec<NV>(ob + po, o);
+            if (op_stores(OP)) store_vec<NV>(ob + po, o);
             D = Cc;
             Cc = U;
         }
     }
-    if (OP == OP_RESIDUAL) {
+    if (op_sums(OP)) {
         const double total = block_sum(acc);
         if (threadIdx.x == 0 && threadIdx.y == 0) partials[blockIdx.x] = total;
     }
@@ -528,9 +531,9 @@ __host__ __device__ constexpr int slot3(int ph, int d) { return (((ph + d) % 3) 
 // one row.  EDGE = false is for steps in which no row and no column involved lies outside the
 // domain: no Dirichlet fix-up is compiled in.
 // level s of one step: row r - 2s + 1 from the window of level s - 1
-template <int T, bool HAS_F, int PH, bool EDGE, int s>
+template <int T, bool HAS_F, bool RES, int PH, bool EDGE, int s>
 __device__ __forceinline__ void temporal_level(Row4 (&win)[T][3], const TemporalCtx& c, const JacGeom& g,
-                                               int r, const RowCursor& out_cur)
+                                               int r, const RowCursor& out_cur, double& acc)
 {
     constexpr bool F_RING = temporal_f_ring(T, HAS_F);
     constexpr int d = -2 * s + 1;              // level s produces row r + d
@@ -559,7 +562,7 @@ __device__ __forceinline__ void temporal_level(Row4 (&win)[T][3], const Temporal
             ff = fill_row4(0.0);
         }
     }
-    Row4 o;
+    Row4 o, res;
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
         const double W = (q == 0) ? w : M.v[q - 1];
@@ -567,6 +570,8 @@ __device__ __forceinline__ void temporal_level(Row4 (&win)[T][3], const Temporal
         double sum = add_rn(add_rn(W, E), add_rn(S.v[q], N.v[q]));
         if (HAS_F) sum = add_rn(sum, ff.v[q]);
         o.v[q] = mul_rn(sum, 0.25);
+        // residual of the state the top level reads (M is that state at this point)
+        if (RES && s == T) res.v[q] = sub_rn(sum, mul_rn(4.0, M.v[q]));
     }
     if (EDGE) {
         if (rs < 0) o = fill_row4(c.c_my);
@@ -577,21 +582,25 @@ __device__ __forceinline__ void temporal_level(Row4 (&win)[T][3], const Temporal
         win[s][slot3(PH, d)] = o;
     } else if (c.store_lane && rs >= c.Y0 && rs < c.Y1) {
         store_row4(c.ob + out_cur.off, o);
+        if (RES) {   // exactly the points this lane stores: every interior point once
+#pragma unroll
+            for (int q = 0; q < 4; ++q) acc = add_rn(acc, mul_rn(res.v[q], res.v[q]));
+        }
     }
 }
 
-template <int T, bool HAS_F, int PH, bool EDGE, int s>
+template <int T, bool HAS_F, bool RES, int PH, bool EDGE, int s>
 struct TemporalLevels {   // levels s, s - 1, ..., 2 (top level first)
     static __device__ __forceinline__ void run(Row4 (&win)[T][3], const TemporalCtx& c, const JacGeom& g, int r,
-                                               const RowCursor& out_cur) {
-        temporal_level<T, HAS_F, PH, EDGE, s>(win, c, g, r, out_cur);
-        TemporalLevels<T, HAS_F, PH, EDGE, s - 1>::run(win, c, g, r, out_cur);
+                                               const RowCursor& out_cur, double& acc) {
+        temporal_level<T, HAS_F, RES, PH, EDGE, s>(win, c, g, r, out_cur, acc);
+        TemporalLevels<T, HAS_F, RES, PH, EDGE, s - 1>::run(win, c, g, r, out_cur, acc);
     }
 };
-template <int T, bool HAS_F, int PH, bool EDGE>
-struct TemporalLevels<T, HAS_F, PH, EDGE, 1> {
+template <int T, bool HAS_F, bool RES, int PH, bool EDGE>
+struct TemporalLevels<T, HAS_F, RES, PH, EDGE, 1> {
     static __device__ __forceinline__ void run(Row4 (&)[T][3], const TemporalCtx&, const JacGeom&, int,
-                                               const RowCursor&) {}
+                                               const RowCursor&, double&) {}
 };
 
 // One pipeline step: input row r arrives (phase PH = (r - r0) mod 3) and every level advances
@@ -599,19 +608,19 @@ struct TemporalLevels<T, HAS_F, PH, EDGE, 1> {
 // the wait for the copy of row r; then the row is taken, its ring stage refilled, and level 1
 // runs.  EDGE = false is for steps in which no row and no column involved lies outside the
 // domain: no Dirichlet fix-up is compiled in.
-template <int T, bool HAS_F, int PH, bool EDGE>
+template <int T, bool HAS_F, bool RES, int PH, bool EDGE>
 __device__ __forceinline__ void temporal_step(Row4 (&win)[T][3], const TemporalCtx& c, const JacGeom& g,
-                                              int r, RowCursor& load_cur, RowCursor& out_cur)
+                                              int r, RowCursor& load_cur, RowCursor& out_cur, double& acc)
 {
     constexpr bool F_RING = temporal_f_ring(T, HAS_F);
-    TemporalLevels<T, HAS_F, PH, EDGE, T>::run(win, c, g, r, out_cur);
+    TemporalLevels<T, HAS_F, RES, PH, EDGE, T>::run(win, c, g, r, out_cur, acc);
     cp_async_wait<kTemporalDepth - 1>();
     __syncwarp();                                    // the other lanes' chunks of row r have landed too
     win[0][PH] = take_row<EDGE>(c, r);
     __syncwarp();                                    // everyone has read the stage before it is refilled
     issue_row<HAS_F, F_RING>(c, r + kTemporalDepth, load_cur);
     load_cur.advance(g, c.brs);
-    temporal_level<T, HAS_F, PH, EDGE, 1>(win, c, g, r, out_cur);
+    temporal_level<T, HAS_F, RES, PH, EDGE, 1>(win, c, g, r, out_cur, acc);
     out_cur.advance(g, c.brs);
 }
 
@@ -621,20 +630,23 @@ __device__ __forceinline__ long long column_base(const JacGeom& g, long long gx)
     return bxi * g.block_stride + g.origin + (gx - bxi * g.bx);
 }
 
-template <int T, bool HAS_F, int PH>
+template <int T, bool HAS_F, bool RES, int PH>
 __device__ __forceinline__ void temporal_step_any(Row4 (&win)[T][3], const TemporalCtx& c, const JacGeom& g,
-                                                  int r, RowCursor& load_cur, RowCursor& out_cur)
+                                                  int r, RowCursor& load_cur, RowCursor& out_cur, double& acc)
 {
     // warp-uniform: does this step see a row outside [0, ny) or a column outside [0, nx)?
     const bool edge = c.edge_x || (r - 2 * T < 0) || (r >= c.ny);
-    if (edge) temporal_step<T, HAS_F, PH, true>(win, c, g, r, load_cur, out_cur);
-    else temporal_step<T, HAS_F, PH, false>(win, c, g, r, load_cur, out_cur);
+    if (edge) temporal_step<T, HAS_F, RES, PH, true>(win, c, g, r, load_cur, out_cur, acc);
+    else temporal_step<T, HAS_F, RES, PH, false>(win, c, g, r, load_cur, out_cur, acc);
 }
 
-template <int T, bool HAS_F>
+// RES: the top level also accumulates the squared residual of the state it reads (the state
+// before the last sweep of the launch); every warp writes its partial sum to partials[warp id].
+template <int T, bool HAS_F, bool RES>
 __global__ void __launch_bounds__(kTemporalWarps * 32, ((T > 4 || temporal_f_ring(T, HAS_F)) ? 2 : JAC_TOCC))
 temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const double* __restrict__ f,
-                  const JacGeom g, const int strips_x, const int strips_y, const int rows_per_strip)
+                  double* __restrict__ partials, const JacGeom g, const int strips_x, const int strips_y,
+                  const int rows_per_strip)
 {
     extern __shared__ __align__(16) double2 t2_ring_mem[];   // [warp][u stages, then f stages][64]
     constexpr bool F_RING = temporal_f_ring(T, HAS_F);
@@ -691,12 +703,18 @@ temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
         load_cur.advance(g, c.brs);
     }
 
+    double acc = 0.0;
     for (int r = c.r0; r < r_end; r += 3) {
-        temporal_step_any<T, HAS_F, 0>(win, c, g, r, load_cur, out_cur);
-        if (r + 1 < r_end) temporal_step_any<T, HAS_F, 1>(win, c, g, r + 1, load_cur, out_cur);
-        if (r + 2 < r_end) temporal_step_any<T, HAS_F, 2>(win, c, g, r + 2, load_cur, out_cur);
+        temporal_step_any<T, HAS_F, RES, 0>(win, c, g, r, load_cur, out_cur, acc);
+        if (r + 1 < r_end) temporal_step_any<T, HAS_F, RES, 1>(win, c, g, r + 1, load_cur, out_cur, acc);
+        if (r + 2 < r_end) temporal_step_any<T, HAS_F, RES, 2>(win, c, g, r + 2, load_cur, out_cur, acc);
     }
     cp_async_wait<0>();
+    if (RES) {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) acc = add_rn(acc, __shfl_down_sync(0xffffffffu, acc, off));
+        if (lane == 0) partials[wid] = acc;
+    }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -810,11 +828,12 @@ __device__ __forceinline__ bool t3_outside(const T3Ctx& c, int plane, bool row_l
 }
 
 // one level: plane `q` of the level from the window (D, M, U) of the level below
-template <bool HAS_F, bool EDGE>
+// RES: rows whose bit is set in res_rows also add the squared residual of M (s - 6 M) to acc
+template <bool HAS_F, bool EDGE, bool RES>
 __device__ __forceinline__ void t3_level(const T3Ctx& c, const Plane6& D, const Plane6& M, const Plane6& U,
                                          const Row2& below, const Row2& above, int q,
                                          const double* fplane /* ring stage of f plane q, this warp's rows */,
-                                         Plane6& out)
+                                         Plane6& out, unsigned res_rows, double& acc)
 {
     const double c6 = 1.0 / 6.0;
 #pragma unroll
@@ -836,15 +855,19 @@ __device__ __forceinline__ void t3_level(const T3Ctx& c, const Plane6& D, const 
             s = add_rn(s, add_rn(D.row[r].v[i], U.row[r].v[i]));
             if (HAS_F) s = add_rn(s, ff.v[i]);
             out.row[r].v[i] = mul_rn(s, c6);
+            if (RES && ((res_rows >> r) & 1u)) {
+                const double rr = sub_rn(s, mul_rn(6.0, M.row[r].v[i]));
+                acc = add_rn(acc, mul_rn(rr, rr));
+            }
         }
         if (EDGE && outside) out.row[r] = fill_row2(cval);
     }
 }
 
-template <int T, bool HAS_F, int PH, bool EDGE>
+template <int T, bool HAS_F, bool RES, int PH, bool EDGE>
 __device__ __forceinline__ void t3_step(Plane6 (&L0)[3], Plane6 (&L1)[3], const T3Ctx& c, const JacGeom& g,
                                         int p, PlaneCursor& load_cur, PlaneCursor& fload_cur,
-                                        PlaneCursor& l1_cur, PlaneCursor& l2_cur)
+                                        PlaneCursor& l1_cur, PlaneCursor& l2_cur, double& acc)
 {
     constexpr int NST = k3d_stages(HAS_F);
     constexpr int LEAD = NST - 2;          // u planes issued ahead of the one being consumed
@@ -859,9 +882,11 @@ __device__ __forceinline__ void t3_step(Plane6 (&L0)[3], Plane6 (&L1)[3], const 
         Row2 below = lds_row2(ex + (wlo * 2 + 1) * 64);   // last row of the warp below
         Row2 above = lds_row2(ex + (whi * 2 + 0) * 64);   // first row of the warp above
         Plane6 o;
-        t3_level<HAS_F, EDGE>(c, L1[slot3(PH, -4)], L1[slot3(PH, -3)], L1[slot3(PH, -2)], below, above, q,
-                              HAS_F ? fmine + ((q - c.p0 + 2 * k3dFStages) % k3dFStages) * k3dPlaneElems : nullptr, o);
-        if (c.store_lane && q >= c.Z0 && q < c.Z1) {
+        const bool live = c.store_lane && q >= c.Z0 && q < c.Z1;   // the points this lane stores
+        t3_level<HAS_F, EDGE, RES>(c, L1[slot3(PH, -4)], L1[slot3(PH, -3)], L1[slot3(PH, -2)], below, above, q,
+                                   HAS_F ? fmine + ((q - c.p0 + 2 * k3dFStages) % k3dFStages) * k3dPlaneElems : nullptr,
+                                   o, live ? c.row_store : 0u, acc);
+        if (live) {
 #pragma unroll
             for (int r = 0; r < k3dRows; ++r)
                 if ((c.row_store >> r) & 1u)
@@ -902,8 +927,10 @@ __device__ __forceinline__ void t3_step(Plane6 (&L0)[3], Plane6 (&L1)[3], const 
         else above = lds_row2(st + min(c.warp * k3dRows + k3dRows, k3dTileRows - 1) * 64);
         if (T == 1) {
             Plane6 o;
-            t3_level<HAS_F, EDGE>(c, L0[slot3(PH, -2)], L0[slot3(PH, -1)], L0[PH], below, above, q, f1, o);
-            if (c.store_lane && q >= c.Z0 && q < c.Z1) {
+            const bool live = c.store_lane && q >= c.Z0 && q < c.Z1;
+            t3_level<HAS_F, EDGE, RES>(c, L0[slot3(PH, -2)], L0[slot3(PH, -1)], L0[PH], below, above, q, f1, o,
+                                       live ? c.row_store : 0u, acc);
+            if (live) {
 #pragma unroll
                 for (int r = 0; r < k3dRows; ++r)
                     if ((c.row_store >> r) & 1u)
@@ -911,7 +938,8 @@ __device__ __forceinline__ void t3_step(Plane6 (&L0)[3], Plane6 (&L1)[3], const 
             }
         } else {
             Plane6& o = L1[slot3(PH, -1)];
-            t3_level<HAS_F, EDGE>(c, L0[slot3(PH, -2)], L0[slot3(PH, -1)], L0[PH], below, above, q, f1, o);
+            t3_level<HAS_F, EDGE, false>(c, L0[slot3(PH, -2)], L0[slot3(PH, -1)], L0[PH], below, above, q, f1, o,
+                                         0u, acc);
             double* ex = c.exch + PH * (k3dWarps * 2 * 64) + (c.warp * 2) * 64 + 2 * c.lane;
             *reinterpret_cast<double2*>(ex) = make_double2(o.row[0].v[0], o.row[0].v[1]);
             *reinterpret_cast<double2*>(ex + 64) = make_double2(o.row[k3dRows - 1].v[0], o.row[k3dRows - 1].v[1]);
@@ -921,10 +949,13 @@ __device__ __forceinline__ void t3_step(Plane6 (&L0)[3], Plane6 (&L1)[3], const 
     __syncthreads();
 }
 
-template <int T, bool HAS_F>
+// RES as for the 2D kernel: partials[CTA * 8 + warp] gets the warp's sum of squared residuals of
+// the state before the last sweep of the launch.
+template <int T, bool HAS_F, bool RES>
 __global__ void __launch_bounds__(k3dWarps * 32, 1)
 temporal3d_kernel(const double* __restrict__ u, double* __restrict__ un, const double* __restrict__ f,
-                  const JacGeom g, const int tiles_x, const int tiles_y, const int tiles_z, const int zchunk)
+                  double* __restrict__ partials, const JacGeom g, const int tiles_x, const int tiles_y,
+                  const int tiles_z, const int zchunk)
 {
     extern __shared__ __align__(16) double t3_smem[];
     T3Ctx c;
@@ -1007,10 +1038,11 @@ temporal3d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
 #define JAC_T3_STEP(PHASE, PL)                                                                   \
     do {                                                                                         \
         const bool edge = edge_xy || ((PL) - 2 * T - 1 < 0) || ((PL) >= c.nz);                   \
-        if (edge) t3_step<T, HAS_F, PHASE, true>(L0, L1, c, g, (PL), load_cur, fload_cur, l1_cur, l2_cur);  \
-        else t3_step<T, HAS_F, PHASE, false>(L0, L1, c, g, (PL), load_cur, fload_cur, l1_cur, l2_cur);      \
+        if (edge) t3_step<T, HAS_F, RES, PHASE, true>(L0, L1, c, g, (PL), load_cur, fload_cur, l1_cur, l2_cur, acc);  \
+        else t3_step<T, HAS_F, RES, PHASE, false>(L0, L1, c, g, (PL), load_cur, fload_cur, l1_cur, l2_cur, acc);      \
     } while (0)
 
+    double acc = 0.0;
     for (int p = c.p0; p < p_end; p += 3) {
         JAC_T3_STEP(0, p);
         if (p + 1 < p_end) JAC_T3_STEP(1, p + 1);
@@ -1018,6 +1050,11 @@ temporal3d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
     }
 #undef JAC_T3_STEP
     cp_async_wait<0>();
+    if (RES) {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) acc = add_rn(acc, __shfl_down_sync(0xffffffffu, acc, off));
+        if (c.lane == 0) partials[(long long)blockIdx.x * k3dWarps + c.warp] = acc;
+    }
 }
 
 }  // namespace jac

@@ -33,6 +33,7 @@ EXPORTS = [
     "jac_get_u_device", "jac_set_boundary", "jac_get_block_padded", "jac_get_halo_buffer",
     "jac_pack_halos", "jac_unpack_halos", "jac_pack_faces", "jac_unpack_faces", "jac_sweep", "jac_residual", "jac_launch_count",
     "jac_last_cuda_error", "jac_strerror", "jac_residual_dense_static", "jac_sweeps_per_launch",
+    "jac_sweep_residual", "jac_solve",
 ]
 
 
@@ -84,6 +85,8 @@ def lib() -> C.CDLL:
         L.jac_unpack_faces.argtypes = [vp, C.c_uint]
         L.jac_sweep.argtypes = [vp, C.c_int]
         L.jac_residual.argtypes = [vp, dp]
+        L.jac_sweep_residual.argtypes = [vp, C.c_int, dp]
+        L.jac_solve.argtypes = [vp, C.c_int, C.c_int, C.c_double, C.POINTER(C.c_int), dp]
         L.jac_launch_count.argtypes = [vp, C.POINTER(C.c_int64)]
         L.jac_sweeps_per_launch.argtypes = [vp, C.POINTER(C.c_int)]
         L.jac_last_cuda_error.argtypes = [vp]
@@ -301,6 +304,19 @@ class Jacobi:
 
     def sweep(self, nsweeps: int = 1):
         self._call("jac_sweep", lib().jac_sweep(self._ctx, int(nsweeps)))
+
+    def sweep_residual(self, nsweeps: int) -> float:
+        """nsweeps sweeps; returns the residual norm of the state before the last of them."""
+        out = C.c_double(0.0)
+        self._call("jac_sweep_residual", lib().jac_sweep_residual(self._ctx, int(nsweeps), C.byref(out)))
+        return out.value
+
+    def solve(self, max_sweeps: int, check_every: int, tol: float):
+        """Sweeps until the lagged residual norm is <= tol; returns (sweeps done, last norm)."""
+        done, res = C.c_int(0), C.c_double(0.0)
+        self._call("jac_solve", lib().jac_solve(self._ctx, int(max_sweeps), int(check_every), float(tol),
+                                                C.byref(done), C.byref(res)))
+        return done.value, res.value
 
     def residual(self) -> float:
         out = C.c_double(0.0)

@@ -289,3 +289,56 @@ def test_sweeps_per_launch_query(jac):
     for kw, want in cases:
         with jac.Jacobi(**kw) as J:
             assert J.sweeps_per_launch() == want, kw
+
+
+FUSED_RESIDUAL_CASES = [((36, 24), (12, 8), 1), ((256, 100), (64, 25), 1), ((1100, 200), (220, 50), 2),
+                        ((24, 18, 12), (8, 6, 4), 1), ((130, 100, 36), (130, 50, 18), 1),
+                        ((64, 48, 40), (32, 24, 20), 2)]
+
+
+@pytest.mark.parametrize("n,b,h", FUSED_RESIDUAL_CASES)
+@pytest.mark.parametrize("mode", ["fused", "exchange", "pertask", "temporal"])
+@pytest.mark.parametrize("has_f", [False, True])
+def test_sweep_with_fused_residual(jac, orc, n, b, h, mode, has_f):
+    """jac_sweep_residual(k): state after k sweeps, norm of the residual of the state after k - 1."""
+    J, B = _setup_pair(jac, orc, n, b, h, has_f, mode, seed=6)
+    for k in (1, 3, 6):
+        B.sweep(k - 1)
+        want_r = B.residual()
+        B.sweep(1)
+        got_r = J.sweep_residual(k)
+        assert abs(got_r - want_r) <= RESID_TOL * want_r, (k, got_r, want_r)
+        _assert_sweep_close(J.get_u(), B.get_u())
+    # an ordinary residual afterwards still works and agrees
+    assert abs(J.residual() - B.residual()) <= RESID_TOL * B.residual()
+    J.close()
+    B.close()
+
+
+def test_solve_stops_at_the_tolerance(jac, orc):
+    n, b = (48, 40), (24, 20)
+    u0, f = _random_problem(n, 9)
+    for mode in ("temporal", "fused"):
+        J = jac.Jacobi(n, b, 1, True, mode)
+        J.set_u(u0)
+        J.set_f(f)
+        r0 = J.residual()
+        done, res = J.solve(100000, 50, 1e-6 * r0)
+        assert res <= 1e-6 * r0 and done % 50 == 0 and 50 <= done < 100000
+        # the oracle at the same sweep count: the reported norm is that of the state one sweep earlier
+        B = orc.Blocked(n, b, 1, True)
+        B.set_u(u0)
+        B.set_f(f)
+        B.sweep(done - 1)
+        want = B.residual()
+        B.sweep(1)
+        assert abs(res - want) <= RESID_TOL * want
+        assert np.array_equal(J.get_u(), B.get_u())
+        # a cap below convergence is honoured
+        J.set_u(u0)
+        done2, res2 = J.solve(30, 8, 0.0)
+        assert done2 == 30 and res2 > 0.0
+        with pytest.raises(jac.JacError):
+            J.solve(0, 8, 1.0)
+        J.close()
+        B.close()
