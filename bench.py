@@ -48,14 +48,14 @@ L2_BYTES = 126e6
 # part of the grid once per launch.
 NCU_TRAFFIC = {
     # profiles/temporal2d_eigenmode_8192.md
-    ("temporal", 8, 2, False): {"bytes_per_point_per_launch": (625.100032e6 + 490.793728e6) / 8192 ** 2,
-                                "src_sha": "a067f0d0087e06c8"},
+    ("temporal", 8, 2, False): {"bytes_per_point_per_launch": (625.295616e6 + 491.547136e6) / 8192 ** 2,
+                                "src_sha": "eeb19b9bd151abe8"},
     # profiles/temporal3d_poisson_512.md
-    ("temporal", 2, 3, True): {"bytes_per_point_per_launch": (2.497591e9 + 1.047600e9) / 512 ** 3,
-                               "src_sha": "a067f0d0087e06c8"},
+    ("temporal", 2, 3, True): {"bytes_per_point_per_launch": (2.496113e9 + 1.047960e9) / 512 ** 3,
+                               "src_sha": "eeb19b9bd151abe8"},
     # profiles/exchange_schedule_eigenmode_8192.md (the update launch alone)
-    ("exchange", 1, 2, False): {"bytes_per_point_per_launch": (574.281984e6 + 494.291200e6) / 8192 ** 2,
-                                "src_sha": "a067f0d0087e06c8"},
+    ("exchange", 1, 2, False): {"bytes_per_point_per_launch": (574.288384e6 + 494.364160e6) / 8192 ** 2,
+                                "src_sha": "eeb19b9bd151abe8"},
 }
 KERNEL_NAMES = {("temporal", 2): "temporal2d_kernel", ("temporal", 3): "temporal3d_kernel", ("fused", 2): "sweep2d_kernel (update pulling neighbour interiors)",
                 ("exchange", 2): "sweep2d_kernel", ("pertask", 2): "sweep2d_kernel (one launch per block)",
