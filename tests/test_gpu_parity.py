@@ -17,10 +17,11 @@ BVALS = [0.5, -1.0, 2.0, 3.0, -0.25, 1.5]
 # CTA tile (x tiles), more rows than one strip (y tiles), halo 1..4
 SHAPES_2D = [((12, 8), (12, 8), 1), ((12, 8), (4, 4), 1), ((12, 8), (1, 1), 1), ((15, 9), (5, 3), 1),
              ((15, 9), (5, 3), 3), ((64, 48), (16, 8), 4), ((640, 72), (640, 72), 1),
-             ((1100, 200), (550, 100), 2), ((130, 210), (130, 70), 1), ((36, 24), (12, 8), 2)]
+             ((1100, 200), (550, 100), 2), ((130, 210), (130, 70), 1), ((36, 24), (12, 8), 2),
+             ((32, 24), (16, 8), 8), ((30, 21), (10, 7), 7)]
 SHAPES_3D = [((6, 4, 8), (3, 2, 4), 1), ((6, 4, 8), (1, 1, 1), 1), ((6, 4, 8), (6, 4, 8), 2),
              ((20, 12, 40), (10, 12, 20), 1), ((132, 20, 36), (132, 10, 18), 1),
-             ((24, 18, 12), (8, 6, 4), 3), ((48, 40, 20), (24, 20, 10), 2)]
+             ((24, 18, 12), (8, 6, 4), 3), ((48, 40, 20), (24, 20, 10), 2), ((16, 16, 16), (8, 8, 8), 8)]
 MODES = ["fused", "exchange", "pertask"]
 
 

@@ -9,13 +9,13 @@ from paper_2210_01238_b200 import inputs
 EPS = np.finfo(np.float64).eps
 
 SHAPES_2D = [((12, 8), (12, 8)), ((12, 8), (4, 4)), ((12, 8), (1, 1)), ((12, 8), (3, 2)),
-             ((12, 8), (12, 1)), ((12, 8), (1, 8)), ((12, 8), (6, 4))]
+             ((12, 8), (12, 1)), ((12, 8), (1, 8)), ((12, 8), (6, 4)), ((32, 24), (16, 8))]
 SHAPES_3D = [((6, 4, 8), (3, 2, 4)), ((6, 4, 8), (1, 1, 1)), ((6, 4, 8), (6, 4, 8)),
              ((6, 4, 8), (2, 4, 2)), ((6, 4, 8), (6, 1, 4))]
 
 
 def _halos(b):
-    return [h for h in (1, 2, 3, 4) if h <= min(b)]
+    return [h for h in (1, 2, 3, 4, 8) if h <= min(b)]
 
 
 def _block_box(B, blk):
