@@ -404,6 +404,11 @@ dense_copy_kernel(double* __restrict__ blocks, double* __restrict__ dense, const
 #ifndef JAC_TOCC
 #define JAC_TOCC 3    // CTAs per SM the register allocation aims for
 #endif
+// points per lane for T > 4.  2 was measured: 12 warps per SM instead of 8, but 1364 against
+// 1702 GLUP/s at T = 8 (more halo lanes and more shuffles per point).
+#ifndef JAC_TP_DEEP
+#define JAC_TP_DEEP 4
+#endif
 constexpr int kTemporalWarps = JAC_TW;
 constexpr int kTemporalDepth = JAC_TD;
 // Right-hand side rows of the 2D temporal kernel: up to T = 4 they travel through a second
@@ -414,12 +419,21 @@ __host__ __device__ constexpr bool temporal_f_ring(int T, bool has_f) { return h
 __host__ __device__ constexpr int temporal_stages_per_warp(int T, bool has_f) {
     return kTemporalDepth + (temporal_f_ring(T, has_f) ? kTemporalFDepth : 0);
 }
+// A lane holds P consecutive points (4; the code also runs with 2, which halves the window
+// registers of deep pipelines but was measured slower).  A ring stage is one row of the strip: 16 P chunks of 16 bytes.
+__host__ __device__ constexpr int temporal_points(int T) { return T > 4 ? JAC_TP_DEEP : 4; }
+__host__ __device__ constexpr int temporal_stage_chunks(int P) { return 16 * P; }
 __host__ __device__ constexpr size_t temporal_smem_bytes(int T, bool has_f) {
-    return (size_t)kTemporalWarps * temporal_stages_per_warp(T, has_f) * 64 * sizeof(double2);
+    return (size_t)kTemporalWarps * temporal_stages_per_warp(T, has_f) *
+           temporal_stage_chunks(temporal_points(T)) * sizeof(double2);
 }
-// lanes at each end of a warp whose points are no longer exact after T levels (4 points per lane)
-__host__ __device__ constexpr int temporal_halo_lanes(int T) { return (T + 3) / 4; }
-__host__ __device__ constexpr int temporal_strip_cols(int T) { return 128 - 8 * temporal_halo_lanes(T); }
+// lanes at each end of a warp whose points are no longer exact after T levels
+__host__ __device__ constexpr int temporal_halo_lanes(int T) {
+    return (T + temporal_points(T) - 1) / temporal_points(T);
+}
+__host__ __device__ constexpr int temporal_strip_cols(int T) {
+    return (32 - 2 * temporal_halo_lanes(T)) * temporal_points(T);
+}
 
 struct RowCursor {
     long long off;  // element offset of the row within the array, relative to a lane's column base
@@ -439,18 +453,28 @@ struct RowCursor {
     }
 };
 
-struct Row4 { double v[4]; };
+template <int P> struct RowN { double v[P]; };
 
-__device__ __forceinline__ Row4 load_row4(const double* p) {
-    const double2 a = *reinterpret_cast<const double2*>(p);
-    const double2 b = *reinterpret_cast<const double2*>(p + 2);
-    Row4 r; r.v[0] = a.x; r.v[1] = a.y; r.v[2] = b.x; r.v[3] = b.y; return r;
+// P consecutive doubles as P/2 128-bit accesses (global or shared memory)
+template <int P> __device__ __forceinline__ RowN<P> load_rown(const double* p) {
+    RowN<P> r;
+#pragma unroll
+    for (int k = 0; k < P / 2; ++k) {
+        const double2 a = reinterpret_cast<const double2*>(p)[k];
+        r.v[2 * k] = a.x; r.v[2 * k + 1] = a.y;
+    }
+    return r;
 }
-__device__ __forceinline__ void store_row4(double* p, const Row4& r) {
-    *reinterpret_cast<double2*>(p) = make_double2(r.v[0], r.v[1]);
-    *reinterpret_cast<double2*>(p + 2) = make_double2(r.v[2], r.v[3]);
+template <int P> __device__ __forceinline__ void store_rown(double* p, const RowN<P>& r) {
+#pragma unroll
+    for (int k = 0; k < P / 2; ++k) reinterpret_cast<double2*>(p)[k] = make_double2(r.v[2 * k], r.v[2 * k + 1]);
 }
-__device__ __forceinline__ Row4 fill_row4(double c) { Row4 r; r.v[0] = r.v[1] = r.v[2] = r.v[3] = c; return r; }
+template <int P> __device__ __forceinline__ RowN<P> fill_rown(double c) {
+    RowN<P> r;
+#pragma unroll
+    for (int k = 0; k < P; ++k) r.v[k] = c;
+    return r;
+}
 
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
     const unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
@@ -494,16 +518,17 @@ struct TemporalCtx {
 // start the copy of input row r into its ring stage (nothing to copy outside the domain).  With a
 // right-hand side, f row r goes into the f ring (F_RING: stages follow the u stages of the warp),
 // or is at least requested into L2 for the loads that follow DEPTH steps later.
-template <bool HAS_F, bool F_RING>
+template <int P, bool HAS_F, bool F_RING>
 __device__ __forceinline__ void issue_row(const TemporalCtx& c, int r, const RowCursor& cur) {
+    constexpr int SC = temporal_stage_chunks(P);
     if (r >= 0 && r < c.ny && r < c.in_end) {
-        const int st = ((r - c.r0) % kTemporalDepth) * 64;
+        const int st = ((r - c.r0) % kTemporalDepth) * SC;
         if (c.copy_a) cp_async16(c.dst_a + st, c.src_a + cur.off);
-        if (c.copy_b) cp_async16(c.dst_b + st, c.src_b + cur.off);
+        if (P == 4 && c.copy_b) cp_async16(c.dst_b + st, c.src_b + cur.off);
         if (F_RING) {
-            const int fs = (kTemporalDepth + ((r - c.r0) % kTemporalFDepth)) * 64;
+            const int fs = (kTemporalDepth + ((r - c.r0) % kTemporalFDepth)) * SC;
             if (c.copy_a) cp_async16(c.dst_a + fs, c.src_a + c.fdelta + cur.off);
-            if (c.copy_b) cp_async16(c.dst_b + fs, c.src_b + c.fdelta + cur.off);
+            if (P == 4 && c.copy_b) cp_async16(c.dst_b + fs, c.src_b + c.fdelta + cur.off);
         } else if (HAS_F && !c.xout) {
             prefetch_line(c.fb + cur.off);
         }
@@ -512,17 +537,15 @@ __device__ __forceinline__ void issue_row(const TemporalCtx& c, int r, const Row
 }
 
 // input row r for this lane once its copy has landed
-template <bool EDGE>
-__device__ __forceinline__ Row4 take_row(const TemporalCtx& c, int r) {
+template <int P, bool EDGE>
+__device__ __forceinline__ RowN<P> take_row(const TemporalCtx& c, int r) {
     if (EDGE) {   // Dirichlet value outside the domain
-        if (r < 0) return fill_row4(c.xout ? c.cx : c.c_my);
-        if (r >= c.ny) return fill_row4(c.xout ? c.cx : c.c_py);
-        if (c.xout) return fill_row4(c.cx);
+        if (r < 0) return fill_rown<P>(c.xout ? c.cx : c.c_my);
+        if (r >= c.ny) return fill_rown<P>(c.xout ? c.cx : c.c_py);
+        if (c.xout) return fill_rown<P>(c.cx);
     }
-    const double2* st = c.mine + ((r - c.r0) % kTemporalDepth) * 64;
-    const double2 a = st[0], b = st[1];
-    Row4 o; o.v[0] = a.x; o.v[1] = a.y; o.v[2] = b.x; o.v[3] = b.y;
-    return o;
+    const double2* st = c.mine + ((r - c.r0) % kTemporalDepth) * temporal_stage_chunks(P);
+    return load_rown<P>(reinterpret_cast<const double*>(st));
 }
 
 __host__ __device__ constexpr int slot3(int ph, int d) { return (((ph + d) % 3) + 3) % 3; }
@@ -532,41 +555,43 @@ __host__ __device__ constexpr int slot3(int ph, int d) { return (((ph + d) % 3) 
 // domain: no Dirichlet fix-up is compiled in.
 // level s of one step: row r - 2s + 1 from the window of level s - 1
 template <int T, bool HAS_F, bool RES, int PH, bool EDGE, int s>
-__device__ __forceinline__ void temporal_level(Row4 (&win)[T][3], const TemporalCtx& c, const JacGeom& g,
-                                               int r, const RowCursor& out_cur, double& acc)
+__device__ __forceinline__ void temporal_level(RowN<temporal_points(T)> (&win)[T][3], const TemporalCtx& c,
+                                               const JacGeom& g, int r, const RowCursor& out_cur, double& acc)
 {
+    constexpr int P = temporal_points(T);
+    using Row = RowN<P>;
     constexpr bool F_RING = temporal_f_ring(T, HAS_F);
     constexpr int d = -2 * s + 1;              // level s produces row r + d
     const int rs = r + d;
-    const Row4& S = win[s - 1][slot3(PH, d - 1)];
-    const Row4& M = win[s - 1][slot3(PH, d)];
-    const Row4& N = win[s - 1][slot3(PH, d + 1)];
-    const double w = __shfl_up_sync(0xffffffffu, M.v[3], 1);
+    const Row& S = win[s - 1][slot3(PH, d - 1)];
+    const Row& M = win[s - 1][slot3(PH, d)];
+    const Row& N = win[s - 1][slot3(PH, d + 1)];
+    const double w = __shfl_up_sync(0xffffffffu, M.v[P - 1], 1);
     const double e = __shfl_down_sync(0xffffffffu, M.v[0], 1);
-    Row4 ff;
+    Row ff;
     if (HAS_F) {
         const bool ok = EDGE ? (rs >= 0 && rs < c.ny && !c.xout) : true;
         if (ok && F_RING) {
             // copied DEPTH + 2s - 1 steps ago; the warp-wide barriers of the steps in between
             // made the other lanes' chunks visible
-            const double2* fr = c.mine + (kTemporalDepth + ((rs - c.r0) & (kTemporalFDepth - 1))) * 64;
-            const double2 a = fr[0], b = fr[1];
-            ff.v[0] = a.x; ff.v[1] = a.y; ff.v[2] = b.x; ff.v[3] = b.y;
+            const double2* fr = c.mine + (kTemporalDepth + ((rs - c.r0) & (kTemporalFDepth - 1))) *
+                                             temporal_stage_chunks(P);
+            ff = load_rown<P>(reinterpret_cast<const double*>(fr));
         } else if (ok) {
             // f of row rs: the output cursor points at row r - 2T + 1, i.e. (T - s) * 2 rows below rs
             RowCursor fc = out_cur;
 #pragma unroll
             for (int k = 0; k < 2 * (T - s); ++k) fc.advance(g, c.brs);
-            ff = load_row4(c.fb + fc.off);
+            ff = load_rown<P>(c.fb + fc.off);
         } else {
-            ff = fill_row4(0.0);
+            ff = fill_rown<P>(0.0);
         }
     }
-    Row4 o, res;
+    Row o, res;
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
+    for (int q = 0; q < P; ++q) {
         const double W = (q == 0) ? w : M.v[q - 1];
-        const double E = (q == 3) ? e : M.v[q + 1];
+        const double E = (q == P - 1) ? e : M.v[q + 1];
         double sum = add_rn(add_rn(W, E), add_rn(S.v[q], N.v[q]));
         if (HAS_F) sum = add_rn(sum, ff.v[q]);
         o.v[q] = mul_rn(sum, 0.25);
@@ -574,24 +599,24 @@ __device__ __forceinline__ void temporal_level(Row4 (&win)[T][3], const Temporal
         if (RES && s == T) res.v[q] = sub_rn(sum, mul_rn(4.0, M.v[q]));
     }
     if (EDGE) {
-        if (rs < 0) o = fill_row4(c.c_my);
-        if (rs >= c.ny) o = fill_row4(c.c_py);
-        if (c.xout) o = fill_row4(c.cx);
+        if (rs < 0) o = fill_rown<P>(c.c_my);
+        if (rs >= c.ny) o = fill_rown<P>(c.c_py);
+        if (c.xout) o = fill_rown<P>(c.cx);
     }
     if (s < T) {
         win[s][slot3(PH, d)] = o;
     } else if (c.store_lane && rs >= c.Y0 && rs < c.Y1) {
-        store_row4(c.ob + out_cur.off, o);
+        store_rown<P>(c.ob + out_cur.off, o);
         if (RES) {   // exactly the points this lane stores: every interior point once
 #pragma unroll
-            for (int q = 0; q < 4; ++q) acc = add_rn(acc, mul_rn(res.v[q], res.v[q]));
+            for (int q = 0; q < P; ++q) acc = add_rn(acc, mul_rn(res.v[q], res.v[q]));
         }
     }
 }
 
 template <int T, bool HAS_F, bool RES, int PH, bool EDGE, int s>
 struct TemporalLevels {   // levels s, s - 1, ..., 2 (top level first)
-    static __device__ __forceinline__ void run(Row4 (&win)[T][3], const TemporalCtx& c, const JacGeom& g, int r,
+    static __device__ __forceinline__ void run(RowN<temporal_points(T)> (&win)[T][3], const TemporalCtx& c, const JacGeom& g, int r,
                                                const RowCursor& out_cur, double& acc) {
         temporal_level<T, HAS_F, RES, PH, EDGE, s>(win, c, g, r, out_cur, acc);
         TemporalLevels<T, HAS_F, RES, PH, EDGE, s - 1>::run(win, c, g, r, out_cur, acc);
@@ -599,7 +624,7 @@ struct TemporalLevels {   // levels s, s - 1, ..., 2 (top level first)
 };
 template <int T, bool HAS_F, bool RES, int PH, bool EDGE>
 struct TemporalLevels<T, HAS_F, RES, PH, EDGE, 1> {
-    static __device__ __forceinline__ void run(Row4 (&)[T][3], const TemporalCtx&, const JacGeom&, int,
+    static __device__ __forceinline__ void run(RowN<temporal_points(T)> (&)[T][3], const TemporalCtx&, const JacGeom&, int,
                                                const RowCursor&, double&) {}
 };
 
@@ -609,16 +634,16 @@ struct TemporalLevels<T, HAS_F, RES, PH, EDGE, 1> {
 // runs.  EDGE = false is for steps in which no row and no column involved lies outside the
 // domain: no Dirichlet fix-up is compiled in.
 template <int T, bool HAS_F, bool RES, int PH, bool EDGE>
-__device__ __forceinline__ void temporal_step(Row4 (&win)[T][3], const TemporalCtx& c, const JacGeom& g,
+__device__ __forceinline__ void temporal_step(RowN<temporal_points(T)> (&win)[T][3], const TemporalCtx& c, const JacGeom& g,
                                               int r, RowCursor& load_cur, RowCursor& out_cur, double& acc)
 {
     constexpr bool F_RING = temporal_f_ring(T, HAS_F);
     TemporalLevels<T, HAS_F, RES, PH, EDGE, T>::run(win, c, g, r, out_cur, acc);
     cp_async_wait<kTemporalDepth - 1>();
     __syncwarp();                                    // the other lanes' chunks of row r have landed too
-    win[0][PH] = take_row<EDGE>(c, r);
+    win[0][PH] = take_row<temporal_points(T), EDGE>(c, r);
     __syncwarp();                                    // everyone has read the stage before it is refilled
-    issue_row<HAS_F, F_RING>(c, r + kTemporalDepth, load_cur);
+    issue_row<temporal_points(T), HAS_F, F_RING>(c, r + kTemporalDepth, load_cur);
     load_cur.advance(g, c.brs);
     temporal_level<T, HAS_F, RES, PH, EDGE, 1>(win, c, g, r, out_cur, acc);
     out_cur.advance(g, c.brs);
@@ -631,7 +656,7 @@ __device__ __forceinline__ long long column_base(const JacGeom& g, long long gx)
 }
 
 template <int T, bool HAS_F, bool RES, int PH>
-__device__ __forceinline__ void temporal_step_any(Row4 (&win)[T][3], const TemporalCtx& c, const JacGeom& g,
+__device__ __forceinline__ void temporal_step_any(RowN<temporal_points(T)> (&win)[T][3], const TemporalCtx& c, const JacGeom& g,
                                                   int r, RowCursor& load_cur, RowCursor& out_cur, double& acc)
 {
     // warp-uniform: does this step see a row outside [0, ny) or a column outside [0, nx)?
@@ -643,7 +668,8 @@ __device__ __forceinline__ void temporal_step_any(Row4 (&win)[T][3], const Tempo
 // RES: the top level also accumulates the squared residual of the state it reads (the state
 // before the last sweep of the launch); every warp writes its partial sum to partials[warp id].
 template <int T, bool HAS_F, bool RES>
-__global__ void __launch_bounds__(kTemporalWarps * 32, ((T > 4 || temporal_f_ring(T, HAS_F)) ? 2 : JAC_TOCC))
+__global__ void __launch_bounds__(kTemporalWarps * 32,
+                                  (((T > 4 && temporal_points(T) == 4) || temporal_f_ring(T, HAS_F)) ? 2 : JAC_TOCC))
 temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const double* __restrict__ f,
                   double* __restrict__ partials, const JacGeom g, const int strips_x, const int strips_y,
                   const int rows_per_strip)
@@ -657,27 +683,30 @@ temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
 
     TemporalCtx c;
     constexpr int HL = temporal_halo_lanes(T);
-    const long long X0 = (long long)sx * temporal_strip_cols(T) - 4 * HL;
-    const long long gx = X0 + 4 * lane;
+    constexpr int P = temporal_points(T);
+    constexpr int SC = temporal_stage_chunks(P);
+    const long long X0 = (long long)sx * temporal_strip_cols(T) - P * HL;
+    const long long gx = X0 + P * lane;
     c.xout = gx < 0 || gx >= g.nx;
     c.cx = gx < 0 ? g.bval[0] : g.bval[1];
     c.c_my = g.bval[2];
     c.c_py = g.bval[3];
-    c.edge_x = (sx == 0) || (X0 + 128 > g.nx);
+    c.edge_x = (sx == 0) || (X0 + 32 * P > g.nx);
     c.store_lane = lane >= HL && lane <= 31 - HL && !c.xout;
     const long long col = c.xout ? g.origin : column_base(g, gx);
     c.fb = HAS_F ? f + col : nullptr;
     c.ob = un + col;
+    // copy duty: chunk `lane` (and, with 4 points per lane, chunk `32 + lane`) of every row
     const long long xa = X0 + 2 * lane, xb = X0 + 64 + 2 * lane;
     c.copy_a = xa >= 0 && xa < g.nx;
-    c.copy_b = xb >= 0 && xb < g.nx;
+    c.copy_b = P == 4 && xb >= 0 && xb < g.nx;
     c.src_a = u + (c.copy_a ? column_base(g, xa) : g.origin);
     c.src_b = u + (c.copy_b ? column_base(g, xb) : g.origin);
-    double2* ring = t2_ring_mem + warp * temporal_stages_per_warp(T, HAS_F) * 64;
+    double2* ring = t2_ring_mem + warp * temporal_stages_per_warp(T, HAS_F) * SC;
     c.fdelta = HAS_F ? (long long)(f - u) : 0;
     c.dst_a = ring + lane;        // chunk k = lane
     c.dst_b = ring + 32 + lane;   // chunk k = 32 + lane
-    c.mine = ring + 2 * lane;     // chunks 2*lane and 2*lane + 1
+    c.mine = ring + (P / 2) * lane;   // this lane's own P points: P/2 consecutive chunks
     c.brs = g.block_stride * g.gx;
     c.ny = (int)g.ny;
     c.Y0 = sy * rows_per_strip;
@@ -686,11 +715,11 @@ temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
     c.in_end = c.Y1 + T;
     const int r_end = c.Y1 + 2 * T - 1;   // the top level trails the input by 2T - 1 rows
 
-    Row4 win[T][3];
+    RowN<P> win[T][3];
 #pragma unroll
     for (int s = 0; s < T; ++s)
 #pragma unroll
-        for (int k = 0; k < 3; ++k) win[s][k] = fill_row4(0.0);
+        for (int k = 0; k < 3; ++k) win[s][k] = fill_rown<P>(0.0);
 
     RowCursor load_cur, out_cur;
     load_cur.init(c.r0, g, c.brs);
@@ -699,7 +728,7 @@ temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
     // fill the ring with the first DEPTH rows
 #pragma unroll 1
     for (int k = 0; k < kTemporalDepth; ++k) {
-        issue_row<HAS_F, F_RING>(c, c.r0 + k, load_cur);
+        issue_row<P, HAS_F, F_RING>(c, c.r0 + k, load_cur);
         load_cur.advance(g, c.brs);
     }
 
