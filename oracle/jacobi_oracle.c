@@ -28,6 +28,8 @@
  *            restricted to the strip (x fastest, then y, then z).
  *            Faces on the domain boundary are neither packed nor unpacked.
  *   exchange comes before the update in every sweep.
+ *   wide     (last part of this file; not in the paper) one exchange of all h ghost layers with
+ *            edges and corners, then up to h sweeps on shrinking extents: same bits.
  *
  * Index conventions: x is the fastest-varying axis, then y, then z.  In 2D, nz = bz = 1
  * and there is no padding along z.
@@ -36,7 +38,9 @@
  * factor per sweep; tiny grids against exact rational arithmetic on the textbook
  * matrix form; random-walk path enumeration for the heated-edge problem; blocked
  * run is bit-identical to the monolithic run; packed buffers equal numpy slices of
- * the dense array; residual identities (r = 4(u_{k+1}-u_k) in 2D, ||r|| = ||f|| at u = 0).
+ * the dense array; residual identities (r = 4(u_{k+1}-u_k) in 2D, ||r|| = ||f|| at u = 0);
+ * wide exchange: every ghost equals the padded global field, k sweeps per exchange are
+ * bit-identical to the monolithic run for every k <= h.
  */
 #include <math.h>
 #include <stdint.h>
@@ -453,5 +457,175 @@ int orc_blocked_residual(orc_blocked *s, double *out_l2)
         total += acc;
     }
     *out_l2 = (double)sqrtl(total);
+    return ORC_OK;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Wide exchange: h ghost layers license up to h sweeps per exchange.        */
+/*                                                                           */
+/* Not in the paper, which exchanges before every update (Section V-C); this */
+/* is the same pack -> transfer -> unpack step made once per group of sweeps.*/
+/* A radius-1 stencil applied t times reaches t cells in every axis at once, */
+/* so the ghost layers must also hold edge and corner data.  They are filled */
+/* axis by axis: phase x, then y, then z.  In phase a the strip of a face is */
+/* the h layers next to it along a, over the WHOLE padded extent (-h .. b+h) */
+/* of every other axis, so what an earlier phase delivered travels on.       */
+/* After the last phase every ghost cell whose position lies inside the      */
+/* domain holds the owner's current value, and every ghost cell outside the  */
+/* domain in exactly one axis holds that face's Dirichlet value (cells       */
+/* outside in two or more axes are never read).                              */
+/*                                                                           */
+/* A group of t <= h sweeps then runs with no further exchange: sweep number */
+/* m (m = 1..t) updates every block's interior extended by e = t - m layers  */
+/* on every side; positions outside the domain keep their value.  The last   */
+/* sweep of a group (e = 0) is the ordinary update.  Interiors end up bit    */
+/* for bit as with an exchange before every sweep.                           */
+/* ------------------------------------------------------------------------- */
+
+/* index range of the wide strip on `face`: h layers along the face's axis (interior layers if
+ * ghost == 0, ghost layers if ghost == 1), the whole padded extent along the other axes */
+static void wide_strip_range(const orc_blocked *s, int face, int ghost, int64_t lo[3], int64_t hi[3])
+{
+    strip_range(s, face, ghost, lo, hi);
+    const int axis = face / 2;
+    for (int a = 0; a < s->ndim; ++a)
+        if (a != axis) { lo[a] = -s->h; hi[a] = s->b[a] + s->h; }
+}
+
+int64_t orc_blocked_wide_face_elems(const orc_blocked *s, int face)
+{
+    if (!s || face < 0 || face >= 2 * s->ndim) return ORC_EINVAL;
+    int64_t lo[3], hi[3];
+    wide_strip_range(s, face, 0, lo, hi);
+    return (hi[0] - lo[0]) * (hi[1] - lo[1]) * (hi[2] - lo[2]);
+}
+
+static int64_t wide_max_face(const orc_blocked *s)
+{
+    int64_t m = 0;
+    for (int fc = 0; fc < 2 * s->ndim; ++fc) {
+        const int64_t e = orc_blocked_wide_face_elems(s, fc);
+        if (e > m) m = e;
+    }
+    return m;
+}
+
+/* One phase (one axis) of the wide exchange on the padded arrays `arr` (nblocks * pad_elems):
+ * pack both faces of every block that have a neighbour, then unpack. `wsend` holds
+ * nblocks * 6 * wmax doubles. */
+static void wide_phase(const orc_blocked *s, double *arr, double *wsend, int64_t wmax, int axis)
+{
+    for (int64_t blk = 0; blk < s->nblocks; ++blk) {
+        const double *u = arr + blk * s->pad_elems;
+        for (int face = 2 * axis; face < 2 * axis + 2; ++face) {
+            if (blk_neighbour(s, blk, face) < 0) continue;
+            int64_t lo[3], hi[3];
+            wide_strip_range(s, face, 0, lo, hi);
+            double *buf = wsend + (blk * 6 + face) * wmax;
+            int64_t q = 0;
+            for (int64_t k = lo[2]; k < hi[2]; ++k)
+                for (int64_t j = lo[1]; j < hi[1]; ++j)
+                    for (int64_t i = lo[0]; i < hi[0]; ++i)
+                        buf[q++] = u[pad_index(s, i, j, k)];
+        }
+    }
+    for (int64_t blk = 0; blk < s->nblocks; ++blk) {
+        double *u = arr + blk * s->pad_elems;
+        for (int face = 2 * axis; face < 2 * axis + 2; ++face) {
+            const int64_t nb = blk_neighbour(s, blk, face);
+            if (nb < 0) continue;
+            int64_t lo[3], hi[3];
+            wide_strip_range(s, face, 1, lo, hi);
+            const double *buf = wsend + (nb * 6 + (face ^ 1)) * wmax;
+            int64_t q = 0;
+            for (int64_t k = lo[2]; k < hi[2]; ++k)
+                for (int64_t j = lo[1]; j < hi[1]; ++j)
+                    for (int64_t i = lo[0]; i < hi[0]; ++i)
+                        u[pad_index(s, i, j, k)] = buf[q++];
+        }
+    }
+}
+
+/* Wide exchange of the current state.  If wide_bufs is not NULL it receives the packed wide
+ * faces as each phase left them: nblocks * 6 slots of orc_blocked_wide_max_face() doubles. */
+int orc_blocked_exchange_wide(orc_blocked *s, double *wide_bufs)
+{
+    if (!s) return ORC_EINVAL;
+    const int64_t wmax = wide_max_face(s);
+    double *wsend = wide_bufs ? wide_bufs
+                              : (double *)calloc((size_t)(s->nblocks * 6 * wmax), sizeof(double));
+    if (!wsend) return ORC_ENOMEM;
+    for (int axis = 0; axis < s->ndim; ++axis)
+        wide_phase(s, s->u[s->cur], wsend, wmax, axis);
+    if (!wide_bufs) free(wsend);
+    return ORC_OK;
+}
+
+int64_t orc_blocked_wide_max_face(const orc_blocked *s)
+{
+    return s ? wide_max_face(s) : ORC_EINVAL;
+}
+
+/* f at block-relative position (i, j, k) of block `blk`, which may lie in a neighbouring
+ * block: f is one global field, looked up by global coordinates */
+static double f_global(const orc_blocked *s, const int64_t c[3], int64_t i, int64_t j, int64_t k)
+{
+    const int64_t rel[3] = {i, j, k};
+    int64_t bc[3], in[3];
+    for (int a = 0; a < 3; ++a) {
+        const int64_t gpos = c[a] * s->b[a] + rel[a];
+        bc[a] = gpos / s->b[a];
+        in[a] = gpos - bc[a] * s->b[a];
+    }
+    int64_t owner = (bc[2] * s->g[1] + bc[1]) * s->g[0] + bc[0];
+    return s->f[owner * s->blk_elems + (in[2] * s->b[1] + in[1]) * s->b[0] + in[0]];
+}
+
+/* The update over every block's interior extended by e layers on every side (0 <= e < h),
+ * reading the padded array as it is.  Positions outside the domain keep their value. */
+int orc_blocked_update_ext(orc_blocked *s, int64_t e)
+{
+    if (!s || e < 0 || e >= s->h) return ORC_EINVAL;
+    const int64_t px = s->p[0], pxy = s->p[0] * s->p[1];
+    const int64_t ez = (s->ndim == 3) ? e : 0;
+    const double c6 = 1.0 / 6.0;
+#pragma omp parallel for schedule(static)
+    for (int64_t blk = 0; blk < s->nblocks; ++blk) {
+        const double *u = blk_u(s, s->cur, blk);
+        double *o = blk_u(s, s->cur ^ 1, blk);
+        int64_t c[3];
+        blk_coords(s, blk, c);
+        for (int64_t k = -ez; k < s->b[2] + ez; ++k)
+            for (int64_t j = -e; j < s->b[1] + e; ++j)
+                for (int64_t i = -e; i < s->b[0] + e; ++i) {
+                    const int64_t p = pad_index(s, i, j, k);
+                    const int64_t gi = c[0] * s->b[0] + i, gj = c[1] * s->b[1] + j,
+                                  gk = c[2] * s->b[2] + k;
+                    if (gi < 0 || gi >= s->n[0] || gj < 0 || gj >= s->n[1] || gk < 0 || gk >= s->n[2]) {
+                        o[p] = u[p];
+                        continue;
+                    }
+                    double sum = (u[p - 1] + u[p + 1]) + (u[p - px] + u[p + px]);
+                    if (s->ndim == 3) sum = sum + (u[p - pxy] + u[p + pxy]);
+                    if (s->f) sum = sum + f_global(s, c, i, j, k);
+                    o[p] = (s->ndim == 3) ? sum * c6 : sum * 0.25;
+                }
+    }
+    s->cur ^= 1;
+    return ORC_OK;
+}
+
+/* nsweeps sweeps in groups of at most k (1 <= k <= h): wide exchange, then the group's
+ * updates on extents shrinking to the interior. */
+int orc_blocked_sweep_wide(orc_blocked *s, int64_t nsweeps, int64_t k)
+{
+    if (!s || nsweeps < 0 || k < 1 || k > s->h) return ORC_EINVAL;
+    for (int64_t left = nsweeps; left > 0;) {
+        const int64_t t = left < k ? left : k;
+        const int rc = orc_blocked_exchange_wide(s, NULL);
+        if (rc) return rc;
+        for (int64_t m = 1; m <= t; ++m) orc_blocked_update_ext(s, t - m);
+        left -= t;
+    }
     return ORC_OK;
 }

@@ -66,6 +66,13 @@ def lib() -> C.CDLL:
         L.orc_blocked_update.argtypes = [C.c_void_p]
         L.orc_blocked_sweep.argtypes = [C.c_void_p, C.c_int64]
         L.orc_blocked_residual.argtypes = [C.c_void_p, _f64p]
+        L.orc_blocked_exchange_wide.argtypes = [C.c_void_p, _f64p]
+        L.orc_blocked_update_ext.argtypes = [C.c_void_p, C.c_int64]
+        L.orc_blocked_sweep_wide.argtypes = [C.c_void_p, C.c_int64, C.c_int64]
+        L.orc_blocked_wide_face_elems.argtypes = [C.c_void_p, C.c_int]
+        L.orc_blocked_wide_face_elems.restype = C.c_int64
+        L.orc_blocked_wide_max_face.argtypes = [C.c_void_p]
+        L.orc_blocked_wide_max_face.restype = C.c_int64
         _lib = L
     return _lib
 
@@ -235,6 +242,40 @@ class Blocked:
         out = C.c_double(0.0)
         _check(lib().orc_blocked_residual(self._p, C.byref(out)), "residual")
         return out.value
+
+    # ---- wide exchange: all h ghost layers including edges and corners, axis by axis
+    def wide_face_shape(self, face: int):
+        """numpy shape of a packed wide face: h layers along the face's axis, b + 2h along the others."""
+        dims = [x + 2 * self.h for x in self.b]
+        dims[face // 2] = self.h
+        return tuple(reversed(dims))
+
+    def exchange_wide(self, keep_buffers: bool = False):
+        """Wide exchange of the current state; with ``keep_buffers`` returns {(blk, face): packed wide face}."""
+        if not keep_buffers:
+            _check(lib().orc_blocked_exchange_wide(self._p, None), "exchange_wide")
+            return None
+        wmax = int(lib().orc_blocked_wide_max_face(self._p))
+        raw = np.zeros((self.nblocks, 6, wmax), dtype=np.float64)
+        _check(lib().orc_blocked_exchange_wide(self._p, _ptr(raw)), "exchange_wide")
+        out = {}
+        for blk in range(self.nblocks):
+            for face in range(2 * self.ndim):
+                if self.neighbour(blk, face) < 0:
+                    continue
+                shp = self.wide_face_shape(face)
+                ne = int(lib().orc_blocked_wide_face_elems(self._p, face))
+                assert ne == int(np.prod(shp))
+                out[(blk, face)] = raw[blk, face, :ne].reshape(shp).copy()
+        return out
+
+    def update_ext(self, e: int):
+        """The update over every block's interior extended by e layers (no exchange)."""
+        _check(lib().orc_blocked_update_ext(self._p, int(e)), "update_ext")
+
+    def sweep_wide(self, nsweeps: int, k: int | None = None):
+        """nsweeps sweeps with one wide exchange per group of k (default h) sweeps."""
+        _check(lib().orc_blocked_sweep_wide(self._p, int(nsweeps), int(self.h if k is None else k)), "sweep_wide")
 
     def neighbour(self, blk: int, face: int) -> int:
         """Block across ``face`` or -1 at the domain boundary (host-side convenience for tests)."""

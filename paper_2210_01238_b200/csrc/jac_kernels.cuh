@@ -761,8 +761,14 @@ temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
 // per plane are stored.  Tiles read across block borders directly; Dirichlet values are
 // injected outside the domain at every level (EDGE variant only).  Requires bx % 2 == 0.
 // ---------------------------------------------------------------------------------------
-constexpr int k3dWarps = 8;          // warps per CTA, stacked along y
-constexpr int k3dRows = 6;           // rows per warp
+#ifndef JAC_T3W
+#define JAC_T3W 8     // warps per CTA, stacked along y
+#endif
+#ifndef JAC_T3R
+#define JAC_T3R 6     // rows per warp
+#endif
+constexpr int k3dWarps = JAC_T3W;
+constexpr int k3dRows = JAC_T3R;
 constexpr int k3dTileRows = k3dWarps * k3dRows;   // 48
 constexpr int k3dPlaneElems = k3dTileRows * 64;   // doubles per ring stage
 constexpr int k3dFStages = 4;        // f planes resident (levels 1 and 2 read planes p-1 and p-3)

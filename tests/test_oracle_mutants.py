@@ -32,6 +32,16 @@ MUTANTS = {
                               "        orc_blocked_update(s);",
                               "        orc_blocked_update(s);\n        orc_blocked_pack(s);\n"
                               "        orc_blocked_unpack(s);", 1),
+    "wide_strips_leave_out_the_ghost_extent": ("if (a != axis) { lo[a] = -s->h; hi[a] = s->b[a] + s->h; }",
+                                               "if (a != axis) { lo[a] = 0; hi[a] = s->b[a]; }", 1),
+    "group_updates_do_not_shrink": ("orc_blocked_update_ext(s, t - m);", "orc_blocked_update_ext(s, 0);", 1),
+    "extended_update_moves_dirichlet_cells": ("                        o[p] = u[p];\n                        continue;\n",
+                                              "", 1),
+    "extended_update_reads_own_f": ("return s->f[owner * s->blk_elems +",
+                                    "owner = (c[2] * s->g[1] + c[1]) * s->g[0] + c[0]; return s->f[owner * s->blk_elems +", 1),
+    "wide_unpack_reads_same_side": ("wsend + (nb * 6 + (face ^ 1)) * wmax", "wsend + (nb * 6 + face) * wmax", 1),
+    "wide_exchange_skips_last_axis": ("for (int axis = 0; axis < s->ndim; ++axis)\n        wide_phase",
+                                      "for (int axis = 0; axis + 1 < s->ndim; ++axis)\n        wide_phase", 1),
 }
 
 
@@ -50,7 +60,8 @@ def test_planted_mistake_is_caught(name, tmp_path):
     env = dict(os.environ, ORC_LIB=str(so))
     r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider",
                         str(ROOT / "tests" / "test_oracle_sweep.py"),
-                        str(ROOT / "tests" / "test_oracle_blocks.py")],
+                        str(ROOT / "tests" / "test_oracle_blocks.py"),
+                        str(ROOT / "tests" / "test_oracle_wide.py")],
                        cwd=ROOT, env=env, capture_output=True, text=True)
     assert r.returncode == 1, f"mutant {name} survived the pins:\n{r.stdout[-2000:]}"
     assert "failed" in r.stdout
