@@ -60,7 +60,9 @@ NCU_TRAFFIC = {
 KERNEL_NAMES = {("temporal", 2): "temporal2d_kernel", ("temporal", 3): "temporal3d_kernel", ("fused", 2): "sweep2d_kernel (update pulling neighbour interiors)",
                 ("exchange", 2): "sweep2d_kernel", ("pertask", 2): "sweep2d_kernel (one launch per block)",
                 ("fused", 3): "sweep3d_kernel (update pulling neighbour interiors)", ("exchange", 3): "sweep3d_kernel",
-                ("pertask", 3): "sweep3d_kernel (one launch per block)"}
+                ("pertask", 3): "sweep3d_kernel (one launch per block)",
+                ("wide", 2): "sweep2d_kernel (grown boxes between wide exchanges)",
+                ("wide", 3): "sweep3d_kernel (grown boxes between wide exchanges)"}
 
 
 def log(*a):
@@ -254,7 +256,9 @@ def run_ours(args, w: inputs.Workload):
     peak, peak_kind = measured_peak_gbs()
 
     def make_ctx(mode, tsteps):
-        J = jac.Jacobi(w.n, w.b, w.halo, w.has_f, mode, tsteps)
+        # the wide schedule needs as many ghost layers as sweeps per exchange
+        halo = max(w.halo, tsteps) if mode == "wide" else w.halo
+        J = jac.Jacobi(w.n, w.b, halo, w.has_f, mode, tsteps)
         for face, v in enumerate(w.boundary()):
             J.set_boundary(face, v)
         if f is not None:
@@ -300,10 +304,13 @@ def run_ours(args, w: inputs.Workload):
     mode, tsteps = args.mode, args.tsteps
     if mode == "auto":
         mode, tsteps = default_schedule(w)
-    if mode != "temporal":
+    if mode == "wide":
+        tsteps = tsteps or 4
+    elif mode != "temporal":
         tsteps = 1
     J = make_ctx(mode, tsteps)
-    tsteps = J.sweeps_per_launch()
+    if mode != "wide":
+        tsteps = J.sweeps_per_launch()
     main_run = time_schedule(J, mode, tsteps, args.steps, args.warmup, True)
     value = main_run["glups"]
 
@@ -359,7 +366,7 @@ def run_ours(args, w: inputs.Workload):
     # ---- the other schedules, briefly, for context (same job, fewer steps)
     others = {}
     if not args.no_others and world == 1:
-        alts = [("exchange", 1), ("fused", 1)]
+        alts = [("exchange", 1), ("fused", 1), ("wide", 4)]   # wide: 4 ghost layers, 4 sweeps per exchange
         if w.ndim == 2 and w.b[0] % 4 == 0:
             alts += [("temporal", 1), ("temporal", 2), ("temporal", 4), ("temporal", 8)]
         if w.ndim == 3 and w.b[0] % 2 == 0:
@@ -370,7 +377,7 @@ def run_ours(args, w: inputs.Workload):
             Jo = make_ctx(m, t)
             r = time_schedule(Jo, m, t, 2, 1, False)
             Jo.close()
-            others[f"{m}{t if m == 'temporal' else ''}"] = {
+            others[f"{m}{t if m in ('temporal', 'wide') else ''}"] = {
                 "glups": r["glups"], "effective_gbs": r["glups"] * w.bytes_per_point,
                 "launch_ms": r["launch_ms"], "launches": r["launches"]}
     del u0_dev
@@ -389,7 +396,8 @@ def run_ours(args, w: inputs.Workload):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": main_run["ms_total"] / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name, "grid": list(w.n), "block": list(w.b), "halo": w.halo,
+            "config": {"workload": w.name, "grid": list(w.n), "block": list(w.b),
+                       "halo": max(w.halo, tsteps) if mode == "wide" else w.halo,
                        "has_f": w.has_f, "sweeps_per_step": sweeps, "residuals_per_step": 1,
                        "schedule": mode, "tsteps": tsteps,
                        "l2": f"arrays of {w.points * 8 / 1e6:.0f} MB each exceed the {L2_BYTES / 1e6:.0f} MB L2"
@@ -414,7 +422,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3_eigenmode_16384", choices=sorted(inputs.CONFIGS))
-    ap.add_argument("--mode", default="auto", choices=["auto", "fused", "exchange", "pertask", "temporal"],
+    ap.add_argument("--mode", default="auto", choices=["auto", "fused", "exchange", "pertask", "temporal", "wide"],
                     help="schedule of jac_sweep; auto = the fastest one the library has for the workload")
     ap.add_argument("--tsteps", type=int, default=0)
     ap.add_argument("--sweeps", type=int, default=0, help="sweeps per step (default: the workload's)")

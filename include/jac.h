@@ -62,6 +62,12 @@ extern "C" {
                                2D: b[0] % 4 == 0, tsteps <= 8; 3D: b[0] % 2 == 0, tsteps <= 2;
                                jac_create returns JAC_EINVAL otherwise                           */
 #define JAC_MODE_EXCHANGE 3 /* per sweep three launches over all blocks: pack, unpack, update    */
+#define JAC_MODE_WIDE     4 /* one wide exchange (jac_exchange_wide: all h ghost layers, edges and
+                               corners included) per group of `tsteps` <= h sweeps (0 = h); the
+                               group's sweeps update boxes shrinking from the interior grown by
+                               tsteps - 1 layers down to the interior, so neighbours are computed
+                               redundantly instead of being exchanged.  2 * ndim + tsteps launches
+                               per group                                                         */
 
 typedef struct jac_ctx jac_ctx; /* opaque, host memory, owned by the library */
 
@@ -70,7 +76,8 @@ typedef struct jac_desc {
     int32_t halo;    /* ghost width h, 1 <= h <= min(b[a]) and h <= 8                            */
     int32_t has_f;   /* 0: f == 0 and is never read (16 B/point/sweep); 1: f present (24 B)      */
     int32_t mode;    /* JAC_MODE_*                                                               */
-    int32_t tsteps;  /* JAC_MODE_TEMPORAL: sweeps per launch; 0 = the library chooses             */
+    int32_t tsteps;  /* JAC_MODE_TEMPORAL: sweeps per launch; JAC_MODE_WIDE: sweeps per exchange
+                        (<= halo); 0 = the library chooses                                       */
     int32_t reserved;/* must be 0                                                                */
     int64_t n[3];    /* global interior points; n[2] ignored (taken as 1) when ndim == 2         */
     int64_t b[3];    /* block interior points; n[a] % b[a] == 0                                  */
@@ -95,6 +102,8 @@ typedef struct jac_layout {
     int64_t off_send;      /*   send buffers,                                                    */
     int64_t off_scratch;   /*   reduction scratch + result word                                  */
     int64_t total_bytes;
+    int64_t wide_face_elems[6]; /* elements of one packed wide face (jac_exchange_wide); in
+                                   JAC_MODE_WIDE the send slots are sized for these              */
 } jac_layout;
 
 /* Workspace size in bytes for `desc` (pure host computation, no CUDA call).
@@ -156,6 +165,23 @@ int jac_unpack_halos(jac_ctx *ctx);
  * be timed apart.  Errors: JAC_EINVAL for bits beyond 2*ndim. */
 int jac_pack_faces(jac_ctx *ctx, unsigned face_mask);
 int jac_unpack_faces(jac_ctx *ctx, unsigned face_mask);
+
+/* Wide exchange (JAC_MODE_WIDE contexts only, else JAC_EINVAL): fills ALL h ghost layers of the
+ * current state, edges and corners included, so that up to h sweeps can follow without another
+ * exchange (a radius-1 stencil applied t times reaches t cells along every axis at once).  The
+ * paper exchanges before every update (Section V-C); this is the same pack -> transfer -> unpack
+ * step made once per group of sweeps, the usual way to trade redundant computation for fewer,
+ * larger messages.  It runs axis by axis, x then y then z, one pack and one unpack launch each:
+ * the strip of a face is the h layers next to it along its axis over the WHOLE padded extent
+ * (b + 2h) of the other axes, so data delivered for an earlier axis travels on into the edges
+ * and corners.  A packed wide face is in source memory order: an x face is [bz+2h][by+2h][h], a y
+ * face [bz+2h][h][bx+2h], a z face [h][by+2h][bx+2h] (2D: no z extent).  Afterwards every ghost
+ * cell whose position lies inside the domain holds its owner's current value, and every ghost cell
+ * outside the domain in exactly one axis holds that face's Dirichlet value.  Asynchronous.
+ * jac_get_wide_buffer: the packed wide face of (block, face) as the exchange left it (HOST output,
+ * synchronous; wide_face_elems[face] doubles). */
+int jac_exchange_wide(jac_ctx *ctx);
+int jac_get_wide_buffer(jac_ctx *ctx, int64_t block, int face, double *host);
 
 /* nsweeps Jacobi iterations, each "exchange halos, then update every block" (paper Section
  * V-C), scheduled as desc.mode says.  Afterwards the interiors hold the new state; the

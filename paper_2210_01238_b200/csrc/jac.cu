@@ -30,10 +30,12 @@ struct Tiling {
     long long ctas_per_block;
 };
 
-Tiling make_tiling(const JacGeom& g)
+// force_nv = 1: one point per thread although the width is even (rows that do not start on a
+// 16-byte boundary)
+Tiling make_tiling(const JacGeom& g, int force_nv = 0)
 {
     Tiling t{};
-    t.nv = (g.bx % 2 == 0) ? 2 : 1;
+    t.nv = force_nv ? force_nv : ((g.bx % 2 == 0) ? 2 : 1);
     const long long need = ceil_div(g.bx, t.nv);
     const long long want_ctas = (long long)kNumSMs * 16;
     if (g.ndim == 2) {
@@ -116,7 +118,7 @@ int build_geometry(const jac_desc* d, JacGeom* g, jac_layout* L)
     if (d->ndim != 2 && d->ndim != 3) return JAC_EINVAL;
     if (d->halo < 1 || d->halo > 8) return JAC_EINVAL;
     if (d->has_f != 0 && d->has_f != 1) return JAC_EINVAL;
-    if (d->mode < JAC_MODE_FUSED || d->mode > JAC_MODE_EXCHANGE) return JAC_EINVAL;
+    if (d->mode < JAC_MODE_FUSED || d->mode > JAC_MODE_WIDE) return JAC_EINVAL;
     if (d->tsteps < 0 || d->tsteps > 8 || d->reserved != 0) return JAC_EINVAL;
     long long n[3] = {1, 1, 1}, b[3] = {1, 1, 1}, gr[3] = {1, 1, 1};
     for (int a = 0; a < d->ndim; ++a) {
@@ -148,10 +150,17 @@ int build_geometry(const jac_desc* d, JacGeom* g, jac_layout* L)
     g->face_elems[0] = g->face_elems[1] = h * b[1] * b[2];
     g->face_elems[2] = g->face_elems[3] = h * b[0] * b[2];
     g->face_elems[4] = g->face_elems[5] = (d->ndim == 3) ? h * b[0] * b[1] : 0;
+    const long long wx = b[0] + 2 * h, wy = b[1] + 2 * h, wz = b[2] + 2 * hz;
+    g->wface_elems[0] = g->wface_elems[1] = h * wy * wz;
+    g->wface_elems[2] = g->wface_elems[3] = h * wx * wz;
+    g->wface_elems[4] = g->wface_elems[5] = (d->ndim == 3) ? h * wx * wy : 0;
+    // the send slots hold wide faces in the schedule that exchanges them, else the plain faces
+    const bool wide = d->mode == JAC_MODE_WIDE;
+    if (wide && d->tsteps > d->halo) return JAC_EINVAL;   // sweeps per exchange <= ghost layers
     long long off = 0;
     for (int fc = 0; fc < 6; ++fc) {
         g->face_off[fc] = off;
-        off += round_up(g->face_elems[fc], 16);  // every face buffer starts on a 128-byte line
+        off += round_up(wide ? g->wface_elems[fc] : g->face_elems[fc], 16);  // 128-byte lines
     }
     g->send_stride = off;
 
@@ -159,8 +168,9 @@ int build_geometry(const jac_desc* d, JacGeom* g, jac_layout* L)
     const long long ctas = g->nblocks * t.ctas_per_block;
     if (ctas > kMaxGrid) return JAC_EINVAL;
     long long max_face = 0;
-    for (int fc = 0; fc < 6; ++fc) max_face = std::max(max_face, g->face_elems[fc]);
+    for (int fc = 0; fc < 6; ++fc) max_face = std::max(max_face, wide ? g->wface_elems[fc] : g->face_elems[fc]);
     if (max_face >= (1LL << 31)) return JAC_EINVAL;
+    if (wide && 2 * g->nblocks * ceil_div(round_up(max_face, 32), 256) > kMaxGrid) return JAC_EINVAL;
     if (g->nblocks * g->nfaces * ceil_div(round_up(ceil_div(max_face, 2), 32), 256) > kMaxGrid) return JAC_EINVAL;
 
     if (L) {
@@ -176,6 +186,7 @@ int build_geometry(const jac_desc* d, JacGeom* g, jac_layout* L)
             L->face_offset[fc] = g->face_off[fc];
         }
         L->send_stride = g->send_stride;
+        for (int fc = 0; fc < 6; ++fc) L->wide_face_elems[fc] = g->wface_elems[fc];
         L->partials = round_up(max_partials(*g, ctas), 32);
         const long long arr_bytes = round_up(g->nblocks * g->block_stride * 8, 256);
         long long o = 0;
@@ -205,6 +216,7 @@ struct jac_ctx {
     int cur;            // which of u[] holds the current state
     bool ghosts_fresh;  // inter-block ghosts of u[cur] equal the neighbours' current faces
     bool packed_current;  // the send buffers hold the faces of the current state
+    bool f_ghosts_fresh;  // JAC_MODE_WIDE: the ghost layers of f hold the neighbours' f
     cudaStream_t stream;
     int device;
     int cuda_err;       // sticky
@@ -325,6 +337,63 @@ int do_exchange(jac_ctx* c)
     if (rc) return rc;
     c->ghosts_fresh = true;
     return JAC_OK;
+}
+
+// ---- wide exchange and the updates between two of them ------------------------------
+// all h ghost layers of `arr`, edges and corners included: per axis one pack and one unpack launch
+int do_exchange_wide(jac_ctx* c, double* arr)
+{
+    for (int axis = 0; axis < c->g.ndim; ++axis) {
+        const long long n = c->g.wface_elems[2 * axis];
+        const int slots = (int)round_up(n, 32);
+        const long long ctas = ceil_div(2 * c->g.nblocks * slots, 256);
+        if (ctas > kMaxGrid) return JAC_EINVAL;
+        jac::halo_wide_kernel<false><<<(unsigned)ctas, 256, 0, c->stream>>>(arr, c->send, c->g, axis, slots);
+        int rc = check_launch(c);
+        if (rc) return rc;
+        jac::halo_wide_kernel<true><<<(unsigned)ctas, 256, 0, c->stream>>>(arr, c->send, c->g, axis, slots);
+        if ((rc = check_launch(c))) return rc;
+    }
+    return JAC_OK;
+}
+
+// the update over every block's interior grown by e >= 1 layers (positions outside the domain keep
+// their value): the ordinary sweep kernels on a geometry whose block box is the grown one
+template <int NV, bool HAS_F>
+void launch_ext_t(jac_ctx* c, const JacGeom& ge, const Tiling& t, const double* u, double* un)
+{
+    const unsigned grid = (unsigned)(ge.nblocks * t.ctas_per_block);
+    if (ge.ndim == 2)
+        jac::sweep2d_kernel<NV, HAS_F, jac::OP_UPDATE_EXT><<<grid, t.block, 0, c->stream>>>(
+            u, un, c->f, nullptr, ge, 0, t.tiles_x, t.tiles_y, t.march);
+    else
+        jac::sweep3d_kernel<NV, HAS_F, jac::OP_UPDATE_EXT><<<grid, t.block, 0, c->stream>>>(
+            u, un, c->f, nullptr, ge, 0, t.tiles_x, t.tiles_y, t.tiles_z, t.march);
+}
+
+int launch_ext(jac_ctx* c, int e, const double* u, double* un)
+{
+    JacGeom ge = c->g;
+    ge.ext = e;
+    ge.bx += 2 * e;
+    ge.by += 2 * e;
+    ge.origin -= (long long)e * ge.PX + e;
+    if (ge.ndim == 3) {
+        ge.bz += 2 * e;
+        ge.origin -= (long long)e * ge.PXY;
+    }
+    // 128-bit accesses need the first column of the grown box on a 16-byte boundary: e even
+    const Tiling t = make_tiling(ge, (e % 2 != 0) ? 1 : 0);
+    if (ge.nblocks * t.ctas_per_block > kMaxGrid) return JAC_EINVAL;
+    const bool f = c->desc.has_f != 0;
+    if (t.nv == 2) {
+        if (f) launch_ext_t<2, true>(c, ge, t, u, un);
+        else launch_ext_t<2, false>(c, ge, t, u, un);
+    } else {
+        if (f) launch_ext_t<1, true>(c, ge, t, u, un);
+        else launch_ext_t<1, false>(c, ge, t, u, un);
+    }
+    return check_launch(c);
 }
 
 // ---- strided box copies between a dense array and the padded blocks ------------------
@@ -529,6 +598,33 @@ int run_sweeps(jac_ctx* c, int nsweeps, bool res, long long* nparts)
             c->packed_current = false;
             break;
         }
+        case JAC_MODE_WIDE: {
+            // groups of up to K sweeps (K <= h): one wide exchange, then updates on boxes shrinking
+            // from the interior grown by t - 1 layers down to the interior itself
+            const int K = c->desc.tsteps > 0 ? c->desc.tsteps : g.h;
+            if (c->f && !c->f_ghosts_fresh) {
+                if ((rc = do_exchange_wide(c, c->f))) return rc;
+                c->f_ghosts_fresh = true;
+            }
+            for (int left = nsweeps; left > 0;) {
+                const int t = std::min(K, left);
+                if ((rc = do_exchange_wide(c, c->u[c->cur]))) return rc;
+                for (int m = 1; m <= t; ++m) {
+                    const int e = t - m;
+                    const bool last = res && left == t && e == 0;
+                    if (e > 0) rc = launch_ext(c, e, c->u[c->cur], c->u[c->cur ^ 1]);
+                    else rc = last ? launch_sweep<jac::OP_UPDATE_RES>(c, c->u[c->cur], c->u[c->cur ^ 1], 0, g.nblocks)
+                                   : launch_sweep<jac::OP_UPDATE>(c, c->u[c->cur], c->u[c->cur ^ 1], 0, g.nblocks);
+                    if (rc) return rc;
+                    c->cur ^= 1;
+                }
+                left -= t;
+            }
+            if (res) *nparts = sweep_parts;
+            c->ghosts_fresh = false;
+            c->packed_current = false;
+            break;
+        }
         default:
             return JAC_EINVAL;
     }
@@ -613,6 +709,7 @@ int jac_create(const jac_desc* desc, void* dev_workspace, size_t bytes, jac_ctx*
     c->cur = 0;
     c->ghosts_fresh = false;
     c->packed_current = false;
+    c->f_ghosts_fresh = false;
     c->stream = static_cast<cudaStream_t>(desc->stream);
     c->device = dev;
     c->cuda_err = 0;
@@ -649,6 +746,7 @@ int jac_set_f(jac_ctx* c, const double* host_dense)
     int rc = usable(c);
     if (rc) return rc;
     if (!host_dense || !c->f) return JAC_EINVAL;
+    c->f_ghosts_fresh = false;
     return copy_dense_host(c, c->f, const_cast<double*>(host_dense), true);
 }
 
@@ -675,6 +773,7 @@ int jac_set_f_device(jac_ctx* c, const double* dev_dense)
     int rc = usable(c);
     if (rc) return rc;
     if (!dev_dense || !c->f) return JAC_EINVAL;
+    c->f_ghosts_fresh = false;
     return copy_dense_device<true>(c, c->f, const_cast<double*>(dev_dense));
 }
 
@@ -818,6 +917,29 @@ int jac_residual(jac_ctx* c, double* host_out_l2)
     if (!c->ghosts_fresh && (rc = do_exchange(c))) return rc;
     if ((rc = launch_sweep<jac::OP_RESIDUAL>(c, c->u[c->cur], nullptr, 0, c->g.nblocks))) return rc;
     return finish_norm(c, c->g.nblocks * c->tile.ctas_per_block, host_out_l2);
+}
+
+int jac_exchange_wide(jac_ctx* c)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    if (c->desc.mode != JAC_MODE_WIDE) return JAC_EINVAL;
+    if ((rc = do_exchange_wide(c, c->u[c->cur]))) return rc;
+    c->packed_current = false;   // the send slots now hold wide faces
+    c->ghosts_fresh = true;      // the face ghosts are among the cells just filled
+    return JAC_OK;
+}
+
+int jac_get_wide_buffer(jac_ctx* c, int64_t block, int face, double* host)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    if (c->desc.mode != JAC_MODE_WIDE) return JAC_EINVAL;
+    if (!host || block < 0 || block >= c->g.nblocks || face < 0 || face >= c->g.nfaces) return JAC_EINVAL;
+    const double* src = c->send + block * c->g.send_stride + c->g.face_off[face];
+    JAC_CK(c, cudaMemcpyAsync(host, src, (size_t)c->g.wface_elems[face] * 8, cudaMemcpyDeviceToHost, c->stream));
+    JAC_CK(c, cudaStreamSynchronize(c->stream));
+    return JAC_OK;
 }
 
 int jac_sweeps_per_launch(const jac_ctx* c, int* host_out)

@@ -24,4 +24,10 @@ struct JacGeom {
     long long face_off[6];
     long long send_stride;
     double bval[6];
+    // wide exchange: a wide face is h layers along its axis and the whole padded extent
+    // (b + 2h) along the other axes
+    long long wface_elems[6];
+    // extended update: the kernel is handed a geometry whose block box is the interior grown by
+    // `ext` layers on every side (bx, by, bz and origin adjusted; 0 in the context's own geometry)
+    int ext;
 };

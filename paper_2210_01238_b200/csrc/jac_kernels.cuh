@@ -13,10 +13,12 @@
 
 namespace jac {
 
-enum : int { OP_UPDATE = 0, OP_UPDATE_PULL = 1, OP_RESIDUAL = 2, OP_UPDATE_RES = 3, OP_UPDATE_PULL_RES = 4 };
+enum : int { OP_UPDATE = 0, OP_UPDATE_PULL = 1, OP_RESIDUAL = 2, OP_UPDATE_RES = 3, OP_UPDATE_PULL_RES = 4,
+             OP_UPDATE_EXT = 5 };
 __host__ __device__ constexpr bool op_stores(int op) { return op != OP_RESIDUAL; }
 __host__ __device__ constexpr bool op_pulls(int op) { return op == OP_UPDATE_PULL || op == OP_UPDATE_PULL_RES; }
 __host__ __device__ constexpr bool op_sums(int op) { return op == OP_RESIDUAL || op == OP_UPDATE_RES || op == OP_UPDATE_PULL_RES; }
+__host__ __device__ constexpr bool op_ext(int op) { return op == OP_UPDATE_EXT; }
 
 __device__ __forceinline__ double add_rn(double a, double b) { return __dadd_rn(a, b); }
 __device__ __forceinline__ double sub_rn(double a, double b) { return __dsub_rn(a, b); }
@@ -71,6 +73,9 @@ __device__ __forceinline__ double block_sum(double v) {
 // OP_RESIDUAL     per-CTA partial of sum r^2, r = s - 4u (ghost-reading)
 // OP_UPDATE_RES, OP_UPDATE_PULL_RES  the update, and in the same pass the partial of sum r^2 of the
 //                 state being read (s is in a register anyway): the residual at no extra traffic
+// OP_UPDATE_EXT   the update over a block box that is the interior grown by g.ext layers on every
+//                 side (the geometry passed in describes the grown box); positions outside the
+//                 domain keep their value.  Used between wide exchanges.
 // ---------------------------------------------------------------------------------------
 template <int NV, bool HAS_F, int OP>
 __global__ void __launch_bounds__(256)
@@ -106,6 +111,16 @@ sweep2d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
             if (byi + 1 < g.gy) off_n1 = bs * g.gx - (long long)(g.by - 1) * PX;  // block above, row 0
         }
 
+        // grown box: which of this thread's columns / which rows lie inside the domain
+        bool xin[NV];
+        long long gy0 = 0;
+        if (op_ext(OP)) {
+            const long long gx0 = (blk % g.gx) * (long long)(g.bx - 2 * g.ext) + x - g.ext;
+#pragma unroll
+            for (int q = 0; q < NV; ++q) xin[q] = gx0 + q >= 0 && gx0 + q < g.nx;
+            gy0 = (blk / g.gx) * (long long)(g.by - 2 * g.ext) - g.ext;
+        }
+
         Vec<NV> S = load_vec<NV>(ub + (j0 == 0 ? off_s0 : (long long)(j0 - 1) * PX));
         Vec<NV> Cc = load_vec<NV>(ub + (long long)j0 * PX);
 #pragma unroll 4
@@ -128,6 +143,7 @@ sweep2d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
                     acc = add_rn(acc, mul_rn(r, r));
                 }
                 if (op_stores(OP)) o.v[q] = mul_rn(s, 0.25);
+                if (op_ext(OP) && !(xin[q] && gy0 + j >= 0 && gy0 + j < g.ny)) o.v[q] = Cc.v[q];
             }
             if (op_stores(OP)) store_vec<NV>(ob + ro, o);
             S = Cc;
@@ -188,6 +204,17 @@ sweep3d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
             if (bzi + 1 < g.gz) off_u1 = bsz - (long long)(g.bz - 1) * PXY;
         }
 
+        // grown box (OP_UPDATE_EXT): is this thread's column inside the domain in x and y; first plane
+        bool xyin[NV];
+        long long gz0 = 0;
+        if (op_ext(OP)) {
+            const long long gx0 = (blk % g.gx) * (long long)(g.bx - 2 * g.ext) + x - g.ext;
+            const long long gy = ((blk / g.gx) % g.gy) * (long long)(g.by - 2 * g.ext) + y - g.ext;
+#pragma unroll
+            for (int q = 0; q < NV; ++q) xyin[q] = gx0 + q >= 0 && gx0 + q < g.nx && gy >= 0 && gy < g.ny;
+            gz0 = (blk / ((long long)g.gx * g.gy)) * (long long)(g.bz - 2 * g.ext) - g.ext;
+        }
+
         Vec<NV> D = load_vec<NV>(ub + (k0 == 0 ? off_d0 : (long long)(k0 - 1) * PXY));
         Vec<NV> Cc = load_vec<NV>(ub + (long long)k0 * PXY);
 #pragma unroll 2
@@ -213,6 +240,7 @@ sweep3d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
                     acc = add_rn(acc, mul_rn(r, r));
                 }
                 if (op_stores(OP)) o.v[q] = mul_rn(s, c6);
+                if (op_ext(OP) && !(xyin[q] && gz0 + k >= 0 && gz0 + k < g.nz)) o.v[q] = Cc.v[q];
             }
             if (op_stores(OP)) store_vec<NV>(ob + po, o);
             D = Cc;
@@ -318,6 +346,43 @@ halo_kernel(double* __restrict__ u, double* __restrict__ send, const JacGeom g,
             if (UNPACK) *c1 = buf[e + 1]; else buf[e + 1] = *c1;
         }
     }
+}
+
+// Wide exchange, one axis per launch: the strip of a face is h layers along `axis` (interior
+// layers for pack, ghost layers for unpack) over the whole padded extent (-h .. b + h) of the other
+// axes, so edge and corner data delivered by the launches of earlier axes travels on.  Element e
+// of a wide face, source memory order (wx = bx + 2h, wy = by + 2h, wz = bz + 2h or 1):
+//   x face: e = (k*wy + j)*h + c      y face: e = (k*h + r)*wx + i      z face: e = (p*wy + j)*wx + i
+// One thread per element; `slots` threads (whole warps) per (block, side) pair.
+template <bool UNPACK>
+__global__ void __launch_bounds__(256)
+halo_wide_kernel(double* __restrict__ arr, double* __restrict__ send, const JacGeom g, const int axis,
+                 const int slots)
+{
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long pr = t / slots;
+    if (pr >= 2 * g.nblocks) return;
+    const long long e = t - pr * slots;
+    const long long blk = pr >> 1;
+    const int face = 2 * axis + (int)(pr & 1);
+    if (e >= g.wface_elems[face]) return;
+    const long long nb = neighbour_block(g, blk, face);
+    if (nb < 0) return;
+    const int h = g.h, hz = g.ndim == 3 ? g.h : 0;
+    const int wx = g.bx + 2 * h, wy = g.by + 2 * h;
+    const int ext = axis == 0 ? g.bx : (axis == 1 ? g.by : g.bz);
+    const int lo = UNPACK ? ((face & 1) ? ext : -h) : ((face & 1) ? ext - h : 0);
+    long long x, y, z;
+    if (axis == 0) {
+        x = e % h + lo; const long long q = e / h; y = q % wy - h; z = q / wy - hz;
+    } else if (axis == 1) {
+        x = e % wx - h; const long long q = e / wx; y = q % h + lo; z = q / h - hz;
+    } else {
+        x = e % wx - h; const long long q = e / wx; y = q % wy - h; z = q / wy + lo;
+    }
+    double* cell = arr + blk * g.block_stride + g.origin + z * g.PXY + y * g.PX + x;
+    if (UNPACK) *cell = send[nb * g.send_stride + g.face_off[face ^ 1] + e];
+    else send[blk * g.send_stride + g.face_off[face] + e] = *cell;
 }
 
 // Dirichlet value into the ghost strip of `face` of every block on that domain face, in both

@@ -21,9 +21,9 @@ _PKG = Path(__file__).resolve().parent
 # JAC_LIB selects another build of the same library (e.g. one compiled with different tile sizes)
 LIB_PATH = Path(os.environ["JAC_LIB"]) if os.environ.get("JAC_LIB") else _PKG / "libjac.so"
 
-MODE_FUSED, MODE_PERTASK, MODE_TEMPORAL, MODE_EXCHANGE = 0, 1, 2, 3
+MODE_FUSED, MODE_PERTASK, MODE_TEMPORAL, MODE_EXCHANGE, MODE_WIDE = 0, 1, 2, 3, 4
 MODES = {"fused": MODE_FUSED, "pertask": MODE_PERTASK, "temporal": MODE_TEMPORAL,
-         "exchange": MODE_EXCHANGE}
+         "exchange": MODE_EXCHANGE, "wide": MODE_WIDE}
 
 OK, EINVAL, ENOMEM, ECUDA, ENODEV, ELIMIT = 0, -1, -2, -3, -4, -5
 
@@ -33,7 +33,7 @@ EXPORTS = [
     "jac_get_u_device", "jac_set_boundary", "jac_get_block_padded", "jac_get_halo_buffer",
     "jac_pack_halos", "jac_unpack_halos", "jac_pack_faces", "jac_unpack_faces", "jac_sweep", "jac_residual", "jac_launch_count",
     "jac_last_cuda_error", "jac_strerror", "jac_residual_dense_static", "jac_sweeps_per_launch",
-    "jac_sweep_residual", "jac_solve",
+    "jac_sweep_residual", "jac_solve", "jac_exchange_wide", "jac_get_wide_buffer",
 ]
 
 
@@ -49,7 +49,7 @@ class Layout(C.Structure):
                 ("face_elems", C.c_int64 * 6), ("face_offset", C.c_int64 * 6),
                 ("send_stride", C.c_int64), ("partials", C.c_int64), ("off_u", C.c_int64 * 2),
                 ("off_f", C.c_int64), ("off_send", C.c_int64), ("off_scratch", C.c_int64),
-                ("total_bytes", C.c_int64)]
+                ("total_bytes", C.c_int64), ("wide_face_elems", C.c_int64 * 6)]
 
 
 class JacError(RuntimeError):
@@ -79,6 +79,8 @@ def lib() -> C.CDLL:
         L.jac_set_boundary.argtypes = [vp, C.c_int, C.c_double]
         L.jac_get_block_padded.argtypes = [vp, C.c_int64, vp]
         L.jac_get_halo_buffer.argtypes = [vp, C.c_int64, C.c_int, vp]
+        L.jac_exchange_wide.argtypes = [vp]
+        L.jac_get_wide_buffer.argtypes = [vp, C.c_int64, C.c_int, vp]
         L.jac_pack_halos.argtypes = [vp]
         L.jac_unpack_halos.argtypes = [vp]
         L.jac_pack_faces.argtypes = [vp, C.c_uint]
@@ -301,6 +303,19 @@ class Jacobi:
 
     def unpack_faces(self, face_mask: int):
         self._call("jac_unpack_faces", lib().jac_unpack_faces(self._ctx, int(face_mask)))
+
+    def exchange_wide(self):
+        """All h ghost layers, edges and corners included (contexts created with mode "wide")."""
+        self._call("jac_exchange_wide", lib().jac_exchange_wide(self._ctx))
+
+    def get_wide_buffer(self, blk: int, face: int) -> np.ndarray:
+        h = self.desc.halo
+        dims = [x + 2 * h for x in self.b]
+        dims[face // 2] = h
+        out = np.empty(tuple(reversed(dims)), dtype=np.float64)
+        self._call("jac_get_wide_buffer",
+                   lib().jac_get_wide_buffer(self._ctx, int(blk), int(face), _host_ptr(out)))
+        return out
 
     def sweep(self, nsweeps: int = 1):
         self._call("jac_sweep", lib().jac_sweep(self._ctx, int(nsweeps)))

@@ -51,6 +51,7 @@ def test_strerror(jac):
     dict(n=(12, 8), b=(4, 4), mode=7),
     dict(n=(12, 8), b=(4, 4), tsteps=9),
     dict(n=(12,), b=(4,)),                # ndim 1
+    dict(n=(12, 8), b=(4, 4), halo=2, mode="wide", tsteps=3),   # more sweeps per exchange than ghost layers
 ])
 def test_invalid_descriptors_are_rejected(jac, kw):
     d = jac.make_desc(**kw)
@@ -100,6 +101,24 @@ def test_layout_is_aligned_and_disjoint(jac, n, b, h, has_f):
         assert L.face_elems[fc] == want
         assert L.face_offset[fc] % 16 == 0
     assert L.send_stride >= sum(L.face_elems)
+
+
+@pytest.mark.parametrize("n,b,h", [((12, 8), (3, 2), 2), ((9, 5, 7), (3, 5, 1), 1), ((256, 256), (64, 64), 4),
+                                   ((1024, 1024, 1024), (128, 128, 128), 2)])
+def test_wide_layout_holds_the_wide_faces(jac, n, b, h):
+    ndim = len(n)
+    narrow = jac.get_layout(jac.make_desc(n, b, h, False, "exchange"))
+    L = jac.get_layout(jac.make_desc(n, b, h, False, "wide"))
+    for fc in range(6):
+        axis = fc // 2
+        want = 0 if axis >= ndim else h * int(np.prod([b[a] + 2 * h for a in range(ndim) if a != axis]))
+        assert L.wide_face_elems[fc] == want == narrow.wide_face_elems[fc]
+        assert L.face_elems[fc] == narrow.face_elems[fc]       # the plain faces are what they were
+        assert L.face_offset[fc] % 16 == 0
+        if fc < 2 * ndim - 1:
+            assert L.face_offset[fc + 1] - L.face_offset[fc] >= L.wide_face_elems[fc]
+    assert L.send_stride >= sum(L.wide_face_elems) and L.send_stride >= narrow.send_stride
+    assert L.off_scratch - L.off_send >= L.nblocks * L.send_stride * 8
 
 
 def test_footprints_of_the_named_configs(jac):
