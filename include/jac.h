@@ -68,6 +68,15 @@ extern "C" {
                                tsteps - 1 layers down to the interior, so neighbours are computed
                                redundantly instead of being exchanged.  2 * ndim + tsteps launches
                                per group                                                         */
+#define JAC_MODE_RESIDENT 5 /* small 2D grids: all sweeps of a jac_sweep call in ONE launch of one
+                               thread-block cluster (8 or 16 CTAs) that keeps the whole grid in
+                               shared memory, slabs of rows per CTA, neighbouring slabs exchanging
+                               their edge rows through distributed shared memory, one cluster
+                               barrier per sweep.  Needs ndim == 2, b[0] % 2 == 0 and
+                               (2*(r+2) + (has_f ? r : 0)) * (n[0]+4) * 8 bytes <= 227 KB for
+                               r = ceil(n[1]/8) or ceil(n[1]/16) (e.g. 256 x 256 with f);
+                               JAC_EINVAL otherwise, also when the device cannot co-schedule a
+                               cluster of that size                                              */
 
 typedef struct jac_ctx jac_ctx; /* opaque, host memory, owned by the library */
 

@@ -11,6 +11,7 @@
 #include "jac.h"
 #include "jac_geom.h"
 #include "jac_kernels.cuh"
+#include "jac_resident.cuh"
 
 namespace {
 
@@ -103,6 +104,30 @@ TemporalGrid temporal_grid_3d(const JacGeom& g, int T)
     return t;
 }
 
+// The resident schedule: the grid is cut into one slab of rows per CTA of a single cluster; 8 CTAs
+// if the slabs then fit the shared memory of an SM, else 16 (pure host arithmetic).
+struct ResidentPlan {
+    int cluster, rows;
+    size_t smem;
+};
+constexpr size_t kMaxSmemPerCta = 227 * 1024;
+
+int plan_resident(const JacGeom& g, bool has_f, ResidentPlan* p)
+{
+    if (g.ndim != 2 || g.bx % 2 != 0 || g.nx >= (1LL << 24) || g.ny >= (1LL << 24)) return JAC_EINVAL;
+    for (int cl = 8; cl <= 16; cl *= 2) {
+        const int rows = (int)ceil_div(g.ny, cl);
+        const size_t smem = jac::resident_smem_bytes(g.nx, rows, has_f);
+        if (smem <= kMaxSmemPerCta) {
+            p->cluster = cl;
+            p->rows = rows;
+            p->smem = smem;
+            return JAC_OK;
+        }
+    }
+    return JAC_EINVAL;
+}
+
 // largest number of partial sums any launch of this geometry can write
 long long max_partials(const JacGeom& g, long long sweep_ctas)
 {
@@ -118,7 +143,7 @@ int build_geometry(const jac_desc* d, JacGeom* g, jac_layout* L)
     if (d->ndim != 2 && d->ndim != 3) return JAC_EINVAL;
     if (d->halo < 1 || d->halo > 8) return JAC_EINVAL;
     if (d->has_f != 0 && d->has_f != 1) return JAC_EINVAL;
-    if (d->mode < JAC_MODE_FUSED || d->mode > JAC_MODE_WIDE) return JAC_EINVAL;
+    if (d->mode < JAC_MODE_FUSED || d->mode > JAC_MODE_RESIDENT) return JAC_EINVAL;
     if (d->tsteps < 0 || d->tsteps > 8 || d->reserved != 0) return JAC_EINVAL;
     long long n[3] = {1, 1, 1}, b[3] = {1, 1, 1}, gr[3] = {1, 1, 1};
     for (int a = 0; a < d->ndim; ++a) {
@@ -164,6 +189,10 @@ int build_geometry(const jac_desc* d, JacGeom* g, jac_layout* L)
     }
     g->send_stride = off;
 
+    if (d->mode == JAC_MODE_RESIDENT) {
+        ResidentPlan rp;
+        if (plan_resident(*g, d->has_f != 0, &rp)) return JAC_EINVAL;   // 3D, odd bx, or too large
+    }
     const Tiling t = make_tiling(*g);
     const long long ctas = g->nblocks * t.ctas_per_block;
     if (ctas > kMaxGrid) return JAC_EINVAL;
@@ -535,6 +564,65 @@ int launch_temporal_n(jac_ctx* c, int t, const double* u, double* un, bool res, 
     }
 }
 
+// nsweeps sweeps in ONE launch of one thread-block cluster that keeps the grid in shared memory
+template <bool HAS_F>
+int launch_resident_t(jac_ctx* c, const ResidentPlan& rp, const double* u, double* un, int nsweeps)
+{
+    auto kern = jac::resident2d_kernel<HAS_F>;
+    JAC_CK(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rp.smem));
+    if (rp.cluster > 8) JAC_CK(c, cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)rp.cluster, 1, 1);
+    cfg.blockDim = dim3(jac::kResThreads, 1, 1);
+    cfg.dynamicSmemBytes = rp.smem;
+    cfg.stream = c->stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)rp.cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    JAC_CK(c, cudaLaunchKernelEx(&cfg, kern, u, un, (const double*)c->f, c->g, nsweeps, rp.rows));
+    return check_launch(c);
+}
+
+int launch_resident(jac_ctx* c, const double* u, double* un, int nsweeps)
+{
+    ResidentPlan rp;
+    if (plan_resident(c->g, c->desc.has_f != 0, &rp)) return JAC_EINVAL;
+    return c->desc.has_f ? launch_resident_t<true>(c, rp, u, un, nsweeps)
+                         : launch_resident_t<false>(c, rp, u, un, nsweeps);
+}
+
+// can a cluster of the planned size be scheduled on this device at all? (16 CTAs with most of an
+// SM's shared memory each need a GPC with 16 free SMs)
+int check_resident_fits_device(jac_ctx* c)
+{
+    ResidentPlan rp;
+    if (plan_resident(c->g, c->desc.has_f != 0, &rp)) return JAC_EINVAL;
+    const void* kern = c->desc.has_f ? (const void*)jac::resident2d_kernel<true>
+                                     : (const void*)jac::resident2d_kernel<false>;
+    JAC_CK(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rp.smem));
+    if (rp.cluster > 8) JAC_CK(c, cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)rp.cluster, 1, 1);
+    cfg.blockDim = dim3(jac::kResThreads, 1, 1);
+    cfg.dynamicSmemBytes = rp.smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)rp.cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int nclusters = 0;
+    JAC_CK(c, cudaOccupancyMaxActiveClusters(&nclusters, kern, &cfg));
+    return nclusters >= 1 ? JAC_OK : JAC_EINVAL;
+}
+
 // nsweeps iterations in the context's schedule.  With `res`, the last sweep also leaves partial
 // sums of the squared residual of the state it reads in the scratch (*nparts of them).
 int run_sweeps(jac_ctx* c, int nsweeps, bool res, long long* nparts)
@@ -593,6 +681,23 @@ int run_sweeps(jac_ctx* c, int nsweeps, bool res, long long* nparts)
                 if (rc) return rc;
                 c->cur ^= 1;
                 left -= t;
+            }
+            c->ghosts_fresh = false;
+            c->packed_current = false;
+            break;
+        }
+        case JAC_MODE_RESIDENT: {
+            // all sweeps in one launch; a residual-carrying last sweep runs as one ordinary launch
+            const int n_res = res ? nsweeps - 1 : nsweeps;
+            if (n_res > 0) {
+                if ((rc = launch_resident(c, c->u[c->cur], c->u[c->cur ^ 1], n_res))) return rc;
+                c->cur ^= 1;
+            }
+            if (res) {
+                if ((rc = launch_sweep<jac::OP_UPDATE_PULL_RES>(c, c->u[c->cur], c->u[c->cur ^ 1], 0, g.nblocks)))
+                    return rc;
+                c->cur ^= 1;
+                *nparts = sweep_parts;
             }
             c->ghosts_fresh = false;
             c->packed_current = false;
@@ -718,6 +823,10 @@ int jac_create(const jac_desc* desc, void* dev_workspace, size_t bytes, jac_ctx*
     if (e != cudaSuccess) {
         delete c;
         return JAC_ECUDA;
+    }
+    if (desc->mode == JAC_MODE_RESIDENT && (rc = check_resident_fits_device(c))) {
+        delete c;
+        return rc;
     }
     *out = c;
     return JAC_OK;

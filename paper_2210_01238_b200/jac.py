@@ -21,9 +21,9 @@ _PKG = Path(__file__).resolve().parent
 # JAC_LIB selects another build of the same library (e.g. one compiled with different tile sizes)
 LIB_PATH = Path(os.environ["JAC_LIB"]) if os.environ.get("JAC_LIB") else _PKG / "libjac.so"
 
-MODE_FUSED, MODE_PERTASK, MODE_TEMPORAL, MODE_EXCHANGE, MODE_WIDE = 0, 1, 2, 3, 4
+MODE_FUSED, MODE_PERTASK, MODE_TEMPORAL, MODE_EXCHANGE, MODE_WIDE, MODE_RESIDENT = 0, 1, 2, 3, 4, 5
 MODES = {"fused": MODE_FUSED, "pertask": MODE_PERTASK, "temporal": MODE_TEMPORAL,
-         "exchange": MODE_EXCHANGE, "wide": MODE_WIDE}
+         "exchange": MODE_EXCHANGE, "wide": MODE_WIDE, "resident": MODE_RESIDENT}
 
 OK, EINVAL, ENOMEM, ECUDA, ENODEV, ELIMIT = 0, -1, -2, -3, -4, -5
 

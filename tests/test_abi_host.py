@@ -52,6 +52,9 @@ def test_strerror(jac):
     dict(n=(12, 8), b=(4, 4), tsteps=9),
     dict(n=(12,), b=(4,)),                # ndim 1
     dict(n=(12, 8), b=(4, 4), halo=2, mode="wide", tsteps=3),   # more sweeps per exchange than ghost layers
+    dict(n=(12, 8, 8), b=(4, 4, 4), mode="resident"),           # the resident schedule is 2D only,
+    dict(n=(15, 8), b=(5, 4), mode="resident"),                 # wants an even block width
+    dict(n=(1024, 1024), b=(512, 512), mode="resident"),        # and a grid that fits a cluster's shared memory
 ])
 def test_invalid_descriptors_are_rejected(jac, kw):
     d = jac.make_desc(**kw)
@@ -119,6 +122,12 @@ def test_wide_layout_holds_the_wide_faces(jac, n, b, h):
             assert L.face_offset[fc + 1] - L.face_offset[fc] >= L.wide_face_elems[fc]
     assert L.send_stride >= sum(L.wide_face_elems) and L.send_stride >= narrow.send_stride
     assert L.off_scratch - L.off_send >= L.nblocks * L.send_stride * 8
+
+
+def test_resident_schedule_accepts_what_fits_a_cluster(jac):
+    # 256 x 256 with f: slabs of 32 rows in 8 CTAs; 512 x 256 needs 16 CTAs; both are accepted
+    for n, b, f in [((256, 256), (256, 256), True), ((512, 256), (128, 64), False), ((12, 4), (4, 4), True)]:
+        assert jac.workspace_bytes(jac.make_desc(n, b, 1, f, "resident")) > 0
 
 
 def test_footprints_of_the_named_configs(jac):
