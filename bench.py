@@ -61,6 +61,7 @@ KERNEL_NAMES = {("temporal", 2): "temporal2d_kernel", ("temporal", 3): "temporal
                 ("exchange", 2): "sweep2d_kernel", ("pertask", 2): "sweep2d_kernel (one launch per block)",
                 ("fused", 3): "sweep3d_kernel (update pulling neighbour interiors)", ("exchange", 3): "sweep3d_kernel",
                 ("pertask", 3): "sweep3d_kernel (one launch per block)",
+                ("resident", 2): "resident2d_kernel (one cluster, grid in shared memory)",
                 ("wide", 2): "sweep2d_kernel (grown boxes between wide exchanges)",
                 ("wide", 3): "sweep3d_kernel (grown boxes between wide exchanges)"}
 
@@ -215,8 +216,20 @@ def replicated_glups(updates_per_rank: float, world: int, ms: float) -> float:
     return updates_per_rank * world / (ms * 1e-3) / 1e9
 
 
+def resident_fits(w: inputs.Workload) -> bool:
+    """Does the library accept the resident schedule for this grid (pure host query)?"""
+    from paper_2210_01238_b200 import jac
+    try:
+        jac.workspace_bytes(jac.make_desc(w.n, w.b, w.halo, w.has_f, "resident"))
+        return True
+    except jac.JacError:
+        return False
+
+
 def default_schedule(w: inputs.Workload):
     """Fastest schedule the library has for the workload (all schedules give identical bits)."""
+    if resident_fits(w):
+        return "resident", 0          # small 2D grids: all sweeps of a call in one launch
     if (w.ndim == 2 and w.b[0] % 4 == 0) or (w.ndim == 3 and w.b[0] % 2 == 0):
         return "temporal", 0          # 0: the library picks the sweeps per launch
     return "exchange", 1
@@ -295,7 +308,7 @@ def run_ours(args, w: inputs.Workload):
         clocks = sampler.stop() if sampler else None
         ms_total = max_over_ranks(ev0.elapsed_time(ev1))
         sweep_ms = sum(a.elapsed_time(b) for a, b in pairs)
-        n_launch = -(-sweeps // tsteps) if mode == "temporal" else sweeps
+        n_launch = -(-sweeps // tsteps) if mode == "temporal" else (1 if mode == "resident" else sweeps)
         glups = replicated_glups(job_updates(w, sweeps) * steps, world, ms_total)
         return {"glups": glups, "ms_total": ms_total, "launch_ms": sweep_ms / (steps * n_launch),
                 "sweeps_per_launch": sweeps / n_launch, "launches": int(launches), "residual": res,
@@ -306,10 +319,10 @@ def run_ours(args, w: inputs.Workload):
         mode, tsteps = default_schedule(w)
     if mode == "wide":
         tsteps = tsteps or 4
-    elif mode != "temporal":
+    elif mode not in ("temporal", "resident"):      # resident: tsteps is the cluster size (0 = library's)
         tsteps = 1
     J = make_ctx(mode, tsteps)
-    if mode != "wide":
+    if mode not in ("wide", "resident"):
         tsteps = J.sweeps_per_launch()
     main_run = time_schedule(J, mode, tsteps, args.steps, args.warmup, True)
     value = main_run["glups"]
@@ -367,6 +380,8 @@ def run_ours(args, w: inputs.Workload):
     others = {}
     if not args.no_others and world == 1:
         alts = [("exchange", 1), ("fused", 1), ("wide", 4)]   # wide: 4 ghost layers, 4 sweeps per exchange
+        if resident_fits(w):
+            alts += [("resident", 8), ("resident", 16)]   # cluster sizes
         if w.ndim == 2 and w.b[0] % 4 == 0:
             alts += [("temporal", 1), ("temporal", 2), ("temporal", 4), ("temporal", 8)]
         if w.ndim == 3 and w.b[0] % 2 == 0:
@@ -374,10 +389,20 @@ def run_ours(args, w: inputs.Workload):
         for m, t in alts:
             if (m, t) == (mode, tsteps):
                 continue
-            Jo = make_ctx(m, t)
+            if m == "resident":
+                try:
+                    jac.workspace_bytes(jac.make_desc(w.n, w.b, w.halo, w.has_f, m, t))
+                except jac.JacError:
+                    continue      # the grid does not fit a cluster of this size
+            try:
+                Jo = make_ctx(m, t)
+            except jac.JacError:
+                if m == "resident":
+                    continue      # the device cannot co-schedule a cluster of this size
+                raise
             r = time_schedule(Jo, m, t, 2, 1, False)
             Jo.close()
-            others[f"{m}{t if m in ('temporal', 'wide') else ''}"] = {
+            others[f"{m}{t if m in ('temporal', 'wide', 'resident') else ''}"] = {
                 "glups": r["glups"], "effective_gbs": r["glups"] * w.bytes_per_point,
                 "launch_ms": r["launch_ms"], "launches": r["launches"]}
     del u0_dev
@@ -422,7 +447,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3_eigenmode_16384", choices=sorted(inputs.CONFIGS))
-    ap.add_argument("--mode", default="auto", choices=["auto", "fused", "exchange", "pertask", "temporal", "wide"],
+    ap.add_argument("--mode", default="auto", choices=["auto", "fused", "exchange", "pertask", "temporal", "wide", "resident"],
                     help="schedule of jac_sweep; auto = the fastest one the library has for the workload")
     ap.add_argument("--tsteps", type=int, default=0)
     ap.add_argument("--sweeps", type=int, default=0, help="sweeps per step (default: the workload's)")

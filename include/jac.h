@@ -76,7 +76,8 @@ extern "C" {
                                (2*(r+2) + (has_f ? r : 0)) * (n[0]+4) * 8 bytes <= 227 KB for
                                r = ceil(n[1]/8) or ceil(n[1]/16) (e.g. 256 x 256 with f);
                                JAC_EINVAL otherwise, also when the device cannot co-schedule a
-                               cluster of that size                                              */
+                               cluster of that size.  desc.tsteps = 8 or 16 fixes the cluster
+                               size (0: 8 if the slabs fit, else 16)                             */
 
 typedef struct jac_ctx jac_ctx; /* opaque, host memory, owned by the library */
 
@@ -86,7 +87,8 @@ typedef struct jac_desc {
     int32_t has_f;   /* 0: f == 0 and is never read (16 B/point/sweep); 1: f present (24 B)      */
     int32_t mode;    /* JAC_MODE_*                                                               */
     int32_t tsteps;  /* JAC_MODE_TEMPORAL: sweeps per launch; JAC_MODE_WIDE: sweeps per exchange
-                        (<= halo); 0 = the library chooses                                       */
+                        (<= halo); JAC_MODE_RESIDENT: CTAs in the cluster (8 or 16); 0 = the
+                        library chooses                                                          */
     int32_t reserved;/* must be 0                                                                */
     int64_t n[3];    /* global interior points; n[2] ignored (taken as 1) when ndim == 2         */
     int64_t b[3];    /* block interior points; n[a] % b[a] == 0                                  */

@@ -112,10 +112,11 @@ struct ResidentPlan {
 };
 constexpr size_t kMaxSmemPerCta = 227 * 1024;
 
-int plan_resident(const JacGeom& g, bool has_f, ResidentPlan* p)
+int plan_resident(const JacGeom& g, bool has_f, int want_cluster, ResidentPlan* p)
 {
     if (g.ndim != 2 || g.bx % 2 != 0 || g.nx >= (1LL << 24) || g.ny >= (1LL << 24)) return JAC_EINVAL;
-    for (int cl = 8; cl <= 16; cl *= 2) {
+    if (want_cluster != 0 && want_cluster != 8 && want_cluster != 16) return JAC_EINVAL;
+    for (int cl = want_cluster ? want_cluster : 8; cl <= (want_cluster ? want_cluster : 16); cl *= 2) {
         const int rows = (int)ceil_div(g.ny, cl);
         const size_t smem = jac::resident_smem_bytes(g.nx, rows, has_f);
         if (smem <= kMaxSmemPerCta) {
@@ -144,7 +145,7 @@ int build_geometry(const jac_desc* d, JacGeom* g, jac_layout* L)
     if (d->halo < 1 || d->halo > 8) return JAC_EINVAL;
     if (d->has_f != 0 && d->has_f != 1) return JAC_EINVAL;
     if (d->mode < JAC_MODE_FUSED || d->mode > JAC_MODE_RESIDENT) return JAC_EINVAL;
-    if (d->tsteps < 0 || d->tsteps > 8 || d->reserved != 0) return JAC_EINVAL;
+    if (d->tsteps < 0 || d->tsteps > (d->mode == JAC_MODE_RESIDENT ? 16 : 8) || d->reserved != 0) return JAC_EINVAL;
     long long n[3] = {1, 1, 1}, b[3] = {1, 1, 1}, gr[3] = {1, 1, 1};
     for (int a = 0; a < d->ndim; ++a) {
         n[a] = d->n[a];
@@ -191,7 +192,7 @@ int build_geometry(const jac_desc* d, JacGeom* g, jac_layout* L)
 
     if (d->mode == JAC_MODE_RESIDENT) {
         ResidentPlan rp;
-        if (plan_resident(*g, d->has_f != 0, &rp)) return JAC_EINVAL;   // 3D, odd bx, or too large
+        if (plan_resident(*g, d->has_f != 0, d->tsteps, &rp)) return JAC_EINVAL;   // 3D, odd bx, or too large
     }
     const Tiling t = make_tiling(*g);
     const long long ctas = g->nblocks * t.ctas_per_block;
@@ -591,7 +592,7 @@ int launch_resident_t(jac_ctx* c, const ResidentPlan& rp, const double* u, doubl
 int launch_resident(jac_ctx* c, const double* u, double* un, int nsweeps)
 {
     ResidentPlan rp;
-    if (plan_resident(c->g, c->desc.has_f != 0, &rp)) return JAC_EINVAL;
+    if (plan_resident(c->g, c->desc.has_f != 0, c->desc.tsteps, &rp)) return JAC_EINVAL;
     return c->desc.has_f ? launch_resident_t<true>(c, rp, u, un, nsweeps)
                          : launch_resident_t<false>(c, rp, u, un, nsweeps);
 }
@@ -601,7 +602,7 @@ int launch_resident(jac_ctx* c, const double* u, double* un, int nsweeps)
 int check_resident_fits_device(jac_ctx* c)
 {
     ResidentPlan rp;
-    if (plan_resident(c->g, c->desc.has_f != 0, &rp)) return JAC_EINVAL;
+    if (plan_resident(c->g, c->desc.has_f != 0, c->desc.tsteps, &rp)) return JAC_EINVAL;
     const void* kern = c->desc.has_f ? (const void*)jac::resident2d_kernel<true>
                                      : (const void*)jac::resident2d_kernel<false>;
     JAC_CK(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rp.smem));

@@ -6,7 +6,8 @@
 // Here CTA c of the cluster owns a slab of `rows` consecutive grid rows in two shared-memory
 // buffers (plus the slab's right-hand side), sweeps from one buffer into the other, writes its
 // first and last new row straight into the neighbouring CTAs' halo rows through distributed
-// shared memory, and meets the other CTAs at one cluster barrier per sweep.  Global memory is
+// shared memory, and meets the other CTAs at one cluster barrier per sweep (arrive after the edge
+// rows, wait after the inner rows, so the barrier's latency is covered by work).  Global memory is
 // read once before the first sweep and written once after the last.
 //
 // Slab layout (doubles): row pitch RP = nx + 4; grid column i sits at index i + 2 (so pairs of
@@ -24,7 +25,6 @@
 namespace jac {
 
 constexpr int kResThreads = 512;
-constexpr int kResSegRows = 8;      // consecutive rows one thread marches through per work item
 
 __host__ __device__ constexpr long long resident_pitch(long long nx) { return nx + 4; }
 // shared-memory bytes of one CTA whose slab has `rows` rows
@@ -94,13 +94,43 @@ resident2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
     }
     cluster.sync();
 
-    // ---- sweeps: buf[cur] -> buf[cur ^ 1]; work item = (column pair, segment of rows)
-    const int nseg = (mine + kResSegRows - 1) / kResSegRows;
+    // ---- sweeps: A -> B.  The slab's first and last row go first: they are what the neighbours
+    // wait for, and the only rows that read this slab's halo rows.  Once they are written (here and
+    // into the neighbours' halo rows) the CTA arrives at the cluster barrier, computes its inner
+    // rows while the barrier completes, and waits before the next sweep.  The inner rows are
+    // marched through in segments (rows below and above a thread's pair stay in registers).
+    const int nedge = mine >= 2 ? 2 : mine;                   // edge rows: 1 and `mine`
+    const int inner = max(0, mine - 2);                       // rows 2 .. mine - 1
+    const int groups = max(1, kResThreads / max(1, npairs));  // row segments that run side by side
+    const int segrows = max(1, (inner + groups - 1) / groups);
+    const int nseg = (inner + segrows - 1) / segrows;
     double *A = buf[0], *B = buf[1];
     for (int s = 0; s < nsweeps; ++s) {
+        for (int it = tid; it < nedge * npairs; it += kResThreads) {
+            const int which = it / npairs, cp = it - which * npairs;
+            const int l = which == 0 ? 1 : mine;
+            const int col = 2 + 2 * cp;
+            const double2 S = *reinterpret_cast<const double2*>(A + (l - 1) * RP + col);
+            const double2 M = *reinterpret_cast<const double2*>(A + l * RP + col);
+            const double2 N = *reinterpret_cast<const double2*>(A + (l + 1) * RP + col);
+            const double w = A[l * RP + col - 1];
+            const double e = A[l * RP + col + 2];
+            double s0 = add_rn(add_rn(w, M.y), add_rn(S.x, N.x));
+            double s1 = add_rn(add_rn(M.x, e), add_rn(S.y, N.y));
+            if (HAS_F) {
+                const double2 ff = *reinterpret_cast<const double2*>(fs + (l - 1) * RP + col);
+                s0 = add_rn(s0, ff.x);
+                s1 = add_rn(s1, ff.y);
+            }
+            const double2 o = make_double2(mul_rn(s0, 0.25), mul_rn(s1, 0.25));
+            *reinterpret_cast<double2*>(B + l * RP + col) = o;
+            if (l == 1 && has_lo) *reinterpret_cast<double2*>(lo_B + col) = o;
+            if (l == mine && has_hi) *reinterpret_cast<double2*>(hi_B + col) = o;
+        }
+        cluster.barrier_arrive();   // release: this CTA's halo reads and edge-row writes are done
         for (int it = tid; it < nseg * npairs; it += kResThreads) {
             const int seg = it / npairs, cp = it - seg * npairs;
-            const int l0 = 1 + seg * kResSegRows, l1 = min(mine + 1, l0 + kResSegRows);
+            const int l0 = 2 + seg * segrows, l1 = min(mine, l0 + segrows);
             const int col = 2 + 2 * cp;
             double2 S = *reinterpret_cast<const double2*>(A + (l0 - 1) * RP + col);
             double2 M = *reinterpret_cast<const double2*>(A + l0 * RP + col);
@@ -116,15 +146,13 @@ resident2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
                     s0 = add_rn(s0, ff.x);
                     s1 = add_rn(s1, ff.y);
                 }
-                const double2 o = make_double2(mul_rn(s0, 0.25), mul_rn(s1, 0.25));
-                *reinterpret_cast<double2*>(B + l * RP + col) = o;
-                if (l == 1 && has_lo) *reinterpret_cast<double2*>(lo_B + col) = o;
-                if (l == mine && has_hi) *reinterpret_cast<double2*>(hi_B + col) = o;
+                *reinterpret_cast<double2*>(B + l * RP + col) = make_double2(mul_rn(s0, 0.25), mul_rn(s1, 0.25));
                 S = M;
                 M = N;
             }
         }
-        cluster.sync();   // every slab and every halo row of the new state is complete and visible
+        __syncthreads();            // nobody in this CTA still reads A (the next sweep writes it)
+        cluster.barrier_wait();     // acquire: the neighbours' rows have arrived in B's halo rows
         double* t = A; A = B; B = t;
         t = lo_A; lo_A = lo_B; lo_B = t;
         t = hi_A; hi_A = hi_B; hi_B = t;
