@@ -71,17 +71,48 @@ struct TemporalGrid {
     long long ctas;
 };
 
-TemporalGrid temporal_grid_2d(const JacGeom& g, int T)
+// Rows per strip of the 2D temporal kernel.  A strip of R rows costs R + 4T - 1 pipeline steps
+// (2T rows of fill, 2T - 1 of drain); the GPU runs `capacity` strips at a time (148 SMs x CTAs per
+// SM, as the kernel's launch bounds ask for, x warps per CTA); w = strips / capacity.  Strips are
+// handed out dynamically, so a launch of many strips takes about
+//     (R + 4T - 1) x (w + alpha):  all pipeline steps at full occupancy, plus a tail of part of one strip;
+// alpha = 0.7 up to T = 4 and 0.45 beyond, fitted to launches of 2048^2 .. 16384^2 (deep pipelines
+// are bound by issue and suffer less from an idle memory system in the tail).  With fewer than six
+// rounds of strips the rounds count whole: a warp was measured to run no faster on a half-empty
+// SM, so a round that is 3 % full costs as much as a full one.  R is the value in 8..256
+// that minimises this estimate; longer strips were measured slower (512 rows lose 8 % at 16384^2,
+// T = 8).  Measured against the earlier fixed rule (32 rows below 7104 strips): 4096^2 with f,
+// T = 4: 0.107 ms per launch instead of 0.113; 8192^2, T = 4: 0.211 instead of 0.226; 2048^2,
+// T = 8: 0.049 instead of 0.064; 16384^2 unchanged.
+int temporal_rows_2d(const JacGeom& g, int T, bool has_f)
+{
+#ifdef JAC_FORCE_ROWS
+    return JAC_FORCE_ROWS;
+#endif
+    const long long strips_x = ceil_div(g.nx, jac::temporal_strip_cols(T));
+    const int ctas_per_sm = ((T > 4 && jac::temporal_points(T) == 4) || jac::temporal_f_ring(T, has_f)) ? 2 : JAC_TOCC;
+    const double capacity = (double)kNumSMs * ctas_per_sm * jac::kTemporalWarps;
+    const double alpha = T > 4 ? 0.45 : 0.7;
+    int best = 8;
+    double best_cost = 1e300;
+    for (int rows = 8; rows <= 256; ++rows) {
+        if (rows > g.ny && rows > 8) break;
+        const double w = (double)(strips_x * ceil_div(g.ny, rows)) / capacity;
+        const double rounds = w < 6.0 ? std::ceil(w - 1e-9) : w;
+        const double cost = (rows + 4 * T - 1) * (rounds + alpha);
+        if (cost <= best_cost) {   // ties go to the longer strip (less redundant work)
+            best_cost = cost;
+            best = rows;
+        }
+    }
+    return best;
+}
+
+TemporalGrid temporal_grid_2d(const JacGeom& g, int T, bool has_f)
 {
     TemporalGrid t{};
     t.a = (int)ceil_div(g.nx, jac::temporal_strip_cols(T));
-    // strips of 256 rows amortise the 4T - 1 steps of pipeline fill; shorter ones when the grid
-    // would otherwise give fewer than four rounds of resident warps (longer strips were measured
-    // slower at 16384^2: 512 rows lose 8 % at T = 8)
-    int rows = 256;
-    while (rows > 32 && (long long)t.a * ceil_div(g.ny, rows) < (long long)kNumSMs * 48) rows /= 2;
-    // tiny grids: not even one warp per scheduler; shorter strips cut the serial length of a launch
-    while (rows > 8 && (long long)t.a * ceil_div(g.ny, rows) < (long long)kNumSMs * 4) rows /= 2;
+    const int rows = temporal_rows_2d(g, T, has_f);
     t.chunk = rows;
     t.b = (int)ceil_div(g.ny, rows);
     t.c = 1;
@@ -130,10 +161,10 @@ int plan_resident(const JacGeom& g, bool has_f, int want_cluster, ResidentPlan* 
 }
 
 // largest number of partial sums any launch of this geometry can write
-long long max_partials(const JacGeom& g, long long sweep_ctas)
+long long max_partials(const JacGeom& g, long long sweep_ctas, bool has_f)
 {
     long long m = sweep_ctas;
-    if (g.ndim == 2) for (int T = 1; T <= 8; ++T) m = std::max(m, temporal_grid_2d(g, T).warps);
+    if (g.ndim == 2) for (int T = 1; T <= 8; ++T) m = std::max(m, temporal_grid_2d(g, T, has_f).warps);
     else for (int T = 1; T <= 2; ++T) m = std::max(m, temporal_grid_3d(g, T).warps);
     return m;
 }
@@ -217,7 +248,7 @@ int build_geometry(const jac_desc* d, JacGeom* g, jac_layout* L)
         }
         L->send_stride = g->send_stride;
         for (int fc = 0; fc < 6; ++fc) L->wide_face_elems[fc] = g->wface_elems[fc];
-        L->partials = round_up(max_partials(*g, ctas), 32);
+        L->partials = round_up(max_partials(*g, ctas, d->has_f != 0), 32);
         const long long arr_bytes = round_up(g->nblocks * g->block_stride * 8, 256);
         long long o = 0;
         L->off_u[0] = o; o += arr_bytes;
@@ -530,7 +561,7 @@ int launch_temporal3d_n(jac_ctx* c, int t, const double* u, double* un, bool res
 template <int T, bool HAS_F, bool RES>
 int launch_temporal_t(jac_ctx* c, const double* u, double* un, long long* nparts)
 {
-    const TemporalGrid t = temporal_grid_2d(c->g, T);
+    const TemporalGrid t = temporal_grid_2d(c->g, T, HAS_F);
     auto kern = jac::temporal2d_kernel<T, HAS_F, RES>;
     const size_t smem = jac::temporal_smem_bytes(T, HAS_F);
     if (smem > 48 * 1024)
