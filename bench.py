@@ -40,22 +40,26 @@ UNIT = "GLUP/s"
 L2_BYTES = 126e6
 
 # DRAM bytes per launch of the dominant kernel from an ncu capture (profiles/), and the hash of
-# the kernel sources the capture was taken with; reported as null once the sources changed.
+# the sources that define that kernel and its launch geometry at the time of the capture; reported
+# as null once any of them changed.
 # key: (schedule, tsteps, ndim, has_f)
 # bytes_per_point_per_launch: (dram__bytes_read.sum + dram__bytes_write.sum) / points of the captured
 # launch (a smaller case of the same workload, named beside each entry), scaled to the workload by
 # its points -- traffic is proportional to the points: every strip or tile reads and writes its own
 # part of the grid once per launch.
+SWEEP_SOURCES = ("jac_kernels.cuh", "jac_geom.h", "jac.cu")
 NCU_TRAFFIC = {
     # profiles/temporal2d_eigenmode_8192.md
-    ("temporal", 8, 2, False): {"bytes_per_point_per_launch": (625.295616e6 + 491.547136e6) / 8192 ** 2,
-                                "src_sha": "eeb19b9bd151abe8"},
+    ("temporal", 8, 2, False): {"bytes_per_point_per_launch": (592.291840e6 + 492.135680e6) / 8192 ** 2,
+                                "src": SWEEP_SOURCES, "src_sha": "f3ca0801f96a9574"},
+    ("temporal", 4, 2, False): {"bytes_per_point_per_launch": (607.004672e6 + 488.668416e6) / 8192 ** 2,
+                                "src": SWEEP_SOURCES, "src_sha": "f3ca0801f96a9574"},
     # profiles/temporal3d_poisson_512.md
-    ("temporal", 2, 3, True): {"bytes_per_point_per_launch": (2.496113e9 + 1.047960e9) / 512 ** 3,
-                               "src_sha": "eeb19b9bd151abe8"},
+    ("temporal", 2, 3, True): {"bytes_per_point_per_launch": (2.499134e9 + 1.047790e9) / 512 ** 3,
+                               "src": SWEEP_SOURCES, "src_sha": "f3ca0801f96a9574"},
     # profiles/exchange_schedule_eigenmode_8192.md (the update launch alone)
-    ("exchange", 1, 2, False): {"bytes_per_point_per_launch": (574.288384e6 + 494.364160e6) / 8192 ** 2,
-                                "src_sha": "eeb19b9bd151abe8"},
+    ("exchange", 1, 2, False): {"bytes_per_point_per_launch": (574.283008e6 + 496.649216e6) / 8192 ** 2,
+                                "src": SWEEP_SOURCES, "src_sha": "f3ca0801f96a9574"},
 }
 KERNEL_NAMES = {("temporal", 2): "temporal2d_kernel", ("temporal", 3): "temporal3d_kernel", ("fused", 2): "sweep2d_kernel (update pulling neighbour interiors)",
                 ("exchange", 2): "sweep2d_kernel", ("pertask", 2): "sweep2d_kernel (one launch per block)",
@@ -70,10 +74,10 @@ def log(*a):
     print(*a, file=sys.stderr, flush=True)
 
 
-def kernel_src_sha() -> str:
+def kernel_src_sha(names=SWEEP_SOURCES) -> str:
     h = hashlib.sha256()
-    for p in sorted((ROOT / "paper_2210_01238_b200" / "csrc").glob("*")):
-        h.update(p.read_bytes())
+    for name in names:
+        h.update((ROOT / "paper_2210_01238_b200" / "csrc" / name).read_bytes())
     return h.hexdigest()[:16]
 
 
@@ -332,7 +336,7 @@ def run_ours(args, w: inputs.Workload):
     achieved = alg_bytes_per_launch / (main_run["launch_ms"] * 1e-3) / 1e9
     traffic = None
     rec = NCU_TRAFFIC.get((mode, tsteps, w.ndim, w.has_f))
-    if rec and rec["src_sha"] == kernel_src_sha():
+    if rec and rec["src_sha"] == kernel_src_sha(rec["src"]):
         traffic = rec["bytes_per_point_per_launch"] * w.points
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
