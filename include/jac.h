@@ -77,7 +77,8 @@ extern "C" {
                                r = ceil(n[1]/8) or ceil(n[1]/16) (e.g. 256 x 256 with f);
                                JAC_EINVAL otherwise, also when the device cannot co-schedule a
                                cluster of that size.  desc.tsteps = 8 or 16 fixes the cluster
-                               size (0: 8 if the slabs fit, else 16)                             */
+                               size (0: 16 for grids of 128 rows or more, else 8; the other
+                               size if that one does not fit or cannot be scheduled)             */
 
 typedef struct jac_ctx jac_ctx; /* opaque, host memory, owned by the library */
 

@@ -135,8 +135,12 @@ TemporalGrid temporal_grid_3d(const JacGeom& g, int T)
     return t;
 }
 
-// The resident schedule: the grid is cut into one slab of rows per CTA of a single cluster; 8 CTAs
-// if the slabs then fit the shared memory of an SM, else 16 (pure host arithmetic).
+// The resident schedule: the grid is cut into one slab of rows per CTA of a single cluster of 8 or
+// 16 CTAs (pure host arithmetic).  A sweep is bound by the cluster barrier and the edge rows'
+// trip through distributed shared memory, not by arithmetic, but halving the slabs still pays
+// once they have a few rows each (256 rows: 1.17 us per sweep with 16 CTAs, 1.65 us with 8), so
+// grids of 128 rows or more ask for 16 first.  jac_create falls back to the other size when the
+// device cannot co-schedule the first choice.
 struct ResidentPlan {
     int cluster, rows;
     size_t smem;
@@ -147,7 +151,10 @@ int plan_resident(const JacGeom& g, bool has_f, int want_cluster, ResidentPlan* 
 {
     if (g.ndim != 2 || g.bx % 2 != 0 || g.nx >= (1LL << 24) || g.ny >= (1LL << 24)) return JAC_EINVAL;
     if (want_cluster != 0 && want_cluster != 8 && want_cluster != 16) return JAC_EINVAL;
-    for (int cl = want_cluster ? want_cluster : 8; cl <= (want_cluster ? want_cluster : 16); cl *= 2) {
+    const int first = want_cluster ? want_cluster : (g.ny >= 128 ? 16 : 8);
+    const int order[2] = {first, want_cluster ? first : 24 - first};
+    for (int k = 0; k < 2; ++k) {
+        const int cl = order[k];
         const int rows = (int)ceil_div(g.ny, cl);
         const size_t smem = jac::resident_smem_bytes(g.nx, rows, has_f);
         if (smem <= kMaxSmemPerCta) {
@@ -278,6 +285,7 @@ struct jac_ctx {
     bool ghosts_fresh;  // inter-block ghosts of u[cur] equal the neighbours' current faces
     bool packed_current;  // the send buffers hold the faces of the current state
     bool f_ghosts_fresh;  // JAC_MODE_WIDE: the ghost layers of f hold the neighbours' f
+    int res_cluster;      // JAC_MODE_RESIDENT: CTAs per cluster settled at creation
     cudaStream_t stream;
     int device;
     int cuda_err;       // sticky
@@ -623,17 +631,18 @@ int launch_resident_t(jac_ctx* c, const ResidentPlan& rp, const double* u, doubl
 int launch_resident(jac_ctx* c, const double* u, double* un, int nsweeps)
 {
     ResidentPlan rp;
-    if (plan_resident(c->g, c->desc.has_f != 0, c->desc.tsteps, &rp)) return JAC_EINVAL;
+    if (plan_resident(c->g, c->desc.has_f != 0, c->res_cluster, &rp)) return JAC_EINVAL;
     return c->desc.has_f ? launch_resident_t<true>(c, rp, u, un, nsweeps)
                          : launch_resident_t<false>(c, rp, u, un, nsweeps);
 }
 
-// can a cluster of the planned size be scheduled on this device at all? (16 CTAs with most of an
+// can a cluster of `cluster` CTAs be scheduled on this device at all? (16 CTAs with most of an
 // SM's shared memory each need a GPC with 16 free SMs)
-int check_resident_fits_device(jac_ctx* c)
+int resident_cluster_schedulable(jac_ctx* c, int cluster, bool* ok)
 {
     ResidentPlan rp;
-    if (plan_resident(c->g, c->desc.has_f != 0, c->desc.tsteps, &rp)) return JAC_EINVAL;
+    *ok = false;
+    if (plan_resident(c->g, c->desc.has_f != 0, cluster, &rp)) return JAC_OK;   // does not fit shared memory
     const void* kern = c->desc.has_f ? (const void*)jac::resident2d_kernel<true>
                                      : (const void*)jac::resident2d_kernel<false>;
     JAC_CK(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rp.smem));
@@ -652,7 +661,27 @@ int check_resident_fits_device(jac_ctx* c)
     cfg.numAttrs = 1;
     int nclusters = 0;
     JAC_CK(c, cudaOccupancyMaxActiveClusters(&nclusters, kern, &cfg));
-    return nclusters >= 1 ? JAC_OK : JAC_EINVAL;
+    *ok = nclusters >= 1;
+    return JAC_OK;
+}
+
+// settles the cluster size of a resident context: the caller's, or the planner's first choice
+// that the device can schedule
+int choose_resident_cluster(jac_ctx* c)
+{
+    ResidentPlan rp;
+    if (plan_resident(c->g, c->desc.has_f != 0, c->desc.tsteps, &rp)) return JAC_EINVAL;
+    const int tries[2] = {rp.cluster, c->desc.tsteps ? rp.cluster : 24 - rp.cluster};
+    for (int k = 0; k < 2; ++k) {
+        bool ok = false;
+        const int rc = resident_cluster_schedulable(c, tries[k], &ok);
+        if (rc) return rc;
+        if (ok) {
+            c->res_cluster = tries[k];
+            return JAC_OK;
+        }
+    }
+    return JAC_EINVAL;
 }
 
 // nsweeps iterations in the context's schedule.  With `res`, the last sweep also leaves partial
@@ -847,6 +876,7 @@ int jac_create(const jac_desc* desc, void* dev_workspace, size_t bytes, jac_ctx*
     c->ghosts_fresh = false;
     c->packed_current = false;
     c->f_ghosts_fresh = false;
+    c->res_cluster = 0;
     c->stream = static_cast<cudaStream_t>(desc->stream);
     c->device = dev;
     c->cuda_err = 0;
@@ -856,7 +886,7 @@ int jac_create(const jac_desc* desc, void* dev_workspace, size_t bytes, jac_ctx*
         delete c;
         return JAC_ECUDA;
     }
-    if (desc->mode == JAC_MODE_RESIDENT && (rc = check_resident_fits_device(c))) {
+    if (desc->mode == JAC_MODE_RESIDENT && (rc = choose_resident_cluster(c))) {
         delete c;
         return rc;
     }

@@ -99,56 +99,66 @@ resident2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
     // into the neighbours' halo rows) the CTA arrives at the cluster barrier, computes its inner
     // rows while the barrier completes, and waits before the next sweep.  The inner rows are
     // marched through in segments (rows below and above a thread's pair stay in registers).
-    const int nedge = mine >= 2 ? 2 : mine;                   // edge rows: 1 and `mine`
+    // The assignment of work to threads is the same in every sweep, so it is fixed here: a thread
+    // owns the column pairs cp0, cp0 + pw, ... and row group `grp`; group 0 also computes edge row 1
+    // and another group (the same one if there is only one) edge row `mine`.
+    const int pw = min(npairs, kResThreads);                  // column pairs side by side
+    const int groups = max(1, kResThreads / pw);              // row groups side by side
+    const int cp0 = tid % pw, grp = tid / pw;
     const int inner = max(0, mine - 2);                       // rows 2 .. mine - 1
-    const int groups = max(1, kResThreads / max(1, npairs));  // row segments that run side by side
-    const int segrows = max(1, (inner + groups - 1) / groups);
-    const int nseg = (inner + segrows - 1) / segrows;
+    const int segrows = (inner + groups - 1) / groups;
+    const int l0 = 2 + grp * segrows;
+    const int l1 = grp < groups ? min(mine, l0 + segrows) : l0;
+    const bool does_lo = grp == 0 && mine >= 1;
+    const bool does_hi = grp == min(groups, 2) - 1 && mine >= 2;
     double *A = buf[0], *B = buf[1];
     for (int s = 0; s < nsweeps; ++s) {
-        for (int it = tid; it < nedge * npairs; it += kResThreads) {
-            const int which = it / npairs, cp = it - which * npairs;
-            const int l = which == 0 ? 1 : mine;
-            const int col = 2 + 2 * cp;
-            const double2 S = *reinterpret_cast<const double2*>(A + (l - 1) * RP + col);
-            const double2 M = *reinterpret_cast<const double2*>(A + l * RP + col);
-            const double2 N = *reinterpret_cast<const double2*>(A + (l + 1) * RP + col);
-            const double w = A[l * RP + col - 1];
-            const double e = A[l * RP + col + 2];
-            double s0 = add_rn(add_rn(w, M.y), add_rn(S.x, N.x));
-            double s1 = add_rn(add_rn(M.x, e), add_rn(S.y, N.y));
-            if (HAS_F) {
-                const double2 ff = *reinterpret_cast<const double2*>(fs + (l - 1) * RP + col);
-                s0 = add_rn(s0, ff.x);
-                s1 = add_rn(s1, ff.y);
-            }
-            const double2 o = make_double2(mul_rn(s0, 0.25), mul_rn(s1, 0.25));
-            *reinterpret_cast<double2*>(B + l * RP + col) = o;
-            if (l == 1 && has_lo) *reinterpret_cast<double2*>(lo_B + col) = o;
-            if (l == mine && has_hi) *reinterpret_cast<double2*>(hi_B + col) = o;
-        }
-        cluster.barrier_arrive();   // release: this CTA's halo reads and edge-row writes are done
-        for (int it = tid; it < nseg * npairs; it += kResThreads) {
-            const int seg = it / npairs, cp = it - seg * npairs;
-            const int l0 = 2 + seg * segrows, l1 = min(mine, l0 + segrows);
-            const int col = 2 + 2 * cp;
-            double2 S = *reinterpret_cast<const double2*>(A + (l0 - 1) * RP + col);
-            double2 M = *reinterpret_cast<const double2*>(A + l0 * RP + col);
-#pragma unroll 4
-            for (int l = l0; l < l1; ++l) {
-                const double2 N = *reinterpret_cast<const double2*>(A + (l + 1) * RP + col);
-                const double w = A[l * RP + col - 1];
-                const double e = A[l * RP + col + 2];
+#pragma unroll 1
+        for (int side = 0; side < 2; ++side) {
+            if (side == 0 ? !does_lo : !does_hi) continue;
+            const int l = side == 0 ? 1 : mine;
+            for (int cp = cp0; cp < npairs; cp += pw) {
+                const int at = l * RP + 2 + 2 * cp;
+                const double2 S = *reinterpret_cast<const double2*>(A + at - RP);
+                const double2 M = *reinterpret_cast<const double2*>(A + at);
+                const double2 N = *reinterpret_cast<const double2*>(A + at + RP);
+                const double w = A[at - 1];
+                const double e = A[at + 2];
                 double s0 = add_rn(add_rn(w, M.y), add_rn(S.x, N.x));
                 double s1 = add_rn(add_rn(M.x, e), add_rn(S.y, N.y));
                 if (HAS_F) {
-                    const double2 ff = *reinterpret_cast<const double2*>(fs + (l - 1) * RP + col);
+                    const double2 ff = *reinterpret_cast<const double2*>(fs + at - RP);
                     s0 = add_rn(s0, ff.x);
                     s1 = add_rn(s1, ff.y);
                 }
-                *reinterpret_cast<double2*>(B + l * RP + col) = make_double2(mul_rn(s0, 0.25), mul_rn(s1, 0.25));
-                S = M;
-                M = N;
+                const double2 o = make_double2(mul_rn(s0, 0.25), mul_rn(s1, 0.25));
+                *reinterpret_cast<double2*>(B + at) = o;
+                if (l == 1 && has_lo) *reinterpret_cast<double2*>(lo_B + 2 + 2 * cp) = o;
+                if (l == mine && has_hi) *reinterpret_cast<double2*>(hi_B + 2 + 2 * cp) = o;
+            }
+        }
+        cluster.barrier_arrive();   // release: this CTA's halo reads and edge-row writes are done
+        if (l0 < l1) {
+            for (int cp = cp0; cp < npairs; cp += pw) {
+                int at = l0 * RP + 2 + 2 * cp;
+                double2 S = *reinterpret_cast<const double2*>(A + at - RP);
+                double2 M = *reinterpret_cast<const double2*>(A + at);
+#pragma unroll 4
+                for (int l = l0; l < l1; ++l, at += RP) {
+                    const double2 N = *reinterpret_cast<const double2*>(A + at + RP);
+                    const double w = A[at - 1];
+                    const double e = A[at + 2];
+                    double s0 = add_rn(add_rn(w, M.y), add_rn(S.x, N.x));
+                    double s1 = add_rn(add_rn(M.x, e), add_rn(S.y, N.y));
+                    if (HAS_F) {
+                        const double2 ff = *reinterpret_cast<const double2*>(fs + at - RP);
+                        s0 = add_rn(s0, ff.x);
+                        s1 = add_rn(s1, ff.y);
+                    }
+                    *reinterpret_cast<double2*>(B + at) = make_double2(mul_rn(s0, 0.25), mul_rn(s1, 0.25));
+                    S = M;
+                    M = N;
+                }
             }
         }
         __syncthreads();            // nobody in this CTA still reads A (the next sweep writes it)
