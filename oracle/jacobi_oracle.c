@@ -27,6 +27,10 @@
  *            (no edges, no corners).  Packed order = source memory order
  *            restricted to the strip (x fastest, then y, then z).
  *            Faces on the domain boundary are neither packed nor unpacked.
+ *   blocks   g = ceil(n / b) per axis.  When n is not a multiple of b the last block along that
+ *            axis is a remainder block of n - (g-1)*b >= h points; it keeps a full-size padded
+ *            array, its interior in the low corner, its +ghost layers right after its interior.
+ *            (The paper's decomposition is into equal cuboids; remainder blocks are an extension.)
  *   exchange comes before the update in every sweep.
  *   wide     (last part of this file; not in the paper) one exchange of all h ghost layers with
  *            edges and corners, then up to h sweeps on shrinking extents: same bits.
@@ -173,6 +177,19 @@ static void blk_coords(const orc_blocked *s, int64_t blk, int64_t c[3])
     c[2] = blk / (s->g[0] * s->g[1]);
 }
 
+/* interior extent of block `blk`: b, except for the last block along an axis when the grid is
+ * not a multiple of the block size (then the remainder n - (g-1)*b; it still owns a full-size
+ * padded array, its interior is the low corner and its +ghost layers follow the interior) */
+static void blk_extent(const orc_blocked *s, int64_t blk, int64_t e[3])
+{
+    int64_t c[3];
+    blk_coords(s, blk, c);
+    for (int a = 0; a < 3; ++a) {
+        const int64_t left = s->n[a] - c[a] * s->b[a];
+        e[a] = left < s->b[a] ? left : s->b[a];
+    }
+}
+
 /* neighbour block across `face`, or -1 if that side is the domain boundary */
 static int64_t blk_neighbour(const orc_blocked *s, int64_t blk, int face)
 {
@@ -194,8 +211,10 @@ static void fill_boundary_ghosts(orc_blocked *s)
         for (int face = 0; face < 2 * s->ndim; ++face) {
             if (blk_neighbour(s, blk, face) >= 0) continue;
             const int axis = face / 2;
-            int64_t lo[3] = {0, 0, 0}, hi[3] = {s->b[0], s->b[1], s->b[2]};
-            if (face & 1) { lo[axis] = s->b[axis]; hi[axis] = s->b[axis] + s->h; }
+            int64_t ext[3];
+            blk_extent(s, blk, ext);
+            int64_t lo[3] = {0, 0, 0}, hi[3] = {ext[0], ext[1], ext[2]};
+            if (face & 1) { lo[axis] = ext[axis]; hi[axis] = ext[axis] + s->h; }
             else          { lo[axis] = -s->h;      hi[axis] = 0; }
             for (int w = 0; w < 2; ++w) {
                 double *u = blk_u(s, w, blk);
@@ -228,11 +247,16 @@ int orc_blocked_create(int ndim, const int64_t *n, const int64_t *b, int64_t h, 
     for (int a = 0; a < 3; ++a) {
         s->n[a] = (a < ndim) ? n[a] : 1;
         s->b[a] = (a < ndim) ? b[a] : 1;
-        if (s->n[a] < 1 || s->b[a] < 1 || s->n[a] % s->b[a] != 0 || (a < ndim && h > s->b[a])) {
+        if (s->n[a] < 1 || s->b[a] < 1 || s->b[a] > s->n[a] || (a < ndim && h > s->b[a])) {
             free(s);
             return ORC_EINVAL;
         }
-        s->g[a] = s->n[a] / s->b[a];
+        s->g[a] = (s->n[a] + s->b[a] - 1) / s->b[a];
+        /* a remainder block must still be at least h wide: its face strips are h layers */
+        if (a < ndim && s->n[a] - (s->g[a] - 1) * s->b[a] < h) {
+            free(s);
+            return ORC_EINVAL;
+        }
         s->p[a] = (a < ndim) ? s->b[a] + 2 * h : 1;
         s->nblocks *= s->g[a];
     }
@@ -269,11 +293,12 @@ static void scatter_dense(const orc_blocked *s, const double *dense, double *dst
 {
 #pragma omp parallel for schedule(static)
     for (int64_t blk = 0; blk < s->nblocks; ++blk) {
-        int64_t c[3];
+        int64_t c[3], ext[3];
         blk_coords(s, blk, c);
-        for (int64_t k = 0; k < s->b[2]; ++k)
-            for (int64_t j = 0; j < s->b[1]; ++j)
-                for (int64_t i = 0; i < s->b[0]; ++i) {
+        blk_extent(s, blk, ext);
+        for (int64_t k = 0; k < ext[2]; ++k)
+            for (int64_t j = 0; j < ext[1]; ++j)
+                for (int64_t i = 0; i < ext[0]; ++i) {
                     const int64_t gi = c[0] * s->b[0] + i, gj = c[1] * s->b[1] + j,
                                   gk = c[2] * s->b[2] + k;
                     const double v = dense[(gk * s->n[1] + gj) * s->n[0] + gi];
@@ -302,12 +327,13 @@ int orc_blocked_get_u(const orc_blocked *s, double *dense)
     if (!s || !dense) return ORC_EINVAL;
 #pragma omp parallel for schedule(static)
     for (int64_t blk = 0; blk < s->nblocks; ++blk) {
-        int64_t c[3];
+        int64_t c[3], ext[3];
         blk_coords(s, blk, c);
+        blk_extent(s, blk, ext);
         const double *u = blk_u(s, s->cur, blk);
-        for (int64_t k = 0; k < s->b[2]; ++k)
-            for (int64_t j = 0; j < s->b[1]; ++j)
-                for (int64_t i = 0; i < s->b[0]; ++i) {
+        for (int64_t k = 0; k < ext[2]; ++k)
+            for (int64_t j = 0; j < ext[1]; ++j)
+                for (int64_t i = 0; i < ext[0]; ++i) {
                     const int64_t gi = c[0] * s->b[0] + i, gj = c[1] * s->b[1] + j,
                                   gk = c[2] * s->b[2] + k;
                     dense[(gk * s->n[1] + gj) * s->n[0] + gi] = u[pad_index(s, i, j, k)];
@@ -324,23 +350,35 @@ int orc_blocked_get_block_padded(const orc_blocked *s, int64_t blk, double *out)
     return ORC_OK;
 }
 
+/* elements of the packed face of (block, face): h layers times the block's extent on the other axes */
+int64_t orc_blocked_face_elems(const orc_blocked *s, int64_t blk, int face)
+{
+    if (!s || blk < 0 || blk >= s->nblocks || face < 0 || face >= 2 * s->ndim) return ORC_EINVAL;
+    int64_t e[3];
+    blk_extent(s, blk, e);
+    e[face / 2] = s->h;
+    return e[0] * e[1] * e[2];
+}
+
 /* the packed send buffer of (block, face) as left by the last pack */
 int orc_blocked_get_halo_buffer(const orc_blocked *s, int64_t blk, int face, double *out)
 {
     if (!s || !out || blk < 0 || blk >= s->nblocks || face < 0 || face >= 2 * s->ndim)
         return ORC_EINVAL;
-    memcpy(out, blk_send(s, blk, face), (size_t)s->face_elems[face] * sizeof(double));
+    memcpy(out, blk_send(s, blk, face), (size_t)orc_blocked_face_elems(s, blk, face) * sizeof(double));
     return ORC_OK;
 }
 
 /* interior-relative index range of the h-wide strip on `face`:
  * ghost == 0: the interior layers next to the face; ghost == 1: the ghost layers */
-static void strip_range(const orc_blocked *s, int face, int ghost, int64_t lo[3], int64_t hi[3])
+static void strip_range(const orc_blocked *s, int64_t blk, int face, int ghost, int64_t lo[3], int64_t hi[3])
 {
     const int axis = face / 2;
-    for (int a = 0; a < 3; ++a) { lo[a] = 0; hi[a] = s->b[a]; }
+    int64_t ext[3];
+    blk_extent(s, blk, ext);
+    for (int a = 0; a < 3; ++a) { lo[a] = 0; hi[a] = ext[a]; }
     if (face & 1) {
-        lo[axis] = ghost ? s->b[axis] : s->b[axis] - s->h;
+        lo[axis] = ghost ? ext[axis] : ext[axis] - s->h;
         hi[axis] = lo[axis] + s->h;
     } else {
         lo[axis] = ghost ? -s->h : 0;
@@ -358,7 +396,7 @@ int orc_blocked_pack(orc_blocked *s)
         for (int face = 0; face < 2 * s->ndim; ++face) {
             if (blk_neighbour(s, blk, face) < 0) continue;
             int64_t lo[3], hi[3];
-            strip_range(s, face, 0, lo, hi);
+            strip_range(s, blk, face, 0, lo, hi);
             double *buf = blk_send(s, blk, face);
             int64_t q = 0;
             for (int64_t k = lo[2]; k < hi[2]; ++k)
@@ -382,7 +420,7 @@ int orc_blocked_unpack(orc_blocked *s)
             const int64_t nb = blk_neighbour(s, blk, face);
             if (nb < 0) continue;
             int64_t lo[3], hi[3];
-            strip_range(s, face, 1, lo, hi);
+            strip_range(s, blk, face, 1, lo, hi);
             const double *buf = blk_send(s, nb, face ^ 1);
             int64_t q = 0;
             for (int64_t k = lo[2]; k < hi[2]; ++k)
@@ -405,9 +443,11 @@ int orc_blocked_update(orc_blocked *s)
         const double *u = blk_u(s, s->cur, blk);
         double *o = blk_u(s, s->cur ^ 1, blk);
         const double *f = s->f ? s->f + blk * s->blk_elems : NULL;
-        for (int64_t k = 0; k < s->b[2]; ++k)
-            for (int64_t j = 0; j < s->b[1]; ++j)
-                for (int64_t i = 0; i < s->b[0]; ++i) {
+        int64_t ext[3];
+        blk_extent(s, blk, ext);
+        for (int64_t k = 0; k < ext[2]; ++k)
+            for (int64_t j = 0; j < ext[1]; ++j)
+                for (int64_t i = 0; i < ext[0]; ++i) {
                     const int64_t p = pad_index(s, i, j, k);
                     double sum = (u[p - 1] + u[p + 1]) + (u[p - px] + u[p + px]);
                     if (s->ndim == 3) sum = sum + (u[p - pxy] + u[p + pxy]);
@@ -443,9 +483,11 @@ int orc_blocked_residual(orc_blocked *s, double *out_l2)
         const double *u = blk_u(s, s->cur, blk);
         const double *f = s->f ? s->f + blk * s->blk_elems : NULL;
         long double acc = 0.0L;
-        for (int64_t k = 0; k < s->b[2]; ++k)
-            for (int64_t j = 0; j < s->b[1]; ++j)
-                for (int64_t i = 0; i < s->b[0]; ++i) {
+        int64_t ext[3];
+        blk_extent(s, blk, ext);
+        for (int64_t k = 0; k < ext[2]; ++k)
+            for (int64_t j = 0; j < ext[1]; ++j)
+                for (int64_t i = 0; i < ext[0]; ++i) {
                     const int64_t p = pad_index(s, i, j, k);
                     double sum = (u[p - 1] + u[p + 1]) + (u[p - px] + u[p + px]);
                     if (s->ndim == 3) sum = sum + (u[p - pxy] + u[p + pxy]);
@@ -484,19 +526,19 @@ int orc_blocked_residual(orc_blocked *s, double *out_l2)
 
 /* index range of the wide strip on `face`: h layers along the face's axis (interior layers if
  * ghost == 0, ghost layers if ghost == 1), the whole padded extent along the other axes */
-static void wide_strip_range(const orc_blocked *s, int face, int ghost, int64_t lo[3], int64_t hi[3])
+static void wide_strip_range(const orc_blocked *s, int64_t blk, int face, int ghost, int64_t lo[3], int64_t hi[3])
 {
-    strip_range(s, face, ghost, lo, hi);
+    strip_range(s, blk, face, ghost, lo, hi);
     const int axis = face / 2;
     for (int a = 0; a < s->ndim; ++a)
-        if (a != axis) { lo[a] = -s->h; hi[a] = s->b[a] + s->h; }
+        if (a != axis) { lo[a] = -s->h; hi[a] = hi[a] + s->h; }
 }
 
-int64_t orc_blocked_wide_face_elems(const orc_blocked *s, int face)
+int64_t orc_blocked_wide_face_elems(const orc_blocked *s, int64_t blk, int face)
 {
-    if (!s || face < 0 || face >= 2 * s->ndim) return ORC_EINVAL;
+    if (!s || blk < 0 || blk >= s->nblocks || face < 0 || face >= 2 * s->ndim) return ORC_EINVAL;
     int64_t lo[3], hi[3];
-    wide_strip_range(s, face, 0, lo, hi);
+    wide_strip_range(s, blk, face, 0, lo, hi);
     return (hi[0] - lo[0]) * (hi[1] - lo[1]) * (hi[2] - lo[2]);
 }
 
@@ -504,7 +546,7 @@ static int64_t wide_max_face(const orc_blocked *s)
 {
     int64_t m = 0;
     for (int fc = 0; fc < 2 * s->ndim; ++fc) {
-        const int64_t e = orc_blocked_wide_face_elems(s, fc);
+        const int64_t e = orc_blocked_wide_face_elems(s, 0, fc);   /* block 0 is never a remainder block unless it is the only one */
         if (e > m) m = e;
     }
     return m;
@@ -520,7 +562,7 @@ static void wide_phase(const orc_blocked *s, double *arr, double *wsend, int64_t
         for (int face = 2 * axis; face < 2 * axis + 2; ++face) {
             if (blk_neighbour(s, blk, face) < 0) continue;
             int64_t lo[3], hi[3];
-            wide_strip_range(s, face, 0, lo, hi);
+            wide_strip_range(s, blk, face, 0, lo, hi);
             double *buf = wsend + (blk * 6 + face) * wmax;
             int64_t q = 0;
             for (int64_t k = lo[2]; k < hi[2]; ++k)
@@ -535,7 +577,7 @@ static void wide_phase(const orc_blocked *s, double *arr, double *wsend, int64_t
             const int64_t nb = blk_neighbour(s, blk, face);
             if (nb < 0) continue;
             int64_t lo[3], hi[3];
-            wide_strip_range(s, face, 1, lo, hi);
+            wide_strip_range(s, blk, face, 1, lo, hi);
             const double *buf = wsend + (nb * 6 + (face ^ 1)) * wmax;
             int64_t q = 0;
             for (int64_t k = lo[2]; k < hi[2]; ++k)
@@ -593,11 +635,12 @@ int orc_blocked_update_ext(orc_blocked *s, int64_t e)
     for (int64_t blk = 0; blk < s->nblocks; ++blk) {
         const double *u = blk_u(s, s->cur, blk);
         double *o = blk_u(s, s->cur ^ 1, blk);
-        int64_t c[3];
+        int64_t c[3], ext[3];
         blk_coords(s, blk, c);
-        for (int64_t k = -ez; k < s->b[2] + ez; ++k)
-            for (int64_t j = -e; j < s->b[1] + e; ++j)
-                for (int64_t i = -e; i < s->b[0] + e; ++i) {
+        blk_extent(s, blk, ext);
+        for (int64_t k = -ez; k < ext[2] + ez; ++k)
+            for (int64_t j = -e; j < ext[1] + e; ++j)
+                for (int64_t i = -e; i < ext[0] + e; ++i) {
                     const int64_t p = pad_index(s, i, j, k);
                     const int64_t gi = c[0] * s->b[0] + i, gj = c[1] * s->b[1] + j,
                                   gk = c[2] * s->b[2] + k;

@@ -69,7 +69,9 @@ def lib() -> C.CDLL:
         L.orc_blocked_exchange_wide.argtypes = [C.c_void_p, _f64p]
         L.orc_blocked_update_ext.argtypes = [C.c_void_p, C.c_int64]
         L.orc_blocked_sweep_wide.argtypes = [C.c_void_p, C.c_int64, C.c_int64]
-        L.orc_blocked_wide_face_elems.argtypes = [C.c_void_p, C.c_int]
+        L.orc_blocked_wide_face_elems.argtypes = [C.c_void_p, C.c_int64, C.c_int]
+        L.orc_blocked_face_elems.argtypes = [C.c_void_p, C.c_int64, C.c_int]
+        L.orc_blocked_face_elems.restype = C.c_int64
         L.orc_blocked_wide_face_elems.restype = C.c_int64
         L.orc_blocked_wide_max_face.argtypes = [C.c_void_p]
         L.orc_blocked_wide_max_face.restype = C.c_int64
@@ -172,7 +174,7 @@ class Blocked:
         self._p = C.c_void_p()
         _check(lib().orc_blocked_create(self.ndim, _dims(n, self.ndim), _dims(b, self.ndim),
                                         self.h, int(has_f), C.byref(self._p)), "create")
-        self.g = [nn // bb for nn, bb in zip(self.n, self.b)]
+        self.g = [-(-nn // bb) for nn, bb in zip(self.n, self.b)]
         self.nblocks = int(np.prod(self.g))
 
     def close(self):
@@ -192,9 +194,18 @@ class Blocked:
     def padded_shape(self):
         return tuple(x + 2 * self.h for x in reversed(self.b))
 
-    def face_shape(self, face: int):
-        """numpy shape of a packed face: (bz, by, h) for x, (bz, h, bx) for y, (h, by, bx) for z (2D drops bz)."""
-        dims = list(self.b)
+    def coords(self, blk: int):
+        g = self.g + [1] * (3 - self.ndim)
+        return [blk % g[0], (blk // g[0]) % g[1], blk // (g[0] * g[1])][: self.ndim]
+
+    def extent(self, blk: int):
+        """Interior points of block ``blk`` per axis: b, or the remainder for the last block of an axis."""
+        return [min(bb, nn - c * bb) for nn, bb, c in zip(self.n, self.b, self.coords(blk))]
+
+    def face_shape(self, face: int, blk: int = 0):
+        """numpy shape of a packed face: (ez, ey, h) for x, (ez, h, ex) for y, (h, ey, ex) for z (2D drops z),
+        e = the block's interior extent."""
+        dims = self.extent(blk)
         dims[face // 2] = self.h
         return tuple(reversed(dims))
 
@@ -222,7 +233,8 @@ class Blocked:
         return out
 
     def get_halo_buffer(self, blk: int, face: int) -> np.ndarray:
-        out = np.empty(self.face_shape(face), dtype=np.float64)
+        out = np.empty(self.face_shape(face, blk), dtype=np.float64)
+        assert out.size == int(lib().orc_blocked_face_elems(self._p, blk, face))
         _check(lib().orc_blocked_get_halo_buffer(self._p, blk, face, _ptr(out)), "get_halo_buffer")
         return out
 
@@ -244,9 +256,9 @@ class Blocked:
         return out.value
 
     # ---- wide exchange: all h ghost layers including edges and corners, axis by axis
-    def wide_face_shape(self, face: int):
-        """numpy shape of a packed wide face: h layers along the face's axis, b + 2h along the others."""
-        dims = [x + 2 * self.h for x in self.b]
+    def wide_face_shape(self, face: int, blk: int = 0):
+        """numpy shape of a packed wide face: h layers along the face's axis, extent + 2h along the others."""
+        dims = [x + 2 * self.h for x in self.extent(blk)]
         dims[face // 2] = self.h
         return tuple(reversed(dims))
 
@@ -263,8 +275,8 @@ class Blocked:
             for face in range(2 * self.ndim):
                 if self.neighbour(blk, face) < 0:
                     continue
-                shp = self.wide_face_shape(face)
-                ne = int(lib().orc_blocked_wide_face_elems(self._p, face))
+                shp = self.wide_face_shape(face, blk)
+                ne = int(lib().orc_blocked_wide_face_elems(self._p, blk, face))
                 assert ne == int(np.prod(shp))
                 out[(blk, face)] = raw[blk, face, :ne].reshape(shp).copy()
         return out

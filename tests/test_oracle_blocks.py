@@ -126,8 +126,9 @@ def test_pack_then_unpack_is_idempotent(orc):
 
 
 def test_create_rejects_bad_shapes(orc):
-    for n, b, h in [((12, 8), (5, 4), 1), ((12, 8), (4, 4), 0), ((12, 8), (4, 4), 5),
-                    ((12, 8), (0, 4), 1)]:
+    # a remainder block narrower than the halo (13 = 3 * 4 + 1 < 2), h = 0, h > b, b = 0, b > n
+    for n, b, h in [((13, 8), (4, 4), 2), ((12, 8), (4, 4), 0), ((12, 8), (4, 4), 5),
+                    ((12, 8), (0, 4), 1), ((12, 8), (16, 4), 1)]:
         with pytest.raises(ValueError):
             orc.Blocked(n, b, h)
 

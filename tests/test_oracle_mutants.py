@@ -32,8 +32,8 @@ MUTANTS = {
                               "        orc_blocked_update(s);",
                               "        orc_blocked_update(s);\n        orc_blocked_pack(s);\n"
                               "        orc_blocked_unpack(s);", 1),
-    "wide_strips_leave_out_the_ghost_extent": ("if (a != axis) { lo[a] = -s->h; hi[a] = s->b[a] + s->h; }",
-                                               "if (a != axis) { lo[a] = 0; hi[a] = s->b[a]; }", 1),
+    "wide_strips_leave_out_the_ghost_extent": ("if (a != axis) { lo[a] = -s->h; hi[a] = hi[a] + s->h; }",
+                                               "if (a != axis) { lo[a] = 0; }", 1),
     "group_updates_do_not_shrink": ("orc_blocked_update_ext(s, t - m);", "orc_blocked_update_ext(s, 0);", 1),
     "extended_update_moves_dirichlet_cells": ("                        o[p] = u[p];\n                        continue;\n",
                                               "", 1),
@@ -42,6 +42,14 @@ MUTANTS = {
     "wide_unpack_reads_same_side": ("wsend + (nb * 6 + (face ^ 1)) * wmax", "wsend + (nb * 6 + face) * wmax", 1),
     "wide_exchange_skips_last_axis": ("for (int axis = 0; axis < s->ndim; ++axis)\n        wide_phase",
                                       "for (int axis = 0; axis + 1 < s->ndim; ++axis)\n        wide_phase", 1),
+    "dirichlet_of_remainder_block_at_full_size_position": (
+        "if (face & 1) { lo[axis] = ext[axis]; hi[axis] = ext[axis] + s->h; }",
+        "if (face & 1) { lo[axis] = s->b[axis]; hi[axis] = s->b[axis] + s->h; }", 1),
+    "update_runs_over_the_full_block_size": (
+        "        for (int64_t k = 0; k < ext[2]; ++k)\n            for (int64_t j = 0; j < ext[1]; ++j)\n"
+        "                for (int64_t i = 0; i < ext[0]; ++i) {\n                    const int64_t p = pad_index(s, i, j, k);",
+        "        for (int64_t k = 0; k < s->b[2]; ++k)\n            for (int64_t j = 0; j < s->b[1]; ++j)\n"
+        "                for (int64_t i = 0; i < s->b[0]; ++i) {\n                    const int64_t p = pad_index(s, i, j, k);", 1),
 }
 
 
@@ -61,7 +69,8 @@ def test_planted_mistake_is_caught(name, tmp_path):
     r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider",
                         str(ROOT / "tests" / "test_oracle_sweep.py"),
                         str(ROOT / "tests" / "test_oracle_blocks.py"),
-                        str(ROOT / "tests" / "test_oracle_wide.py")],
+                        str(ROOT / "tests" / "test_oracle_wide.py"),
+                        str(ROOT / "tests" / "test_oracle_remainder.py")],
                        cwd=ROOT, env=env, capture_output=True, text=True)
     assert r.returncode == 1, f"mutant {name} survived the pins:\n{r.stdout[-2000:]}"
     assert "failed" in r.stdout
