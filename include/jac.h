@@ -18,7 +18,12 @@
  * Conventions
  *   - x is the fastest-varying axis, then y, then z.  "Dense" arrays are n[0]*n[1]*n[2]
  *     doubles in that order (in 2D n[2] = 1).
- *   - Blocks are numbered x-fastest over the block grid g[a] = n[a] / b[a].
+ *   - Blocks are numbered x-fastest over the block grid g[a] = ceil(n[a] / b[a]).  When n[a] is
+ *     not a multiple of b[a] the last block along that axis is a remainder block of
+ *     n[a] - (g[a]-1)*b[a] points (at least `halo`, else JAC_EINVAL).  It keeps the full-size
+ *     placement of every block; its interior is the low corner of it and its +ghost layers come
+ *     right after its interior; its packed faces are correspondingly smaller.  (The paper's
+ *     decomposition is into equal cuboids; remainder blocks are an extension of this library.)
  *   - Faces: 0:-x 1:+x 2:-y 3:+y 4:-z 5:+z.  A face is the `halo` interior layers next to
  *     that side over the interior extent of the other axes (no edges, no corners).  A packed
  *     face holds those elements in source memory order: an x face is [bz][by][halo], a y face
@@ -59,7 +64,8 @@ extern "C" {
                                launch per block                                                  */
 #define JAC_MODE_TEMPORAL 2 /* `tsteps` sweeps per launch; tiles read across block borders
                                directly (equivalent to an exchange before every sweep).
-                               2D: b[0] % 4 == 0, tsteps <= 8; 3D: b[0] % 2 == 0, tsteps <= 2;
+                               2D: b[0] % 4 == 0 and n[0] % 4 == 0, tsteps <= 8;
+                               3D: b[0] % 2 == 0 and n[0] % 2 == 0, tsteps <= 2;
                                jac_create returns JAC_EINVAL otherwise                           */
 #define JAC_MODE_EXCHANGE 3 /* per sweep three launches over all blocks: pack, unpack, update    */
 #define JAC_MODE_WIDE     4 /* one wide exchange (jac_exchange_wide: all h ghost layers, edges and
@@ -72,7 +78,7 @@ extern "C" {
                                thread-block cluster (8 or 16 CTAs) that keeps the whole grid in
                                shared memory, slabs of rows per CTA, neighbouring slabs exchanging
                                their edge rows through distributed shared memory, one cluster
-                               barrier per sweep.  Needs ndim == 2, b[0] % 2 == 0 and
+                               barrier per sweep.  Needs ndim == 2, b[0] and n[0] even and
                                (2*(r+2) + (has_f ? r : 0)) * (n[0]+4) * 8 bytes <= 227 KB for
                                r = ceil(n[1]/8) or ceil(n[1]/16) (e.g. 256 x 256 with f);
                                JAC_EINVAL otherwise, also when the device cannot co-schedule a
@@ -92,7 +98,7 @@ typedef struct jac_desc {
                         library chooses                                                          */
     int32_t reserved;/* must be 0                                                                */
     int64_t n[3];    /* global interior points; n[2] ignored (taken as 1) when ndim == 2         */
-    int64_t b[3];    /* block interior points; n[a] % b[a] == 0                                  */
+    int64_t b[3];    /* block interior points, 1 <= b[a] <= n[a]                                 */
     void   *stream;  /* cudaStream_t of the caller (NULL = the legacy default stream)            */
 } jac_desc;
 
@@ -105,7 +111,7 @@ typedef struct jac_layout {
     int64_t xpad;          /* ghost columns are the innermost h of an xpad-wide margin           */
     int64_t origin;        /* element offset of interior point (0,0,0) inside a padded block     */
     int64_t block_stride;  /* elements between consecutive blocks of one array                   */
-    int64_t face_elems[6]; /* elements of one packed face                                        */
+    int64_t face_elems[6]; /* elements of one packed face of a full-size block                   */
     int64_t face_offset[6];/* element offset of each face inside a block's send region           */
     int64_t send_stride;   /* elements of one block's send region                                */
     int64_t partials;      /* doubles of reduction scratch                                       */
@@ -154,7 +160,9 @@ int jac_set_boundary(jac_ctx *ctx, int face, double value);
 /* Inspection (synchronous, HOST output).
  * jac_get_block_padded: the canonical padded block (b+2h)^d of the current state, x fastest,
  *   ghost cells as they currently are (edge/corner ghosts are never written: they stay 0).
- * jac_get_halo_buffer: the packed face of (block, face) as the last pack left it. */
+ * jac_get_halo_buffer: the packed face of (block, face) as the last pack left it; always
+ *   face_elems[face] doubles are copied, of which a remainder block's face fills only the first
+ *   h * (its extents on the other two axes). */
 int jac_get_block_padded(jac_ctx *ctx, int64_t block, double *host);
 int jac_get_halo_buffer(jac_ctx *ctx, int64_t block, int face, double *host);
 

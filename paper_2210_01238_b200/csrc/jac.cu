@@ -36,7 +36,7 @@ struct Tiling {
 Tiling make_tiling(const JacGeom& g, int force_nv = 0)
 {
     Tiling t{};
-    t.nv = force_nv ? force_nv : ((g.bx % 2 == 0) ? 2 : 1);
+    t.nv = force_nv ? force_nv : ((g.bx % 2 == 0 && g.rx % 2 == 0) ? 2 : 1);
     const long long need = ceil_div(g.bx, t.nv);
     const long long want_ctas = (long long)kNumSMs * 16;
     if (g.ndim == 2) {
@@ -149,7 +149,7 @@ constexpr size_t kMaxSmemPerCta = 227 * 1024;
 
 int plan_resident(const JacGeom& g, bool has_f, int want_cluster, ResidentPlan* p)
 {
-    if (g.ndim != 2 || g.bx % 2 != 0 || g.nx >= (1LL << 24) || g.ny >= (1LL << 24)) return JAC_EINVAL;
+    if (g.ndim != 2 || g.bx % 2 != 0 || g.rx % 2 != 0 || g.nx >= (1LL << 24) || g.ny >= (1LL << 24)) return JAC_EINVAL;
     if (want_cluster != 0 && want_cluster != 8 && want_cluster != 16) return JAC_EINVAL;
     const int first = want_cluster ? want_cluster : (g.ny >= 128 ? 16 : 8);
     const int order[2] = {first, want_cluster ? first : 24 - first};
@@ -188,10 +188,11 @@ int build_geometry(const jac_desc* d, JacGeom* g, jac_layout* L)
     for (int a = 0; a < d->ndim; ++a) {
         n[a] = d->n[a];
         b[a] = d->b[a];
-        if (n[a] < 1 || b[a] < 1 || b[a] > n[a] || n[a] % b[a] != 0) return JAC_EINVAL;
+        if (n[a] < 1 || b[a] < 1 || b[a] > n[a]) return JAC_EINVAL;
         if (d->halo > b[a]) return JAC_EINVAL;
         if (b[a] > (1LL << 30) || n[a] > (1LL << 40)) return JAC_EINVAL;
-        gr[a] = n[a] / b[a];
+        gr[a] = ceil_div(n[a], b[a]);
+        if (n[a] - (gr[a] - 1) * b[a] < d->halo) return JAC_EINVAL;   // a remainder block narrower than a face strip
         if (gr[a] > (1LL << 30)) return JAC_EINVAL;
     }
     std::memset(g, 0, sizeof(*g));
@@ -201,6 +202,9 @@ int build_geometry(const jac_desc* d, JacGeom* g, jac_layout* L)
     g->nfaces = 2 * d->ndim;
     g->bx = (int)b[0]; g->by = (int)b[1]; g->bz = (int)b[2];
     g->gx = (int)gr[0]; g->gy = (int)gr[1]; g->gz = (int)gr[2];
+    g->rx = (int)(n[0] - (gr[0] - 1) * b[0]);
+    g->ry = (int)(n[1] - (gr[1] - 1) * b[1]);
+    g->rz = (int)(n[2] - (gr[2] - 1) * b[2]);
     g->nx = n[0]; g->ny = n[1]; g->nz = n[2];
     const long long hz = (d->ndim == 3) ? d->halo : 0;
     const long long PY = b[1] + 2 * d->halo, PZ = b[2] + 2 * hz;
@@ -228,6 +232,13 @@ int build_geometry(const jac_desc* d, JacGeom* g, jac_layout* L)
     }
     g->send_stride = off;
 
+    if (d->mode == JAC_MODE_TEMPORAL) {
+        // whole lanes lie inside or outside the domain: 4 points per lane in 2D, 2 in 3D
+        if (n[1] >= (1LL << 30)) return JAC_EINVAL;
+        if (d->ndim == 2 && (b[0] % 4 != 0 || n[0] % 4 != 0)) return JAC_EINVAL;
+        if (d->ndim == 3 && (b[0] % 2 != 0 || n[0] % 2 != 0 || d->tsteps > 2 || n[2] >= (1LL << 30)))
+            return JAC_EINVAL;
+    }
     if (d->mode == JAC_MODE_RESIDENT) {
         ResidentPlan rp;
         if (plan_resident(*g, d->has_f != 0, d->tsteps, &rp)) return JAC_EINVAL;   // 3D, odd bx, or too large
@@ -444,11 +455,11 @@ int launch_ext(jac_ctx* c, int e, const double* u, double* un)
 {
     JacGeom ge = c->g;
     ge.ext = e;
-    ge.bx += 2 * e;
-    ge.by += 2 * e;
+    ge.bx += 2 * e; ge.rx += 2 * e;
+    ge.by += 2 * e; ge.ry += 2 * e;
     ge.origin -= (long long)e * ge.PX + e;
     if (ge.ndim == 3) {
-        ge.bz += 2 * e;
+        ge.bz += 2 * e; ge.rz += 2 * e;
         ge.origin -= (long long)e * ge.PXY;
     }
     // 128-bit accesses need the first column of the grown box on a 16-byte boundary: e even
@@ -488,12 +499,15 @@ int copy_dense_host(jac_ctx* c, double* arr, double* host, bool to_device)
         const long long bxi = blk % g.gx, byi = (blk / g.gx) % g.gy, bzi = blk / ((long long)g.gx * g.gy);
         double* dev = arr + blk * g.block_stride + g.origin;
         double* hp = host + ((bzi * g.bz) * g.ny + byi * g.by) * g.nx + bxi * g.bx;
+        // interior extent of this block (the last one along an axis may be a remainder block)
+        const size_t ex = bxi + 1 == g.gx ? g.rx : g.bx, ey = byi + 1 == g.gy ? g.ry : g.by,
+                     ez = bzi + 1 == g.gz ? g.rz : g.bz;
         cudaError_t e;
         if (to_device)
-            e = copy_box(dev, g.PX * 8, PY, hp, g.nx * 8, g.ny, (size_t)g.bx * 8, g.by, g.bz,
+            e = copy_box(dev, g.PX * 8, PY, hp, g.nx * 8, g.ny, ex * 8, ey, ez,
                          cudaMemcpyHostToDevice, c->stream);
         else
-            e = copy_box(hp, g.nx * 8, g.ny, dev, g.PX * 8, PY, (size_t)g.bx * 8, g.by, g.bz,
+            e = copy_box(hp, g.nx * 8, g.ny, dev, g.PX * 8, PY, ex * 8, ey, ez,
                          cudaMemcpyDeviceToHost, c->stream);
         JAC_CK(c, e);
     }
@@ -505,7 +519,7 @@ template <bool TO_BLOCKS>
 int copy_dense_device(jac_ctx* c, double* arr, double* dense)
 {
     const JacGeom& g = c->g;
-    const int nv = ((g.bx % 2 == 0) && (((uintptr_t)dense & 15u) == 0)) ? 2 : 1;
+    const int nv = ((g.bx % 2 == 0) && (g.nx % 2 == 0) && (((uintptr_t)dense & 15u) == 0)) ? 2 : 1;
     const int segs = (int)ceil_div(ceil_div(g.nx, nv), 256);
     const long long ctas = g.ny * g.nz * segs;
     if (ctas > kMaxGrid) return JAC_EINVAL;
@@ -846,12 +860,6 @@ int jac_create(const jac_desc* desc, void* dev_workspace, size_t bytes, jac_ctx*
     jac_layout L;
     int rc = build_geometry(desc, &g, &L);
     if (rc) return rc;
-    if (desc->mode == JAC_MODE_TEMPORAL) {
-        if (desc->n[1] >= (1LL << 30)) return JAC_EINVAL;
-        if (desc->ndim == 2 && desc->b[0] % 4 != 0) return JAC_EINVAL;
-        if (desc->ndim == 3 && (desc->b[0] % 2 != 0 || desc->tsteps > 2 || desc->n[2] >= (1LL << 30)))
-            return JAC_EINVAL;
-    }
     if (!dev_workspace || bytes < (size_t)L.total_bytes || ((uintptr_t)dev_workspace & 255u))
         return JAC_ENOMEM;
     int dev = -1;

@@ -16,6 +16,9 @@
 struct JacGeom {
     int ndim, h, xpad, nfaces;
     int bx, by, bz;  // block interior
+    int rx, ry, rz;  // interior of the last block along each axis: b, or the remainder n - (g-1)*b when
+                     // the grid is not a multiple of the block size (the block keeps full-size storage,
+                     // its interior in the low corner, its +ghost layers right after its interior)
     int gx, gy, gz;  // block grid
     long long nx, ny, nz;
     long long PX, PXY, block_stride, origin;

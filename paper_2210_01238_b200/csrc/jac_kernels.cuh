@@ -60,6 +60,20 @@ __device__ __forceinline__ double block_sum(double v) {
     return total;
 }
 
+// interior extent of a block: the last block along an axis may be a remainder block
+struct BlockExtent { int x, y, z; };
+__device__ __forceinline__ BlockExtent block_extent(const JacGeom& g, long long blk)
+{
+    const int bxi = (int)(blk % g.gx);
+    const int byi = (int)((blk / g.gx) % g.gy);
+    const int bzi = (int)(blk / ((long long)g.gx * g.gy));
+    BlockExtent e;
+    e.x = bxi + 1 == g.gx ? g.rx : g.bx;
+    e.y = byi + 1 == g.gy ? g.ry : g.by;
+    e.z = bzi + 1 == g.gz ? g.rz : g.bz;
+    return e;
+}
+
 // ---------------------------------------------------------------------------------------
 // 2D: one CTA owns a strip of `rows` rows x (blockDim.x * NV) columns of one block and
 // marches along y.  The rows j-1, j, j+1 of a thread's own columns live in registers; the
@@ -88,12 +102,13 @@ sweep2d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
     const int yt = (int)((t / tiles_x) % tiles_y);
     const long long blk = blk0 + t / ((long long)tiles_x * tiles_y);
     const int x = (xt * blockDim.x + threadIdx.x) * NV;
+    const BlockExtent ext = block_extent(g, blk);
     const int j0 = yt * rows;
-    const int j1 = min(g.by, j0 + rows);
+    const int j1 = min(ext.y, j0 + rows);
     const long long PX = g.PX;
     double acc = 0.0;
 
-    if (x < g.bx) {
+    if (x < ext.x && j0 < j1) {
         const long long base = blk * g.block_stride + g.origin + x;
         const double* ub = u + base;
         const double* fb = HAS_F ? f + base : nullptr;
@@ -176,13 +191,14 @@ sweep3d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
     const long long blk = blk0 + t / ((long long)tiles_x * tiles_y * tiles_z);
     const int x = (xt * blockDim.x + threadIdx.x) * NV;
     const int y = yt * blockDim.y + threadIdx.y;
+    const BlockExtent ext = block_extent(g, blk);
     const int k0 = zt * planes;
-    const int k1 = min(g.bz, k0 + planes);
+    const int k1 = min(ext.z, k0 + planes);
     const long long PX = g.PX, PXY = g.PXY;
     const double c6 = 1.0 / 6.0;
     double acc = 0.0;
 
-    if (x < g.bx && y < g.by) {
+    if (x < ext.x && y < ext.y && k0 < k1) {
         const long long base = blk * g.block_stride + g.origin + (long long)y * PX + x;
         const double* ub = u + base;
         const double* fb = HAS_F ? f + base : nullptr;
@@ -290,18 +306,27 @@ __device__ __forceinline__ long long neighbour_block(const JacGeom& g, long long
 
 // offset (relative to the block's interior origin) of element e of the strip on `face`;
 // lo = first layer of the strip along the face's axis (interior-relative)
-__device__ __forceinline__ long long strip_offset(const JacGeom& g, int face, long long e, int lo)
+// (ext = the block's interior extent; the strip spans it on the axes other than the face's)
+__device__ __forceinline__ long long strip_offset(const JacGeom& g, const BlockExtent& ext, int face, long long e, int lo)
 {
     const int axis = face >> 1;
     long long x, y, z;
     if (axis == 0) {
-        x = e % g.h + lo; const long long t = e / g.h; y = t % g.by; z = t / g.by;
+        x = e % g.h + lo; const long long t = e / g.h; y = t % ext.y; z = t / ext.y;
     } else if (axis == 1) {
-        x = e % g.bx; const long long t = e / g.bx; y = t % g.h + lo; z = t / g.h;
+        x = e % ext.x; const long long t = e / ext.x; y = t % g.h + lo; z = t / g.h;
     } else {
-        x = e % g.bx; const long long t = e / g.bx; y = t % g.by; z = t / g.by + lo;
+        x = e % ext.x; const long long t = e / ext.x; y = t % ext.y; z = t / ext.y + lo;
     }
     return z * g.PXY + y * g.PX + x;
+}
+
+// elements of the packed face of a block with interior extent `ext`
+__device__ __forceinline__ long long face_elems_of(const JacGeom& g, const BlockExtent& ext, int face)
+{
+    const int axis = face >> 1;
+    const long long h = g.h;
+    return axis == 0 ? h * ext.y * ext.z : (axis == 1 ? h * ext.x * ext.z : h * ext.x * ext.y);
 }
 
 // A thread moves two consecutive elements of one face; `slots` threads (a multiple of 32, so a
@@ -322,27 +347,28 @@ halo_kernel(double* __restrict__ u, double* __restrict__ send, const JacGeom g,
     const long long blk = pair / g.nfaces;
     const int face = (int)(pair - blk * g.nfaces);
     if (!((face_mask >> face) & 1u)) return;
-    const long long n = g.face_elems[face];
+    const BlockExtent be = block_extent(g, blk);
+    const long long n = face_elems_of(g, be, face);
     if (e >= n) return;
     const long long nb = neighbour_block(g, blk, face);
     if (nb < 0) return;
     const int axis = face >> 1;
-    const int ext = axis == 0 ? g.bx : (axis == 1 ? g.by : g.bz);
+    const int ext = axis == 0 ? be.x : (axis == 1 ? be.y : be.z);
     double* ub = u + blk * g.block_stride + g.origin;
     // pack reads the interior strip next to the face; unpack writes the ghost strip
     const int lo = UNPACK ? ((face & 1) ? ext : -g.h) : ((face & 1) ? ext - g.h : 0);
     double* buf = UNPACK ? send + nb * g.send_stride + g.face_off[face ^ 1]
                          : send + blk * g.send_stride + g.face_off[face];
     const bool pair_ok = e + 1 < n;
-    if (axis != 0 && (g.bx & 1) == 0) {
-        double2* cell = reinterpret_cast<double2*>(ub + strip_offset(g, face, e, lo));
+    if (axis != 0 && (be.x & 1) == 0) {
+        double2* cell = reinterpret_cast<double2*>(ub + strip_offset(g, be, face, e, lo));
         double2* slot = reinterpret_cast<double2*>(buf + e);
         if (UNPACK) *cell = *slot; else *slot = *cell;
     } else {
-        double* c0 = ub + strip_offset(g, face, e, lo);
+        double* c0 = ub + strip_offset(g, be, face, e, lo);
         if (UNPACK) *c0 = buf[e]; else buf[e] = *c0;
         if (pair_ok) {
-            double* c1 = ub + strip_offset(g, face, e + 1, lo);
+            double* c1 = ub + strip_offset(g, be, face, e + 1, lo);
             if (UNPACK) *c1 = buf[e + 1]; else buf[e + 1] = *c1;
         }
     }
@@ -365,12 +391,14 @@ halo_wide_kernel(double* __restrict__ arr, double* __restrict__ send, const JacG
     const long long e = t - pr * slots;
     const long long blk = pr >> 1;
     const int face = 2 * axis + (int)(pr & 1);
-    if (e >= g.wface_elems[face]) return;
     const long long nb = neighbour_block(g, blk, face);
     if (nb < 0) return;
+    const BlockExtent be = block_extent(g, blk);
     const int h = g.h, hz = g.ndim == 3 ? g.h : 0;
-    const int wx = g.bx + 2 * h, wy = g.by + 2 * h;
-    const int ext = axis == 0 ? g.bx : (axis == 1 ? g.by : g.bz);
+    const int wx = be.x + 2 * h, wy = be.y + 2 * h, wz = be.z + 2 * hz;
+    const long long n = axis == 0 ? (long long)h * wy * wz : (axis == 1 ? (long long)h * wx * wz : (long long)h * wx * wy);
+    if (e >= n) return;
+    const int ext = axis == 0 ? be.x : (axis == 1 ? be.y : be.z);
     const int lo = UNPACK ? ((face & 1) ? ext : -h) : ((face & 1) ? ext - h : 0);
     long long x, y, z;
     if (axis == 0) {
@@ -405,13 +433,14 @@ fill_boundary_kernel(double* __restrict__ u0, double* __restrict__ u1, const Jac
         rem /= ga[a];
     }
     const long long blk = (c[2] * g.gy + c[1]) * g.gx + c[0];
-    const int ext = axis == 0 ? g.bx : (axis == 1 ? g.by : g.bz);
+    const BlockExtent be = block_extent(g, blk);
+    const int ext = axis == 0 ? be.x : (axis == 1 ? be.y : be.z);
     const int lo = (face & 1) ? ext : -g.h;
-    const long long n = g.face_elems[face];
+    const long long n = face_elems_of(g, be, face);
     const long long base = blk * g.block_stride + g.origin;
     for (long long e = (long long)chunk * blockDim.x + threadIdx.x; e < n;
          e += (long long)chunks * blockDim.x) {
-        const long long off = base + strip_offset(g, face, e, lo);
+        const long long off = base + strip_offset(g, be, face, e, lo);
         u0[off] = value;
         u1[off] = value;
     }

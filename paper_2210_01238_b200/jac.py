@@ -283,13 +283,20 @@ class Jacobi:
                    lib().jac_get_block_padded(self._ctx, int(blk), _host_ptr(out)))
         return out
 
+    def extent(self, blk: int):
+        """Interior points of block ``blk`` per axis: b, or the remainder for the last block of an axis."""
+        g = [int(self.layout.g[a]) for a in range(3)]
+        c = [blk % g[0], (blk // g[0]) % g[1], blk // (g[0] * g[1])][: self.ndim]
+        return [min(bb, nn - cc * bb) for nn, bb, cc in zip(self.n, self.b, c)]
+
     def get_halo_buffer(self, blk: int, face: int) -> np.ndarray:
-        dims = list(self.b)
-        dims[face // 2] = self.desc.halo
-        out = np.empty(tuple(reversed(dims)), dtype=np.float64)
+        """Packed face of (block, face); a remainder block's face is correspondingly smaller."""
+        raw = np.empty(int(self.layout.face_elems[face]), dtype=np.float64)
         self._call("jac_get_halo_buffer",
-                   lib().jac_get_halo_buffer(self._ctx, int(blk), int(face), _host_ptr(out)))
-        return out
+                   lib().jac_get_halo_buffer(self._ctx, int(blk), int(face), _host_ptr(raw)))
+        dims = self.extent(blk)
+        dims[face // 2] = self.desc.halo
+        return raw[: int(np.prod(dims))].reshape(tuple(reversed(dims))).copy()
 
     # ---- the hot path
     def pack_halos(self):
@@ -310,12 +317,12 @@ class Jacobi:
 
     def get_wide_buffer(self, blk: int, face: int) -> np.ndarray:
         h = self.desc.halo
-        dims = [x + 2 * h for x in self.b]
-        dims[face // 2] = h
-        out = np.empty(tuple(reversed(dims)), dtype=np.float64)
+        raw = np.empty(int(self.layout.wide_face_elems[face]), dtype=np.float64)
         self._call("jac_get_wide_buffer",
-                   lib().jac_get_wide_buffer(self._ctx, int(blk), int(face), _host_ptr(out)))
-        return out
+                   lib().jac_get_wide_buffer(self._ctx, int(blk), int(face), _host_ptr(raw)))
+        dims = [x + 2 * h for x in self.extent(blk)]
+        dims[face // 2] = h
+        return raw[: int(np.prod(dims))].reshape(tuple(reversed(dims))).copy()
 
     def sweep(self, nsweeps: int = 1):
         self._call("jac_sweep", lib().jac_sweep(self._ctx, int(nsweeps)))

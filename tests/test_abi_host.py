@@ -42,7 +42,9 @@ def test_strerror(jac):
 
 
 @pytest.mark.parametrize("kw", [
-    dict(n=(12, 8), b=(5, 4)),            # not divisible
+    dict(n=(13, 8), b=(4, 4), halo=2),    # remainder block (1 point) narrower than the halo
+    dict(n=(14, 8), b=(4, 4), mode="temporal"),                 # temporal 2D wants n[0] % 4 == 0 ...
+    dict(n=(14, 8), b=(4, 4), mode="resident", halo=1, tsteps=3),  # a cluster size that is neither 8 nor 16
     dict(n=(12, 8), b=(4, 4), halo=0),
     dict(n=(12, 8), b=(4, 4), halo=5),    # wider than the block
     dict(n=(12, 8), b=(4, 4), halo=9),
@@ -81,12 +83,13 @@ def test_null_arguments(jac):
                                           ((4096, 4096), (512, 512), 1, True),
                                           ((1024, 1024, 1024), (128, 128, 128), 1, True),
                                           ((12, 8), (3, 2), 2, True), ((9, 5, 7), (3, 5, 1), 1, False),
+                                          ((14, 11), (4, 4), 2, True), ((10, 9, 7), (4, 4, 3), 1, False),
                                           ((256, 256), (64, 64), 4, False)])
 def test_layout_is_aligned_and_disjoint(jac, n, b, h, has_f):
     d = jac.make_desc(n, b, h, has_f)
     L = jac.get_layout(d)
     ndim = len(n)
-    assert L.nblocks == int(np.prod([nn // bb for nn, bb in zip(n, b)]))
+    assert L.nblocks == int(np.prod([-(-nn // bb) for nn, bb in zip(n, b)]))
     assert L.xpad >= h and L.xpad % 4 == 0
     assert L.pad[0] == b[0] + 2 * L.xpad and L.pad[1] == b[1] + 2 * h
     assert L.pad[2] == (b[2] + 2 * h if ndim == 3 else 1)
