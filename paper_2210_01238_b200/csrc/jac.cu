@@ -366,8 +366,13 @@ int launch_halo(jac_ctx* c, long long pair0, long long npairs, unsigned face_mas
     const int slots = halo_slots(c, face_mask);
     const long long ctas = ceil_div(npairs * slots, 256);
     if (ctas > kMaxGrid) return JAC_EINVAL;
-    jac::halo_kernel<UNPACK><<<(unsigned)ctas, 256, 0, c->stream>>>(c->u[c->cur], c->send, c->g, pair0, npairs,
-                                                                  slots, face_mask);
+    // 32-bit index arithmetic when thread and pair numbers fit (they do for any grid that fits a GPU)
+    if (ctas * 256 < (1LL << 32) && c->g.nblocks * c->g.nfaces < (1LL << 31))
+        jac::halo_kernel<UNPACK, unsigned><<<(unsigned)ctas, 256, 0, c->stream>>>(c->u[c->cur], c->send, c->g, pair0,
+                                                                                npairs, slots, face_mask);
+    else
+        jac::halo_kernel<UNPACK, long long><<<(unsigned)ctas, 256, 0, c->stream>>>(c->u[c->cur], c->send, c->g, pair0,
+                                                                                 npairs, slots, face_mask);
     return check_launch(c);
 }
 
@@ -428,10 +433,13 @@ int do_exchange_wide(jac_ctx* c, double* arr)
         const int slots = (int)round_up(n, 32);
         const long long ctas = ceil_div(2 * c->g.nblocks * slots, 256);
         if (ctas > kMaxGrid) return JAC_EINVAL;
-        jac::halo_wide_kernel<false><<<(unsigned)ctas, 256, 0, c->stream>>>(arr, c->send, c->g, axis, slots);
+        const bool narrow = ctas * 256 < (1LL << 32) && 2 * c->g.nblocks < (1LL << 31);
+        if (narrow) jac::halo_wide_kernel<false, unsigned><<<(unsigned)ctas, 256, 0, c->stream>>>(arr, c->send, c->g, axis, slots);
+        else jac::halo_wide_kernel<false, long long><<<(unsigned)ctas, 256, 0, c->stream>>>(arr, c->send, c->g, axis, slots);
         int rc = check_launch(c);
         if (rc) return rc;
-        jac::halo_wide_kernel<true><<<(unsigned)ctas, 256, 0, c->stream>>>(arr, c->send, c->g, axis, slots);
+        if (narrow) jac::halo_wide_kernel<true, unsigned><<<(unsigned)ctas, 256, 0, c->stream>>>(arr, c->send, c->g, axis, slots);
+        else jac::halo_wide_kernel<true, long long><<<(unsigned)ctas, 256, 0, c->stream>>>(arr, c->send, c->g, axis, slots);
         if ((rc = check_launch(c))) return rc;
     }
     return JAC_OK;

@@ -289,34 +289,62 @@ reduce_partials_kernel(const double* __restrict__ partials, const long long n, d
 // Pack reads the interior strip next to the face; unpack writes the ghost strip of the same
 // face from the neighbour's opposite-face buffer.
 // ---------------------------------------------------------------------------------------
+// Block coordinates, the neighbour across a face and the block's interior extent, from one
+// decomposition of the block number.  IT is the integer type the arithmetic runs in: 32-bit
+// whenever block, pair and thread counts fit (the host checks), since 64-bit divisions are what
+// these short kernels would otherwise spend most of their instructions on.
+template <typename IT>
+struct BlockPlace {
+    IT nb;            // neighbour across the face (valid if has_nb)
+    bool has_nb;
+    BlockExtent ext;
+};
+template <typename IT>
+__device__ __forceinline__ BlockPlace<IT> block_place(const JacGeom& g, IT blk, int face)
+{
+    const IT gx = (IT)g.gx, gy = (IT)g.gy;
+    const IT q = blk / gx;
+    const int bxi = (int)(blk - q * gx);
+    const IT bzi_ = q / gy;
+    const int byi = (int)(q - bzi_ * gy);
+    const int bzi = (int)bzi_;
+    BlockPlace<IT> p;
+    p.ext.x = bxi + 1 == g.gx ? g.rx : g.bx;
+    p.ext.y = byi + 1 == g.gy ? g.ry : g.by;
+    p.ext.z = bzi + 1 == g.gz ? g.rz : g.bz;
+    switch (face) {
+        case 0: p.has_nb = bxi > 0; p.nb = blk - 1; break;
+        case 1: p.has_nb = bxi + 1 < g.gx; p.nb = blk + 1; break;
+        case 2: p.has_nb = byi > 0; p.nb = blk - gx; break;
+        case 3: p.has_nb = byi + 1 < g.gy; p.nb = blk + gx; break;
+        case 4: p.has_nb = bzi > 0; p.nb = blk - gx * gy; break;
+        default: p.has_nb = bzi + 1 < g.gz; p.nb = blk + gx * gy; break;
+    }
+    return p;
+}
+
 __device__ __forceinline__ long long neighbour_block(const JacGeom& g, long long blk, int face)
 {
-    const int bxi = (int)(blk % g.gx);
-    const int byi = (int)((blk / g.gx) % g.gy);
-    const int bzi = (int)(blk / ((long long)g.gx * g.gy));
-    switch (face) {
-        case 0: return bxi > 0 ? blk - 1 : -1;
-        case 1: return bxi + 1 < g.gx ? blk + 1 : -1;
-        case 2: return byi > 0 ? blk - g.gx : -1;
-        case 3: return byi + 1 < g.gy ? blk + g.gx : -1;
-        case 4: return bzi > 0 ? blk - (long long)g.gx * g.gy : -1;
-        default: return bzi + 1 < g.gz ? blk + (long long)g.gx * g.gy : -1;
-    }
+    const BlockPlace<long long> p = block_place<long long>(g, blk, face);
+    return p.has_nb ? p.nb : -1;
 }
 
 // offset (relative to the block's interior origin) of element e of the strip on `face`;
-// lo = first layer of the strip along the face's axis (interior-relative)
-// (ext = the block's interior extent; the strip spans it on the axes other than the face's)
-__device__ __forceinline__ long long strip_offset(const JacGeom& g, const BlockExtent& ext, int face, long long e, int lo)
+// lo = first layer of the strip along the face's axis (interior-relative); ext = the block's
+// interior extent, which the strip spans on the axes other than the face's.  e < 2^31.
+__device__ __forceinline__ long long strip_offset(const JacGeom& g, const BlockExtent& ext, int face, unsigned e, int lo)
 {
     const int axis = face >> 1;
     long long x, y, z;
     if (axis == 0) {
-        x = e % g.h + lo; const long long t = e / g.h; y = t % ext.y; z = t / ext.y;
+        const unsigned t = e / (unsigned)g.h; x = (int)(e - t * g.h) + lo;
+        z = t / (unsigned)ext.y; y = t - (unsigned)z * ext.y;
     } else if (axis == 1) {
-        x = e % ext.x; const long long t = e / ext.x; y = t % g.h + lo; z = t / g.h;
+        const unsigned t = e / (unsigned)ext.x; x = e - t * ext.x;
+        z = t / (unsigned)g.h; y = (int)(t - (unsigned)z * g.h) + lo;
     } else {
-        x = e % ext.x; const long long t = e / ext.x; y = t % ext.y; z = t / ext.y + lo;
+        const unsigned t = e / (unsigned)ext.x; x = e - t * ext.x;
+        const unsigned p = t / (unsigned)ext.y; y = t - p * ext.y; z = (int)p + lo;
     }
     return z * g.PXY + y * g.PX + x;
 }
@@ -334,31 +362,31 @@ __device__ __forceinline__ long long face_elems_of(const JacGeom& g, const Block
 // threads, not faces: small faces do not leave CTAs mostly idle.  On y and z faces with an even
 // block width the two elements are adjacent in memory on both sides and move as one 128-bit
 // access; on x faces they are two strided cells.
-template <bool UNPACK>
+template <bool UNPACK, typename IT>
 __global__ void __launch_bounds__(256)
 halo_kernel(double* __restrict__ u, double* __restrict__ send, const JacGeom g,
             const long long pair0, const long long npairs, const int slots, const unsigned face_mask)
 {
-    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    const long long pr = t / slots;
-    if (pr >= npairs) return;
-    const long long e = 2 * (t - pr * slots);
-    const long long pair = pair0 + pr;
-    const long long blk = pair / g.nfaces;
-    const int face = (int)(pair - blk * g.nfaces);
+    const IT t = (IT)blockIdx.x * (IT)blockDim.x + (IT)threadIdx.x;
+    const IT pr = t / (IT)slots;
+    if (pr >= (IT)npairs) return;
+    const unsigned e = 2u * (unsigned)(t - pr * (IT)slots);
+    const IT pair = (IT)pair0 + pr;
+    const IT blk = pair / (IT)g.nfaces;
+    const int face = (int)(pair - blk * (IT)g.nfaces);
     if (!((face_mask >> face) & 1u)) return;
-    const BlockExtent be = block_extent(g, blk);
+    const BlockPlace<IT> bp = block_place<IT>(g, blk, face);
+    if (!bp.has_nb) return;
+    const BlockExtent& be = bp.ext;
     const long long n = face_elems_of(g, be, face);
     if (e >= n) return;
-    const long long nb = neighbour_block(g, blk, face);
-    if (nb < 0) return;
     const int axis = face >> 1;
     const int ext = axis == 0 ? be.x : (axis == 1 ? be.y : be.z);
-    double* ub = u + blk * g.block_stride + g.origin;
+    double* ub = u + (long long)blk * g.block_stride + g.origin;
     // pack reads the interior strip next to the face; unpack writes the ghost strip
     const int lo = UNPACK ? ((face & 1) ? ext : -g.h) : ((face & 1) ? ext - g.h : 0);
-    double* buf = UNPACK ? send + nb * g.send_stride + g.face_off[face ^ 1]
-                         : send + blk * g.send_stride + g.face_off[face];
+    double* buf = UNPACK ? send + (long long)bp.nb * g.send_stride + g.face_off[face ^ 1]
+                         : send + (long long)blk * g.send_stride + g.face_off[face];
     const bool pair_ok = e + 1 < n;
     if (axis != 0 && (be.x & 1) == 0) {
         double2* cell = reinterpret_cast<double2*>(ub + strip_offset(g, be, face, e, lo));
@@ -375,42 +403,45 @@ halo_kernel(double* __restrict__ u, double* __restrict__ send, const JacGeom g,
 }
 
 // Wide exchange, one axis per launch: the strip of a face is h layers along `axis` (interior
-// layers for pack, ghost layers for unpack) over the whole padded extent (-h .. b + h) of the other
-// axes, so edge and corner data delivered by the launches of earlier axes travels on.  Element e
-// of a wide face, source memory order (wx = bx + 2h, wy = by + 2h, wz = bz + 2h or 1):
+// layers for pack, ghost layers for unpack) over the whole padded extent (-h .. extent + h) of the
+// other axes, so edge and corner data delivered by the launches of earlier axes travels on.
+// Element e of a wide face, source memory order (wx, wy, wz = the block's extent + 2h; wz = 1 in 2D):
 //   x face: e = (k*wy + j)*h + c      y face: e = (k*h + r)*wx + i      z face: e = (p*wy + j)*wx + i
 // One thread per element; `slots` threads (whole warps) per (block, side) pair.
-template <bool UNPACK>
+template <bool UNPACK, typename IT>
 __global__ void __launch_bounds__(256)
 halo_wide_kernel(double* __restrict__ arr, double* __restrict__ send, const JacGeom g, const int axis,
                  const int slots)
 {
-    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    const long long pr = t / slots;
-    if (pr >= 2 * g.nblocks) return;
-    const long long e = t - pr * slots;
-    const long long blk = pr >> 1;
+    const IT t = (IT)blockIdx.x * (IT)blockDim.x + (IT)threadIdx.x;
+    const IT pr = t / (IT)slots;
+    if (pr >= (IT)(2 * g.nblocks)) return;
+    const unsigned e = (unsigned)(t - pr * (IT)slots);
+    const IT blk = pr >> 1;
     const int face = 2 * axis + (int)(pr & 1);
-    const long long nb = neighbour_block(g, blk, face);
-    if (nb < 0) return;
-    const BlockExtent be = block_extent(g, blk);
+    const BlockPlace<IT> bp = block_place<IT>(g, blk, face);
+    if (!bp.has_nb) return;
+    const BlockExtent& be = bp.ext;
     const int h = g.h, hz = g.ndim == 3 ? g.h : 0;
-    const int wx = be.x + 2 * h, wy = be.y + 2 * h, wz = be.z + 2 * hz;
+    const unsigned wx = be.x + 2 * h, wy = be.y + 2 * h, wz = be.z + 2 * hz;
     const long long n = axis == 0 ? (long long)h * wy * wz : (axis == 1 ? (long long)h * wx * wz : (long long)h * wx * wy);
     if (e >= n) return;
     const int ext = axis == 0 ? be.x : (axis == 1 ? be.y : be.z);
     const int lo = UNPACK ? ((face & 1) ? ext : -h) : ((face & 1) ? ext - h : 0);
     long long x, y, z;
     if (axis == 0) {
-        x = e % h + lo; const long long q = e / h; y = q % wy - h; z = q / wy - hz;
+        const unsigned q = e / (unsigned)h; x = (int)(e - q * h) + lo;
+        const unsigned k = q / wy; y = (int)(q - k * wy) - h; z = (int)k - hz;
     } else if (axis == 1) {
-        x = e % wx - h; const long long q = e / wx; y = q % h + lo; z = q / h - hz;
+        const unsigned q = e / wx; x = (int)(e - q * wx) - h;
+        const unsigned k = q / (unsigned)h; y = (int)(q - k * h) + lo; z = (int)k - hz;
     } else {
-        x = e % wx - h; const long long q = e / wx; y = q % wy - h; z = q / wy + lo;
+        const unsigned q = e / wx; x = (int)(e - q * wx) - h;
+        const unsigned k = q / wy; y = (int)(q - k * wy) - h; z = (int)k + lo;
     }
-    double* cell = arr + blk * g.block_stride + g.origin + z * g.PXY + y * g.PX + x;
-    if (UNPACK) *cell = send[nb * g.send_stride + g.face_off[face ^ 1] + e];
-    else send[blk * g.send_stride + g.face_off[face] + e] = *cell;
+    double* cell = arr + (long long)blk * g.block_stride + g.origin + z * g.PXY + y * g.PX + x;
+    if (UNPACK) *cell = send[(long long)bp.nb * g.send_stride + g.face_off[face ^ 1] + e];
+    else send[(long long)blk * g.send_stride + g.face_off[face] + e] = *cell;
 }
 
 // Dirichlet value into the ghost strip of `face` of every block on that domain face, in both
@@ -1081,7 +1112,7 @@ __device__ __forceinline__ void t3_step(Plane6 (&L0)[3], Plane6 (&L1)[3], const 
 // RES as for the 2D kernel: partials[CTA * 8 + warp] gets the warp's sum of squared residuals of
 // the state before the last sweep of the launch.
 template <int T, bool HAS_F, bool RES>
-__global__ void __launch_bounds__(k3dWarps * 32, 1)
+__global__ void __launch_bounds__(k3dWarps * 32, k3dWarps <= 4 ? 2 : 1)
 temporal3d_kernel(const double* __restrict__ u, double* __restrict__ un, const double* __restrict__ f,
                   double* __restrict__ partials, const JacGeom g, const int tiles_x, const int tiles_y,
                   const int tiles_z, const int zchunk)
