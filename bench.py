@@ -415,7 +415,7 @@ def run_ours(args, w: inputs.Workload):
     # ---- the oracle on the host cores, bounded sample (rank 0, single-GPU runs only)
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        g, osw, dt, threads = oracle_time_job(w, u0, f, 12.0, w.sweeps)
+        g, osw, dt, threads = oracle_time_job(w, u0, f, 20.0, w.sweeps)
         cpu_baseline = {"value": g, "unit": UNIT, "cores": threads, "kind": "oracle",
                         "sample": f"{osw} of {w.sweeps} sweeps (+1 residual) of the full "
                                   f"{'x'.join(map(str, w.n))} grid, {dt:.1f} s"}
