@@ -343,3 +343,27 @@ def test_solve_stops_at_the_tolerance(jac, orc):
             J.solve(0, 8, 1.0)
         J.close()
         B.close()
+
+
+def test_work_is_issued_on_the_callers_stream(jac, orc):
+    """A context created on a side stream runs there: results are right, and two contexts on two
+    streams do not disturb each other."""
+    import torch
+    n, b, h = (130, 70), (130, 70), 1
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    u0, f = _random_problem(n, 3)
+    B = orc.Blocked(n, b, h, True)
+    B.set_u(u0); B.set_f(f)
+    J1 = jac.Jacobi(n, b, h, True, "fused", stream=s1)
+    J2 = jac.Jacobi(n, b, h, True, "exchange", stream=s2)
+    assert J1.desc.stream == s1.cuda_stream and J2.desc.stream == s2.cuda_stream
+    for J in (J1, J2):
+        J.set_u(u0); J.set_f(f)
+    for _ in range(5):          # interleave the two streams' launches
+        J1.sweep(1); J2.sweep(1)
+    B.sweep(5)
+    want = B.get_u()
+    assert np.array_equal(J1.get_u(), want) and np.array_equal(J2.get_u(), want)
+    r = B.residual()
+    assert abs(J1.residual() - r) <= RESID_TOL * r and abs(J2.residual() - r) <= RESID_TOL * r
+    J1.close(); J2.close(); B.close()
