@@ -419,6 +419,12 @@ def run_ours(args, w: inputs.Workload):
         cpu_baseline = {"value": g, "unit": UNIT, "cores": threads, "kind": "oracle",
                         "sample": f"{osw} of {w.sweeps} sweeps (+1 residual) of the full "
                                   f"{'x'.join(map(str, w.n))} grid, {dt:.1f} s"}
+        if w.points <= 2 ** 24:      # the small grids also on one core
+            from oracle import orc
+            orc.set_threads(1)
+            g1, osw1, dt1, _ = oracle_time_job(w, u0, f, 5.0, w.sweeps)
+            orc.set_threads(threads)
+            cpu_baseline["one_core"] = {"value": g1, "sample": f"{osw1} sweeps, {dt1:.1f} s"}
 
     if rank == 0:
         line = {
