@@ -153,6 +153,19 @@ int jac_set_u_device(jac_ctx *ctx, const double *dev_dense);
 int jac_set_f_device(jac_ctx *ctx, const double *dev_dense);
 int jac_get_u_device(jac_ctx *ctx, double *dev_dense);
 
+/* The same copies and the same residual without waiting for them: the work is queued on the
+ * stream and the call returns.  For callers that keep several contexts busy at once, e.g. two
+ * contexts on two streams so that the input copy of one job, the sweeps of another and the output
+ * copy of a third overlap (the two copy directions and the SMs are separate engines).  The host
+ * array must stay alive and untouched until the stream has passed the call, and should be pinned:
+ * pageable memory makes the copies synchronous again.  jac_residual_async writes the norm to
+ * *host_out_l2 when the stream gets there (pinned memory; synchronise the stream before reading);
+ * its value has the bits jac_residual would return.  (No counterpart in the paper, whose proxy
+ * keeps its data on the GPUs between iterations.) */
+int jac_set_u_async(jac_ctx *ctx, const double *host_dense);
+int jac_get_u_async(jac_ctx *ctx, double *host_dense);
+int jac_residual_async(jac_ctx *ctx, double *host_out_l2);
+
 /* Dirichlet value of one domain face: written into the ghost layers (all h of them, interior
  * extent) of every block touching that face, in both solution arrays.  Asynchronous. */
 int jac_set_boundary(jac_ctx *ctx, int face, double value);

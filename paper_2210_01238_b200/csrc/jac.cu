@@ -499,7 +499,7 @@ cudaError_t copy_box(void* dst, size_t dpitch, size_t drows, const void* src, si
 }
 
 // host dense <-> interiors of all blocks of `arr`
-int copy_dense_host(jac_ctx* c, double* arr, double* host, bool to_device)
+int copy_dense_host(jac_ctx* c, double* arr, double* host, bool to_device, bool wait = true)
 {
     const JacGeom& g = c->g;
     const size_t PY = (size_t)(g.PXY / g.PX);
@@ -519,7 +519,7 @@ int copy_dense_host(jac_ctx* c, double* arr, double* host, bool to_device)
                          cudaMemcpyDeviceToHost, c->stream);
         JAC_CK(c, e);
     }
-    JAC_CK(c, cudaStreamSynchronize(c->stream));
+    if (wait) JAC_CK(c, cudaStreamSynchronize(c->stream));
     return JAC_OK;
 }
 
@@ -818,6 +818,9 @@ int run_sweeps(jac_ctx* c, int nsweeps, bool res, long long* nparts)
     }
     return JAC_OK;
 }
+
+// the square root of one device double, in place (correctly rounded, as std::sqrt on the host)
+__global__ void sqrt_in_place_kernel(double* v) { *v = sqrt(*v); }
 
 // fixed-order sum of the first nparts partial sums -> host, as a norm
 int finish_norm(jac_ctx* c, long long nparts, double* host_out_l2)
@@ -1126,6 +1129,39 @@ int jac_get_wide_buffer(jac_ctx* c, int64_t block, int face, double* host)
     const double* src = c->send + block * c->g.send_stride + c->g.face_off[face];
     JAC_CK(c, cudaMemcpyAsync(host, src, (size_t)c->g.wface_elems[face] * 8, cudaMemcpyDeviceToHost, c->stream));
     JAC_CK(c, cudaStreamSynchronize(c->stream));
+    return JAC_OK;
+}
+
+int jac_set_u_async(jac_ctx* c, const double* host_dense)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    if (!host_dense) return JAC_EINVAL;
+    c->ghosts_fresh = false;
+    c->packed_current = false;
+    return copy_dense_host(c, c->u[c->cur], const_cast<double*>(host_dense), true, false);
+}
+
+int jac_get_u_async(jac_ctx* c, double* host_dense)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    if (!host_dense) return JAC_EINVAL;
+    return copy_dense_host(c, c->u[c->cur], host_dense, false, false);
+}
+
+int jac_residual_async(jac_ctx* c, double* host_out_l2)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    if (!host_out_l2) return JAC_EINVAL;
+    if (!c->ghosts_fresh && (rc = do_exchange(c))) return rc;
+    if ((rc = launch_sweep<jac::OP_RESIDUAL>(c, c->u[c->cur], nullptr, 0, c->g.nblocks))) return rc;
+    jac::reduce_partials_kernel<<<1, 1024, 0, c->stream>>>(c->partials, c->g.nblocks * c->tile.ctas_per_block, c->result);
+    if ((rc = check_launch(c))) return rc;
+    sqrt_in_place_kernel<<<1, 1, 0, c->stream>>>(c->result);
+    if ((rc = check_launch(c))) return rc;
+    JAC_CK(c, cudaMemcpyAsync(host_out_l2, c->result, sizeof(double), cudaMemcpyDeviceToHost, c->stream));
     return JAC_OK;
 }
 

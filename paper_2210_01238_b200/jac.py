@@ -34,6 +34,7 @@ EXPORTS = [
     "jac_pack_halos", "jac_unpack_halos", "jac_pack_faces", "jac_unpack_faces", "jac_sweep", "jac_residual", "jac_launch_count",
     "jac_last_cuda_error", "jac_strerror", "jac_residual_dense_static", "jac_sweeps_per_launch",
     "jac_sweep_residual", "jac_solve", "jac_exchange_wide", "jac_get_wide_buffer",
+    "jac_set_u_async", "jac_get_u_async", "jac_residual_async",
 ]
 
 
@@ -74,7 +75,8 @@ def lib() -> C.CDLL:
         L.jac_create.argtypes = [C.POINTER(Desc), vp, C.c_size_t, C.POINTER(vp)]
         L.jac_destroy.argtypes = [vp]
         for name in ("jac_set_u", "jac_set_f", "jac_get_u", "jac_set_u_device",
-                     "jac_set_f_device", "jac_get_u_device"):
+                     "jac_set_f_device", "jac_get_u_device", "jac_set_u_async", "jac_get_u_async",
+                     "jac_residual_async"):
             getattr(L, name).argtypes = [vp, vp]
         L.jac_set_boundary.argtypes = [vp, C.c_int, C.c_double]
         L.jac_get_block_padded.argtypes = [vp, C.c_int64, vp]
@@ -272,6 +274,25 @@ class Jacobi:
         assert not t.is_cuda and t.dtype == self._torch.float64 and t.is_contiguous()
         self._call("jac_get_u", lib().jac_get_u(self._ctx, t.data_ptr()))
         return t
+
+    # ---- the same without waiting (pinned host tensors; synchronise the stream before reuse)
+    def _pinned_ptr(self, t, shape=None):
+        assert not t.is_cuda and t.is_pinned() and t.dtype == self._torch.float64 and t.is_contiguous()
+        assert shape is None or tuple(t.shape) == shape
+        return t.data_ptr()
+
+    def set_u_async(self, t):
+        self._call("jac_set_u_async", lib().jac_set_u_async(self._ctx, self._pinned_ptr(t, self.dense_shape)))
+
+    def get_u_async(self, t):
+        self._call("jac_get_u_async", lib().jac_get_u_async(self._ctx, self._pinned_ptr(t, self.dense_shape)))
+        return t
+
+    def residual_async(self, out):
+        """``out``: pinned float64 tensor with one element; holds the norm once the stream got there."""
+        assert out.numel() == 1
+        self._call("jac_residual_async", lib().jac_residual_async(self._ctx, self._pinned_ptr(out)))
+        return out
 
     def set_boundary(self, face: int, value: float):
         self._call("jac_set_boundary", lib().jac_set_boundary(self._ctx, int(face), float(value)))

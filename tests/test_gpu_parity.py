@@ -367,3 +367,47 @@ def test_work_is_issued_on_the_callers_stream(jac, orc):
     r = B.residual()
     assert abs(J1.residual() - r) <= RESID_TOL * r and abs(J2.residual() - r) <= RESID_TOL * r
     J1.close(); J2.close(); B.close()
+
+
+def test_asynchronous_copies_and_residual_pipeline(jac, orc):
+    """jac_set_u_async / jac_get_u_async / jac_residual_async on two contexts and two streams,
+    several jobs in flight with no host wait in between: every job's solution and norm are those
+    of the blocking calls, bit for bit."""
+    import torch
+    n, b, h = (256, 140), (128, 70), 1
+    rng = np.random.default_rng(5)
+    f = rng.uniform(-1, 1, (140, 256))
+    inputs_u = [rng.uniform(-1, 1, (140, 256)) for _ in range(4)]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    ctxs = [jac.Jacobi(n, b, h, True, "temporal", stream=s) for s in streams]
+    for J in ctxs:
+        J.set_f(f)
+    host_in = [torch.from_numpy(u).pin_memory() for u in inputs_u]
+    host_out = [torch.empty(140, 256, dtype=torch.float64).pin_memory() for _ in range(4)]
+    norms = [torch.zeros(1, dtype=torch.float64).pin_memory() for _ in range(4)]
+    for k in range(4):
+        J = ctxs[k % 2]
+        J.set_u_async(host_in[k])
+        J.sweep(9)
+        J.residual_async(norms[k])
+        J.get_u_async(host_out[k])
+    for s in streams:
+        s.synchronize()
+    for k in range(4):
+        B = orc.Blocked(n, b, h, True)
+        B.set_u(inputs_u[k]); B.set_f(f)
+        B.sweep(9)
+        assert np.array_equal(host_out[k].numpy(), B.get_u()), k
+        want = B.residual()
+        assert abs(float(norms[k][0]) - want) <= RESID_TOL * want
+        B.close()
+    # the asynchronous norm has the bits of the blocking one
+    J = ctxs[0]
+    J.set_u(inputs_u[0]); J.sweep(3)
+    r = J.residual()
+    J.residual_async(norms[0]); streams[0].synchronize()
+    assert float(norms[0][0]) == r
+    with pytest.raises(AssertionError):
+        J.set_u_async(torch.from_numpy(inputs_u[0]))      # pageable memory is refused by the binding
+    for J in ctxs:
+        J.close()
