@@ -383,7 +383,8 @@ def run_ours(args, w: inputs.Workload):
         # directions and the SMs are separate engines; a step is three stages long, so three
         # contexts keep all of them busy).  Every step still copies its input in and its solution
         # and residual out inside the timed region.
-        if u0.nbytes <= 4 * 2 ** 30:
+        # (single-process runs only: every rank of a multi-GPU run would pin another 8 GiB of host memory)
+        if u0.nbytes <= 4 * 2 ** 30 and world == 1:
             J.close()
             J = None
             depth = 3
