@@ -24,6 +24,9 @@ __device__ __forceinline__ double add_rn(double a, double b) { return __dadd_rn(
 __device__ __forceinline__ double sub_rn(double a, double b) { return __dsub_rn(a, b); }
 __device__ __forceinline__ double mul_rn(double a, double b) { return __dmul_rn(a, b); }
 
+// ask for a line to be brought into L2
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];\n" ::"l"(p)); }
+
 // NV consecutive doubles held by one thread (NV = 1 or 2; NV = 2 uses one 128-bit access).
 template <int NV> struct Vec { double v[NV]; };
 
@@ -136,11 +139,20 @@ sweep2d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
             gy0 = (blk / g.gx) * (long long)(g.by - 2 * g.ext) - g.ext;
         }
 
+        // a thread at a block border reads its west / east neighbour from the next block: one
+        // 32-byte sector per row that no other thread touches; asked for a few rows ahead, or the
+        // whole warp waits for DRAM in every row
+        const bool far_w = op_pulls(OP) && off_w != -1, far_e = op_pulls(OP) && off_e != NV;
+
         Vec<NV> S = load_vec<NV>(ub + (j0 == 0 ? off_s0 : (long long)(j0 - 1) * PX));
         Vec<NV> Cc = load_vec<NV>(ub + (long long)j0 * PX);
 #pragma unroll 4
         for (int j = j0; j < j1; ++j) {
             const long long ro = (long long)j * PX;
+            if (op_pulls(OP) && j + 8 < j1) {
+                if (far_w) prefetch_l2(ub + ro + 8 * PX + off_w);
+                if (far_e) prefetch_l2(ub + ro + 8 * PX + off_e);
+            }
             const Vec<NV> N = load_vec<NV>(ub + ro + ((op_pulls(OP) && j + 1 == g.by) ? off_n1 : PX));
             const double w = ub[ro + off_w];
             const double e = ub[ro + off_e];
@@ -231,11 +243,18 @@ sweep3d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
             gz0 = (blk / ((long long)g.gx * g.gy)) * (long long)(g.bz - 2 * g.ext) - g.ext;
         }
 
+        // far west / east neighbours (the next block's column): asked for a few planes ahead, as in 2D
+        const bool far_w = op_pulls(OP) && off_w != -1, far_e = op_pulls(OP) && off_e != NV;
+
         Vec<NV> D = load_vec<NV>(ub + (k0 == 0 ? off_d0 : (long long)(k0 - 1) * PXY));
         Vec<NV> Cc = load_vec<NV>(ub + (long long)k0 * PXY);
 #pragma unroll 2
         for (int k = k0; k < k1; ++k) {
             const long long po = (long long)k * PXY;
+            if (op_pulls(OP) && k + 4 < k1) {
+                if (far_w) prefetch_l2(ub + po + 4 * PXY + off_w);
+                if (far_e) prefetch_l2(ub + po + 4 * PXY + off_e);
+            }
             const Vec<NV> U = load_vec<NV>(ub + po + ((op_pulls(OP) && k + 1 == g.bz) ? off_u1 : PXY));
             const Vec<NV> S = load_vec<NV>(ub + po + off_s);
             const Vec<NV> N = load_vec<NV>(ub + po + off_n);
