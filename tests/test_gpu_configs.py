@@ -273,3 +273,45 @@ def test_offsets_beyond_2_to_31_elements(jac, orc):
         got = np.array([float(out[p[1], p[0]]) for p in pts])
         assert np.array_equal(got, want), (mode, got - want)
         del out
+
+
+# ------------------------------------------------------------------ the later schedules at full size
+def test_full_size_wide_schedule_and_remainder_blocks(jac, orc):
+    """16384^2 in 1024^2 blocks with four ghost layers and one wide exchange per four sweeps, and a
+    16000 x 15000 grid in 1024^2 blocks (remainder blocks of 640 and 664 points) in the exchange,
+    fused and temporal schedules: whole fields against the oracle."""
+    rng = np.random.default_rng(12)
+    n, b, sweeps = (16384, 16384), (1024, 1024), 24
+    u0 = rng.uniform(-1, 1, (n[1], n[0]))
+    B = orc.Blocked(n, b, 4)
+    B.set_boundary(3, 1.0)
+    B.set_u(u0)
+    B.sweep(sweeps)
+    want, want_r = B.get_u(), B.residual()
+    B.close()
+    with jac.Jacobi(n, b, 4, False, "wide", 4) as J:
+        J.set_boundary(3, 1.0)
+        J.set_u(u0)
+        J.sweep(sweeps)
+        assert np.array_equal(J.get_u(), want)
+        r = J.residual()
+        assert abs(r - want_r) <= RESID_TOL * want_r
+    del want
+
+    n = (16000, 15000)
+    u0 = np.ascontiguousarray(u0[: n[1], : n[0]])
+    f = rng.uniform(-1, 1, (n[1], n[0]))
+    B = orc.Blocked(n, b, 1, True)
+    B.set_boundary(0, -0.5)
+    B.set_u(u0); B.set_f(f)
+    B.sweep(sweeps)
+    want, want_r = B.get_u(), B.residual()
+    B.close()
+    for mode, ts in (("temporal", 0), ("temporal", 8), ("fused", 0), ("exchange", 0)):
+        with jac.Jacobi(n, b, 1, True, mode, ts) as J:
+            J.set_boundary(0, -0.5)
+            J.set_u(u0); J.set_f(f)
+            J.sweep(sweeps)
+            assert np.array_equal(J.get_u(), want), mode
+            r = J.residual()
+            assert abs(r - want_r) <= RESID_TOL * want_r
