@@ -327,7 +327,13 @@ def run_ours(args, w: inputs.Workload):
         tsteps = tsteps or 4
     elif mode not in ("temporal", "resident"):      # resident: tsteps is the cluster size (0 = library's)
         tsteps = 1
-    J = make_ctx(mode, tsteps)
+    try:
+        J = make_ctx(mode, tsteps)
+    except jac.JacError:
+        if mode != "resident" or args.mode != "auto":
+            raise
+        mode, tsteps = "temporal", 0      # the device cannot co-schedule the cluster: next best schedule
+        J = make_ctx(mode, tsteps)
     if mode not in ("wide", "resident"):
         tsteps = J.sweeps_per_launch()
     main_run = time_schedule(J, mode, tsteps, args.steps, args.warmup, True)
