@@ -191,6 +191,14 @@ int jac_pack_halos(jac_ctx *ctx);
  * unpack is the neighbour reading the send buffer in place. */
 int jac_unpack_halos(jac_ctx *ctx);
 
+/* jac_pack_halos followed by jac_unpack_halos as ONE launch: the thread that fills a ghost cell
+ * reads the neighbour's interior cell and also leaves it in the neighbour's send slot, so the send
+ * buffers and the ghosts are afterwards exactly what the two calls leave (one read and two writes
+ * per face cell instead of two and two).  On one GPU, where the "transfer" between pack and unpack
+ * (paper Section V-C) is a read in place, nothing is lost by not stopping in between; jac_residual
+ * uses it when the ghosts are stale. */
+int jac_exchange_halos(jac_ctx *ctx);
+
 /* Pack / unpack only the faces whose bit is set in face_mask (bit i = face i).  Same kernels
  * and buffers as jac_pack_halos / jac_unpack_halos, one launch over all blocks; a mask with all
  * 2*ndim bits set is exactly those calls.  A partial exchange never marks the ghosts as current.
@@ -243,7 +251,8 @@ int jac_solve(jac_ctx *ctx, int max_sweeps, int check_every, double tol, int *ho
 /* L2 norm of the residual of the current state, sqrt( sum_p ( s(p) - c*u(p) )^2 ) with s as in
  * the update (including + f), over all interior points, not normalised.  (The paper runs a
  * fixed iteration count and has no residual; this is the convergence measure of the same
- * Jacobi method.)  Exchanges halos first if the ghosts are stale, reduces on the device in a
+ * Jacobi method.)  Exchanges halos first if the ghosts are stale (jac_exchange_halos; pack and
+ * unpack per block face in JAC_MODE_PERTASK), reduces on the device in a
  * fixed order (repeatable bit for bit), synchronises the stream and writes one HOST double. */
 int jac_residual(jac_ctx *ctx, double *host_out_l2);
 

@@ -413,6 +413,24 @@ int do_unpack(jac_ctx* c)
     return c->desc.mode == JAC_MODE_PERTASK ? launch_halo_pertask<true>(c) : launch_halo_all<true>(c);
 }
 
+// pack and unpack of all faces in one launch (same buffers and ghosts afterwards)
+int do_exchange_fused(jac_ctx* c)
+{
+    const int slots = halo_slots(c, 0x3fu);
+    const long long npairs = c->g.nblocks * c->g.nfaces;
+    const long long ctas = ceil_div(npairs * slots, 256);
+    if (ctas > kMaxGrid) return JAC_EINVAL;
+    if (ctas * 256 < (1LL << 32) && npairs < (1LL << 31))
+        jac::halo_exchange_kernel<unsigned><<<(unsigned)ctas, 256, 0, c->stream>>>(c->u[c->cur], c->send, c->g, npairs, slots);
+    else
+        jac::halo_exchange_kernel<long long><<<(unsigned)ctas, 256, 0, c->stream>>>(c->u[c->cur], c->send, c->g, npairs, slots);
+    const int rc = check_launch(c);
+    if (rc) return rc;
+    c->packed_current = true;
+    c->ghosts_fresh = true;
+    return JAC_OK;
+}
+
 int do_exchange(jac_ctx* c)
 {
     int rc = do_pack(c);
@@ -1036,6 +1054,13 @@ int jac_unpack_halos(jac_ctx* c)
     return JAC_OK;
 }
 
+int jac_exchange_halos(jac_ctx* c)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    return do_exchange_fused(c);
+}
+
 int jac_pack_faces(jac_ctx* c, unsigned face_mask)
 {
     int rc = usable(c);
@@ -1104,7 +1129,7 @@ int jac_residual(jac_ctx* c, double* host_out_l2)
     int rc = usable(c);
     if (rc) return rc;
     if (!host_out_l2) return JAC_EINVAL;
-    if (!c->ghosts_fresh && (rc = do_exchange(c))) return rc;
+    if (!c->ghosts_fresh && (rc = (c->desc.mode == JAC_MODE_PERTASK ? do_exchange(c) : do_exchange_fused(c)))) return rc;
     if ((rc = launch_sweep<jac::OP_RESIDUAL>(c, c->u[c->cur], nullptr, 0, c->g.nblocks))) return rc;
     return finish_norm(c, c->g.nblocks * c->tile.ctas_per_block, host_out_l2);
 }
@@ -1155,7 +1180,7 @@ int jac_residual_async(jac_ctx* c, double* host_out_l2)
     int rc = usable(c);
     if (rc) return rc;
     if (!host_out_l2) return JAC_EINVAL;
-    if (!c->ghosts_fresh && (rc = do_exchange(c))) return rc;
+    if (!c->ghosts_fresh && (rc = (c->desc.mode == JAC_MODE_PERTASK ? do_exchange(c) : do_exchange_fused(c)))) return rc;
     if ((rc = launch_sweep<jac::OP_RESIDUAL>(c, c->u[c->cur], nullptr, 0, c->g.nblocks))) return rc;
     jac::reduce_partials_kernel<<<1, 1024, 0, c->stream>>>(c->partials, c->g.nblocks * c->tile.ctas_per_block, c->result);
     if ((rc = check_launch(c))) return rc;

@@ -421,6 +421,50 @@ halo_kernel(double* __restrict__ u, double* __restrict__ send, const JacGeom g,
     }
 }
 
+// Pack and unpack in one launch: the thread that fills ghost cells of (block, face) reads them from
+// the neighbour's interior strip and also leaves them in the neighbour's send slot, so that the
+// buffers and the ghosts end up exactly as after halo_kernel<false> followed by halo_kernel<true>.
+// One read and two writes per face cell instead of two reads and two writes, and one launch.
+template <typename IT>
+__global__ void __launch_bounds__(256)
+halo_exchange_kernel(double* __restrict__ u, double* __restrict__ send, const JacGeom g, const long long npairs,
+                     const int slots)
+{
+    const IT t = (IT)blockIdx.x * (IT)blockDim.x + (IT)threadIdx.x;
+    const IT pr = t / (IT)slots;
+    if (pr >= (IT)npairs) return;
+    const unsigned e = 2u * (unsigned)(t - pr * (IT)slots);
+    const IT blk = pr / (IT)g.nfaces;
+    const int face = (int)(pr - blk * (IT)g.nfaces);
+    const BlockPlace<IT> bp = block_place<IT>(g, blk, face);
+    if (!bp.has_nb) return;
+    const BlockExtent& be = bp.ext;      // the neighbour has the same extent on the axes the strip spans
+    const long long n = face_elems_of(g, be, face);
+    if (e >= n) return;
+    const int axis = face >> 1;
+    const int full = axis == 0 ? g.bx : (axis == 1 ? g.by : g.bz);   // both blocks of such a pair are
+    // full along the axis, or the one at the high end is the remainder block: its strip starts at 0
+    const int lo_src = (face & 1) ? 0 : full - g.h;                  // the neighbour's interior strip facing us
+    const int lo_dst = (face & 1) ? (axis == 0 ? be.x : (axis == 1 ? be.y : be.z)) : -g.h;   // our ghost strip
+    const double* src = u + (long long)bp.nb * g.block_stride + g.origin;
+    double* dst = u + (long long)blk * g.block_stride + g.origin;
+    double* buf = send + (long long)bp.nb * g.send_stride + g.face_off[face ^ 1];
+    if (axis != 0 && (be.x & 1) == 0) {
+        const double2 v = *reinterpret_cast<const double2*>(src + strip_offset(g, be, face, e, lo_src));
+        *reinterpret_cast<double2*>(buf + e) = v;
+        *reinterpret_cast<double2*>(dst + strip_offset(g, be, face, e, lo_dst)) = v;
+    } else {
+        const double v0 = src[strip_offset(g, be, face, e, lo_src)];
+        buf[e] = v0;
+        dst[strip_offset(g, be, face, e, lo_dst)] = v0;
+        if (e + 1 < n) {
+            const double v1 = src[strip_offset(g, be, face, e + 1, lo_src)];
+            buf[e + 1] = v1;
+            dst[strip_offset(g, be, face, e + 1, lo_dst)] = v1;
+        }
+    }
+}
+
 // Wide exchange, one axis per launch: the strip of a face is h layers along `axis` (interior
 // layers for pack, ghost layers for unpack) over the whole padded extent (-h .. extent + h) of the
 // other axes, so edge and corner data delivered by the launches of earlier axes travels on.

@@ -5,7 +5,8 @@
 For a block edge B the domain is a G x G grid of blocks (G = 64, 32, 8, 4) so that every kind of
 face has interior instances: 4 G (G-1) faces are exchanged per call.  Data: Uniform[-1,1], seed 2.
 Each operation (pack, unpack, pack+unpack; x faces = strided columns, y faces = contiguous rows,
-all faces) is repeated until `--total-gib` of face payload has moved, and reported as
+all faces; for all faces also the exchange that does pack and unpack in one launch, counted with
+the bytes of pack + unpack) is repeated until `--total-gib` of face payload has moved, and reported as
 
     GB/s = 2 x payload x repetitions / time          (read + write of every face cell)
 
@@ -75,8 +76,10 @@ def run(sizes, widths, total_gib):
                     ops = {"pack": lambda m=mask: J.pack_faces(m),
                            "unpack": lambda m=mask: J.unpack_faces(m),
                            "pack+unpack": lambda m=mask: (J.pack_faces(m), J.unpack_faces(m))}
+                    if kind == "all":     # the same end state from one launch; counted like pack + unpack
+                        ops["exchange"] = lambda: J.exchange_halos()
                     for name, fn in ops.items():
-                        mult = 2 if name == "pack+unpack" else 1
+                        mult = 2 if name in ("pack+unpack", "exchange") else 1
                         th = _time_hot(torch, stream, fn, reps)
                         tc = _time_cold(torch, stream, fn, reps, flush)
                         rec[f"{kind}:{name}"] = {
@@ -86,10 +89,11 @@ def run(sizes, widths, total_gib):
                 rows.append(rec)
                 print(json.dumps(rec), flush=True)
     hdr = f"{'block':>6} {'h':>2} {'faces':>6} {'payload MB':>10} | " + " | ".join(
-        f"{k:>22}" for k in ("x pack hot/cold GB/s", "y pack hot/cold GB/s", "all p+u hot/cold GB/s"))
+        f"{k:>22}" for k in ("x pack hot/cold GB/s", "y pack hot/cold GB/s", "all p+u hot/cold GB/s",
+                             "one launch hot/cold"))
     print(hdr, file=sys.stderr)
     for r in rows:
-        cells = [r["x:pack"], r["y:pack"], r["all:pack+unpack"]]
+        cells = [r["x:pack"], r["y:pack"], r["all:pack+unpack"], r["all:exchange"]]
         print(f"{r['block']:>6} {r['halo']:>2} {4 * r['grid'] * (r['grid'] - 1):>6} "
               f"{r['payload_bytes_per_call'] / 1e6:>10.2f} | " +
               " | ".join(f"{c['hot_gbs']:>10.0f} /{c['cold_gbs']:>9.0f}" for c in cells), file=sys.stderr)

@@ -34,7 +34,7 @@ EXPORTS = [
     "jac_pack_halos", "jac_unpack_halos", "jac_pack_faces", "jac_unpack_faces", "jac_sweep", "jac_residual", "jac_launch_count",
     "jac_last_cuda_error", "jac_strerror", "jac_residual_dense_static", "jac_sweeps_per_launch",
     "jac_sweep_residual", "jac_solve", "jac_exchange_wide", "jac_get_wide_buffer",
-    "jac_set_u_async", "jac_get_u_async", "jac_residual_async",
+    "jac_set_u_async", "jac_get_u_async", "jac_residual_async", "jac_exchange_halos",
 ]
 
 
@@ -83,6 +83,7 @@ def lib() -> C.CDLL:
         L.jac_get_halo_buffer.argtypes = [vp, C.c_int64, C.c_int, vp]
         L.jac_exchange_wide.argtypes = [vp]
         L.jac_get_wide_buffer.argtypes = [vp, C.c_int64, C.c_int, vp]
+        L.jac_exchange_halos.argtypes = [vp]
         L.jac_pack_halos.argtypes = [vp]
         L.jac_unpack_halos.argtypes = [vp]
         L.jac_pack_faces.argtypes = [vp, C.c_uint]
@@ -325,6 +326,10 @@ class Jacobi:
 
     def unpack_halos(self):
         self._call("jac_unpack_halos", lib().jac_unpack_halos(self._ctx))
+
+    def exchange_halos(self):
+        """pack_halos + unpack_halos as one launch."""
+        self._call("jac_exchange_halos", lib().jac_exchange_halos(self._ctx))
 
     def pack_faces(self, face_mask: int):
         self._call("jac_pack_faces", lib().jac_pack_faces(self._ctx, int(face_mask)))

@@ -411,3 +411,23 @@ def test_asynchronous_copies_and_residual_pipeline(jac, orc):
         J.set_u_async(torch.from_numpy(inputs_u[0]))      # pageable memory is refused by the binding
     for J in ctxs:
         J.close()
+
+
+@pytest.mark.parametrize("n,b,h", SHAPES_2D + SHAPES_3D + [((14, 11), (4, 4), 2), ((9, 5, 7), (4, 2, 3), 1)])
+def test_one_launch_exchange_leaves_what_pack_and_unpack_leave(jac, orc, n, b, h):
+    ndim = len(n)
+    dense = inputs.linear_index_field(n)
+    A = jac.Jacobi(n, b, h, False, "exchange")
+    B = orc.Blocked(n, b, h)
+    for face in range(2 * ndim):
+        A.set_boundary(face, BVALS[face]); B.set_boundary(face, BVALS[face])
+    A.set_u(dense); B.set_u(dense)
+    A.exchange_halos()
+    B.pack(); B.unpack()
+    for blk in range(B.nblocks):
+        for face in range(2 * ndim):
+            if B.neighbour(blk, face) >= 0:
+                assert np.array_equal(A.get_halo_buffer(blk, face), B.get_halo_buffer(blk, face)), (blk, face)
+        assert np.array_equal(A.get_block_padded(blk), B.get_block_padded(blk)), blk
+    assert np.array_equal(A.get_u(), dense)
+    A.close(); B.close()
