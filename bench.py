@@ -50,16 +50,16 @@ L2_BYTES = 126e6
 SWEEP_SOURCES = ("jac_kernels.cuh", "jac_geom.h", "jac.cu")
 NCU_TRAFFIC = {
     # profiles/temporal2d_eigenmode_8192.md
-    ("temporal", 8, 2, False): {"bytes_per_point_per_launch": (592.694528e6 + 491.509248e6) / 8192 ** 2,
-                                "src": SWEEP_SOURCES, "src_sha": "247781e3c6c69f24"},
-    ("temporal", 4, 2, False): {"bytes_per_point_per_launch": (606.842368e6 + 488.531712e6) / 8192 ** 2,
-                                "src": SWEEP_SOURCES, "src_sha": "247781e3c6c69f24"},
+    ("temporal", 8, 2, False): {"bytes_per_point_per_launch": (592.426752e6 + 492.332288e6) / 8192 ** 2,
+                                "src": SWEEP_SOURCES, "src_sha": "6926e351d1db4903"},
+    ("temporal", 4, 2, False): {"bytes_per_point_per_launch": (606.767616e6 + 489.245952e6) / 8192 ** 2,
+                                "src": SWEEP_SOURCES, "src_sha": "6926e351d1db4903"},
     # profiles/temporal3d_poisson_512.md
-    ("temporal", 2, 3, True): {"bytes_per_point_per_launch": (2.495436e9 + 1.047913e9) / 512 ** 3,
-                               "src": SWEEP_SOURCES, "src_sha": "247781e3c6c69f24"},
+    ("temporal", 2, 3, True): {"bytes_per_point_per_launch": (2.497970e9 + 1.048288e9) / 512 ** 3,
+                               "src": SWEEP_SOURCES, "src_sha": "6926e351d1db4903"},
     # profiles/exchange_schedule_eigenmode_8192.md (the update launch alone)
-    ("exchange", 1, 2, False): {"bytes_per_point_per_launch": (574.365696e6 + 494.292480e6) / 8192 ** 2,
-                                "src": SWEEP_SOURCES, "src_sha": "247781e3c6c69f24"},
+    ("exchange", 1, 2, False): {"bytes_per_point_per_launch": (574.306816e6 + 495.150336e6) / 8192 ** 2,
+                                "src": SWEEP_SOURCES, "src_sha": "6926e351d1db4903"},
 }
 KERNEL_NAMES = {("temporal", 2): "temporal2d_kernel", ("temporal", 3): "temporal3d_kernel", ("fused", 2): "sweep2d_kernel (update pulling neighbour interiors)",
                 ("exchange", 2): "sweep2d_kernel", ("pertask", 2): "sweep2d_kernel (one launch per block)",
