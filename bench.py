@@ -166,9 +166,17 @@ def oracle_time_job(w: inputs.Workload, u0, f, target_seconds: float, max_sweeps
     B.sweep(1)
     t1 = time.perf_counter() - t0
     sweeps = int(max(1, min(max_sweeps, target_seconds / max(t1, 1e-9))))
+    every = w.residual_every if w.residual_every > 0 else 0
+    if every:
+        sweeps = max(every, sweeps // every * every)     # whole groups: `every` sweeps, then the residual
     t0 = time.perf_counter()
-    B.sweep(sweeps)
-    B.residual()
+    if every:
+        for _ in range(sweeps // every):
+            B.sweep(every)
+            B.residual()
+    else:
+        B.sweep(sweeps)
+        B.residual()
     dt = time.perf_counter() - t0
     B.close()
     return job_updates(w, sweeps) / dt / 1e9, sweeps, dt, orc.max_threads()
@@ -282,43 +290,59 @@ def run_ours(args, w: inputs.Workload):
             J.set_f(f)
         return J
 
+    # the workload's cadence: a residual after every `every` sweeps (0: only after the last sweep)
+    every = w.residual_every if 0 < w.residual_every <= sweeps else sweeps
+    groups = [every] * (sweeps // every) + ([sweeps % every] if sweeps % every else [])
+    norms = torch.zeros(len(groups), dtype=torch.float64).pin_memory()
+
+    def one_job(J, pairs=None):
+        """The sweeps of one step with the residual after every group (queued, nothing waits)."""
+        for k, n_sw in enumerate(groups):
+            if pairs is not None:
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+            J.sweep(n_sw)
+            if pairs is not None:
+                b.record(stream)
+                pairs.append((a, b))
+            J.residual_async(norms[k:k + 1])
+
     def time_schedule(J, mode, tsteps, steps, warmup, sample_clocks):
-        """K steps (each: input -> blocks, the sweeps, the residual) between two barriers, timed
-        with CUDA events on the launch stream; the sweep calls are also timed on their own."""
-        res = None
+        """K steps (each: input -> blocks, the sweeps, a residual after every group of sweeps the
+        workload names) between two barriers, timed with CUDA events on the launch stream; the sweep
+        calls are also timed on their own."""
         for _ in range(warmup):
             J.set_u_device(u0_dev)
-            J.sweep(sweeps)
-            res = J.residual()
+            one_job(J)
         barrier()
         sampler = ClockSampler(uuid) if sample_clocks else None
         if sampler:
             sampler.start()
         l0 = J.launch_count()
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        pairs = []
+        step_pairs = []
         ev0.record(stream)
         for _ in range(steps):
             J.set_u_device(u0_dev)
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            J.sweep(sweeps)
-            b.record(stream)
-            res = J.residual()
-            pairs.append((a, b))
+            pairs = []
+            one_job(J, pairs)
+            step_pairs.append(pairs)
         ev1.record(stream)
         barrier()
         launches = J.launch_count() - l0
         clocks = sampler.stop() if sampler else None
         ms_total = max_over_ranks(ev0.elapsed_time(ev1))
-        per_step = sorted(a.elapsed_time(b) for a, b in pairs)
+        per_step = sorted(sum(a.elapsed_time(b) for a, b in pairs) for pairs in step_pairs)
         sweep_ms = sum(per_step)
-        n_launch = -(-sweeps // tsteps) if mode == "temporal" else (1 if mode == "resident" else sweeps)
+        if mode == "temporal":
+            n_launch = sum(-(-n_sw // tsteps) for n_sw in groups)
+        else:
+            n_launch = len(groups) if mode == "resident" else sweeps
         glups = replicated_glups(job_updates(w, sweeps) * steps, world, ms_total)
         return {"glups": glups, "ms_total": ms_total, "launch_ms": sweep_ms / (steps * n_launch),
                 "launch_ms_best": per_step[0] / n_launch, "launch_ms_median": statistics.median(per_step) / n_launch,
-                "sweeps_per_launch": sweeps / n_launch, "launches": int(launches), "residual": res,
-                "clocks": clocks}
+                "sweeps_per_launch": sweeps / n_launch, "launches": int(launches), "residual": float(norms[-1]),
+                "residuals_per_step": len(groups), "clocks": clocks}
 
     mode, tsteps = args.mode, args.tsteps
     if mode == "auto":
@@ -361,88 +385,92 @@ def run_ours(args, w: inputs.Workload):
                          "launch time is the mean over the timed jac_sweep calls"
                          + (" and includes the pack and unpack launches" if mode == "exchange" else ""))}
 
-    # ---- end to end through the C ABI with host buffers: H2D of u0, the job, D2H of the solution
+    # ---- end to end through the C ABI with HOST buffers: every step copies its input from pinned
+    # host memory into the context (jac_set_u_async), runs the job, and copies the solution and
+    # the residual norms back (jac_get_u_async, jac_residual_async) inside the timed region.  The
+    # contexts carry JAC_FLAG_HOST_STAGING: one contiguous copy per direction plus a kernel
+    # between the dense staging array and the blocks; the copy in runs on the context's own copy
+    # stream and overlaps the previous step's sweeps and copy out.
+    J.close()
+    J = None
     e2e = None
     if not args.no_e2e:
         host_in = torch.from_numpy(u0).pin_memory()
-        host_out = torch.empty_like(host_in).pin_memory()
-        e2e_steps = max(1, min(args.steps, 3))
-        J.set_u_pinned(host_in); J.sweep(1); J.get_u_pinned(host_out)   # warm the path
-        barrier()
-        t0 = time.perf_counter()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(e2e_steps):
-            J.set_u_pinned(host_in)
-            J.sweep(sweeps)
-            J.residual()
-            J.get_u_pinned(host_out)
-        e1.record(stream)
-        barrier()
-        wall = time.perf_counter() - t0
-        # the copies run on the stream, so the events see them; host-side gaps count too
-        ms_e2e = max_over_ranks(max(e0.elapsed_time(e1), wall * 1e3))
-        e2e = {"value": job_updates(w, sweeps) * e2e_steps * world / (ms_e2e * 1e-3) / 1e9, "unit": UNIT,
-               "h2d_bytes_per_step": int(u0.nbytes), "d2h_bytes_per_step": int(u0.nbytes) + 8,
-               "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps,
-               "what": "jac_set_u(pinned host) + jac_sweep + jac_residual + jac_get_u(pinned host)"}
-        # The same job as a pipeline: three contexts on three streams, steps going round them,
-        # nothing waits on the host until the end.  The input copy of one step, the sweeps of the
-        # previous one and the output copy of the one before run at the same time (the two copy
-        # directions and the SMs are separate engines; a step is three stages long, so three
-        # contexts keep all of them busy).  Every step still copies its input in and its solution
-        # and residual out inside the timed region.
-        # (single-process runs only: every rank of a multi-GPU run would pin another 8 GiB of host memory)
-        if u0.nbytes <= 4 * 2 ** 30 and world == 1:
-            J.close()
-            J = None
-            depth = 3
+        nbytes = int(u0.nbytes)
+
+        def job_norms():
+            return torch.zeros(len(groups), dtype=torch.float64).pin_memory()
+
+        def staged_ctx(on_stream):
+            halo = max(w.halo, tsteps) if mode == "wide" else w.halo
+            Jc = jac.Jacobi(w.n, w.b, halo, w.has_f, mode, tsteps, stream=on_stream, flags=jac.FLAG_HOST_STAGING)
+            for face, v in enumerate(w.boundary()):
+                Jc.set_boundary(face, v)
+            if f is not None:
+                Jc.set_f(f)
+            return Jc
+
+        def e2e_step(Jc, out, nrm):
+            Jc.set_u_async(host_in)
+            for k, n_sw in enumerate(groups):
+                Jc.sweep(n_sw)
+                Jc.residual_async(nrm[k:k + 1])
+            Jc.get_u_async(out)
+
+        def run_pipeline(depth, count):
+            """`count` steps going round `depth` contexts on `depth` streams; host clock between
+            synchronisations of all streams (fill and drain of the pipeline inside the timed region)."""
             streams = [torch.cuda.Stream() for _ in range(depth)]
-            ctxs = [make_ctx(mode, tsteps, st) for st in streams]
+            ctxs = [staged_ctx(st) for st in streams]
             outs = [torch.empty_like(host_in).pin_memory() for _ in range(depth)]
-            norms = [torch.zeros(1, dtype=torch.float64).pin_memory() for _ in range(depth)]
-
-            # dense device arrays between the host and the blocks: one contiguous copy per direction
-            # (the per-block strided copies of jac_set_u_async were measured not to overlap as well)
-            stage_in = [torch.empty_like(u0_dev) for _ in range(depth)]
-            stage_out = [torch.empty_like(u0_dev) for _ in range(depth)]
-
-            def pipelined_steps(count):
-                for k in range(count):
-                    i = k % depth
-                    Jp = ctxs[i]
-                    with torch.cuda.stream(streams[i]):
-                        stage_in[i].copy_(host_in, non_blocking=True)
-                        Jp.set_u_device(stage_in[i])
-                        Jp.sweep(sweeps)
-                        Jp.residual_async(norms[i])
-                        Jp.get_u_device(stage_out[i])
-                        outs[i].copy_(stage_out[i], non_blocking=True)
-
-            pipe_steps = max(2 * depth, args.steps)   # fill and drain of the pipeline are inside the timed region
-            pipelined_steps(depth)                   # warm every context
-            barrier()
-            t0 = time.perf_counter()
-            pipelined_steps(pipe_steps)
+            nrms = [job_norms() for _ in range(depth)]
+            for i in range(depth):                                   # warm every context
+                e2e_step(ctxs[i], outs[i], nrms[i])
             for st in streams:
                 st.synchronize()
             barrier()
-            ms_pipe = max_over_ranks((time.perf_counter() - t0) * 1e3)
-            assert abs(float(norms[0][0]) - main_run["residual"]) <= 1e-10 * main_run["residual"]
-            e2e = {"value": job_updates(w, sweeps) * pipe_steps * world / (ms_pipe * 1e-3) / 1e9, "unit": UNIT,
-                   "h2d_bytes_per_step": int(u0.nbytes), "d2h_bytes_per_step": int(u0.nbytes) + 8,
-                   "steps": pipe_steps, "ms_per_step": ms_pipe / pipe_steps,
-                   "what": "three contexts on three streams, steps going round them: pinned host -> dense device array "
-                           "(one copy) + jac_set_u_device + jac_sweep + jac_residual_async + jac_get_u_device + dense "
-                           "device array -> pinned host; timed by the host clock between synchronisations of all streams",
-                   "one_context": {"value": e2e["value"], "ms_per_step": e2e["ms_per_step"], "steps": e2e["steps"],
-                                   "what": e2e["what"]}}
-            for Jp in ctxs:
-                Jp.close()
-            del outs, norms, stage_in, stage_out
-        del host_in, host_out
-    if J is not None:
-        J.close()
+            t0 = time.perf_counter()
+            for k in range(count):
+                i = k % depth
+                e2e_step(ctxs[i], outs[i], nrms[i])
+            for st in streams:
+                st.synchronize()
+            barrier()
+            ms = max_over_ranks((time.perf_counter() - t0) * 1e3)
+            last = float(nrms[(count - 1) % depth][-1])
+            assert abs(last - main_run["residual"]) <= 1e-10 * main_run["residual"], (last, main_run["residual"])
+            for Jc in ctxs:
+                Jc.close()
+            return ms
+
+        def e2e_record(ms, count, what):
+            return {"value": job_updates(w, sweeps) * count * world / (ms * 1e-3) / 1e9, "unit": UNIT,
+                    "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": nbytes + 8 * len(groups),
+                    "steps": count, "ms_per_step": ms / count,
+                    "pcie_gbs_per_direction": nbytes / (ms / count * 1e-3) / 1e9, "what": what}
+
+        one_steps = max(3, min(args.steps, 6))
+        one = e2e_record(run_pipeline(1, one_steps), one_steps,
+                         "one context, steps queued back to back on one stream: jac_set_u_async(pinned host) + jac_sweep + "
+                         "jac_residual_async per group + jac_get_u_async(pinned host)")
+        e2e = one
+        # several contexts on as many streams, steps going round them: the copy in of one step, the
+        # sweeps of another and the copy out of a third run at the same time (the two copy directions
+        # and the SMs are separate engines).  Single-process runs only: every rank of a multi-GPU run
+        # would pin several more GiB of host memory.
+        if nbytes <= 4 * 2 ** 30 and world == 1:
+            depth = 3
+            pipe_steps = max(2 * depth, args.steps)
+            e2e = e2e_record(run_pipeline(depth, pipe_steps), pipe_steps,
+                             f"{depth} contexts on {depth} streams, steps going round them; every step is jac_set_u_async(pinned "
+                             "host) + jac_sweep + jac_residual_async per group + jac_get_u_async(pinned host); timed by the host "
+                             "clock between synchronisations of all streams")
+            e2e["one_context"] = one
+        bound_ms = 2 * nbytes / 55e9 * 1e3
+        e2e["note"] = ("bound by the host link when the copies take longer than the sweeps: at about 55 GB/s per direction "
+                       f"{nbytes / 2 ** 30:.2f} GiB in and out are {bound_ms / 2:.1f} ms each against "
+                       f"{main_run['ms_total'] / args.steps:.1f} ms of device work per step")
+        del host_in
 
     # ---- the other schedules, briefly, for context (same job, fewer steps)
     others = {}
@@ -497,7 +525,7 @@ def run_ours(args, w: inputs.Workload):
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": w.name, "grid": list(w.n), "block": list(w.b),
                        "halo": max(w.halo, tsteps) if mode == "wide" else w.halo,
-                       "has_f": w.has_f, "sweeps_per_step": sweeps, "residuals_per_step": 1,
+                       "has_f": w.has_f, "sweeps_per_step": sweeps, "residuals_per_step": main_run["residuals_per_step"],
                        "schedule": mode, "tsteps": tsteps,
                        "l2": f"arrays of {w.points * 8 / 1e6:.0f} MB each exceed the {L2_BYTES / 1e6:.0f} MB L2"
                              if w.points * 8 > L2_BYTES else "arrays fit in L2 (no flush; latency-bound case)",

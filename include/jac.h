@@ -86,6 +86,31 @@ extern "C" {
                                size (0: 16 for grids of 128 rows or more, else 8; the other
                                size if that one does not fit or cannot be scheduled)             */
 
+/* Descriptor flags. */
+#define JAC_FLAG_HOST_STAGING 1 /* the workspace also holds two dense staging arrays (n[0]*n[1]*n[2]
+                                   doubles each, accounted for by jac_workspace_bytes), and jac_set_u,
+                                   jac_set_f, jac_get_u and their *_async forms move the grid as ONE
+                                   contiguous copy per direction between the host and a staging
+                                   array plus one kernel between the staging array and the blocks,
+                                   instead of one strided copy per block.  The copy in runs on a
+                                   stream of the context's own: it starts as soon as the staging
+                                   array is free and overlaps whatever is queued on the caller's
+                                   stream (the previous job's sweeps and copy out); the caller's
+                                   stream waits for it before it touches the blocks.  For callers
+                                   that stream jobs through a context from pinned host memory     */
+
+#define JAC_FLAG_CUT_LO 2       /* the context is one SLAB of a larger domain that is cut into slabs of  */
+#define JAC_FLAG_CUT_HI 4       /* whole block planes along the slowest axis (y in 2D, z in 3D), one slab
+                                   per GPU: the low / high end of that axis is a cut towards a
+                                   neighbouring slab, not a domain face.  n[] is the slab's own extent.
+                                   The ghost layers on a cut hold the neighbouring slab's face, which
+                                   arrives through jac_unpack_cut / jac_sweep_end; the workspace also
+                                   holds the packed cut planes (two send buffers and one receive buffer
+                                   per cut).  Modes JAC_MODE_FUSED and JAC_MODE_EXCHANGE only; a slab
+                                   sweeps through jac_sweep_begin / jac_sweep_end, jac_sweep is
+                                   JAC_EINVAL.  With JAC_FLAG_CUT_HI n[slowest] must be a multiple of
+                                   b[slowest]                                                      */
+
 typedef struct jac_ctx jac_ctx; /* opaque, host memory, owned by the library */
 
 typedef struct jac_desc {
@@ -96,7 +121,7 @@ typedef struct jac_desc {
     int32_t tsteps;  /* JAC_MODE_TEMPORAL: sweeps per launch; JAC_MODE_WIDE: sweeps per exchange
                         (<= halo); JAC_MODE_RESIDENT: CTAs in the cluster (8 or 16); 0 = the
                         library chooses                                                          */
-    int32_t reserved;/* must be 0                                                                */
+    int32_t flags;   /* JAC_FLAG_* bits, 0 for none                                              */
     int64_t n[3];    /* global interior points; n[2] ignored (taken as 1) when ndim == 2         */
     int64_t b[3];    /* block interior points, 1 <= b[a] <= n[a]                                 */
     void   *stream;  /* cudaStream_t of the caller (NULL = the legacy default stream)            */
@@ -122,6 +147,12 @@ typedef struct jac_layout {
     int64_t total_bytes;
     int64_t wide_face_elems[6]; /* elements of one packed wide face (jac_exchange_wide); in
                                    JAC_MODE_WIDE the send slots are sized for these              */
+    int64_t off_stage_in;  /* byte offsets of the dense staging arrays (JAC_FLAG_HOST_STAGING),  */
+    int64_t off_stage_out; /*   -1 without the flag                                              */
+    int64_t cut_elems;     /* doubles of one packed cut plane (JAC_FLAG_CUT_*; else 0): blocks of
+                              the plane in block order, 128-byte aligned slots of face_elems     */
+    int64_t off_cut_send[2][2]; /* [side][buffer] byte offsets of the send buffers of a cut,     */
+    int64_t off_cut_recv[2];    /*   and of its receive buffer; -1 where the side is no cut      */
 } jac_layout;
 
 /* Workspace size in bytes for `desc` (pure host computation, no CUDA call).
@@ -181,13 +212,13 @@ int jac_get_halo_buffer(jac_ctx *ctx, int64_t block, int face, double *host);
 
 /* Halo pack: for every block and every face with a neighbour block, gather the h interior
  * layers next to that face of the current state into the face's contiguous send buffer
- * (paper Section V-C: "packing the GPU data").  One launch over all blocks and faces
+ * (the packing step of paper Section V-C).  One launch over all blocks and faces
  * (JAC_MODE_PERTASK: one launch per block face). */
 int jac_pack_halos(jac_ctx *ctx);
 
 /* Halo unpack: for every block and every face with a neighbour, copy the neighbour's
- * opposite-face send buffer into this block's h ghost layers on that face (paper Section
- * V-C: "the data are unpacked into the GPU").  On one GPU the transfer between pack and
+ * opposite-face send buffer into this block's h ghost layers on that face (the unpacking step
+ * of paper Section V-C).  On one GPU the transfer between pack and
  * unpack is the neighbour reading the send buffer in place. */
 int jac_unpack_halos(jac_ctx *ctx);
 
@@ -256,6 +287,49 @@ int jac_solve(jac_ctx *ctx, int max_sweeps, int check_every, double tol, int *ho
  * fixed order (repeatable bit for bit), synchronises the stream and writes one HOST double. */
 int jac_residual(jac_ctx *ctx, double *host_out_l2);
 
+/* ---- Slab contexts: one domain sharded over several GPUs (JAC_FLAG_CUT_LO / JAC_FLAG_CUT_HI) ----
+ *
+ * The paper's proxy (Section V-C) spreads the blocks over many GPUs and credits its gains to
+ * overlapping the halo messages with kernel work.  Here each GPU owns a slab of whole block planes
+ * along the slowest axis as a context of its own; between slabs only the faces on the cut planes
+ * travel, once per sweep, and the residual needs one 8-byte sum.  The library packs, unpacks and
+ * orders its own streams; MOVING a packed plane to the neighbour is the caller's part -- an NCCL
+ * send/recv between the buffers jac_cut_info names, or nothing at all when the neighbour slab's
+ * send buffer can be read in place (same device, or a peer device mapped into this one: the unpack
+ * kernel reads it with ordinary loads, every CTA its own part).
+ *
+ * jac_pack_cut: packs the cut faces of the CURRENT state into the send buffers (alternating between
+ *   two buffers per cut, so a neighbour may still be reading the previous one).  Asynchronous.
+ * jac_unpack_cut: fills the cut ghost layers of the current state from packed planes: dev_src_lo /
+ *   dev_src_hi are DEVICE pointers to the plane the lower / upper neighbour packed from its face
+ *   towards this slab (NULL: this context's own receive buffer of that side; ignored where the
+ *   side is no cut); ready_lo / ready_hi are cudaEvent_t values the stream waits for before it
+ *   reads (NULL: none; pass the neighbour's event from jac_cut_info when reading its buffer in
+ *   place).  Marks the cut ghosts current.  jac_pack_cut + transfer + jac_unpack_cut is the cut
+ *   exchange of the initial state; after that jac_sweep_begin / jac_sweep_end keep them current.
+ * jac_sweep_begin: first half of one sweep.  Updates the block planes next to a cut first, packs
+ *   their NEW cut faces (as jac_pack_cut does, recording the ready events), and starts the update
+ *   of all other planes on a second stream of the context, so that the faces travel while the bulk
+ *   of the slab is computed.  Needs current cut ghosts (JAC_EINVAL otherwise).
+ * jac_sweep_end: second half.  Unpacks the neighbours' new faces (arguments as jac_unpack_cut) into
+ *   the ghost layers of the new state, joins the second stream and makes the new state current.
+ * jac_cut_info: for cut `side` (0 low, 1 high): the send buffer the LAST pack wrote, the receive
+ *   buffer, their size in bytes and the event recorded after that pack (cudaEvent_t).  Host query;
+ *   any output pointer may be NULL.
+ * jac_residual_sumsq_async: as jac_residual_async, but the SUM OF SQUARES of the slab's residual
+ *   (no square root), so that the sums of all slabs can be added and rooted once.  Works on any
+ *   context.  jac_residual* on a slab need current cut ghosts.
+ * Errors: JAC_EINVAL on a context without cuts, for a call out of order, a side that is no cut. */
+int jac_pack_cut(jac_ctx *ctx);
+int jac_unpack_cut(jac_ctx *ctx, const double *dev_src_lo, void *ready_lo, const double *dev_src_hi,
+                   void *ready_hi);
+int jac_sweep_begin(jac_ctx *ctx);
+int jac_sweep_end(jac_ctx *ctx, const double *dev_src_lo, void *ready_lo, const double *dev_src_hi,
+                  void *ready_hi);
+int jac_cut_info(const jac_ctx *ctx, int side, void **dev_send, void **dev_recv, size_t *bytes,
+                 void **ready_event);
+int jac_residual_sumsq_async(jac_ctx *ctx, double *host_out_sumsq);
+
 /* Residual norm of a DENSE grid without a context, a workspace or any allocation.
  * (The paper has no counterpart: this is a convenience of this library.)
  *
@@ -276,7 +350,8 @@ int jac_residual(jac_ctx *ctx, double *host_out_l2);
  *     part a call uses is cleared first.  Calls whose GPU work overlaps (other streams or
  *     threads) race on it: serialise them;
  *   - the first call on each device looks up the array's device address; make that first call
- *     outside any stream capture.
+ *     before any stream capture begins.  (Every call, the first included, ends by synchronising
+ *     `stream` to hand back the host double.)
  * Calls no cudaMalloc/cudaFree or other allocating routine.
  * Errors: JAC_EINVAL (null u or out, ndim not 2 or 3, a size < 1), JAC_ELIMIT, JAC_ECUDA. */
 int jac_residual_dense_static(int ndim, const int64_t *n, const double *dev_u,

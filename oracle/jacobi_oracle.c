@@ -672,3 +672,80 @@ int orc_blocked_sweep_wide(orc_blocked *s, int64_t nsweeps, int64_t k)
     }
     return ORC_OK;
 }
+
+/* ------------------------------------------------------------------------- */
+/* Slabs: one domain held as several blocked states, cut along the slowest   */
+/* axis into runs of whole block planes (the paper's proxy spreads its       */
+/* blocks over many GPUs, Section V-C; each slab stands for one GPU's part). */
+/*                                                                           */
+/* A slab is an ordinary blocked state over its own extent.  Where its low   */
+/* or high end along the slowest axis is a cut and not a domain face, the    */
+/* ghost layers there hold the neighbouring slab's face instead of a         */
+/* Dirichlet value: before every update the h interior layers next to the    */
+/* cut are packed (all blocks of that plane, block order, each block's face  */
+/* in the order of a packed face, one slot of face_elems[] per block),       */
+/* carried to the neighbour, and unpacked into its ghost layers.  Exactly    */
+/* the pack -> transfer -> unpack of the faces between blocks, for the faces */
+/* that cross a cut.  A run over slabs is bit-identical to the run over the  */
+/* whole domain.                                                             */
+/* ------------------------------------------------------------------------- */
+
+/* blocks of the first (side 0) or last (side 1) plane along the slowest axis */
+static void slab_plane(const orc_blocked *s, int side, int64_t *blk0, int64_t *count)
+{
+    const int sa = s->ndim - 1;
+    *count = s->nblocks / s->g[sa];
+    *blk0 = side ? (s->g[sa] - 1) * *count : 0;
+}
+
+/* doubles of one packed cut plane */
+int64_t orc_blocked_cut_elems(const orc_blocked *s)
+{
+    if (!s) return ORC_EINVAL;
+    int64_t blk0, count;
+    slab_plane(s, 0, &blk0, &count);
+    return count * s->face_elems[2 * (s->ndim - 1)];
+}
+
+/* the h interior layers next to the low / high end of the slowest axis -> out */
+int orc_blocked_pack_cut(const orc_blocked *s, int side, double *out)
+{
+    if (!s || !out || side < 0 || side > 1) return ORC_EINVAL;
+    const int face = 2 * (s->ndim - 1) + side;
+    int64_t blk0, count;
+    slab_plane(s, side, &blk0, &count);
+    for (int64_t m = 0; m < count; ++m) {
+        const double *u = blk_u(s, s->cur, blk0 + m);
+        int64_t lo[3], hi[3];
+        strip_range(s, blk0 + m, face, 0, lo, hi);
+        double *buf = out + m * s->face_elems[face];
+        int64_t q = 0;
+        for (int64_t k = lo[2]; k < hi[2]; ++k)
+            for (int64_t j = lo[1]; j < hi[1]; ++j)
+                for (int64_t i = lo[0]; i < hi[0]; ++i)
+                    buf[q++] = u[pad_index(s, i, j, k)];
+    }
+    return ORC_OK;
+}
+
+/* in (a plane packed by the neighbouring slab from its face towards this one) -> the ghost
+ * layers at the low / high end of the slowest axis */
+int orc_blocked_unpack_cut(orc_blocked *s, int side, const double *in)
+{
+    if (!s || !in || side < 0 || side > 1) return ORC_EINVAL;
+    const int face = 2 * (s->ndim - 1) + side;
+    int64_t blk0, count;
+    slab_plane(s, side, &blk0, &count);
+    for (int64_t m = 0; m < count; ++m) {
+        double *u = blk_u(s, s->cur, blk0 + m);
+        int64_t lo[3], hi[3];
+        strip_range(s, blk0 + m, face, 1, lo, hi);
+        const double *buf = in + m * s->face_elems[face];
+        int64_t q = 0;
+        for (int64_t k = lo[2]; k < hi[2]; ++k)
+            for (int64_t j = lo[1]; j < hi[1]; ++j)
+                for (int64_t i = lo[0]; i < hi[0]; ++i)
+                    u[pad_index(s, i, j, k)] = buf[q++];
+    }
+    return ORC_OK;
+}

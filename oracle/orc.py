@@ -75,6 +75,10 @@ def lib() -> C.CDLL:
         L.orc_blocked_wide_face_elems.restype = C.c_int64
         L.orc_blocked_wide_max_face.argtypes = [C.c_void_p]
         L.orc_blocked_wide_max_face.restype = C.c_int64
+        L.orc_blocked_cut_elems.argtypes = [C.c_void_p]
+        L.orc_blocked_cut_elems.restype = C.c_int64
+        L.orc_blocked_pack_cut.argtypes = [C.c_void_p, C.c_int, _f64p]
+        L.orc_blocked_unpack_cut.argtypes = [C.c_void_p, C.c_int, _f64p]
         _lib = L
     return _lib
 
@@ -288,6 +292,22 @@ class Blocked:
     def sweep_wide(self, nsweeps: int, k: int | None = None):
         """nsweeps sweeps with one wide exchange per group of k (default h) sweeps."""
         _check(lib().orc_blocked_sweep_wide(self._p, int(nsweeps), int(self.h if k is None else k)), "sweep_wide")
+
+    # ---- slabs: the faces that cross a cut along the slowest axis
+    def cut_elems(self) -> int:
+        return int(lib().orc_blocked_cut_elems(self._p))
+
+    def pack_cut(self, side: int) -> np.ndarray:
+        """The h interior layers next to the low (0) / high (1) end of the slowest axis, packed."""
+        out = np.zeros(self.cut_elems(), dtype=np.float64)
+        _check(lib().orc_blocked_pack_cut(self._p, int(side), _ptr(out)), "pack_cut")
+        return out
+
+    def unpack_cut(self, side: int, plane: np.ndarray):
+        """A plane packed by the neighbouring slab -> the ghost layers at that end."""
+        plane = np.ascontiguousarray(plane, dtype=np.float64)
+        assert plane.size == self.cut_elems()
+        _check(lib().orc_blocked_unpack_cut(self._p, int(side), _ptr(plane)), "unpack_cut")
 
     def neighbour(self, blk: int, face: int) -> int:
         """Block across ``face`` or -1 at the domain boundary (host-side convenience for tests)."""

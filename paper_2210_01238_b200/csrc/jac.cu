@@ -50,7 +50,9 @@ Tiling make_tiling(const JacGeom& g, int force_nv = 0)
         t.tiles_y = (int)ceil_div(g.by, rows);
     } else {
         const int tx = std::min(64, pow2_ceil(need));
-        const int ty = std::min(std::max(1, 512 / tx), std::min(8, pow2_ceil(g.by)));
+        // at least one whole warp: the CTA-wide sum shuffles over 32 lanes (threads beyond the block's
+        // rows fail the extent test and contribute 0)
+        const int ty = std::max(std::min(std::max(1, 512 / tx), std::min(8, pow2_ceil(g.by))), 32 / tx);
         t.block = dim3(tx, ty, 1);
         t.tiles_x = (int)ceil_div(need, tx);
         t.tiles_y = (int)ceil_div(g.by, ty);
@@ -183,7 +185,11 @@ int build_geometry(const jac_desc* d, JacGeom* g, jac_layout* L)
     if (d->halo < 1 || d->halo > 8) return JAC_EINVAL;
     if (d->has_f != 0 && d->has_f != 1) return JAC_EINVAL;
     if (d->mode < JAC_MODE_FUSED || d->mode > JAC_MODE_RESIDENT) return JAC_EINVAL;
-    if (d->tsteps < 0 || d->tsteps > (d->mode == JAC_MODE_RESIDENT ? 16 : 8) || d->reserved != 0) return JAC_EINVAL;
+    if (d->tsteps < 0 || d->tsteps > (d->mode == JAC_MODE_RESIDENT ? 16 : 8)) return JAC_EINVAL;
+    if (d->flags & ~(JAC_FLAG_HOST_STAGING | JAC_FLAG_CUT_LO | JAC_FLAG_CUT_HI)) return JAC_EINVAL;
+    const bool has_cut = (d->flags & (JAC_FLAG_CUT_LO | JAC_FLAG_CUT_HI)) != 0;
+    // a slab exchanges its cut faces once per sweep: only the one-sweep-per-exchange schedules
+    if (has_cut && d->mode != JAC_MODE_FUSED && d->mode != JAC_MODE_EXCHANGE) return JAC_EINVAL;
     long long n[3] = {1, 1, 1}, b[3] = {1, 1, 1}, gr[3] = {1, 1, 1};
     for (int a = 0; a < d->ndim; ++a) {
         n[a] = d->n[a];
@@ -195,6 +201,8 @@ int build_geometry(const jac_desc* d, JacGeom* g, jac_layout* L)
         if (n[a] - (gr[a] - 1) * b[a] < d->halo) return JAC_EINVAL;   // a remainder block narrower than a face strip
         if (gr[a] > (1LL << 30)) return JAC_EINVAL;
     }
+    // the blocks on a cut are whole: a remainder block exists only at the far end of the domain
+    if ((d->flags & JAC_FLAG_CUT_HI) && n[d->ndim - 1] % b[d->ndim - 1] != 0) return JAC_EINVAL;
     std::memset(g, 0, sizeof(*g));
     g->ndim = d->ndim;
     g->h = d->halo;
@@ -274,6 +282,25 @@ int build_geometry(const jac_desc* d, JacGeom* g, jac_layout* L)
         if (d->has_f) { L->off_f = o; o += arr_bytes; } else L->off_f = -1;
         L->off_send = o; o += round_up(g->nblocks * g->send_stride * 8, 256);
         L->off_scratch = o; o += round_up((L->partials + 32) * 8, 256);
+        L->cut_elems = 0;
+        for (int sd = 0; sd < 2; ++sd) L->off_cut_send[sd][0] = L->off_cut_send[sd][1] = L->off_cut_recv[sd] = -1;
+        if (has_cut) {
+            const int sa = d->ndim - 1;
+            L->cut_elems = (g->nblocks / gr[sa]) * round_up(g->face_elems[2 * sa], 16);
+            const long long cut_bytes = round_up(L->cut_elems * 8, 256);
+            for (int sd = 0; sd < 2; ++sd) {
+                if (!(d->flags & (sd ? JAC_FLAG_CUT_HI : JAC_FLAG_CUT_LO))) continue;
+                L->off_cut_send[sd][0] = o; o += cut_bytes;
+                L->off_cut_send[sd][1] = o; o += cut_bytes;
+                L->off_cut_recv[sd] = o; o += cut_bytes;
+            }
+        }
+        L->off_stage_in = L->off_stage_out = -1;
+        if (d->flags & JAC_FLAG_HOST_STAGING) {
+            const long long dense_bytes = round_up(n[0] * n[1] * n[2] * 8, 256);
+            L->off_stage_in = o; o += dense_bytes;
+            L->off_stage_out = o; o += dense_bytes;
+        }
         L->total_bytes = o;
     }
     return JAC_OK;
@@ -297,6 +324,23 @@ struct jac_ctx {
     bool packed_current;  // the send buffers hold the faces of the current state
     bool f_ghosts_fresh;  // JAC_MODE_WIDE: the ghost layers of f hold the neighbours' f
     int res_cluster;      // JAC_MODE_RESIDENT: CTAs per cluster settled at creation
+    // JAC_FLAG_HOST_STAGING: dense arrays between the host and the blocks, a copy stream per
+    // direction, and the events that order them against the caller's stream
+    double* stage_in;
+    double* stage_out;
+    cudaStream_t h2d;
+    cudaEvent_t ev_in_ready, ev_in_free, ev_out_done;
+    // JAC_FLAG_CUT_*: the slab's cut planes (side 0 = low, 1 = high end of the slowest axis)
+    bool cut[2];
+    double* cut_send[2][2];   // [side][parity]: packs alternate between two buffers
+    double* cut_recv[2];
+    int cut_parity;           // buffer the last pack wrote
+    bool cut_fresh;           // the cut ghosts of u[cur] hold the neighbour slabs' current faces
+    bool in_sweep;            // jac_sweep_begin without its jac_sweep_end
+    cudaStream_t aux;         // the blocks away from the cuts run here while the cut faces travel
+    cudaEvent_t ev_fork, ev_join, ev_cut_ready[2];
+    const char* d2h_lo;   // host range the last copy out writes (until the stream has passed it)
+    const char* d2h_hi;
     cudaStream_t stream;
     int device;
     int cuda_err;       // sticky
@@ -313,6 +357,23 @@ namespace {
             return JAC_ECUDA;                              \
         }                                                  \
     } while (0)
+
+void release_copy_objects(jac_ctx* c)
+{
+    if (c->ev_in_ready) cudaEventDestroy(c->ev_in_ready);
+    if (c->ev_in_free) cudaEventDestroy(c->ev_in_free);
+    if (c->ev_out_done) cudaEventDestroy(c->ev_out_done);
+    if (c->h2d) cudaStreamDestroy(c->h2d);
+    c->ev_in_ready = c->ev_in_free = c->ev_out_done = nullptr;
+    c->h2d = nullptr;
+    if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+    if (c->ev_join) cudaEventDestroy(c->ev_join);
+    for (int side = 0; side < 2; ++side)
+        if (c->ev_cut_ready[side]) cudaEventDestroy(c->ev_cut_ready[side]);
+    if (c->aux) cudaStreamDestroy(c->aux);
+    c->ev_fork = c->ev_join = c->ev_cut_ready[0] = c->ev_cut_ready[1] = nullptr;
+    c->aux = nullptr;
+}
 
 int check_launch(jac_ctx* c)
 {
@@ -556,6 +617,54 @@ int copy_dense_device(jac_ctx* c, double* arr, double* dense)
     return check_launch(c);
 }
 
+// ---- JAC_FLAG_HOST_STAGING: one contiguous copy per direction through a dense staging array ----
+// Copy in: host -> staging array on the context's own host-to-device stream, then (on the caller's
+// stream, after an event) the kernel that scatters the dense array into the blocks.  The copy does
+// not queue behind the work already on the caller's stream -- the sweeps of the previous job, its
+// copy out -- so it overlaps them (the two copy directions and the SMs are separate engines); it
+// only waits until the staging array is free again and, if the host range is the target of a copy
+// out that is still in flight, for that copy.
+int staged_in(jac_ctx* c, double* arr, const double* host, bool wait)
+{
+    const size_t bytes = (size_t)(c->g.nx * c->g.ny * c->g.nz) * sizeof(double);
+    JAC_CK(c, cudaStreamWaitEvent(c->h2d, c->ev_in_free, 0));
+    const char* lo = reinterpret_cast<const char*>(host);
+    if (c->d2h_lo && lo < c->d2h_hi && c->d2h_lo < lo + bytes) JAC_CK(c, cudaStreamWaitEvent(c->h2d, c->ev_out_done, 0));
+    JAC_CK(c, cudaMemcpyAsync(c->stage_in, host, bytes, cudaMemcpyHostToDevice, c->h2d));
+    JAC_CK(c, cudaEventRecord(c->ev_in_ready, c->h2d));
+    JAC_CK(c, cudaStreamWaitEvent(c->stream, c->ev_in_ready, 0));
+    const int rc = copy_dense_device<true>(c, arr, c->stage_in);
+    if (rc) return rc;
+    JAC_CK(c, cudaEventRecord(c->ev_in_free, c->stream));
+    if (wait) JAC_CK(c, cudaStreamSynchronize(c->stream));
+    return JAC_OK;
+}
+
+// Copy out: the kernel that gathers the blocks into the dense staging array, then one contiguous
+// copy to the host, both on the caller's stream.
+int staged_out(jac_ctx* c, double* arr, double* host, bool wait)
+{
+    const size_t bytes = (size_t)(c->g.nx * c->g.ny * c->g.nz) * sizeof(double);
+    const int rc = copy_dense_device<false>(c, arr, c->stage_out);
+    if (rc) return rc;
+    JAC_CK(c, cudaMemcpyAsync(host, c->stage_out, bytes, cudaMemcpyDeviceToHost, c->stream));
+    JAC_CK(c, cudaEventRecord(c->ev_out_done, c->stream));
+    c->d2h_lo = reinterpret_cast<const char*>(host);
+    c->d2h_hi = c->d2h_lo + bytes;
+    if (wait) JAC_CK(c, cudaStreamSynchronize(c->stream));
+    return JAC_OK;
+}
+
+// dense host array <-> blocks, by whichever route the context has
+int host_to_blocks(jac_ctx* c, double* arr, const double* host, bool wait)
+{
+    return c->stage_in ? staged_in(c, arr, host, wait) : copy_dense_host(c, arr, const_cast<double*>(host), true, wait);
+}
+int blocks_to_host(jac_ctx* c, double* arr, double* host, bool wait)
+{
+    return c->stage_out ? staged_out(c, arr, host, wait) : copy_dense_host(c, arr, host, false, wait);
+}
+
 int usable(jac_ctx* c)
 {
     if (!c) return JAC_EINVAL;
@@ -729,6 +838,7 @@ int choose_resident_cluster(jac_ctx* c)
 int run_sweeps(jac_ctx* c, int nsweeps, bool res, long long* nparts)
 {
     int rc = JAC_OK;
+    if (c->cut[0] || c->cut[1]) return JAC_EINVAL;   // a slab sweeps through jac_sweep_begin / jac_sweep_end
     const JacGeom& g = c->g;
     const long long sweep_parts = g.nblocks * c->tile.ctas_per_block;
     switch (c->desc.mode) {
@@ -853,6 +963,115 @@ int finish_norm(jac_ctx* c, long long nparts, double* host_out_l2)
     return JAC_OK;
 }
 
+// ---- slab contexts (JAC_FLAG_CUT_*): the faces that cross a cut ------------------------------
+bool has_cuts(const jac_ctx* c) { return c->cut[0] || c->cut[1]; }
+
+struct PlaneRange { long long blk0, nblk; };
+
+// the blocks of the slab's first (side 0) or last (side 1) plane along the slowest axis: blocks are
+// numbered x fastest, so a plane is a contiguous range
+PlaneRange cut_plane(const jac_ctx* c, int side)
+{
+    const int gs = c->g.ndim == 2 ? c->g.gy : c->g.gz;
+    const long long per_plane = c->g.nblocks / gs;
+    return PlaneRange{side ? (gs - 1) * per_plane : 0, per_plane};
+}
+
+template <bool UNPACK>
+int launch_cut(jac_ctx* c, int side, double* arr, double* buf)
+{
+    const PlaneRange r = cut_plane(c, side);
+    const int face = 2 * (c->g.ndim - 1) + side;
+    const long long slot = round_up(c->g.face_elems[face], 16);
+    const int slots = (int)round_up(ceil_div(c->g.face_elems[face], 2), 32);
+    const long long ctas = ceil_div(r.nblk * slots, 256);
+    if (ctas > kMaxGrid) return JAC_EINVAL;
+    jac::cut_kernel<UNPACK><<<(unsigned)ctas, 256, 0, c->stream>>>(arr, buf, c->g, r.blk0, r.nblk, slots, face, slot);
+    return check_launch(c);
+}
+
+// the cut faces of `arr` into the send buffers the previous pack did not use; an event per side
+// tells a reader on another stream when its buffer is complete
+int pack_cuts(jac_ctx* c, double* arr)
+{
+    c->cut_parity ^= 1;
+    for (int side = 0; side < 2; ++side) {
+        if (!c->cut[side]) continue;
+        const int rc = launch_cut<false>(c, side, arr, c->cut_send[side][c->cut_parity]);
+        if (rc) return rc;
+        JAC_CK(c, cudaEventRecord(c->ev_cut_ready[side], c->stream));
+    }
+    return JAC_OK;
+}
+
+// the cut ghost layers of `arr` from packed planes: src[side] (a device pointer, e.g. the neighbour
+// slab's send buffer; after `ready[side]` if given) or the context's own receive buffer
+int unpack_cuts(jac_ctx* c, double* arr, const double* const src[2], void* const ready[2])
+{
+    for (int side = 0; side < 2; ++side) {
+        if (!c->cut[side]) continue;
+        if (ready[side]) JAC_CK(c, cudaStreamWaitEvent(c->stream, static_cast<cudaEvent_t>(ready[side]), 0));
+        double* from = src[side] ? const_cast<double*>(src[side]) : c->cut_recv[side];
+        const int rc = launch_cut<true>(c, side, arr, from);
+        if (rc) return rc;
+    }
+    return JAC_OK;
+}
+
+// First half of a sweep of a slab: the planes of blocks next to a cut are updated first and their
+// new cut faces packed, so that they can travel while the rest of the slab is updated on the
+// context's second stream.
+int slab_sweep_begin(jac_ctx* c)
+{
+    const JacGeom& g = c->g;
+    const bool exch = c->desc.mode == JAC_MODE_EXCHANGE;
+    int rc;
+    if (exch && (rc = do_exchange(c))) return rc;       // the faces between the slab's own blocks
+    const double* u = c->u[c->cur];
+    double* un = c->u[c->cur ^ 1];
+    const int gs = g.ndim == 2 ? g.gy : g.gz;
+    const long long per_plane = g.nblocks / gs;
+    JAC_CK(c, cudaEventRecord(c->ev_fork, c->stream));
+    JAC_CK(c, cudaStreamWaitEvent(c->aux, c->ev_fork, 0));
+    // planes next to a cut (one plane may be next to both)
+    for (int side = 0; side < 2; ++side) {
+        if (!c->cut[side] || (side == 1 && gs == 1 && c->cut[0])) continue;
+        const PlaneRange r = cut_plane(c, side);
+        rc = exch ? launch_sweep<jac::OP_UPDATE>(c, u, un, r.blk0, r.nblk)
+                  : launch_sweep<jac::OP_UPDATE_PULL>(c, u, un, r.blk0, r.nblk);
+        if (rc) return rc;
+    }
+    if ((rc = pack_cuts(c, un))) return rc;
+    // the planes in between, meanwhile
+    const long long p0 = c->cut[0] ? 1 : 0, p1 = c->cut[1] ? gs - 1 : gs;
+    if (p1 > p0) {
+        cudaStream_t keep = c->stream;
+        c->stream = c->aux;
+        rc = exch ? launch_sweep<jac::OP_UPDATE>(c, u, un, p0 * per_plane, (p1 - p0) * per_plane)
+                  : launch_sweep<jac::OP_UPDATE_PULL>(c, u, un, p0 * per_plane, (p1 - p0) * per_plane);
+        c->stream = keep;
+        if (rc) return rc;
+    }
+    JAC_CK(c, cudaEventRecord(c->ev_join, c->aux));
+    c->in_sweep = true;
+    return JAC_OK;
+}
+
+// Second half: the neighbours' new cut faces go into the ghost layers of the new state, the
+// second stream joins, and the new state becomes the current one.
+int slab_sweep_end(jac_ctx* c, const double* const src[2], void* const ready[2])
+{
+    int rc;
+    if ((rc = unpack_cuts(c, c->u[c->cur ^ 1], src, ready))) return rc;
+    JAC_CK(c, cudaStreamWaitEvent(c->stream, c->ev_join, 0));
+    c->cur ^= 1;
+    c->in_sweep = false;
+    c->cut_fresh = true;
+    c->ghosts_fresh = false;
+    c->packed_current = false;
+    return JAC_OK;
+}
+
 }  // namespace
 
 // =====================================================================================
@@ -914,6 +1133,21 @@ int jac_create(const jac_desc* desc, void* dev_workspace, size_t bytes, jac_ctx*
     c->packed_current = false;
     c->f_ghosts_fresh = false;
     c->res_cluster = 0;
+    c->stage_in = c->stage_out = nullptr;
+    c->h2d = nullptr;
+    c->ev_in_ready = c->ev_in_free = c->ev_out_done = nullptr;
+    c->d2h_lo = c->d2h_hi = nullptr;
+    c->cut[0] = (desc->flags & JAC_FLAG_CUT_LO) != 0;
+    c->cut[1] = (desc->flags & JAC_FLAG_CUT_HI) != 0;
+    for (int side = 0; side < 2; ++side) {
+        c->cut_send[side][0] = c->cut_send[side][1] = c->cut_recv[side] = nullptr;
+        c->ev_cut_ready[side] = nullptr;
+    }
+    c->cut_parity = 0;
+    c->cut_fresh = false;
+    c->in_sweep = false;
+    c->aux = nullptr;
+    c->ev_fork = c->ev_join = nullptr;
     c->stream = static_cast<cudaStream_t>(desc->stream);
     c->device = dev;
     c->cuda_err = 0;
@@ -927,6 +1161,37 @@ int jac_create(const jac_desc* desc, void* dev_workspace, size_t bytes, jac_ctx*
         delete c;
         return rc;
     }
+    if (desc->flags & JAC_FLAG_HOST_STAGING) {
+        c->stage_in = reinterpret_cast<double*>(c->ws + L.off_stage_in);
+        c->stage_out = reinterpret_cast<double*>(c->ws + L.off_stage_out);
+        if (cudaStreamCreateWithFlags(&c->h2d, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_in_ready, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_in_free, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_out_done, cudaEventDisableTiming) != cudaSuccess) {
+            cudaGetLastError();
+            release_copy_objects(c);
+            delete c;
+            return JAC_ECUDA;
+        }
+    }
+    if (has_cuts(c)) {
+        bool ok = cudaStreamCreateWithFlags(&c->aux, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) == cudaSuccess;
+        for (int side = 0; side < 2 && ok; ++side) {
+            if (!c->cut[side]) continue;
+            c->cut_send[side][0] = reinterpret_cast<double*>(c->ws + L.off_cut_send[side][0]);
+            c->cut_send[side][1] = reinterpret_cast<double*>(c->ws + L.off_cut_send[side][1]);
+            c->cut_recv[side] = reinterpret_cast<double*>(c->ws + L.off_cut_recv[side]);
+            ok = cudaEventCreateWithFlags(&c->ev_cut_ready[side], cudaEventDisableTiming) == cudaSuccess;
+        }
+        if (!ok) {
+            cudaGetLastError();
+            release_copy_objects(c);
+            delete c;
+            return JAC_ECUDA;
+        }
+    }
     *out = c;
     return JAC_OK;
 }
@@ -934,7 +1199,10 @@ int jac_create(const jac_desc* desc, void* dev_workspace, size_t bytes, jac_ctx*
 int jac_destroy(jac_ctx* ctx)
 {
     if (!ctx) return JAC_EINVAL;
+    if (ctx->h2d) cudaStreamSynchronize(ctx->h2d);
+    if (ctx->aux) cudaStreamSynchronize(ctx->aux);
     cudaStreamSynchronize(ctx->stream);
+    release_copy_objects(ctx);
     delete ctx;
     return JAC_OK;
 }
@@ -946,7 +1214,8 @@ int jac_set_u(jac_ctx* c, const double* host_dense)
     if (!host_dense) return JAC_EINVAL;
     c->ghosts_fresh = false;
     c->packed_current = false;
-    return copy_dense_host(c, c->u[c->cur], const_cast<double*>(host_dense), true);
+    c->cut_fresh = false;
+    return host_to_blocks(c, c->u[c->cur], host_dense, true);
 }
 
 int jac_set_f(jac_ctx* c, const double* host_dense)
@@ -955,7 +1224,7 @@ int jac_set_f(jac_ctx* c, const double* host_dense)
     if (rc) return rc;
     if (!host_dense || !c->f) return JAC_EINVAL;
     c->f_ghosts_fresh = false;
-    return copy_dense_host(c, c->f, const_cast<double*>(host_dense), true);
+    return host_to_blocks(c, c->f, host_dense, true);
 }
 
 int jac_get_u(jac_ctx* c, double* host_dense)
@@ -963,7 +1232,7 @@ int jac_get_u(jac_ctx* c, double* host_dense)
     int rc = usable(c);
     if (rc) return rc;
     if (!host_dense) return JAC_EINVAL;
-    return copy_dense_host(c, c->u[c->cur], host_dense, false);
+    return blocks_to_host(c, c->u[c->cur], host_dense, true);
 }
 
 int jac_set_u_device(jac_ctx* c, const double* dev_dense)
@@ -973,6 +1242,7 @@ int jac_set_u_device(jac_ctx* c, const double* dev_dense)
     if (!dev_dense) return JAC_EINVAL;
     c->ghosts_fresh = false;
     c->packed_current = false;
+    c->cut_fresh = false;
     return copy_dense_device<true>(c, c->u[c->cur], const_cast<double*>(dev_dense));
 }
 
@@ -998,6 +1268,7 @@ int jac_set_boundary(jac_ctx* c, int face, double value)
     int rc = usable(c);
     if (rc) return rc;
     if (face < 0 || face >= c->g.nfaces) return JAC_EINVAL;
+    if ((face >> 1) == c->g.ndim - 1 && c->cut[face & 1]) return JAC_EINVAL;   // a cut is not a domain face
     c->g.bval[face] = value;
     const int axis = face >> 1;
     const long long on_face = c->g.nblocks / (axis == 0 ? c->g.gx : axis == 1 ? c->g.gy : c->g.gz);
@@ -1129,6 +1400,7 @@ int jac_residual(jac_ctx* c, double* host_out_l2)
     int rc = usable(c);
     if (rc) return rc;
     if (!host_out_l2) return JAC_EINVAL;
+    if (has_cuts(c) && (!c->cut_fresh || c->in_sweep)) return JAC_EINVAL;
     if (!c->ghosts_fresh && (rc = (c->desc.mode == JAC_MODE_PERTASK ? do_exchange(c) : do_exchange_fused(c)))) return rc;
     if ((rc = launch_sweep<jac::OP_RESIDUAL>(c, c->u[c->cur], nullptr, 0, c->g.nblocks))) return rc;
     return finish_norm(c, c->g.nblocks * c->tile.ctas_per_block, host_out_l2);
@@ -1164,7 +1436,8 @@ int jac_set_u_async(jac_ctx* c, const double* host_dense)
     if (!host_dense) return JAC_EINVAL;
     c->ghosts_fresh = false;
     c->packed_current = false;
-    return copy_dense_host(c, c->u[c->cur], const_cast<double*>(host_dense), true, false);
+    c->cut_fresh = false;
+    return host_to_blocks(c, c->u[c->cur], host_dense, false);
 }
 
 int jac_get_u_async(jac_ctx* c, double* host_dense)
@@ -1172,21 +1445,79 @@ int jac_get_u_async(jac_ctx* c, double* host_dense)
     int rc = usable(c);
     if (rc) return rc;
     if (!host_dense) return JAC_EINVAL;
-    return copy_dense_host(c, c->u[c->cur], host_dense, false, false);
+    return blocks_to_host(c, c->u[c->cur], host_dense, false);
 }
 
-int jac_residual_async(jac_ctx* c, double* host_out_l2)
+namespace {
+// the residual of the current state queued on the stream: its sum of squares, or the norm
+int residual_queued(jac_ctx* c, double* host_out, bool norm)
 {
     int rc = usable(c);
     if (rc) return rc;
-    if (!host_out_l2) return JAC_EINVAL;
+    if (!host_out) return JAC_EINVAL;
+    if (has_cuts(c) && (!c->cut_fresh || c->in_sweep)) return JAC_EINVAL;
     if (!c->ghosts_fresh && (rc = (c->desc.mode == JAC_MODE_PERTASK ? do_exchange(c) : do_exchange_fused(c)))) return rc;
     if ((rc = launch_sweep<jac::OP_RESIDUAL>(c, c->u[c->cur], nullptr, 0, c->g.nblocks))) return rc;
     jac::reduce_partials_kernel<<<1, 1024, 0, c->stream>>>(c->partials, c->g.nblocks * c->tile.ctas_per_block, c->result);
     if ((rc = check_launch(c))) return rc;
-    sqrt_in_place_kernel<<<1, 1, 0, c->stream>>>(c->result);
-    if ((rc = check_launch(c))) return rc;
-    JAC_CK(c, cudaMemcpyAsync(host_out_l2, c->result, sizeof(double), cudaMemcpyDeviceToHost, c->stream));
+    if (norm) {
+        sqrt_in_place_kernel<<<1, 1, 0, c->stream>>>(c->result);
+        if ((rc = check_launch(c))) return rc;
+    }
+    JAC_CK(c, cudaMemcpyAsync(host_out, c->result, sizeof(double), cudaMemcpyDeviceToHost, c->stream));
+    return JAC_OK;
+}
+}  // namespace
+
+int jac_residual_async(jac_ctx* c, double* host_out_l2) { return residual_queued(c, host_out_l2, true); }
+
+int jac_residual_sumsq_async(jac_ctx* c, double* host_out_sumsq) { return residual_queued(c, host_out_sumsq, false); }
+
+int jac_pack_cut(jac_ctx* c)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    if (!has_cuts(c) || c->in_sweep) return JAC_EINVAL;
+    return pack_cuts(c, c->u[c->cur]);
+}
+
+int jac_unpack_cut(jac_ctx* c, const double* dev_src_lo, void* ready_lo, const double* dev_src_hi, void* ready_hi)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    if (!has_cuts(c) || c->in_sweep) return JAC_EINVAL;
+    const double* const src[2] = {dev_src_lo, dev_src_hi};
+    void* const ready[2] = {ready_lo, ready_hi};
+    if ((rc = unpack_cuts(c, c->u[c->cur], src, ready))) return rc;
+    c->cut_fresh = true;
+    return JAC_OK;
+}
+
+int jac_sweep_begin(jac_ctx* c)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    if (!has_cuts(c) || c->in_sweep || !c->cut_fresh) return JAC_EINVAL;
+    return slab_sweep_begin(c);
+}
+
+int jac_sweep_end(jac_ctx* c, const double* dev_src_lo, void* ready_lo, const double* dev_src_hi, void* ready_hi)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    if (!has_cuts(c) || !c->in_sweep) return JAC_EINVAL;
+    const double* const src[2] = {dev_src_lo, dev_src_hi};
+    void* const ready[2] = {ready_lo, ready_hi};
+    return slab_sweep_end(c, src, ready);
+}
+
+int jac_cut_info(const jac_ctx* c, int side, void** dev_send, void** dev_recv, size_t* bytes, void** ready_event)
+{
+    if (!c || side < 0 || side > 1 || !c->cut[side]) return JAC_EINVAL;
+    if (dev_send) *dev_send = c->cut_send[side][c->cut_parity];
+    if (dev_recv) *dev_recv = c->cut_recv[side];
+    if (bytes) *bytes = (size_t)c->L.cut_elems * sizeof(double);
+    if (ready_event) *ready_event = c->ev_cut_ready[side];
     return JAC_OK;
 }
 

@@ -465,6 +465,44 @@ halo_exchange_kernel(double* __restrict__ u, double* __restrict__ send, const Ja
     }
 }
 
+// Cut faces of a slab context: the faces of the blocks on the slab's first or last plane along the
+// slowest axis that look across the cut (they have no neighbour block inside the context).  Pack
+// gathers their h interior layers into one contiguous plane buffer, unpack scatters such a buffer
+// into their ghost layers.  Block m of the plane owns elements [m * slot, m * slot + its face
+// elements) of the buffer, in the order of a packed face.  `slots` threads per block, two
+// consecutive elements per thread (a cut face is a y face in 2D, a z face in 3D: contiguous rows).
+template <bool UNPACK>
+__global__ void __launch_bounds__(256)
+cut_kernel(double* __restrict__ u, double* __restrict__ buf, const JacGeom g, const long long blk0,
+           const long long nblk, const int slots, const int face, const long long slot)
+{
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long m = t / slots;
+    if (m >= nblk) return;
+    const unsigned e = 2u * (unsigned)(t - m * slots);
+    const long long blk = blk0 + m;
+    const BlockExtent be = block_extent(g, blk);
+    const long long n = face_elems_of(g, be, face);
+    if (e >= n) return;
+    const int axis = face >> 1;
+    const int ext = axis == 1 ? be.y : be.z;
+    const int lo = UNPACK ? ((face & 1) ? ext : -g.h) : ((face & 1) ? ext - g.h : 0);
+    double* ub = u + blk * g.block_stride + g.origin;
+    double* bp = buf + m * slot;
+    if ((be.x & 1) == 0) {
+        double2* cell = reinterpret_cast<double2*>(ub + strip_offset(g, be, face, e, lo));
+        double2* sl = reinterpret_cast<double2*>(bp + e);
+        if (UNPACK) *cell = *sl; else *sl = *cell;
+    } else {
+        double* c0 = ub + strip_offset(g, be, face, e, lo);
+        if (UNPACK) *c0 = bp[e]; else bp[e] = *c0;
+        if (e + 1 < n) {
+            double* c1 = ub + strip_offset(g, be, face, e + 1, lo);
+            if (UNPACK) *c1 = bp[e + 1]; else bp[e + 1] = *c1;
+        }
+    }
+}
+
 // Wide exchange, one axis per launch: the strip of a face is h layers along `axis` (interior
 // layers for pack, ghost layers for unpack) over the whole padded extent (-h .. extent + h) of the
 // other axes, so edge and corner data delivered by the launches of earlier axes travels on.

@@ -26,6 +26,7 @@ MODES = {"fused": MODE_FUSED, "pertask": MODE_PERTASK, "temporal": MODE_TEMPORAL
          "exchange": MODE_EXCHANGE, "wide": MODE_WIDE, "resident": MODE_RESIDENT}
 
 OK, EINVAL, ENOMEM, ECUDA, ENODEV, ELIMIT = 0, -1, -2, -3, -4, -5
+FLAG_HOST_STAGING, FLAG_CUT_LO, FLAG_CUT_HI = 1, 2, 4
 
 EXPORTS = [
     "jac_workspace_bytes", "jac_get_layout", "jac_create", "jac_destroy",
@@ -35,12 +36,14 @@ EXPORTS = [
     "jac_last_cuda_error", "jac_strerror", "jac_residual_dense_static", "jac_sweeps_per_launch",
     "jac_sweep_residual", "jac_solve", "jac_exchange_wide", "jac_get_wide_buffer",
     "jac_set_u_async", "jac_get_u_async", "jac_residual_async", "jac_exchange_halos",
+    "jac_pack_cut", "jac_unpack_cut", "jac_sweep_begin", "jac_sweep_end", "jac_cut_info",
+    "jac_residual_sumsq_async",
 ]
 
 
 class Desc(C.Structure):
     _fields_ = [("ndim", C.c_int32), ("halo", C.c_int32), ("has_f", C.c_int32),
-                ("mode", C.c_int32), ("tsteps", C.c_int32), ("reserved", C.c_int32),
+                ("mode", C.c_int32), ("tsteps", C.c_int32), ("flags", C.c_int32),
                 ("n", C.c_int64 * 3), ("b", C.c_int64 * 3), ("stream", C.c_void_p)]
 
 
@@ -50,7 +53,9 @@ class Layout(C.Structure):
                 ("face_elems", C.c_int64 * 6), ("face_offset", C.c_int64 * 6),
                 ("send_stride", C.c_int64), ("partials", C.c_int64), ("off_u", C.c_int64 * 2),
                 ("off_f", C.c_int64), ("off_send", C.c_int64), ("off_scratch", C.c_int64),
-                ("total_bytes", C.c_int64), ("wide_face_elems", C.c_int64 * 6)]
+                ("total_bytes", C.c_int64), ("wide_face_elems", C.c_int64 * 6),
+                ("off_stage_in", C.c_int64), ("off_stage_out", C.c_int64), ("cut_elems", C.c_int64),
+                ("off_cut_send", (C.c_int64 * 2) * 2), ("off_cut_recv", C.c_int64 * 2)]
 
 
 class JacError(RuntimeError):
@@ -76,8 +81,13 @@ def lib() -> C.CDLL:
         L.jac_destroy.argtypes = [vp]
         for name in ("jac_set_u", "jac_set_f", "jac_get_u", "jac_set_u_device",
                      "jac_set_f_device", "jac_get_u_device", "jac_set_u_async", "jac_get_u_async",
-                     "jac_residual_async"):
+                     "jac_residual_async", "jac_residual_sumsq_async"):
             getattr(L, name).argtypes = [vp, vp]
+        L.jac_pack_cut.argtypes = [vp]
+        L.jac_sweep_begin.argtypes = [vp]
+        L.jac_unpack_cut.argtypes = [vp, vp, vp, vp, vp]
+        L.jac_sweep_end.argtypes = [vp, vp, vp, vp, vp]
+        L.jac_cut_info.argtypes = [vp, C.c_int, C.POINTER(vp), C.POINTER(vp), C.POINTER(C.c_size_t), C.POINTER(vp)]
         L.jac_set_boundary.argtypes = [vp, C.c_int, C.c_double]
         L.jac_get_block_padded.argtypes = [vp, C.c_int64, vp]
         L.jac_get_halo_buffer.argtypes = [vp, C.c_int64, C.c_int, vp]
@@ -110,12 +120,12 @@ def strerror(code: int) -> str:
     return lib().jac_strerror(int(code)).decode()
 
 
-def make_desc(n, b, halo=1, has_f=False, mode=MODE_FUSED, tsteps=0, stream=0) -> Desc:
+def make_desc(n, b, halo=1, has_f=False, mode=MODE_FUSED, tsteps=0, stream=0, flags=0) -> Desc:
     ndim = len(n)
     d = Desc()
     d.ndim, d.halo, d.has_f = ndim, int(halo), int(bool(has_f))
     d.mode = MODES[mode] if isinstance(mode, str) else int(mode)
-    d.tsteps, d.reserved = int(tsteps), 0
+    d.tsteps, d.flags = int(tsteps), int(flags)
     for a in range(3):
         d.n[a] = int(n[a]) if a < ndim else 1
         d.b[a] = int(b[a]) if a < ndim else 1
@@ -179,7 +189,7 @@ class Jacobi:
     ``*_device`` calls.
     """
 
-    def __init__(self, n, b, halo=1, has_f=False, mode="fused", tsteps=0, stream=None):
+    def __init__(self, n, b, halo=1, has_f=False, mode="fused", tsteps=0, stream=None, flags=0):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("paper_2210_01238_b200.jac needs a CUDA device; there is no CPU path")
@@ -187,7 +197,7 @@ class Jacobi:
         self.n, self.b = tuple(int(x) for x in n), tuple(int(x) for x in b)
         self.ndim = len(self.n)
         self.stream = stream if stream is not None else torch.cuda.current_stream()
-        self.desc = make_desc(n, b, halo, has_f, mode, tsteps, self.stream.cuda_stream)
+        self.desc = make_desc(n, b, halo, has_f, mode, tsteps, self.stream.cuda_stream, flags)
         self.layout = get_layout(self.desc)
         nbytes = workspace_bytes(self.desc)
         with torch.cuda.stream(self.stream):
@@ -294,6 +304,52 @@ class Jacobi:
         assert out.numel() == 1
         self._call("jac_residual_async", lib().jac_residual_async(self._ctx, self._pinned_ptr(out)))
         return out
+
+    def residual_sumsq_async(self, out):
+        """As residual_async, but the sum of squares (slabs of one domain add theirs, then take the root)."""
+        assert out.numel() == 1
+        self._call("jac_residual_sumsq_async", lib().jac_residual_sumsq_async(self._ctx, self._pinned_ptr(out)))
+        return out
+
+    def residual_sumsq(self) -> float:
+        """Sum of squares of the residual of the current state (waits for the stream)."""
+        out = self._torch.zeros(1, dtype=self._torch.float64).pin_memory()
+        self.residual_sumsq_async(out)
+        self.stream.synchronize()
+        return float(out[0])
+
+    # ---- slab contexts (flags FLAG_CUT_LO / FLAG_CUT_HI)
+    def cut_info(self, side: int):
+        """(send pointer of the last pack, receive pointer, bytes, ready event) of cut ``side``."""
+        send, recv, ev, nbytes = C.c_void_p(), C.c_void_p(), C.c_void_p(), C.c_size_t(0)
+        self._call("jac_cut_info", lib().jac_cut_info(self._ctx, int(side), C.byref(send), C.byref(recv),
+                                                      C.byref(nbytes), C.byref(ev)))
+        return send.value, recv.value, nbytes.value, ev.value
+
+    def _cut_view(self, ptr: int, nbytes: int):
+        """The workspace bytes [ptr, ptr + nbytes) as a float64 tensor (no copy)."""
+        off = ptr - self.workspace.data_ptr()
+        return self.workspace[off:off + nbytes].view(self._torch.float64)
+
+    def cut_send(self, side: int):
+        send, _, nbytes, _ = self.cut_info(side)
+        return self._cut_view(send, nbytes)
+
+    def cut_recv(self, side: int):
+        _, recv, nbytes, _ = self.cut_info(side)
+        return self._cut_view(recv, nbytes)
+
+    def pack_cut(self):
+        self._call("jac_pack_cut", lib().jac_pack_cut(self._ctx))
+
+    def unpack_cut(self, src_lo=None, ready_lo=None, src_hi=None, ready_hi=None):
+        self._call("jac_unpack_cut", lib().jac_unpack_cut(self._ctx, src_lo, ready_lo, src_hi, ready_hi))
+
+    def sweep_begin(self):
+        self._call("jac_sweep_begin", lib().jac_sweep_begin(self._ctx))
+
+    def sweep_end(self, src_lo=None, ready_lo=None, src_hi=None, ready_hi=None):
+        self._call("jac_sweep_end", lib().jac_sweep_end(self._ctx, src_lo, ready_lo, src_hi, ready_hi))
 
     def set_boundary(self, face: int, value: float):
         self._call("jac_set_boundary", lib().jac_set_boundary(self._ctx, int(face), float(value)))

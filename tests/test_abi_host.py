@@ -127,6 +127,24 @@ def test_wide_layout_holds_the_wide_faces(jac, n, b, h):
     assert L.off_scratch - L.off_send >= L.nblocks * L.send_stride * 8
 
 
+@pytest.mark.parametrize("n,b,has_f", [((16384, 16384), (1024, 1024), False), ((10, 9, 7), (4, 4, 3), True),
+                                        ((14, 11), (4, 4), True)])
+def test_host_staging_flag_adds_two_dense_arrays(jac, n, b, has_f):
+    plain = jac.get_layout(jac.make_desc(n, b, 1, has_f))
+    L = jac.get_layout(jac.make_desc(n, b, 1, has_f, flags=jac.FLAG_HOST_STAGING))
+    dense = -(-int(np.prod(n)) * 8 // 256) * 256
+    assert plain.off_stage_in == -1 and plain.off_stage_out == -1
+    assert L.off_stage_in == plain.total_bytes and L.off_stage_out == L.off_stage_in + dense
+    assert L.total_bytes == plain.total_bytes + 2 * dense
+    assert L.off_stage_in % 256 == 0 and L.off_stage_out % 256 == 0
+    for name in ("off_u", "off_f", "off_send", "off_scratch", "block_stride", "origin"):
+        a, c = getattr(plain, name), getattr(L, name)
+        assert (list(a) == list(c)) if hasattr(a, "__len__") else (a == c), name
+    with pytest.raises(jac.JacError) as e:          # a flag bit the library does not know
+        jac.workspace_bytes(jac.make_desc(n, b, 1, has_f, flags=2))
+    assert e.value.code == jac.EINVAL
+
+
 def test_resident_schedule_accepts_what_fits_a_cluster(jac):
     # 256 x 256 with f: slabs of 32 rows in 8 CTAs; 512 x 256 needs 16 CTAs; both are accepted
     for n, b, f in [((256, 256), (256, 256), True), ((512, 256), (128, 64), False), ((12, 4), (4, 4), True)]:

@@ -1,10 +1,10 @@
 """The five named configurations at full size, in the launch configurations the benchmark times.
 
-Where the CPU oracle finishes the whole job in seconds (configs 1-3 on the machine's host cores) the
-complete solution and every residual are compared; for the 1024^3 run the oracle evaluates sampled
-outputs one by one (the monolithic sweep on each point's dependency box) and the residuals are
-checked through properties that hold at any size.  Set JAC_FULL_ORACLE=1 to sweep the whole
-1024^3 problem on the CPU as well (minutes, ~50 GB of host memory).
+The complete solution and every residual are compared with the CPU oracle.  The 1024^3 run needs
+about 60 GB of host memory for that (the oracle's three padded arrays, f and the two solutions); a
+host with less falls back to sampled outputs, which the oracle evaluates one by one (the monolithic
+sweep on each point's dependency box), plus properties of the residuals that hold at any size, and
+the test prints which of the two ran.  JAC_FULL_ORACLE=0 / 1 forces one or the other.
 """
 import math
 import os
@@ -138,7 +138,7 @@ def test_c3_eigenmode_16384(jac, orc):
 @pytest.mark.parametrize("B_edge", sorted(inputs.HALO_BENCH_SHAPES))
 @pytest.mark.parametrize("h", inputs.HALO_BENCH_WIDTHS)
 def test_c4_halo_shapes_bit_exact(jac, orc, B_edge, h):
-    """Every send buffer after pack and every padded block after unpack, bit for bit."""
+    """Every send buffer of every block after pack and every padded block after unpack, bit for bit."""
     G = inputs.HALO_BENCH_SHAPES[B_edge]
     n, b = (B_edge * G, B_edge * G), (B_edge, B_edge)
     dense = inputs.uniform_field(n, inputs.HALO_BENCH_SEED)
@@ -148,16 +148,13 @@ def test_c4_halo_shapes_bit_exact(jac, orc, B_edge, h):
     with jac.Jacobi(n, b, h, False, "exchange") as J:
         J.set_u(dense)
         J.pack_halos()
-        # all faces of a sample of blocks that covers corners, edges and the interior of the grid
-        blocks = sorted({0, G - 1, G * G - 1, G * (G - 1), G + 1, (G // 2) * G + G // 2, G * G - G - 2}
-                        | set(range(0, G * G, max(1, G * G // 61))))
-        for blk in blocks:
+        for blk in range(G * G):
             for face in range(4):
                 if O.neighbour(blk, face) >= 0:
                     assert np.array_equal(J.get_halo_buffer(blk, face), O.get_halo_buffer(blk, face)), (blk, face)
         J.unpack_halos()
         O.unpack()
-        for blk in blocks:
+        for blk in range(G * G):
             assert np.array_equal(J.get_block_padded(blk), O.get_block_padded(blk)), blk
         assert np.array_equal(J.get_u(), dense)      # interiors untouched
     O.close()
@@ -168,8 +165,29 @@ def _box(arr):
     return lambda lo, hi: arr[tuple(slice(l, h) for l, h in zip(reversed(lo), reversed(hi)))]
 
 
+def _host_memory_bytes() -> int:
+    try:
+        return os.sysconf("SC_PHYS_PAGES") * os.sysconf("SC_PAGE_SIZE")
+    except (ValueError, OSError):
+        return 0
+
+
+def _available_memory_bytes() -> int:
+    try:
+        with open("/proc/meminfo") as fh:
+            for line in fh:
+                if line.startswith("MemAvailable:"):
+                    return int(line.split()[1]) * 1024
+    except OSError:
+        pass
+    return _host_memory_bytes()
+
+
 def test_c5_poisson3d_1024(jac, orc):
     w = inputs.POISSON3D_1024
+    forced = os.environ.get("JAC_FULL_ORACLE")
+    full = forced == "1" or (forced != "0" and min(_host_memory_bytes(), _available_memory_bytes()) >= 72 * 2 ** 30)
+    print(f"config 5 at 1024^3: {'whole field and all residuals' if full else 'sampled outputs'} against the oracle")
     f = inputs.rhs(w)
     norm_f = float(np.sqrt(np.sum(np.square(f, dtype=np.float64))))
     with _make(jac, w, "temporal", 2) as J:     # the schedule the benchmark times
@@ -194,16 +212,18 @@ def test_c5_poisson3d_1024(jac, orc):
         g = got[p[2], p[1], p[0]]
         assert abs(g - v) <= SWEEP_TOL * max(1.0, abs(v)), (p, g, v)
         assert g == v, p
-    if os.environ.get("JAC_FULL_ORACLE") == "1":
+    if full:
         B = _make_oracle(orc, w)
         B.set_f(f)
+        del f
         want_r = []
         for _ in range(w.sweeps // w.residual_every):
             B.sweep(w.residual_every)
             want_r.append(B.residual())
-        assert np.array_equal(got, B.get_u())
-        assert np.max(np.abs(np.array(got_r) - np.array(want_r)) / np.array(want_r)) <= RESID_TOL
+        want = B.get_u()
         B.close()
+        assert np.array_equal(got, want)
+        assert np.max(np.abs(np.array(got_r) - np.array(want_r)) / np.array(want_r)) <= RESID_TOL
 
 
 def test_c5_scaled_256_whole_field_and_residuals(jac, orc):

@@ -5,11 +5,12 @@ workspace: its scratch is a fixed array inside the library image.  A caller insi
 framework's memory pool, or a monitoring hook that must not stall the solver with a cudaMalloc,
 can therefore still ask how far from converged a grid is.
 
-The check: its result must agree with ``jac_residual`` (the context-based entry point, which
-reduces the same per-point residuals from a caller-provided workspace) within the tolerance the
-other residual tests use, on two calls in a row -- the second call finds the first call's numbers
-still in the shared scratch and must not be disturbed by them.  This file sorts last so that a
-run stopping at the first failure has already gone through every other test.
+The check: its result must agree with the CPU oracle's residual of the same padded grid, and with
+``jac_residual`` (the context-based entry point, which reduces the same per-point residuals from
+a caller-provided workspace), within the tolerance the other residual tests use, on two calls in
+a row -- the second call finds the first call's numbers still in the shared scratch and must not
+be disturbed by them.  This file sorts last so that a run stopping at the first failure has
+already gone through every other test.
 """
 import ctypes as C
 
@@ -47,7 +48,14 @@ CASES = [((300, 170), (100, 85), True), ((1024, 1536), (256, 256), False), ((40,
          ((9, 5), (9, 5), False)]
 
 
-def test_matches_context_residual_on_consecutive_calls(jac):
+def _oracle(orc, n, u, f, bvals):
+    """The oracle's residual norm of the dense grid inside its ring of Dirichlet values."""
+    padded = orc.mono_padded(n, bvals)
+    padded[(slice(1, -1),) * len(n)] = u
+    return orc.mono_residual(padded, f)
+
+
+def test_matches_oracle_and_context_residual_on_consecutive_calls(jac, orc):
     import torch
     for n, b, has_f in CASES:
         rng = np.random.default_rng(21)
@@ -55,13 +63,16 @@ def test_matches_context_residual_on_consecutive_calls(jac):
         u = rng.uniform(-1, 1, shape)
         f = rng.uniform(-1, 1, shape) if has_f else None
         bvals = [0.5, -1.0, 2.0, 3.0, -0.25, 1.5][: 2 * len(n)]
-        want = _reference(jac, n, b, u, f, bvals)
+        want = _oracle(orc, n, u, f, bvals)
+        by_context = _reference(jac, n, b, u, f, bvals)
+        assert abs(by_context - want) <= RESID_TOL * want, (n, by_context, want)
         ud = torch.from_numpy(u).cuda()
         fd = torch.from_numpy(f).cuda() if has_f else None
         first = jac.residual_dense_static(ud, fd, bvals)
         second = jac.residual_dense_static(ud, fd, bvals)
         assert abs(first - want) <= RESID_TOL * want, (n, first, want)
         assert abs(second - want) <= RESID_TOL * want, (n, second, want)
+        assert abs(first - by_context) <= RESID_TOL * by_context, (n, first, by_context)
         assert first == second            # fixed reduction order: repeatable bit for bit
         assert np.array_equal(ud.cpu().numpy(), u)   # inputs are only read
 
