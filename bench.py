@@ -5,7 +5,8 @@
                     [--workload c3_eigenmode_16384] [--mode auto] [--tsteps T]
 
 One *step* is one whole job of the workload: its sweeps (every sweep with its halo exchange:
-pack, unpack, update) followed by the residual reduction.  The metric is Jacobi GLUP/s
+pack, unpack, update, in whatever form the schedule gives them) and the residual norm after every
+group of sweeps the workload names (configs 2 and 5: every 10 sweeps; else after the last sweep).  The metric is Jacobi GLUP/s
 (1e9 lattice-point updates per second); effective GB/s = GLUP/s x compulsory bytes per point
 (16 B: read u, write u'; 24 B with f).
 
@@ -296,16 +297,21 @@ def run_ours(args, w: inputs.Workload):
     norms = torch.zeros(len(groups), dtype=torch.float64).pin_memory()
 
     def one_job(J, pairs=None):
-        """The sweeps of one step with the residual after every group (queued, nothing waits)."""
+        """The sweeps of one step with the residual norm after every group (queued, nothing waits).
+        The norm after group k comes out of the first sweep of group k + 1, which reads that state
+        anyway (jac_residual_sweep_async); only the last one needs a pass of its own."""
         for k, n_sw in enumerate(groups):
             if pairs is not None:
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(stream)
-            J.sweep(n_sw)
+                a.record(J.stream)
+            if k == 0:
+                J.sweep(n_sw)
+            else:
+                J.residual_sweep_async(n_sw, norms[k - 1:k])
             if pairs is not None:
-                b.record(stream)
+                b.record(J.stream)
                 pairs.append((a, b))
-            J.residual_async(norms[k:k + 1])
+        J.residual_async(norms[len(groups) - 1:])
 
     def time_schedule(J, mode, tsteps, steps, warmup, sample_clocks):
         """K steps (each: input -> blocks, the sweeps, a residual after every group of sweeps the
@@ -413,8 +419,11 @@ def run_ours(args, w: inputs.Workload):
         def e2e_step(Jc, out, nrm):
             Jc.set_u_async(host_in)
             for k, n_sw in enumerate(groups):
-                Jc.sweep(n_sw)
-                Jc.residual_async(nrm[k:k + 1])
+                if k == 0:
+                    Jc.sweep(n_sw)
+                else:
+                    Jc.residual_sweep_async(n_sw, nrm[k - 1:k])
+            Jc.residual_async(nrm[len(groups) - 1:])
             Jc.get_u_async(out)
 
         def run_pipeline(depth, count):
@@ -451,8 +460,8 @@ def run_ours(args, w: inputs.Workload):
 
         one_steps = max(3, min(args.steps, 6))
         one = e2e_record(run_pipeline(1, one_steps), one_steps,
-                         "one context, steps queued back to back on one stream: jac_set_u_async(pinned host) + jac_sweep + "
-                         "jac_residual_async per group + jac_get_u_async(pinned host)")
+                         "one context, steps queued back to back on one stream: jac_set_u_async(pinned host) + jac_sweep (jac_residual_sweep_async from the second group on) + "
+                         "jac_residual_async after the last group + jac_get_u_async(pinned host)")
         e2e = one
         # several contexts on as many streams, steps going round them: the copy in of one step, the
         # sweeps of another and the copy out of a third run at the same time (the two copy directions
@@ -463,7 +472,7 @@ def run_ours(args, w: inputs.Workload):
             pipe_steps = max(2 * depth, args.steps)
             e2e = e2e_record(run_pipeline(depth, pipe_steps), pipe_steps,
                              f"{depth} contexts on {depth} streams, steps going round them; every step is jac_set_u_async(pinned "
-                             "host) + jac_sweep + jac_residual_async per group + jac_get_u_async(pinned host); timed by the host "
+                             "host) + jac_sweep (jac_residual_sweep_async from the second group on) + jac_residual_async + jac_get_u_async(pinned host); timed by the host "
                              "clock between synchronisations of all streams")
             e2e["one_context"] = one
         bound_ms = 2 * nbytes / 55e9 * 1e3

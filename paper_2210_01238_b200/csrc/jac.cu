@@ -3,6 +3,7 @@
 // in the caller's workspace.
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -12,6 +13,7 @@
 #include "jac_geom.h"
 #include "jac_kernels.cuh"
 #include "jac_resident.cuh"
+#include "jac_temporal3d.cuh"
 
 namespace {
 
@@ -126,14 +128,16 @@ TemporalGrid temporal_grid_2d(const JacGeom& g, int T, bool has_f)
 TemporalGrid temporal_grid_3d(const JacGeom& g, int T)
 {
     TemporalGrid t{};
-    t.a = (int)ceil_div(g.nx, 60);
-    t.b = (int)ceil_div(g.ny, jac::k3dTileRows - 2 * T);
-    int zchunk = 128;
-    while (zchunk > 16 && (long long)t.a * t.b * ceil_div(g.nz, zchunk) < (long long)kNumSMs * 4) zchunk /= 2;
+    t.a = (int)ceil_div(g.nx, jac::t3_out_cols(T));
+    t.b = (int)ceil_div(g.ny, jac::t3_out_rows(T));
+    // planes per chunk: a chunk of Z planes costs Z + 2T steps; long chunks waste the least, but the
+    // launch should still be several rounds of CTAs (one CTA per SM)
+    int zchunk = 256;
+    while (zchunk > 16 && (long long)t.a * t.b * ceil_div(g.nz, zchunk) < (long long)kNumSMs * 6) zchunk /= 2;
     t.chunk = zchunk;
     t.c = (int)ceil_div(g.nz, zchunk);
     t.ctas = (long long)t.a * t.b * t.c;
-    t.warps = t.ctas * jac::k3dWarps;
+    t.warps = t.ctas * jac::kT3Warps;
     return t;
 }
 
@@ -174,7 +178,7 @@ long long max_partials(const JacGeom& g, long long sweep_ctas, bool has_f)
 {
     long long m = sweep_ctas;
     if (g.ndim == 2) for (int T = 1; T <= 8; ++T) m = std::max(m, temporal_grid_2d(g, T, has_f).warps);
-    else for (int T = 1; T <= 2; ++T) m = std::max(m, temporal_grid_3d(g, T).warps);
+    else for (int T = 1; T <= jac::kT3MaxT; ++T) m = std::max(m, temporal_grid_3d(g, T).warps);
     return m;
 }
 
@@ -244,7 +248,7 @@ int build_geometry(const jac_desc* d, JacGeom* g, jac_layout* L)
         // whole lanes lie inside or outside the domain: 4 points per lane in 2D, 2 in 3D
         if (n[1] >= (1LL << 30)) return JAC_EINVAL;
         if (d->ndim == 2 && (b[0] % 4 != 0 || n[0] % 4 != 0)) return JAC_EINVAL;
-        if (d->ndim == 3 && (b[0] % 2 != 0 || n[0] % 2 != 0 || d->tsteps > 2 || n[2] >= (1LL << 30)))
+        if (d->ndim == 3 && (b[0] % 2 != 0 || n[0] % 2 != 0 || d->tsteps > jac::kT3MaxT || n[2] >= (1LL << 30)))
             return JAC_EINVAL;
     }
     if (d->mode == JAC_MODE_RESIDENT) {
@@ -674,83 +678,115 @@ int usable(jac_ctx* c)
 
 // Sweeps per launch when the caller leaves the choice to the library.  2D: 8 levels pay off only
 // without a right-hand side and on grids large enough to fill the GPU with 256-row strips
-// (measured: 16384^2 1668 vs 1320 GLUP/s; 4096^2 with f 236 vs 326); otherwise 4.  3D: 2.
+// (measured: 16384^2 1668 vs 1320 GLUP/s; 4096^2 with f 236 vs 326); otherwise 4.  3D: 3.
 int default_tsteps(const jac_desc& d)
 {
     if (d.tsteps > 0) return d.tsteps;
-    if (d.ndim == 3) return 2;
+    if (d.ndim == 3) return 3;
     const bool large = d.n[0] * d.n[1] >= (1LL << 26);
     return (!d.has_f && large) ? 8 : 4;
 }
 
-// T sweeps in one launch (3D, tiles of 64 x 48 streamed along z).  RES: the launch also leaves
-// per-warp partial sums of the squared residual of the state before its last sweep.
-template <int T, bool HAS_F, bool RES>
+// The dynamic shared memory a kernel may use is an attribute of the kernel on a device: set it the
+// first time the kernel is launched on that device, not on every launch (the call costs host time,
+// which the launch-bound small grids feel).
+template <auto Kern>
+int ensure_dynamic_smem(jac_ctx* c, size_t smem)
+{
+    static std::atomic<unsigned long long> done{0};      // one bit per device ordinal
+    const unsigned long long bit = 1ULL << (c->device & 63);
+    if (c->device < 64 && (done.load(std::memory_order_acquire) & bit)) return JAC_OK;
+    JAC_CK(c, cudaFuncSetAttribute(Kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    done.fetch_or(bit, std::memory_order_release);
+    return JAC_OK;
+}
+
+// T sweeps in one launch (3D, tiles of 64 x 32 streamed along z).  RES (jac::kRes*): the launch also
+// leaves per-warp partial sums of the squared residual of the state before its last sweep, or of
+// the state it reads.
+template <int T, bool HAS_F, int RES>
 int launch_temporal3d_t(jac_ctx* c, const double* u, double* un, long long* nparts)
 {
     const TemporalGrid t = temporal_grid_3d(c->g, T);
     if (t.ctas > kMaxGrid) return JAC_EINVAL;
-    auto kern = jac::temporal3d_kernel<T, HAS_F, RES>;
-    const size_t smem = jac::k3d_smem_bytes(HAS_F);
-    JAC_CK(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    kern<<<(unsigned)t.ctas, jac::k3dWarps * 32, smem, c->stream>>>(u, un, c->f, c->partials, c->g, t.a, t.b, t.c,
+    constexpr auto kern = jac::temporal3d_kernel<T, HAS_F, RES>;
+    const size_t smem = jac::t3_smem_bytes(T, HAS_F);
+    const int rc = ensure_dynamic_smem<kern>(c, smem);
+    if (rc) return rc;
+    kern<<<(unsigned)t.ctas, jac::kT3Warps * 32, smem, c->stream>>>(u, un, c->f, c->partials, c->g, t.a, t.b, t.c,
                                                                    t.chunk);
-    if (RES) *nparts = t.warps;
+    if (RES != jac::kResNone) *nparts = t.warps;
     return check_launch(c);
 }
 
-int launch_temporal3d_n(jac_ctx* c, int t, const double* u, double* un, bool res, long long* nparts)
+template <int T, int RES>
+int launch_temporal3d(jac_ctx* c, const double* u, double* un, long long* nparts)
 {
-    const bool f = c->desc.has_f != 0;
-    if (res) {
-        if (t == 1) return f ? launch_temporal3d_t<1, true, true>(c, u, un, nparts)
-                             : launch_temporal3d_t<1, false, true>(c, u, un, nparts);
-        return f ? launch_temporal3d_t<2, true, true>(c, u, un, nparts)
-                 : launch_temporal3d_t<2, false, true>(c, u, un, nparts);
+    return c->desc.has_f ? launch_temporal3d_t<T, true, RES>(c, u, un, nparts)
+                         : launch_temporal3d_t<T, false, RES>(c, u, un, nparts);
+}
+
+template <int RES>
+int launch_temporal3d_r(jac_ctx* c, int t, const double* u, double* un, long long* nparts)
+{
+    switch (t) {
+        case 1: return launch_temporal3d<1, RES>(c, u, un, nparts);
+        case 2: return launch_temporal3d<2, RES>(c, u, un, nparts);
+        default: return launch_temporal3d<3, RES>(c, u, un, nparts);
     }
-    if (t == 1) return f ? launch_temporal3d_t<1, true, false>(c, u, un, nparts)
-                         : launch_temporal3d_t<1, false, false>(c, u, un, nparts);
-    return f ? launch_temporal3d_t<2, true, false>(c, u, un, nparts)
-             : launch_temporal3d_t<2, false, false>(c, u, un, nparts);
+}
+
+int launch_temporal3d_n(jac_ctx* c, int t, const double* u, double* un, int res, long long* nparts)
+{
+    if (res == jac::kResBeforeLast) return launch_temporal3d_r<jac::kResBeforeLast>(c, t, u, un, nparts);
+    if (res == jac::kResOfInput) return launch_temporal3d_r<jac::kResOfInput>(c, t, u, un, nparts);
+    return launch_temporal3d_r<jac::kResNone>(c, t, u, un, nparts);
 }
 
 // T sweeps in one launch (2D, register-streaming temporal blocking)
-template <int T, bool HAS_F, bool RES>
+template <int T, bool HAS_F, int RES>
 int launch_temporal_t(jac_ctx* c, const double* u, double* un, long long* nparts)
 {
     const TemporalGrid t = temporal_grid_2d(c->g, T, HAS_F);
-    auto kern = jac::temporal2d_kernel<T, HAS_F, RES>;
+    constexpr auto kern = jac::temporal2d_kernel<T, HAS_F, RES>;
     const size_t smem = jac::temporal_smem_bytes(T, HAS_F);
-    if (smem > 48 * 1024)
-        JAC_CK(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    if (smem > 48 * 1024) {
+        const int rc = ensure_dynamic_smem<kern>(c, smem);
+        if (rc) return rc;
+    }
     kern<<<(unsigned)t.ctas, jac::kTemporalWarps * 32, smem, c->stream>>>(u, un, c->f, c->partials, c->g, t.a, t.b,
                                                                          t.chunk);
-    if (RES) *nparts = t.warps;
+    if (RES != jac::kResNone) *nparts = t.warps;
     return check_launch(c);
 }
 
-template <int T>
-int launch_temporal(jac_ctx* c, const double* u, double* un, bool res, long long* nparts)
+template <int T, int RES>
+int launch_temporal(jac_ctx* c, const double* u, double* un, long long* nparts)
 {
-    const bool f = c->desc.has_f != 0;
-    if (res) return f ? launch_temporal_t<T, true, true>(c, u, un, nparts)
-                      : launch_temporal_t<T, false, true>(c, u, un, nparts);
-    return f ? launch_temporal_t<T, true, false>(c, u, un, nparts)
-             : launch_temporal_t<T, false, false>(c, u, un, nparts);
+    return c->desc.has_f ? launch_temporal_t<T, true, RES>(c, u, un, nparts)
+                         : launch_temporal_t<T, false, RES>(c, u, un, nparts);
 }
 
-int launch_temporal_n(jac_ctx* c, int t, const double* u, double* un, bool res, long long* nparts)
+template <int RES>
+int launch_temporal_r(jac_ctx* c, int t, const double* u, double* un, long long* nparts)
 {
     switch (t) {
-        case 1: return launch_temporal<1>(c, u, un, res, nparts);
-        case 2: return launch_temporal<2>(c, u, un, res, nparts);
-        case 3: return launch_temporal<3>(c, u, un, res, nparts);
-        case 4: return launch_temporal<4>(c, u, un, res, nparts);
-        case 5: return launch_temporal<5>(c, u, un, res, nparts);
-        case 6: return launch_temporal<6>(c, u, un, res, nparts);
-        case 7: return launch_temporal<7>(c, u, un, res, nparts);
-        default: return launch_temporal<8>(c, u, un, res, nparts);
+        case 1: return launch_temporal<1, RES>(c, u, un, nparts);
+        case 2: return launch_temporal<2, RES>(c, u, un, nparts);
+        case 3: return launch_temporal<3, RES>(c, u, un, nparts);
+        case 4: return launch_temporal<4, RES>(c, u, un, nparts);
+        case 5: return launch_temporal<5, RES>(c, u, un, nparts);
+        case 6: return launch_temporal<6, RES>(c, u, un, nparts);
+        case 7: return launch_temporal<7, RES>(c, u, un, nparts);
+        default: return launch_temporal<8, RES>(c, u, un, nparts);
     }
+}
+
+int launch_temporal_n(jac_ctx* c, int t, const double* u, double* un, int res, long long* nparts)
+{
+    if (res == jac::kResBeforeLast) return launch_temporal_r<jac::kResBeforeLast>(c, t, u, un, nparts);
+    if (res == jac::kResOfInput) return launch_temporal_r<jac::kResOfInput>(c, t, u, un, nparts);
+    return launch_temporal_r<jac::kResNone>(c, t, u, un, nparts);
 }
 
 // nsweeps sweeps in ONE launch of one thread-block cluster that keeps the grid in shared memory
@@ -833,20 +869,24 @@ int choose_resident_cluster(jac_ctx* c)
     return JAC_EINVAL;
 }
 
-// nsweeps iterations in the context's schedule.  With `res`, the last sweep also leaves partial
-// sums of the squared residual of the state it reads in the scratch (*nparts of them).
-int run_sweeps(jac_ctx* c, int nsweeps, bool res, long long* nparts)
+// nsweeps iterations in the context's schedule.  res (jac::kRes*): one launch also leaves partial
+// sums of the squared residual in the scratch (*nparts of them) -- kResBeforeLast: the last sweep,
+// of the state it reads; kResOfInput: the first sweep, of the state the call starts from.
+int run_sweeps(jac_ctx* c, int nsweeps, int res, long long* nparts)
 {
     int rc = JAC_OK;
     if (c->cut[0] || c->cut[1]) return JAC_EINVAL;   // a slab sweeps through jac_sweep_begin / jac_sweep_end
     const JacGeom& g = c->g;
     const long long sweep_parts = g.nblocks * c->tile.ctas_per_block;
+    // does sweep number s (0-based) of the call carry the residual?
+    auto carries = [&](int s) {
+        return (res == jac::kResBeforeLast && s + 1 == nsweeps) || (res == jac::kResOfInput && s == 0);
+    };
     switch (c->desc.mode) {
         case JAC_MODE_FUSED:
             for (int s = 0; s < nsweeps; ++s) {
-                const bool last = res && s + 1 == nsweeps;
-                rc = last ? launch_sweep<jac::OP_UPDATE_PULL_RES>(c, c->u[c->cur], c->u[c->cur ^ 1], 0, g.nblocks)
-                          : launch_sweep<jac::OP_UPDATE_PULL>(c, c->u[c->cur], c->u[c->cur ^ 1], 0, g.nblocks);
+                rc = carries(s) ? launch_sweep<jac::OP_UPDATE_PULL_RES>(c, c->u[c->cur], c->u[c->cur ^ 1], 0, g.nblocks)
+                                : launch_sweep<jac::OP_UPDATE_PULL>(c, c->u[c->cur], c->u[c->cur ^ 1], 0, g.nblocks);
                 if (rc) return rc;
                 c->cur ^= 1;
             }
@@ -856,10 +896,9 @@ int run_sweeps(jac_ctx* c, int nsweeps, bool res, long long* nparts)
             break;
         case JAC_MODE_EXCHANGE:
             for (int s = 0; s < nsweeps; ++s) {
-                const bool last = res && s + 1 == nsweeps;
                 if ((rc = do_exchange(c))) return rc;
-                rc = last ? launch_sweep<jac::OP_UPDATE_RES>(c, c->u[c->cur], c->u[c->cur ^ 1], 0, g.nblocks)
-                          : launch_sweep<jac::OP_UPDATE>(c, c->u[c->cur], c->u[c->cur ^ 1], 0, g.nblocks);
+                rc = carries(s) ? launch_sweep<jac::OP_UPDATE_RES>(c, c->u[c->cur], c->u[c->cur ^ 1], 0, g.nblocks)
+                                : launch_sweep<jac::OP_UPDATE>(c, c->u[c->cur], c->u[c->cur ^ 1], 0, g.nblocks);
                 if (rc) return rc;
                 c->cur ^= 1;
                 c->ghosts_fresh = false;
@@ -869,11 +908,10 @@ int run_sweeps(jac_ctx* c, int nsweeps, bool res, long long* nparts)
             break;
         case JAC_MODE_PERTASK:
             for (int s = 0; s < nsweeps; ++s) {
-                const bool last = res && s + 1 == nsweeps;
                 if ((rc = do_exchange(c))) return rc;
                 for (long long blk = 0; blk < g.nblocks; ++blk) {
-                    rc = last ? launch_sweep<jac::OP_UPDATE_RES>(c, c->u[c->cur], c->u[c->cur ^ 1], blk, 1)
-                              : launch_sweep<jac::OP_UPDATE>(c, c->u[c->cur], c->u[c->cur ^ 1], blk, 1);
+                    rc = carries(s) ? launch_sweep<jac::OP_UPDATE_RES>(c, c->u[c->cur], c->u[c->cur ^ 1], blk, 1)
+                                    : launch_sweep<jac::OP_UPDATE>(c, c->u[c->cur], c->u[c->cur ^ 1], blk, 1);
                     if (rc) return rc;
                 }
                 c->cur ^= 1;
@@ -883,12 +921,17 @@ int run_sweeps(jac_ctx* c, int nsweeps, bool res, long long* nparts)
             if (res) *nparts = sweep_parts;
             break;
         case JAC_MODE_TEMPORAL: {
+            // as few launches as the depth allows, and those of equal depth up to one sweep: a
+            // launch of one sweep costs most of what a launch of T does
             const int T = default_tsteps(c->desc);
-            for (int left = nsweeps; left > 0;) {
-                const int t = std::min(T, left);
-                const bool last = res && left == t;
-                rc = (g.ndim == 2) ? launch_temporal_n(c, t, c->u[c->cur], c->u[c->cur ^ 1], last, nparts)
-                                   : launch_temporal3d_n(c, t, c->u[c->cur], c->u[c->cur ^ 1], last, nparts);
+            const int launches = (nsweeps + T - 1) / T;
+            for (int k = 0, left = nsweeps; left > 0; ++k) {
+                const int t = nsweeps / launches + (k < nsweeps % launches ? 1 : 0);
+                const int r = (res == jac::kResBeforeLast && left == t) ? jac::kResBeforeLast
+                              : (res == jac::kResOfInput && k == 0)     ? jac::kResOfInput
+                                                                        : jac::kResNone;
+                rc = (g.ndim == 2) ? launch_temporal_n(c, t, c->u[c->cur], c->u[c->cur ^ 1], r, nparts)
+                                   : launch_temporal3d_n(c, t, c->u[c->cur], c->u[c->cur ^ 1], r, nparts);
                 if (rc) return rc;
                 c->cur ^= 1;
                 left -= t;
@@ -898,13 +941,19 @@ int run_sweeps(jac_ctx* c, int nsweeps, bool res, long long* nparts)
             break;
         }
         case JAC_MODE_RESIDENT: {
-            // all sweeps in one launch; a residual-carrying last sweep runs as one ordinary launch
+            // all sweeps in one launch; a residual-carrying first or last sweep runs as one ordinary launch
             const int n_res = res ? nsweeps - 1 : nsweeps;
+            if (res == jac::kResOfInput) {
+                if ((rc = launch_sweep<jac::OP_UPDATE_PULL_RES>(c, c->u[c->cur], c->u[c->cur ^ 1], 0, g.nblocks)))
+                    return rc;
+                c->cur ^= 1;
+                *nparts = sweep_parts;
+            }
             if (n_res > 0) {
                 if ((rc = launch_resident(c, c->u[c->cur], c->u[c->cur ^ 1], n_res))) return rc;
                 c->cur ^= 1;
             }
-            if (res) {
+            if (res == jac::kResBeforeLast) {
                 if ((rc = launch_sweep<jac::OP_UPDATE_PULL_RES>(c, c->u[c->cur], c->u[c->cur ^ 1], 0, g.nblocks)))
                     return rc;
                 c->cur ^= 1;
@@ -917,6 +966,7 @@ int run_sweeps(jac_ctx* c, int nsweeps, bool res, long long* nparts)
         case JAC_MODE_WIDE: {
             // groups of up to K sweeps (K <= h): one wide exchange, then updates on boxes shrinking
             // from the interior grown by t - 1 layers down to the interior itself
+            if (res == jac::kResOfInput) return JAC_EINVAL;   // the first update of a group runs on a grown box
             const int K = c->desc.tsteps > 0 ? c->desc.tsteps : g.h;
             if (c->f && !c->f_ghosts_fresh) {
                 if ((rc = do_exchange_wide(c, c->f))) return rc;
@@ -1360,7 +1410,7 @@ int jac_sweep(jac_ctx* c, int nsweeps)
     if (rc) return rc;
     if (nsweeps < 0) return JAC_EINVAL;
     if (nsweeps == 0) return JAC_OK;
-    return run_sweeps(c, nsweeps, false, nullptr);
+    return run_sweeps(c, nsweeps, jac::kResNone, nullptr);
 }
 
 int jac_sweep_residual(jac_ctx* c, int nsweeps, double* host_out_l2)
@@ -1369,7 +1419,7 @@ int jac_sweep_residual(jac_ctx* c, int nsweeps, double* host_out_l2)
     if (rc) return rc;
     if (nsweeps < 1 || !host_out_l2) return JAC_EINVAL;
     long long nparts = 0;
-    if ((rc = run_sweeps(c, nsweeps, true, &nparts))) return rc;
+    if ((rc = run_sweeps(c, nsweeps, jac::kResBeforeLast, &nparts))) return rc;
     return finish_norm(c, nparts, host_out_l2);
 }
 
@@ -1385,7 +1435,7 @@ int jac_solve(jac_ctx* c, int max_sweeps, int check_every, double tol, int* host
     while (done < max_sweeps) {
         const int n = std::min(check_every, max_sweeps - done);
         long long nparts = 0;
-        if ((rc = run_sweeps(c, n, true, &nparts))) return rc;
+        if ((rc = run_sweeps(c, n, jac::kResBeforeLast, &nparts))) return rc;
         if ((rc = finish_norm(c, nparts, &res))) return rc;
         done += n;
         if (res <= tol) break;
@@ -1472,6 +1522,26 @@ int residual_queued(jac_ctx* c, double* host_out, bool norm)
 int jac_residual_async(jac_ctx* c, double* host_out_l2) { return residual_queued(c, host_out_l2, true); }
 
 int jac_residual_sumsq_async(jac_ctx* c, double* host_out_sumsq) { return residual_queued(c, host_out_sumsq, false); }
+
+int jac_residual_sweep_async(jac_ctx* c, int nsweeps, double* host_out_l2)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    if (nsweeps < 1 || !host_out_l2 || has_cuts(c)) return JAC_EINVAL;
+    // schedules whose first launch cannot carry the sum: the ordinary residual pass, then the sweeps
+    if (c->desc.mode == JAC_MODE_WIDE) {
+        if ((rc = residual_queued(c, host_out_l2, true))) return rc;
+        return run_sweeps(c, nsweeps, jac::kResNone, nullptr);
+    }
+    long long nparts = 0;
+    if ((rc = run_sweeps(c, nsweeps, jac::kResOfInput, &nparts))) return rc;
+    jac::reduce_partials_kernel<<<1, 1024, 0, c->stream>>>(c->partials, nparts, c->result);
+    if ((rc = check_launch(c))) return rc;
+    sqrt_in_place_kernel<<<1, 1, 0, c->stream>>>(c->result);
+    if ((rc = check_launch(c))) return rc;
+    JAC_CK(c, cudaMemcpyAsync(host_out_l2, c->result, sizeof(double), cudaMemcpyDeviceToHost, c->stream));
+    return JAC_OK;
+}
 
 int jac_pack_cut(jac_ctx* c)
 {

@@ -20,6 +20,11 @@ __host__ __device__ constexpr bool op_pulls(int op) { return op == OP_UPDATE_PUL
 __host__ __device__ constexpr bool op_sums(int op) { return op == OP_RESIDUAL || op == OP_UPDATE_RES || op == OP_UPDATE_PULL_RES; }
 __host__ __device__ constexpr bool op_ext(int op) { return op == OP_UPDATE_EXT; }
 
+// which state a temporal launch also measures the residual of (RES template argument)
+enum : int { kResNone = 0,        // none
+             kResBeforeLast = 1,  // the state before the last sweep of the launch (its top level reads it)
+             kResOfInput = 2 };   // the state the launch reads (its first level reads it)
+
 __device__ __forceinline__ double add_rn(double a, double b) { return __dadd_rn(a, b); }
 __device__ __forceinline__ double sub_rn(double a, double b) { return __dsub_rn(a, b); }
 __device__ __forceinline__ double mul_rn(double a, double b) { return __dmul_rn(a, b); }
@@ -780,7 +785,7 @@ __host__ __device__ constexpr int slot3(int ph, int d) { return (((ph + d) % 3) 
 // one row.  EDGE = false is for steps in which no row and no column involved lies outside the
 // domain: no Dirichlet fix-up is compiled in.
 // level s of one step: row r - 2s + 1 from the window of level s - 1
-template <int T, bool HAS_F, bool RES, int PH, bool EDGE, int s>
+template <int T, bool HAS_F, int RES, int PH, bool EDGE, int s>
 __device__ __forceinline__ void temporal_level(RowN<temporal_points(T)> (&win)[T][3], const TemporalCtx& c,
                                                const JacGeom& g, int r, const RowCursor& out_cur, double& acc)
 {
@@ -821,8 +826,8 @@ __device__ __forceinline__ void temporal_level(RowN<temporal_points(T)> (&win)[T
         double sum = add_rn(add_rn(W, E), add_rn(S.v[q], N.v[q]));
         if (HAS_F) sum = add_rn(sum, ff.v[q]);
         o.v[q] = mul_rn(sum, 0.25);
-        // residual of the state the top level reads (M is that state at this point)
-        if (RES && s == T) res.v[q] = sub_rn(sum, mul_rn(4.0, M.v[q]));
+        // residual of the state this level reads (M is that state at this point)
+        if ((RES == kResBeforeLast && s == T) || (RES == kResOfInput && s == 1)) res.v[q] = sub_rn(sum, mul_rn(4.0, M.v[q]));
     }
     if (EDGE) {
         if (rs < 0) o = fill_rown<P>(c.c_my);
@@ -833,14 +838,16 @@ __device__ __forceinline__ void temporal_level(RowN<temporal_points(T)> (&win)[T
         win[s][slot3(PH, d)] = o;
     } else if (c.store_lane && rs >= c.Y0 && rs < c.Y1) {
         store_rown<P>(c.ob + out_cur.off, o);
-        if (RES) {   // exactly the points this lane stores: every interior point once
+    }
+    // the points of the strip's output region: every interior point is in exactly one, and every
+    // level is exact there
+    if (((RES == kResBeforeLast && s == T) || (RES == kResOfInput && s == 1)) && c.store_lane && rs >= c.Y0 && rs < c.Y1) {
 #pragma unroll
-            for (int q = 0; q < P; ++q) acc = add_rn(acc, mul_rn(res.v[q], res.v[q]));
-        }
+        for (int q = 0; q < P; ++q) acc = add_rn(acc, mul_rn(res.v[q], res.v[q]));
     }
 }
 
-template <int T, bool HAS_F, bool RES, int PH, bool EDGE, int s>
+template <int T, bool HAS_F, int RES, int PH, bool EDGE, int s>
 struct TemporalLevels {   // levels s, s - 1, ..., 2 (top level first)
     static __device__ __forceinline__ void run(RowN<temporal_points(T)> (&win)[T][3], const TemporalCtx& c, const JacGeom& g, int r,
                                                const RowCursor& out_cur, double& acc) {
@@ -848,7 +855,7 @@ struct TemporalLevels {   // levels s, s - 1, ..., 2 (top level first)
         TemporalLevels<T, HAS_F, RES, PH, EDGE, s - 1>::run(win, c, g, r, out_cur, acc);
     }
 };
-template <int T, bool HAS_F, bool RES, int PH, bool EDGE>
+template <int T, bool HAS_F, int RES, int PH, bool EDGE>
 struct TemporalLevels<T, HAS_F, RES, PH, EDGE, 1> {
     static __device__ __forceinline__ void run(RowN<temporal_points(T)> (&)[T][3], const TemporalCtx&, const JacGeom&, int,
                                                const RowCursor&, double&) {}
@@ -859,7 +866,7 @@ struct TemporalLevels<T, HAS_F, RES, PH, EDGE, 1> {
 // the wait for the copy of row r; then the row is taken, its ring stage refilled, and level 1
 // runs.  EDGE = false is for steps in which no row and no column involved lies outside the
 // domain: no Dirichlet fix-up is compiled in.
-template <int T, bool HAS_F, bool RES, int PH, bool EDGE>
+template <int T, bool HAS_F, int RES, int PH, bool EDGE>
 __device__ __forceinline__ void temporal_step(RowN<temporal_points(T)> (&win)[T][3], const TemporalCtx& c, const JacGeom& g,
                                               int r, RowCursor& load_cur, RowCursor& out_cur, double& acc)
 {
@@ -881,7 +888,7 @@ __device__ __forceinline__ long long column_base(const JacGeom& g, long long gx)
     return bxi * g.block_stride + g.origin + (gx - bxi * g.bx);
 }
 
-template <int T, bool HAS_F, bool RES, int PH>
+template <int T, bool HAS_F, int RES, int PH>
 __device__ __forceinline__ void temporal_step_any(RowN<temporal_points(T)> (&win)[T][3], const TemporalCtx& c, const JacGeom& g,
                                                   int r, RowCursor& load_cur, RowCursor& out_cur, double& acc)
 {
@@ -891,9 +898,9 @@ __device__ __forceinline__ void temporal_step_any(RowN<temporal_points(T)> (&win
     else temporal_step<T, HAS_F, RES, PH, false>(win, c, g, r, load_cur, out_cur, acc);
 }
 
-// RES: the top level also accumulates the squared residual of the state it reads (the state
-// before the last sweep of the launch); every warp writes its partial sum to partials[warp id].
-template <int T, bool HAS_F, bool RES>
+// RES: the top level (kResBeforeLast) or the first level (kResOfInput) also accumulates the squared
+// residual of the state it reads; every warp writes its partial sum to partials[warp id].
+template <int T, bool HAS_F, int RES>
 __global__ void __launch_bounds__(kTemporalWarps * 32,
                                   (((T > 4 && temporal_points(T) == 4) || temporal_f_ring(T, HAS_F)) ? 2 : JAC_TOCC))
 temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const double* __restrict__ f,
@@ -965,356 +972,10 @@ temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
         if (r + 2 < r_end) temporal_step_any<T, HAS_F, RES, 2>(win, c, g, r + 2, load_cur, out_cur, acc);
     }
     cp_async_wait<0>();
-    if (RES) {
+    if (RES != kResNone) {
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) acc = add_rn(acc, __shfl_down_sync(0xffffffffu, acc, off));
         if (lane == 0) partials[wid] = acc;
-    }
-}
-
-// ---------------------------------------------------------------------------------------
-// 3D temporal blocking: T (1 or 2) sweeps per launch.
-//
-// A CTA of 8 warps owns a tile of 64 columns x 48 rows and streams it along z.  A lane holds 2
-// consecutive points of each of its warp's 6 rows, so a warp covers 64 x 6 points of a plane.
-// Input plane p enters at level 0; level s produces plane p - 2s + 1 (two planes behind the level
-// below, so the levels of one step are independent).  Each level keeps a 3-plane window of its
-// own rows in registers (3 * 6 * 2 doubles per lane and level).  West/east neighbours come by
-// shuffle, north/south neighbours inside a warp from registers, and across warps from shared
-// memory: level-0 planes sit in the cp.async ring anyway, and every warp publishes the first and
-// last row of its level-1 plane in a small exchange buffer.  One __syncthreads per step.
-// Two columns / two rows at every tile side lose validity (one per level): 60 x (48 - 2T) points
-// per plane are stored.  Tiles read across block borders directly; Dirichlet values are
-// injected outside the domain at every level (EDGE variant only).  Requires bx % 2 == 0.
-// ---------------------------------------------------------------------------------------
-#ifndef JAC_T3W
-#define JAC_T3W 8     // warps per CTA, stacked along y
-#endif
-#ifndef JAC_T3R
-#define JAC_T3R 6     // rows per warp
-#endif
-constexpr int k3dWarps = JAC_T3W;
-constexpr int k3dRows = JAC_T3R;
-constexpr int k3dTileRows = k3dWarps * k3dRows;   // 48
-constexpr int k3dPlaneElems = k3dTileRows * 64;   // doubles per ring stage
-constexpr int k3dFStages = 4;        // f planes resident (levels 1 and 2 read planes p-1 and p-3)
-// u planes resident: p-1 and p are read, the others are in flight.  With f the shared memory
-// is split between the two rings.
-__host__ __device__ constexpr int k3d_stages(bool has_f) { return has_f ? 4 : 5; }
-__host__ __device__ constexpr size_t k3d_smem_bytes(bool has_f) {
-    return (size_t)((k3d_stages(has_f) + (has_f ? k3dFStages : 0)) * k3dPlaneElems + 3 * k3dWarps * 2 * 64) *
-           sizeof(double);
-}
-
-struct Row2 { double v[2]; };
-__device__ __forceinline__ Row2 fill_row2(double c) { Row2 r; r.v[0] = r.v[1] = c; return r; }
-__device__ __forceinline__ Row2 lds_row2(const double* p) {
-    const double2 a = *reinterpret_cast<const double2*>(p);
-    Row2 r; r.v[0] = a.x; r.v[1] = a.y; return r;
-}
-
-struct Plane6 { Row2 row[k3dRows]; };
-
-struct T3Ctx {
-    const double* ub;        // u + lane column base
-    const double* fb;
-    double* ob;
-    long long row_off[k3dRows];   // element offset of each of the warp's rows (valid rows only)
-    long long bsz;           // elements between blocks adjacent in z
-    double* ring;            // shared: [stage][tile row][64]
-    double* fring;           // shared: [stage][tile row][64], right-hand side
-    double* exch;            // shared: [slot][warp][first/last][64]
-    int nz, p0, in_end, Z0, Z1;
-    int warp, lane;
-    unsigned row_out_lo, row_out_hi;   // bit r: the warp's row r lies below / above the domain
-    bool nb_lo_out_lo, nb_lo_out_hi, nb_hi_out_lo, nb_hi_out_hi;  // same for the rows just outside the warp
-    unsigned row_store;      // bit r: row r is an output row of the tile and inside the domain
-    double cx, c_my, c_py, c_mz, c_pz;
-    bool xout, store_lane;
-};
-
-// plane cursor: element offset of global plane gz, block-aware
-struct PlaneCursor {
-    long long off;
-    int k;
-    __device__ __forceinline__ void init(int gz, const JacGeom& g, long long bsz) {
-        if (gz < 0) { k = gz; off = (long long)gz * g.PXY; }
-        else {
-            const int bzi = gz / g.bz;
-            k = gz - bzi * g.bz;
-            off = bzi * bsz + (long long)k * g.PXY;
-        }
-    }
-    __device__ __forceinline__ void advance(const JacGeom& g, long long bsz) {
-        ++k;
-        off += g.PXY;
-        if (k == g.bz) { k = 0; off += bsz - (long long)g.bz * g.PXY; }
-    }
-};
-
-// start the copies of u plane p (and, with f, of f plane p - 1) into their ring stages; one group
-template <bool HAS_F>
-__device__ __forceinline__ void t3_issue_plane(const T3Ctx& c, int p, const PlaneCursor& cur, const PlaneCursor& fcur) {
-    constexpr int NST = k3d_stages(HAS_F);
-    const unsigned rows_out = c.row_out_lo | c.row_out_hi;
-    if (p >= 0 && p < c.nz && p < c.in_end && !c.xout) {
-        double* st = c.ring + ((p - c.p0) % NST) * k3dPlaneElems + (c.warp * k3dRows) * 64 + 2 * c.lane;
-#pragma unroll
-        for (int r = 0; r < k3dRows; ++r)
-            if (!((rows_out >> r) & 1u)) cp_async16(st + r * 64, c.ub + cur.off + c.row_off[r]);
-    }
-    if (HAS_F) {
-        const int q = p - 1;
-        if (q >= 0 && q < c.nz && q < c.in_end && !c.xout) {
-            double* st = c.fring + ((q - c.p0 + 2 * k3dFStages) % k3dFStages) * k3dPlaneElems +
-                         (c.warp * k3dRows) * 64 + 2 * c.lane;
-#pragma unroll
-            for (int r = 0; r < k3dRows; ++r)
-                if (!((rows_out >> r) & 1u)) cp_async16(st + r * 64, c.fb + fcur.off + c.row_off[r]);
-        }
-    }
-    cp_async_commit();
-}
-
-// Dirichlet value of a point that lies outside the domain (plane, then row, then column decide)
-template <bool EDGE>
-__device__ __forceinline__ bool t3_outside(const T3Ctx& c, int plane, bool row_lo, bool row_hi, double* val) {
-    if (!EDGE) return false;
-    if (plane < 0) { *val = c.c_mz; return true; }
-    if (plane >= c.nz) { *val = c.c_pz; return true; }
-    if (row_lo) { *val = c.c_my; return true; }
-    if (row_hi) { *val = c.c_py; return true; }
-    if (c.xout) { *val = c.cx; return true; }
-    return false;
-}
-
-// one level: plane `q` of the level from the window (D, M, U) of the level below
-// RES: rows whose bit is set in res_rows also add the squared residual of M (s - 6 M) to acc
-template <bool HAS_F, bool EDGE, bool RES>
-__device__ __forceinline__ void t3_level(const T3Ctx& c, const Plane6& D, const Plane6& M, const Plane6& U,
-                                         const Row2& below, const Row2& above, int q,
-                                         const double* fplane /* ring stage of f plane q, this warp's rows */,
-                                         Plane6& out, unsigned res_rows, double& acc)
-{
-    const double c6 = 1.0 / 6.0;
-#pragma unroll
-    for (int r = 0; r < k3dRows; ++r) {
-        const Row2& S = (r == 0) ? below : M.row[r - 1];
-        const Row2& N = (r == k3dRows - 1) ? above : M.row[r + 1];
-        const double w = __shfl_up_sync(0xffffffffu, M.row[r].v[1], 1);
-        const double e = __shfl_down_sync(0xffffffffu, M.row[r].v[0], 1);
-        const bool rlo = (c.row_out_lo >> r) & 1u, rhi = (c.row_out_hi >> r) & 1u;
-        double cval = 0.0;
-        const bool outside = t3_outside<EDGE>(c, q, rlo, rhi, &cval);
-        Row2 ff = fill_row2(0.0);
-        if (HAS_F && !outside) ff = lds_row2(fplane + r * 64);   // this lane copied it itself
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-            const double W = (i == 0) ? w : M.row[r].v[0];
-            const double E = (i == 1) ? e : M.row[r].v[1];
-            double s = add_rn(add_rn(W, E), add_rn(S.v[i], N.v[i]));
-            s = add_rn(s, add_rn(D.row[r].v[i], U.row[r].v[i]));
-            if (HAS_F) s = add_rn(s, ff.v[i]);
-            out.row[r].v[i] = mul_rn(s, c6);
-            if (RES && ((res_rows >> r) & 1u)) {
-                const double rr = sub_rn(s, mul_rn(6.0, M.row[r].v[i]));
-                acc = add_rn(acc, mul_rn(rr, rr));
-            }
-        }
-        if (EDGE && outside) out.row[r] = fill_row2(cval);
-    }
-}
-
-template <int T, bool HAS_F, bool RES, int PH, bool EDGE>
-__device__ __forceinline__ void t3_step(Plane6 (&L0)[3], Plane6 (&L1)[3], const T3Ctx& c, const JacGeom& g,
-                                        int p, PlaneCursor& load_cur, PlaneCursor& fload_cur,
-                                        PlaneCursor& l1_cur, PlaneCursor& l2_cur, double& acc)
-{
-    constexpr int NST = k3d_stages(HAS_F);
-    constexpr int LEAD = NST - 2;          // u planes issued ahead of the one being consumed
-    const double* fmine = HAS_F ? c.fring + (c.warp * k3dRows) * 64 + 2 * c.lane : nullptr;
-    const int wlo = c.warp > 0 ? c.warp - 1 : 0;
-    const int whi = c.warp + 1 < k3dWarps ? c.warp + 1 : c.warp;
-
-    // ---- top level first: it only needs planes finished in earlier steps
-    if (T == 2) {
-        const int q = p - 3;
-        const double* ex = c.exch + slot3(PH, -2) * (k3dWarps * 2 * 64) + 2 * c.lane;
-        Row2 below = lds_row2(ex + (wlo * 2 + 1) * 64);   // last row of the warp below
-        Row2 above = lds_row2(ex + (whi * 2 + 0) * 64);   // first row of the warp above
-        Plane6 o;
-        const bool live = c.store_lane && q >= c.Z0 && q < c.Z1;   // the points this lane stores
-        t3_level<HAS_F, EDGE, RES>(c, L1[slot3(PH, -4)], L1[slot3(PH, -3)], L1[slot3(PH, -2)], below, above, q,
-                                   HAS_F ? fmine + ((q - c.p0 + 2 * k3dFStages) % k3dFStages) * k3dPlaneElems : nullptr,
-                                   o, live ? c.row_store : 0u, acc);
-        if (live) {
-#pragma unroll
-            for (int r = 0; r < k3dRows; ++r)
-                if ((c.row_store >> r) & 1u)
-                    *reinterpret_cast<double2*>(c.ob + l2_cur.off + c.row_off[r]) = make_double2(o.row[r].v[0], o.row[r].v[1]);
-        }
-        l2_cur.advance(g, c.bsz);
-    }
-
-    // ---- input plane p: wait for this warp's rows, take them into registers
-    cp_async_wait<LEAD - 1>();
-    {
-        const double* st = c.ring + ((p - c.p0) % NST) * k3dPlaneElems + (c.warp * k3dRows) * 64 + 2 * c.lane;
-#pragma unroll
-        for (int r = 0; r < k3dRows; ++r) {
-            double cval = 0.0;
-            if (t3_outside<EDGE>(c, p, (c.row_out_lo >> r) & 1u, (c.row_out_hi >> r) & 1u, &cval))
-                L0[PH].row[r] = fill_row2(cval);
-            else
-                L0[PH].row[r] = lds_row2(st + r * 64);
-        }
-    }
-    // the stage of u plane p - 2 is no longer read by anyone (barrier of the previous step), and this
-    // thread has just read its part of f plane p - 3: refill both
-    t3_issue_plane<HAS_F>(c, p + LEAD, load_cur, fload_cur);
-    load_cur.advance(g, c.bsz);
-    if (HAS_F) fload_cur.advance(g, c.bsz);
-
-    // ---- level 1: plane p - 1 from level-0 planes p-2, p-1, p
-    {
-        const int q = p - 1;
-        const double* st = c.ring + ((q - c.p0 + NST) % NST) * k3dPlaneElems + 2 * c.lane;
-        const double* f1 = HAS_F ? fmine + ((q - c.p0 + 2 * k3dFStages) % k3dFStages) * k3dPlaneElems : nullptr;
-        Row2 below, above;
-        double cval = 0.0;
-        if (t3_outside<EDGE>(c, q, c.nb_lo_out_lo, c.nb_lo_out_hi, &cval)) below = fill_row2(cval);
-        else below = lds_row2(st + max(c.warp * k3dRows - 1, 0) * 64);
-        if (t3_outside<EDGE>(c, q, c.nb_hi_out_lo, c.nb_hi_out_hi, &cval)) above = fill_row2(cval);
-        else above = lds_row2(st + min(c.warp * k3dRows + k3dRows, k3dTileRows - 1) * 64);
-        if (T == 1) {
-            Plane6 o;
-            const bool live = c.store_lane && q >= c.Z0 && q < c.Z1;
-            t3_level<HAS_F, EDGE, RES>(c, L0[slot3(PH, -2)], L0[slot3(PH, -1)], L0[PH], below, above, q, f1, o,
-                                       live ? c.row_store : 0u, acc);
-            if (live) {
-#pragma unroll
-                for (int r = 0; r < k3dRows; ++r)
-                    if ((c.row_store >> r) & 1u)
-                        *reinterpret_cast<double2*>(c.ob + l1_cur.off + c.row_off[r]) = make_double2(o.row[r].v[0], o.row[r].v[1]);
-            }
-        } else {
-            Plane6& o = L1[slot3(PH, -1)];
-            t3_level<HAS_F, EDGE, false>(c, L0[slot3(PH, -2)], L0[slot3(PH, -1)], L0[PH], below, above, q, f1, o,
-                                         0u, acc);
-            double* ex = c.exch + PH * (k3dWarps * 2 * 64) + (c.warp * 2) * 64 + 2 * c.lane;
-            *reinterpret_cast<double2*>(ex) = make_double2(o.row[0].v[0], o.row[0].v[1]);
-            *reinterpret_cast<double2*>(ex + 64) = make_double2(o.row[k3dRows - 1].v[0], o.row[k3dRows - 1].v[1]);
-        }
-        l1_cur.advance(g, c.bsz);
-    }
-    __syncthreads();
-}
-
-// RES as for the 2D kernel: partials[CTA * 8 + warp] gets the warp's sum of squared residuals of
-// the state before the last sweep of the launch.
-template <int T, bool HAS_F, bool RES>
-__global__ void __launch_bounds__(k3dWarps * 32, k3dWarps <= 4 ? 2 : 1)
-temporal3d_kernel(const double* __restrict__ u, double* __restrict__ un, const double* __restrict__ f,
-                  double* __restrict__ partials, const JacGeom g, const int tiles_x, const int tiles_y,
-                  const int tiles_z, const int zchunk)
-{
-    extern __shared__ __align__(16) double t3_smem[];
-    T3Ctx c;
-    constexpr int NST = k3d_stages(HAS_F);
-    c.ring = t3_smem;
-    c.fring = t3_smem + NST * k3dPlaneElems;
-    c.exch = c.fring + (HAS_F ? k3dFStages : 0) * k3dPlaneElems;
-    c.lane = threadIdx.x & 31;
-    c.warp = threadIdx.x >> 5;
-    const long long tix = blockIdx.x;
-    const int sx = (int)(tix % tiles_x);
-    const int sy = (int)((tix / tiles_x) % tiles_y);
-    const int sz = (int)(tix / ((long long)tiles_x * tiles_y));
-
-    const long long X0 = (long long)sx * 60 - 2;
-    const long long gx = X0 + 2 * c.lane;
-    c.xout = gx < 0 || gx >= g.nx;
-    c.cx = gx < 0 ? g.bval[0] : g.bval[1];
-    c.c_my = g.bval[2]; c.c_py = g.bval[3]; c.c_mz = g.bval[4]; c.c_pz = g.bval[5];
-    c.store_lane = c.lane >= 1 && c.lane <= 30 && !c.xout;
-    const long long col = c.xout ? g.origin : column_base(g, gx);
-    c.ub = u + col;
-    c.fb = HAS_F ? f + col : nullptr;
-    c.ob = un + col;
-
-    const int out_rows = k3dTileRows - 2 * T;
-    const int Yt0 = sy * out_rows - T;                       // global row of tile row 0
-    const long long bsy = g.block_stride * g.gx;
-    c.bsz = bsy * g.gy;
-    c.row_out_lo = c.row_out_hi = c.row_store = 0u;
-#pragma unroll
-    for (int r = 0; r < k3dRows; ++r) {
-        const int trow = c.warp * k3dRows + r;
-        const long long gy = (long long)Yt0 + trow;
-        c.row_off[r] = 0;
-        if (gy < 0) c.row_out_lo |= 1u << r;
-        else if (gy >= g.ny) c.row_out_hi |= 1u << r;
-        else {
-            const long long byi = gy / g.by;
-            c.row_off[r] = byi * bsy + (gy - byi * g.by) * g.PX;
-            if (trow >= T && trow < k3dTileRows - T) c.row_store |= 1u << r;
-        }
-    }
-    {
-        const long long glo = (long long)Yt0 + c.warp * k3dRows - 1, ghi = (long long)Yt0 + c.warp * k3dRows + k3dRows;
-        c.nb_lo_out_lo = glo < 0; c.nb_lo_out_hi = glo >= g.ny;
-        c.nb_hi_out_lo = ghi < 0; c.nb_hi_out_hi = ghi >= g.ny;
-    }
-    c.nz = (int)g.nz;
-    c.Z0 = sz * zchunk;
-    c.Z1 = min(c.nz, c.Z0 + zchunk);
-    c.p0 = c.Z0 - T;
-    c.in_end = c.Z1 + T;
-    const int p_end = c.Z1 + 2 * T - 1;
-
-    // does this tile ever see a point outside the domain in x or y?  (z is checked per step)
-    const bool edge_xy = (sx == 0) || (X0 + 64 > g.nx) || (Yt0 < 0) || ((long long)Yt0 + k3dTileRows > g.ny);
-
-    Plane6 L0[3], L1[3];
-#pragma unroll
-    for (int k = 0; k < 3; ++k)
-#pragma unroll
-        for (int r = 0; r < k3dRows; ++r) { L0[k].row[r] = fill_row2(0.0); L1[k].row[r] = fill_row2(0.0); }
-    // the exchange buffer is read before it is first written: give it defined contents
-    for (int i = threadIdx.x; i < 3 * k3dWarps * 2 * 64; i += blockDim.x) c.exch[i] = 0.0;
-
-    PlaneCursor load_cur, fload_cur, l1_cur, l2_cur;
-    load_cur.init(c.p0, g, c.bsz);
-    fload_cur.init(c.p0 - 1, g, c.bsz);    // the f plane that travels with u plane p is p - 1
-    l1_cur.init(c.p0 - 1, g, c.bsz);       // output plane of level 1 (stores when T == 1)
-    l2_cur.init(c.p0 - 3, g, c.bsz);       // output plane of level 2
-#pragma unroll 1
-    for (int k = 0; k < NST - 2; ++k) {
-        t3_issue_plane<HAS_F>(c, c.p0 + k, load_cur, fload_cur);
-        load_cur.advance(g, c.bsz);
-        if (HAS_F) fload_cur.advance(g, c.bsz);
-    }
-    __syncthreads();
-
-#define JAC_T3_STEP(PHASE, PL)                                                                   \
-    do {                                                                                         \
-        const bool edge = edge_xy || ((PL) - 2 * T - 1 < 0) || ((PL) >= c.nz);                   \
-        if (edge) t3_step<T, HAS_F, RES, PHASE, true>(L0, L1, c, g, (PL), load_cur, fload_cur, l1_cur, l2_cur, acc);  \
-        else t3_step<T, HAS_F, RES, PHASE, false>(L0, L1, c, g, (PL), load_cur, fload_cur, l1_cur, l2_cur, acc);      \
-    } while (0)
-
-    double acc = 0.0;
-    for (int p = c.p0; p < p_end; p += 3) {
-        JAC_T3_STEP(0, p);
-        if (p + 1 < p_end) JAC_T3_STEP(1, p + 1);
-        if (p + 2 < p_end) JAC_T3_STEP(2, p + 2);
-    }
-#undef JAC_T3_STEP
-    cp_async_wait<0>();
-    if (RES) {
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) acc = add_rn(acc, __shfl_down_sync(0xffffffffu, acc, off));
-        if (c.lane == 0) partials[(long long)blockIdx.x * k3dWarps + c.warp] = acc;
     }
 }
 

@@ -37,7 +37,7 @@ EXPORTS = [
     "jac_sweep_residual", "jac_solve", "jac_exchange_wide", "jac_get_wide_buffer",
     "jac_set_u_async", "jac_get_u_async", "jac_residual_async", "jac_exchange_halos",
     "jac_pack_cut", "jac_unpack_cut", "jac_sweep_begin", "jac_sweep_end", "jac_cut_info",
-    "jac_residual_sumsq_async",
+    "jac_residual_sumsq_async", "jac_residual_sweep_async",
 ]
 
 
@@ -101,6 +101,7 @@ def lib() -> C.CDLL:
         L.jac_sweep.argtypes = [vp, C.c_int]
         L.jac_residual.argtypes = [vp, dp]
         L.jac_sweep_residual.argtypes = [vp, C.c_int, dp]
+        L.jac_residual_sweep_async.argtypes = [vp, C.c_int, vp]
         L.jac_solve.argtypes = [vp, C.c_int, C.c_int, C.c_double, C.POINTER(C.c_int), dp]
         L.jac_launch_count.argtypes = [vp, C.POINTER(C.c_int64)]
         L.jac_sweeps_per_launch.argtypes = [vp, C.POINTER(C.c_int)]
@@ -414,6 +415,14 @@ class Jacobi:
         out = C.c_double(0.0)
         self._call("jac_sweep_residual", lib().jac_sweep_residual(self._ctx, int(nsweeps), C.byref(out)))
         return out.value
+
+    def residual_sweep_async(self, nsweeps: int, out):
+        """The residual norm of the current state (into the pinned 1-element tensor ``out`` when the
+        stream gets there), then nsweeps sweeps; the norm comes out of the first sweep's pass."""
+        assert out.numel() == 1
+        self._call("jac_residual_sweep_async",
+                   lib().jac_residual_sweep_async(self._ctx, int(nsweeps), self._pinned_ptr(out)))
+        return out
 
     def solve(self, max_sweeps: int, check_every: int, tol: float):
         """Sweeps until the lagged residual norm is <= tol; returns (sweeps done, last norm)."""

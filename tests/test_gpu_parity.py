@@ -216,15 +216,16 @@ def test_temporal_blocking_matches_oracle(jac, orc, n, b, tsteps, has_f):
     B.close()
 
 
-# 3D: tiles are 60 x (48 - 2T) outputs wide and stream z in chunks: shapes with ragged tiles in
-# x and y, several z chunks, blocks smaller and larger than a tile
+# 3D: tiles are 60 (T = 3: 56) x (32 - 2T) outputs wide and stream z in chunks: shapes with ragged
+# tiles in x and y, several z chunks, blocks smaller and larger than a tile, nonzero Dirichlet values
 TEMPORAL_SHAPES_3D = [((8, 8, 8), (4, 4, 4)), ((24, 18, 12), (8, 6, 4)), ((64, 48, 40), (32, 24, 20)),
                       ((130, 100, 36), (130, 50, 18)), ((132, 20, 70), (66, 10, 35)),
-                      ((256, 128, 24), (128, 128, 8)), ((62, 46, 20), (2, 2, 2))]
+                      ((256, 128, 24), (128, 128, 8)), ((62, 46, 20), (2, 2, 2)), ((120, 56, 300), (60, 28, 100)),
+                      ((58, 27, 9), (58, 27, 9))]
 
 
 @pytest.mark.parametrize("n,b", TEMPORAL_SHAPES_3D)
-@pytest.mark.parametrize("tsteps", [1, 2])
+@pytest.mark.parametrize("tsteps", [1, 2, 3])
 @pytest.mark.parametrize("has_f", [False, True])
 def test_temporal_blocking_3d_matches_oracle(jac, orc, n, b, tsteps, has_f):
     J, B = _setup_pair(jac, orc, n, b, 1, has_f, "temporal", seed=4, tsteps=tsteps)
@@ -247,7 +248,7 @@ def test_temporal_mode_rejects_unsupported_shapes(jac):
     with pytest.raises(jac.JacError):
         jac.Jacobi((9, 8, 8), (3, 4, 4), mode="temporal")     # 3D: bx % 2 != 0
     with pytest.raises(jac.JacError):
-        jac.Jacobi((8, 8, 8), (4, 4, 4), mode="temporal", tsteps=3)   # 3D: at most 2 sweeps per launch
+        jac.Jacobi((8, 8, 8), (4, 4, 4), mode="temporal", tsteps=4)   # 3D: at most 3 sweeps per launch
 
 
 def test_partial_exchange_by_face_mask(jac, orc):
@@ -286,7 +287,7 @@ def test_sweeps_per_launch_query(jac):
              (dict(n=(64, 64), b=(32, 32), mode="temporal", tsteps=3), 3),
              (dict(n=(64, 64), b=(32, 32), mode="temporal"), 4),            # small grid: 4
              (dict(n=(64, 64), b=(32, 32), mode="temporal", has_f=True), 4),
-             (dict(n=(16, 16, 16), b=(8, 8, 8), mode="temporal"), 2)]
+             (dict(n=(16, 16, 16), b=(8, 8, 8), mode="temporal"), 3)]
     for kw, want in cases:
         with jac.Jacobi(**kw) as J:
             assert J.sweeps_per_launch() == want, kw
@@ -311,6 +312,30 @@ def test_sweep_with_fused_residual(jac, orc, n, b, h, mode, has_f):
         assert abs(got_r - want_r) <= RESID_TOL * want_r, (k, got_r, want_r)
         _assert_sweep_close(J.get_u(), B.get_u())
     # an ordinary residual afterwards still works and agrees
+    assert abs(J.residual() - B.residual()) <= RESID_TOL * B.residual()
+    J.close()
+    B.close()
+
+
+@pytest.mark.parametrize("n,b,h", FUSED_RESIDUAL_CASES + [((480, 96), (4, 1), 1), ((120, 56, 70), (60, 28, 35), 1)])
+@pytest.mark.parametrize("mode,tsteps", [("fused", 0), ("exchange", 0), ("pertask", 0), ("temporal", 0), ("temporal", 2),
+                                         ("temporal", 1), ("wide", 0)])
+@pytest.mark.parametrize("has_f", [False, True])
+def test_residual_from_the_first_sweep_s_pass(jac, orc, n, b, h, mode, tsteps, has_f):
+    """jac_residual_sweep_async(k): the norm of the residual of the state BEFORE the k sweeps, then the
+    state after them."""
+    import torch
+    J, B = _setup_pair(jac, orc, n, b, h, has_f, mode, seed=8, tsteps=tsteps)
+    norms = torch.zeros(3, dtype=torch.float64).pin_memory()
+    want = []
+    for i, k in enumerate((1, 4, 10)):
+        want.append(B.residual())
+        B.sweep(k)
+        J.residual_sweep_async(k, norms[i:i + 1])
+    got_u = J.get_u()              # waits for the stream
+    _assert_sweep_close(got_u, B.get_u())
+    for got_r, want_r in zip(norms.tolist(), want):
+        assert abs(got_r - want_r) <= RESID_TOL * want_r, (got_r, want_r)
     assert abs(J.residual() - B.residual()) <= RESID_TOL * B.residual()
     J.close()
     B.close()
