@@ -551,13 +551,63 @@ def run_ours(args, w: inputs.Workload):
         dist.destroy_process_group()
 
 
+# ----------------------------------------------------------------------------- config 4
+def run_halo_microbenchmark(args):
+    """Config 4 (halo pack/unpack microbenchmark): the library's timings per block size and halo
+    width with their roofline fractions, and beside each the CPU oracle's pack and unpack loops of the
+    same decomposition timed on the host cores.  One JSON line."""
+    import torch
+    from paper_2210_01238_b200 import halo_bench
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    peak, peak_kind = measured_peak_gbs()
+    total_gib = args.halo_gib
+    rows = halo_bench.run(sorted(inputs.HALO_BENCH_SHAPES), list(inputs.HALO_BENCH_WIDTHS), total_gib, peak,
+                          with_3d=not args.no_others)
+    torch.cuda.empty_cache()
+    if not args.no_cpu_baseline:
+        from oracle import orc
+        threads = orc.max_threads()
+        for r in rows:
+            n, b, h = r["grid"], r["block"], r["halo"]
+            if len(n) == 3:
+                continue            # 26 GB of oracle state for one number: the 2D cases carry the comparison
+            O = orc.Blocked(n, b, h)
+            O.set_u(inputs.uniform_field(n, inputs.HALO_BENCH_SEED))
+            O.pack(); O.unpack()
+            reps = max(3, min(200, int(2e8 / max(1, r["payload_bytes_per_call"]))))
+            t0 = time.perf_counter()
+            for _ in range(reps):
+                O.pack()
+            t_pack = (time.perf_counter() - t0) / reps
+            t0 = time.perf_counter()
+            for _ in range(reps):
+                O.unpack()
+            t_unpack = (time.perf_counter() - t0) / reps
+            O.close()
+            counted = 2 * r["payload_bytes_per_call"]
+            r["cpu_baseline"] = {"kind": "oracle", "cores": threads, "unit": "GB/s",
+                                 "pack_gbs": counted / t_pack / 1e9, "unpack_gbs": counted / t_unpack / 1e9,
+                                 "pack_us": t_pack * 1e6, "unpack_us": t_unpack * 1e6,
+                                 "sample": f"{reps} repetitions of pack and of unpack of all faces"}
+    big = rows[-1]["all:exchange"]
+    line = {"metric": "halo_exchange_gbs", "unit": "GB/s", "value": big["cold_gbs"], "n_gpus": 1, "higher_is_better": True,
+            "dtype": "f64", "data": "synthetic", "vs_baseline": None,
+            "config": {"workload": "c4_halo_microbenchmark", "value_is": "one-launch exchange of all faces, L2 evicted "
+                       "between repetitions, of the last row", "gib_per_operation": total_gib},
+            "roofline": dict(big["roofline"], peak_kind=f"of {peak_kind}"), "rows": rows}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c3_eigenmode_16384", choices=sorted(inputs.CONFIGS))
+    ap.add_argument("--workload", default="c3_eigenmode_16384", choices=sorted(inputs.CONFIGS) + ["c4_halo"])
+    ap.add_argument("--halo-gib", type=float, default=1.0, help="c4_halo: GiB of face payload per operation")
     ap.add_argument("--mode", default="auto", choices=["auto", "fused", "exchange", "pertask", "temporal", "wide", "resident"],
                     help="schedule of jac_sweep; auto = the fastest one the library has for the workload")
     ap.add_argument("--tsteps", type=int, default=0)
@@ -570,6 +620,10 @@ def main():
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         log("warning: fewer than 3 warm-up steps")
+    if args.workload == "c4_halo":
+        if args.impl == "ours" and int(os.environ.get("RANK", "0")) == 0:
+            run_halo_microbenchmark(args)
+        return
     w = inputs.CONFIGS[args.workload]
     if args.n:
         w = inputs.scaled(w, (args.n,) * w.ndim, name=f"{w.name}_at_{args.n}")

@@ -67,7 +67,10 @@ extern "C" {
                                2D: b[0] % 4 == 0 and n[0] % 4 == 0, tsteps <= 8;
                                3D: b[0] % 2 == 0 and n[0] % 2 == 0, tsteps <= 3;
                                jac_create returns JAC_EINVAL otherwise                           */
-#define JAC_MODE_EXCHANGE 3 /* per sweep three launches over all blocks: pack, unpack, update    */
+#define JAC_MODE_EXCHANGE 3 /* the paper's order made explicit: per sweep every face is packed into
+                               its send buffer and unpacked into the neighbour's ghost cells (both
+                               by one launch over all blocks, as jac_exchange_halos), then one
+                               update launch over all blocks reads the ghosts                    */
 #define JAC_MODE_WIDE     4 /* one wide exchange (jac_exchange_wide: all h ghost layers, edges and
                                corners included) per group of `tsteps` <= h sweeps (0 = h); the
                                group's sweeps update boxes shrinking from the interior grown by
@@ -282,11 +285,15 @@ int jac_sweep_residual(jac_ctx *ctx, int nsweeps, double *host_out_l2);
  * fixed iteration count.) */
 int jac_residual_sweep_async(jac_ctx *ctx, int nsweeps, double *host_out_l2);
 
-/* Iterate until converged: runs sweeps in groups of check_every (each group through
- * jac_sweep_residual) until the lagged residual norm is <= tol or max_sweeps sweeps have run.
- * HOST outputs: the sweeps actually done and the last norm measured (the residual of the state one
- * sweep before the final one).  Errors: JAC_EINVAL for max_sweeps < 1, check_every < 1, tol < 0 or
- * NaN, null outputs. */
+/* Iterate until converged: runs sweeps in groups of check_every (each group as
+ * jac_sweep_residual does) until the lagged residual norm is <= tol or max_sweeps sweeps have run.
+ * The comparison with tol is made on the device: several groups are queued at a time without
+ * waiting, a group whose norm meets tol raises a flag in the workspace, the launches queued behind
+ * it see the flag and return at once, and the host looks at the flag only between batches of
+ * groups (JAC_MODE_WIDE: after every group).  The result is that of stopping exactly after the
+ * group that met tol.  HOST outputs: the sweeps actually done and the last norm measured (the
+ * residual of the state one sweep before the final one).  Errors: JAC_EINVAL for max_sweeps < 1,
+ * check_every < 1, tol < 0 or NaN, null outputs. */
 int jac_solve(jac_ctx *ctx, int max_sweeps, int check_every, double tol, int *host_sweeps_done,
               double *host_residual);
 

@@ -8,6 +8,7 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "jac.h"
 #include "jac_geom.h"
@@ -17,7 +18,11 @@
 
 namespace {
 
-constexpr int kNumSMs = 148;  // B200
+// SMs the launch planners assume when no device has been asked yet (the pure host queries: the
+// workspace layout must not depend on the machine it is computed on).  A context asks its device
+// once, at creation, and plans its launches with that count wherever the scratch sized for the
+// nominal count allows it.
+constexpr int kNominalSMs = 148;  // B200
 constexpr long long kMaxGrid = 2147483647LL;
 
 long long round_up(long long v, long long m) { return (v + m - 1) / m * m; }
@@ -35,12 +40,12 @@ struct Tiling {
 
 // force_nv = 1: one point per thread although the width is even (rows that do not start on a
 // 16-byte boundary)
-Tiling make_tiling(const JacGeom& g, int force_nv = 0)
+Tiling make_tiling(const JacGeom& g, int sms, int force_nv = 0)
 {
     Tiling t{};
     t.nv = force_nv ? force_nv : ((g.bx % 2 == 0 && g.rx % 2 == 0) ? 2 : 1);
     const long long need = ceil_div(g.bx, t.nv);
-    const long long want_ctas = (long long)kNumSMs * 16;
+    const long long want_ctas = (long long)sms * 16;
     if (g.ndim == 2) {
         const int tpb = (int)std::min<long long>(256, round_up(need, 32));
         t.block = dim3(tpb, 1, 1);
@@ -88,14 +93,14 @@ struct TemporalGrid {
 // T = 8).  Measured against the earlier fixed rule (32 rows below 7104 strips): 4096^2 with f,
 // T = 4: 0.107 ms per launch instead of 0.113; 8192^2, T = 4: 0.211 instead of 0.226; 2048^2,
 // T = 8: 0.049 instead of 0.064; 16384^2 unchanged.
-int temporal_rows_2d(const JacGeom& g, int T, bool has_f)
+int temporal_rows_2d(const JacGeom& g, int T, bool has_f, int sms)
 {
 #ifdef JAC_FORCE_ROWS
     return JAC_FORCE_ROWS;
 #endif
     const long long strips_x = ceil_div(g.nx, jac::temporal_strip_cols(T));
     const int ctas_per_sm = ((T > 4 && jac::temporal_points(T) == 4) || jac::temporal_f_ring(T, has_f)) ? 2 : JAC_TOCC;
-    const double capacity = (double)kNumSMs * ctas_per_sm * jac::kTemporalWarps;
+    const double capacity = (double)sms * ctas_per_sm * jac::kTemporalWarps;
     const double alpha = T > 4 ? 0.45 : 0.7;
     int best = 8;
     double best_cost = 1e300;
@@ -112,11 +117,11 @@ int temporal_rows_2d(const JacGeom& g, int T, bool has_f)
     return best;
 }
 
-TemporalGrid temporal_grid_2d(const JacGeom& g, int T, bool has_f)
+TemporalGrid temporal_grid_2d(const JacGeom& g, int T, bool has_f, int sms)
 {
     TemporalGrid t{};
     t.a = (int)ceil_div(g.nx, jac::temporal_strip_cols(T));
-    const int rows = temporal_rows_2d(g, T, has_f);
+    const int rows = temporal_rows_2d(g, T, has_f, sms);
     t.chunk = rows;
     t.b = (int)ceil_div(g.ny, rows);
     t.c = 1;
@@ -125,7 +130,7 @@ TemporalGrid temporal_grid_2d(const JacGeom& g, int T, bool has_f)
     return t;
 }
 
-TemporalGrid temporal_grid_3d(const JacGeom& g, int T)
+TemporalGrid temporal_grid_3d(const JacGeom& g, int T, int sms)
 {
     TemporalGrid t{};
     t.a = (int)ceil_div(g.nx, jac::t3_out_cols(T));
@@ -133,7 +138,7 @@ TemporalGrid temporal_grid_3d(const JacGeom& g, int T)
     // planes per chunk: a chunk of Z planes costs Z + 2T steps; long chunks waste the least, but the
     // launch should still be several rounds of CTAs (one CTA per SM)
     int zchunk = 256;
-    while (zchunk > 16 && (long long)t.a * t.b * ceil_div(g.nz, zchunk) < (long long)kNumSMs * 6) zchunk /= 2;
+    while (zchunk > 16 && (long long)t.a * t.b * ceil_div(g.nz, zchunk) < (long long)sms * 6) zchunk /= 2;
     t.chunk = zchunk;
     t.c = (int)ceil_div(g.nz, zchunk);
     t.ctas = (long long)t.a * t.b * t.c;
@@ -174,11 +179,11 @@ int plan_resident(const JacGeom& g, bool has_f, int want_cluster, ResidentPlan* 
 }
 
 // largest number of partial sums any launch of this geometry can write
-long long max_partials(const JacGeom& g, long long sweep_ctas, bool has_f)
+long long max_partials(const JacGeom& g, long long sweep_ctas, bool has_f, int sms)
 {
     long long m = sweep_ctas;
-    if (g.ndim == 2) for (int T = 1; T <= 8; ++T) m = std::max(m, temporal_grid_2d(g, T, has_f).warps);
-    else for (int T = 1; T <= jac::kT3MaxT; ++T) m = std::max(m, temporal_grid_3d(g, T).warps);
+    if (g.ndim == 2) for (int T = 1; T <= 8; ++T) m = std::max(m, temporal_grid_2d(g, T, has_f, sms).warps);
+    else for (int T = 1; T <= jac::kT3MaxT; ++T) m = std::max(m, temporal_grid_3d(g, T, sms).warps);
     return m;
 }
 
@@ -255,7 +260,7 @@ int build_geometry(const jac_desc* d, JacGeom* g, jac_layout* L)
         ResidentPlan rp;
         if (plan_resident(*g, d->has_f != 0, d->tsteps, &rp)) return JAC_EINVAL;   // 3D, odd bx, or too large
     }
-    const Tiling t = make_tiling(*g);
+    const Tiling t = make_tiling(*g, kNominalSMs);
     const long long ctas = g->nblocks * t.ctas_per_block;
     if (ctas > kMaxGrid) return JAC_EINVAL;
     long long max_face = 0;
@@ -278,7 +283,7 @@ int build_geometry(const jac_desc* d, JacGeom* g, jac_layout* L)
         }
         L->send_stride = g->send_stride;
         for (int fc = 0; fc < 6; ++fc) L->wide_face_elems[fc] = g->wface_elems[fc];
-        L->partials = round_up(max_partials(*g, ctas, d->has_f != 0), 32);
+        L->partials = round_up(max_partials(*g, ctas, d->has_f != 0, kNominalSMs), 32);
         const long long arr_bytes = round_up(g->nblocks * g->block_stride * 8, 256);
         long long o = 0;
         L->off_u[0] = o; o += arr_bytes;
@@ -323,6 +328,7 @@ struct jac_ctx {
     double* send;
     double* partials;
     double* result;
+    int sms;            // SMs of the device, as the launch planners use it
     int cur;            // which of u[] holds the current state
     bool ghosts_fresh;  // inter-block ghosts of u[cur] equal the neighbours' current faces
     bool packed_current;  // the send buffers hold the faces of the current state
@@ -416,16 +422,26 @@ int launch_sweep(jac_ctx* c, const double* u, double* un, long long blk0, long l
     return check_launch(c);
 }
 
-// threads reserved per (block, face) pair: one per two elements of the largest face, whole warps
+// threads reserved per (block, face) pair, whole warps: a thread takes up to kHaloUnits units (a row
+// of an x face, two cells of a line of a y or z face), and there are at least as many threads as a
+// line has units, so that threads keep their column and walk over lines
 int halo_slots(const jac_ctx* c, unsigned face_mask)
 {
-    long long m = 2;
-    for (int fc = 0; fc < c->g.nfaces; ++fc)
-        if ((face_mask >> fc) & 1u) m = std::max(m, c->g.face_elems[fc]);
-    return (int)round_up(ceil_div(m, 2), 32);
+    const JacGeom& g = c->g;
+    const long long vec_per_line = (g.bx % 2 == 0 && g.PX % 2 == 0) ? g.bx / 2 : g.bx;
+    long long units = 1, line = 1;
+    for (int fc = 0; fc < g.nfaces; ++fc) {
+        if (!((face_mask >> fc) & 1u)) continue;
+        if (fc < 2) units = std::max(units, g.face_elems[fc] / g.h);                 // rows
+        else {
+            units = std::max(units, g.face_elems[fc] / g.bx * vec_per_line);
+            line = vec_per_line;
+        }
+    }
+    return (int)round_up(std::max(ceil_div(units, jac::kHaloUnits), std::min<long long>(line, 1 << 20)), 32);
 }
 
-template <bool UNPACK>
+template <int OP>
 int launch_halo(jac_ctx* c, long long pair0, long long npairs, unsigned face_mask)
 {
     const int slots = halo_slots(c, face_mask);
@@ -433,19 +449,19 @@ int launch_halo(jac_ctx* c, long long pair0, long long npairs, unsigned face_mas
     if (ctas > kMaxGrid) return JAC_EINVAL;
     // 32-bit index arithmetic when thread and pair numbers fit (they do for any grid that fits a GPU)
     if (ctas * 256 < (1LL << 32) && c->g.nblocks * c->g.nfaces < (1LL << 31))
-        jac::halo_kernel<UNPACK, unsigned><<<(unsigned)ctas, 256, 0, c->stream>>>(c->u[c->cur], c->send, c->g, pair0,
-                                                                                npairs, slots, face_mask);
+        jac::halo_kernel<OP, unsigned><<<(unsigned)ctas, 256, 0, c->stream>>>(c->u[c->cur], c->send, c->g, pair0,
+                                                                            npairs, slots, face_mask);
     else
-        jac::halo_kernel<UNPACK, long long><<<(unsigned)ctas, 256, 0, c->stream>>>(c->u[c->cur], c->send, c->g, pair0,
-                                                                                 npairs, slots, face_mask);
+        jac::halo_kernel<OP, long long><<<(unsigned)ctas, 256, 0, c->stream>>>(c->u[c->cur], c->send, c->g, pair0,
+                                                                             npairs, slots, face_mask);
     return check_launch(c);
 }
 
 // pack or unpack the faces in face_mask of all blocks in one launch
-template <bool UNPACK>
+template <int OP>
 int launch_halo_all(jac_ctx* c, unsigned face_mask = 0x3fu)
 {
-    return launch_halo<UNPACK>(c, 0, c->g.nblocks * c->g.nfaces, face_mask);
+    return launch_halo<OP>(c, 0, c->g.nblocks * c->g.nfaces, face_mask);
 }
 
 bool has_neighbour(const JacGeom& g, long long blk, int face)
@@ -457,13 +473,13 @@ bool has_neighbour(const JacGeom& g, long long blk, int face)
 }
 
 // one launch per (block, face) that has a neighbour: the task-per-block schedule
-template <bool UNPACK>
+template <int OP>
 int launch_halo_pertask(jac_ctx* c)
 {
     for (long long blk = 0; blk < c->g.nblocks; ++blk)
         for (int face = 0; face < c->g.nfaces; ++face) {
             if (!has_neighbour(c->g, blk, face)) continue;
-            const int rc = launch_halo<UNPACK>(c, blk * c->g.nfaces + face, 1, 1u << face);
+            const int rc = launch_halo<OP>(c, blk * c->g.nfaces + face, 1, 1u << face);
             if (rc) return rc;
         }
     return JAC_OK;
@@ -471,33 +487,28 @@ int launch_halo_pertask(jac_ctx* c)
 
 int do_pack(jac_ctx* c)
 {
-    return c->desc.mode == JAC_MODE_PERTASK ? launch_halo_pertask<false>(c) : launch_halo_all<false>(c);
+    return c->desc.mode == JAC_MODE_PERTASK ? launch_halo_pertask<jac::HALO_PACK>(c) : launch_halo_all<jac::HALO_PACK>(c);
 }
 int do_unpack(jac_ctx* c)
 {
-    return c->desc.mode == JAC_MODE_PERTASK ? launch_halo_pertask<true>(c) : launch_halo_all<true>(c);
+    return c->desc.mode == JAC_MODE_PERTASK ? launch_halo_pertask<jac::HALO_UNPACK>(c) : launch_halo_all<jac::HALO_UNPACK>(c);
 }
 
 // pack and unpack of all faces in one launch (same buffers and ghosts afterwards)
 int do_exchange_fused(jac_ctx* c)
 {
-    const int slots = halo_slots(c, 0x3fu);
-    const long long npairs = c->g.nblocks * c->g.nfaces;
-    const long long ctas = ceil_div(npairs * slots, 256);
-    if (ctas > kMaxGrid) return JAC_EINVAL;
-    if (ctas * 256 < (1LL << 32) && npairs < (1LL << 31))
-        jac::halo_exchange_kernel<unsigned><<<(unsigned)ctas, 256, 0, c->stream>>>(c->u[c->cur], c->send, c->g, npairs, slots);
-    else
-        jac::halo_exchange_kernel<long long><<<(unsigned)ctas, 256, 0, c->stream>>>(c->u[c->cur], c->send, c->g, npairs, slots);
-    const int rc = check_launch(c);
+    const int rc = launch_halo_all<jac::HALO_EXCHANGE>(c);
     if (rc) return rc;
     c->packed_current = true;
     c->ghosts_fresh = true;
     return JAC_OK;
 }
 
+// the exchange before an update: pack and unpack as one launch (the task-per-block schedule keeps
+// them apart, one launch per block face each)
 int do_exchange(jac_ctx* c)
 {
+    if (c->desc.mode != JAC_MODE_PERTASK) return do_exchange_fused(c);
     int rc = do_pack(c);
     if (rc) return rc;
     c->packed_current = true;
@@ -554,7 +565,7 @@ int launch_ext(jac_ctx* c, int e, const double* u, double* un)
         ge.origin -= (long long)e * ge.PXY;
     }
     // 128-bit accesses need the first column of the grown box on a 16-byte boundary: e even
-    const Tiling t = make_tiling(ge, (e % 2 != 0) ? 1 : 0);
+    const Tiling t = make_tiling(ge, c->sms, (e % 2 != 0) ? 1 : 0);
     if (ge.nblocks * t.ctas_per_block > kMaxGrid) return JAC_EINVAL;
     const bool f = c->desc.has_f != 0;
     if (t.nv == 2) {
@@ -707,7 +718,7 @@ int ensure_dynamic_smem(jac_ctx* c, size_t smem)
 template <int T, bool HAS_F, int RES>
 int launch_temporal3d_t(jac_ctx* c, const double* u, double* un, long long* nparts)
 {
-    const TemporalGrid t = temporal_grid_3d(c->g, T);
+    const TemporalGrid t = temporal_grid_3d(c->g, T, c->sms);
     if (t.ctas > kMaxGrid) return JAC_EINVAL;
     constexpr auto kern = jac::temporal3d_kernel<T, HAS_F, RES>;
     const size_t smem = jac::t3_smem_bytes(T, HAS_F);
@@ -747,7 +758,7 @@ int launch_temporal3d_n(jac_ctx* c, int t, const double* u, double* un, int res,
 template <int T, bool HAS_F, int RES>
 int launch_temporal_t(jac_ctx* c, const double* u, double* un, long long* nparts)
 {
-    const TemporalGrid t = temporal_grid_2d(c->g, T, HAS_F);
+    const TemporalGrid t = temporal_grid_2d(c->g, T, HAS_F, c->sms);
     constexpr auto kern = jac::temporal2d_kernel<T, HAS_F, RES>;
     const size_t smem = jac::temporal_smem_bytes(T, HAS_F);
     if (smem > 48 * 1024) {
@@ -793,9 +804,8 @@ int launch_temporal_n(jac_ctx* c, int t, const double* u, double* un, int res, l
 template <bool HAS_F>
 int launch_resident_t(jac_ctx* c, const ResidentPlan& rp, const double* u, double* un, int nsweeps)
 {
+    // the kernel's attributes (shared memory, cluster size) were set when the context was created
     auto kern = jac::resident2d_kernel<HAS_F>;
-    JAC_CK(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rp.smem));
-    if (rp.cluster > 8) JAC_CK(c, cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3((unsigned)rp.cluster, 1, 1);
@@ -830,8 +840,10 @@ int resident_cluster_schedulable(jac_ctx* c, int cluster, bool* ok)
     if (plan_resident(c->g, c->desc.has_f != 0, cluster, &rp)) return JAC_OK;   // does not fit shared memory
     const void* kern = c->desc.has_f ? (const void*)jac::resident2d_kernel<true>
                                      : (const void*)jac::resident2d_kernel<false>;
-    JAC_CK(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rp.smem));
-    if (rp.cluster > 8) JAC_CK(c, cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+    // once per context, and to the largest size any context may ask for, so that contexts of
+    // different grids do not undo each other's setting
+    JAC_CK(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmemPerCta));
+    JAC_CK(c, cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3((unsigned)rp.cluster, 1, 1);
@@ -999,6 +1011,27 @@ int run_sweeps(jac_ctx* c, int nsweeps, int res, long long* nparts)
 
 // the square root of one device double, in place (correctly rounded, as std::sqrt on the host)
 __global__ void sqrt_in_place_kernel(double* v) { *v = sqrt(*v); }
+
+// End of one group of jac_solve's sweeps, on the device: the group's partial sums are added in the
+// usual fixed order, the norm and the sweeps done so far are recorded, and once the norm has met
+// the tolerance a flag goes up that turns every later launch of the call into a no-op.
+// result: [0] sum of squares, [1] its root; stop, done: the flag and the sweep count.
+__global__ void __launch_bounds__(1024)
+solve_check_kernel(const double* __restrict__ partials, const long long n, const double tol, const int group_sweeps,
+                   double* __restrict__ result, int* __restrict__ stop, int* __restrict__ done)
+{
+    if (*stop != 0) return;
+    double acc = 0.0;
+    for (long long i = threadIdx.x; i < n; i += blockDim.x) acc = jac::add_rn(acc, partials[i]);
+    const double total = jac::block_sum(acc);
+    if (threadIdx.x == 0) {
+        const double norm = sqrt(total);          // correctly rounded, as std::sqrt on the host
+        result[0] = total;
+        result[1] = norm;
+        *done += group_sweeps;
+        if (norm <= tol) *stop = 1;
+    }
+}
 
 // fixed-order sum of the first nparts partial sums -> host, as a norm
 int finish_norm(jac_ctx* c, long long nparts, double* host_out_l2)
@@ -1170,7 +1203,18 @@ int jac_create(const jac_desc* desc, void* dev_workspace, size_t bytes, jac_ctx*
     c->desc = *desc;
     c->g = g;
     c->L = L;
-    c->tile = make_tiling(g);
+    // launch plans for the SM count of this device, if the scratch (sized for the nominal count) holds them
+    c->sms = kNominalSMs;
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) {
+        const Tiling t = make_tiling(g, sms);
+        if (max_partials(g, g.nblocks * t.ctas_per_block, desc->has_f != 0, sms) <= L.partials &&
+            g.nblocks * t.ctas_per_block <= kMaxGrid)
+            c->sms = sms;
+    } else {
+        cudaGetLastError();
+    }
+    c->tile = make_tiling(g, c->sms);
     c->ws = static_cast<char*>(dev_workspace);
     c->u[0] = reinterpret_cast<double*>(c->ws + L.off_u[0]);
     c->u[1] = reinterpret_cast<double*>(c->ws + L.off_u[1]);
@@ -1390,7 +1434,7 @@ int jac_pack_faces(jac_ctx* c, unsigned face_mask)
     if (face_mask & ~all) return JAC_EINVAL;
     if (face_mask == all) return jac_pack_halos(c);
     if (!face_mask) return JAC_OK;
-    return launch_halo_all<false>(c, face_mask);
+    return launch_halo_all<jac::HALO_PACK>(c, face_mask);
 }
 
 int jac_unpack_faces(jac_ctx* c, unsigned face_mask)
@@ -1401,7 +1445,7 @@ int jac_unpack_faces(jac_ctx* c, unsigned face_mask)
     if (face_mask & ~all) return JAC_EINVAL;
     if (face_mask == all) return jac_unpack_halos(c);
     if (!face_mask) return JAC_OK;
-    return launch_halo_all<true>(c, face_mask);
+    return launch_halo_all<jac::HALO_UNPACK>(c, face_mask);
 }
 
 int jac_sweep(jac_ctx* c, int nsweeps)
@@ -1430,18 +1474,70 @@ int jac_solve(jac_ctx* c, int max_sweeps, int check_every, double tol, int* host
     if (rc) return rc;
     if (max_sweeps < 1 || check_every < 1 || !(tol >= 0.0) || !host_sweeps_done || !host_residual)
         return JAC_EINVAL;
-    int done = 0;
-    double res = 0.0;
-    while (done < max_sweeps) {
-        const int n = std::min(check_every, max_sweeps - done);
-        long long nparts = 0;
-        if ((rc = run_sweeps(c, n, jac::kResBeforeLast, &nparts))) return rc;
-        if ((rc = finish_norm(c, nparts, &res))) return rc;
-        done += n;
-        if (res <= tol) break;
+    if (c->desc.mode == JAC_MODE_WIDE) {
+        // the wide exchange and the grown-box updates do not look at the flag: ask after every group
+        int done = 0;
+        double res = 0.0;
+        while (done < max_sweeps) {
+            const int n = std::min(check_every, max_sweeps - done);
+            long long nparts = 0;
+            if ((rc = run_sweeps(c, n, jac::kResBeforeLast, &nparts))) return rc;
+            if ((rc = finish_norm(c, nparts, &res))) return rc;
+            done += n;
+            if (res <= tol) break;
+        }
+        *host_sweeps_done = done;
+        *host_residual = res;
+        return JAC_OK;
     }
+    // The test against the tolerance runs on the device.  Groups are queued several at a time without
+    // waiting; once a group's norm meets the tolerance the launches queued behind it return at once,
+    // and the host only looks at the flag between batches.
+    constexpr int kGroupsPerLook = 8;
+    int* stop = reinterpret_cast<int*>(c->result + 2);
+    int* done_dev = reinterpret_cast<int*>(c->result + 3);
+    JAC_CK(c, cudaMemsetAsync(c->result, 0, 4 * sizeof(double), c->stream));
+    const int cur0 = c->cur;
+    std::vector<signed char> cur_after;      // which array is current after each queued group
+    int queued = 0, done = 0;
+    double norm = 0.0;
+    bool stopped = false;
+    c->g.stop = stop;
+    while (queued < max_sweeps && !stopped && rc == JAC_OK) {
+        for (int k = 0; k < kGroupsPerLook && queued < max_sweeps && rc == JAC_OK; ++k) {
+            const int n = std::min(check_every, max_sweeps - queued);
+            long long nparts = 0;
+            if ((rc = run_sweeps(c, n, jac::kResBeforeLast, &nparts))) break;
+            solve_check_kernel<<<1, 1024, 0, c->stream>>>(c->partials, nparts, tol, n, c->result, stop, done_dev);
+            if ((rc = check_launch(c))) break;
+            queued += n;
+            cur_after.push_back((signed char)c->cur);
+        }
+        if (rc) break;
+        double look[4];
+        cudaError_t e = cudaMemcpyAsync(look, c->result, sizeof(look), cudaMemcpyDeviceToHost, c->stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+        if (e != cudaSuccess) {
+            c->cuda_err = (int)e;
+            rc = JAC_ECUDA;
+            break;
+        }
+        int flag = 0;
+        std::memcpy(&flag, &look[2], sizeof(int));
+        std::memcpy(&done, &look[3], sizeof(int));
+        norm = look[1];
+        stopped = flag != 0;
+    }
+    c->g.stop = nullptr;
+    if (rc) return rc;
+    // the launches queued behind the group that met the tolerance did nothing: the current array is
+    // the one that was current after that group
+    const int groups_done = (done + check_every - 1) / check_every;
+    c->cur = groups_done > 0 ? cur_after[(size_t)groups_done - 1] : cur0;
+    c->ghosts_fresh = false;
+    c->packed_current = false;
     *host_sweeps_done = done;
-    *host_residual = res;
+    *host_residual = norm;
     return JAC_OK;
 }
 

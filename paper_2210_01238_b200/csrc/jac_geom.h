@@ -33,4 +33,7 @@ struct JacGeom {
     // extended update: the kernel is handed a geometry whose block box is the interior grown by
     // `ext` layers on every side (bx, by, bz and origin adjusted; 0 in the context's own geometry)
     int ext;
+    // jac_solve: where a call that has met its tolerance raises a flag; the sweep and halo kernels of
+    // the call's later groups look at it first and return at once (null outside jac_solve)
+    const int* stop;
 };

@@ -29,6 +29,10 @@ __device__ __forceinline__ double add_rn(double a, double b) { return __dadd_rn(
 __device__ __forceinline__ double sub_rn(double a, double b) { return __dsub_rn(a, b); }
 __device__ __forceinline__ double mul_rn(double a, double b) { return __dmul_rn(a, b); }
 
+// has the solve this launch belongs to already met its tolerance?  (uniform over the grid: the flag
+// only changes between launches)
+__device__ __forceinline__ bool solve_stopped(const JacGeom& g) { return g.stop != nullptr && *g.stop != 0; }
+
 // ask for a line to be brought into L2
 __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];\n" ::"l"(p)); }
 
@@ -105,6 +109,7 @@ sweep2d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
                double* __restrict__ partials, const JacGeom g, const long long blk0,
                const int tiles_x, const int tiles_y, const int rows)
 {
+    if (solve_stopped(g)) return;
     const long long t = blockIdx.x;
     const int xt = (int)(t % tiles_x);
     const int yt = (int)((t / tiles_x) % tiles_y);
@@ -201,6 +206,7 @@ sweep3d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
                double* __restrict__ partials, const JacGeom g, const long long blk0,
                const int tiles_x, const int tiles_y, const int tiles_z, const int planes)
 {
+    if (solve_stopped(g)) return;
     const long long t = blockIdx.x;
     const int xt = (int)(t % tiles_x);
     const int yt = (int)((t / tiles_x) % tiles_y);
@@ -381,91 +387,185 @@ __device__ __forceinline__ long long face_elems_of(const JacGeom& g, const Block
     return axis == 0 ? h * ext.y * ext.z : (axis == 1 ? h * ext.x * ext.z : h * ext.x * ext.y);
 }
 
-// A thread moves two consecutive elements of one face; `slots` threads (a multiple of 32, so a
-// warp never straddles faces) are reserved per (block, face) pair, and the grid is packed over
-// threads, not faces: small faces do not leave CTAs mostly idle.  On y and z faces with an even
-// block width the two elements are adjacent in memory on both sides and move as one 128-bit
-// access; on x faces they are two strided cells.
-template <bool UNPACK, typename IT>
+// Halo pack, unpack, or both at once.  `slots` threads (a multiple of 32, so a warp never straddles
+// faces) are reserved per (block, face) pair and the grid is packed over threads, not faces: small
+// faces do not leave CTAs mostly idle.  The work of a face is cut into units, up to four per thread,
+// whose loads are all issued before the first store:
+//   x face   a unit is one row (k, j) of the strip: h cells, strided by the row pitch in the block
+//            and contiguous in the buffer; consecutive threads take consecutive rows, so a warp
+//            touches 32 sectors of the block and 32 h contiguous doubles of the buffer.
+//            Ghost columns are the innermost h cells of a four-cell margin that nothing else
+//            uses; for h <= 2 the unpack writes the whole 32-byte sector (the ghost cells and
+//            zeros beside them): a store of a full sector needs no read of the old one, a store
+//            of 8 of its bytes does.
+//   y, z     a unit is two cells of a line of the strip, contiguous on both sides (one 128-bit
+//            access each when the line starts are 16-byte aligned); a thread keeps its column and
+//            walks over lines, so the only division per unit is the line's split into (y, z).
+// HALO_EXCHANGE does pack and unpack in one pass: the thread that fills ghost cells of (block,
+// face) reads them from the neighbour's interior strip and also leaves them in the neighbour's
+// send slot, so the buffers and the ghosts end up exactly as after pack followed by unpack: one
+// read and two writes per face cell instead of two reads and two writes, and one launch.
+enum : int { HALO_PACK = 0, HALO_UNPACK = 1, HALO_EXCHANGE = 2 };
+constexpr int kHaloUnits = 4;     // units per thread
+
+template <int OP, typename IT>
 __global__ void __launch_bounds__(256)
 halo_kernel(double* __restrict__ u, double* __restrict__ send, const JacGeom g,
             const long long pair0, const long long npairs, const int slots, const unsigned face_mask)
 {
+    if (solve_stopped(g)) return;
     const IT t = (IT)blockIdx.x * (IT)blockDim.x + (IT)threadIdx.x;
     const IT pr = t / (IT)slots;
     if (pr >= (IT)npairs) return;
-    const unsigned e = 2u * (unsigned)(t - pr * (IT)slots);
+    const unsigned local = (unsigned)(t - pr * (IT)slots);
     const IT pair = (IT)pair0 + pr;
     const IT blk = pair / (IT)g.nfaces;
     const int face = (int)(pair - blk * (IT)g.nfaces);
     if (!((face_mask >> face) & 1u)) return;
     const BlockPlace<IT> bp = block_place<IT>(g, blk, face);
     if (!bp.has_nb) return;
-    const BlockExtent& be = bp.ext;
-    const long long n = face_elems_of(g, be, face);
-    if (e >= n) return;
+    const BlockExtent& be = bp.ext;          // the neighbour has the same extent on the axes the strip spans
     const int axis = face >> 1;
+    const int h = g.h;
     const int ext = axis == 0 ? be.x : (axis == 1 ? be.y : be.z);
-    double* ub = u + (long long)blk * g.block_stride + g.origin;
-    // pack reads the interior strip next to the face; unpack writes the ghost strip
-    const int lo = UNPACK ? ((face & 1) ? ext : -g.h) : ((face & 1) ? ext - g.h : 0);
-    double* buf = UNPACK ? send + (long long)bp.nb * g.send_stride + g.face_off[face ^ 1]
-                         : send + (long long)blk * g.send_stride + g.face_off[face];
-    const bool pair_ok = e + 1 < n;
-    if (axis != 0 && (be.x & 1) == 0) {
-        double2* cell = reinterpret_cast<double2*>(ub + strip_offset(g, be, face, e, lo));
-        double2* slot = reinterpret_cast<double2*>(buf + e);
-        if (UNPACK) *cell = *slot; else *slot = *cell;
-    } else {
-        double* c0 = ub + strip_offset(g, be, face, e, lo);
-        if (UNPACK) *c0 = buf[e]; else buf[e] = *c0;
-        if (pair_ok) {
-            double* c1 = ub + strip_offset(g, be, face, e + 1, lo);
-            if (UNPACK) *c1 = buf[e + 1]; else buf[e + 1] = *c1;
-        }
-    }
-}
+    const int full = axis == 0 ? g.bx : (axis == 1 ? g.by : g.bz);
+    // first layer of the strip along the face's axis, interior-relative:
+    //   where the data is read (pack: our interior strip; exchange: the neighbour's strip facing us --
+    //   both blocks of such a pair are full along the axis, or the one at the high end is the remainder
+    //   block, whose strip starts at 0)            and where ghost cells are written
+    const int lo_src = OP == HALO_EXCHANGE ? ((face & 1) ? 0 : full - h) : ((face & 1) ? ext - h : 0);
+    const int lo_dst = (face & 1) ? ext : -h;
+    double* own = u + (long long)blk * g.block_stride + g.origin;
+    const double* src_blk = OP == HALO_EXCHANGE ? u + (long long)bp.nb * g.block_stride + g.origin : own;
+    // the send slot involved: ours (pack) or the neighbour's opposite one (unpack, exchange)
+    double* buf = OP == HALO_PACK ? send + (long long)blk * g.send_stride + g.face_off[face]
+                                  : send + (long long)bp.nb * g.send_stride + g.face_off[face ^ 1];
+    const long long PX = g.PX, PXY = g.PXY;
 
-// Pack and unpack in one launch: the thread that fills ghost cells of (block, face) reads them from
-// the neighbour's interior strip and also leaves them in the neighbour's send slot, so that the
-// buffers and the ghosts end up exactly as after halo_kernel<false> followed by halo_kernel<true>.
-// One read and two writes per face cell instead of two reads and two writes, and one launch.
-template <typename IT>
-__global__ void __launch_bounds__(256)
-halo_exchange_kernel(double* __restrict__ u, double* __restrict__ send, const JacGeom g, const long long npairs,
-                     const int slots)
-{
-    const IT t = (IT)blockIdx.x * (IT)blockDim.x + (IT)threadIdx.x;
-    const IT pr = t / (IT)slots;
-    if (pr >= (IT)npairs) return;
-    const unsigned e = 2u * (unsigned)(t - pr * (IT)slots);
-    const IT blk = pr / (IT)g.nfaces;
-    const int face = (int)(pr - blk * (IT)g.nfaces);
-    const BlockPlace<IT> bp = block_place<IT>(g, blk, face);
-    if (!bp.has_nb) return;
-    const BlockExtent& be = bp.ext;      // the neighbour has the same extent on the axes the strip spans
-    const long long n = face_elems_of(g, be, face);
-    if (e >= n) return;
-    const int axis = face >> 1;
-    const int full = axis == 0 ? g.bx : (axis == 1 ? g.by : g.bz);   // both blocks of such a pair are
-    // full along the axis, or the one at the high end is the remainder block: its strip starts at 0
-    const int lo_src = (face & 1) ? 0 : full - g.h;                  // the neighbour's interior strip facing us
-    const int lo_dst = (face & 1) ? (axis == 0 ? be.x : (axis == 1 ? be.y : be.z)) : -g.h;   // our ghost strip
-    const double* src = u + (long long)bp.nb * g.block_stride + g.origin;
-    double* dst = u + (long long)blk * g.block_stride + g.origin;
-    double* buf = send + (long long)bp.nb * g.send_stride + g.face_off[face ^ 1];
-    if (axis != 0 && (be.x & 1) == 0) {
-        const double2 v = *reinterpret_cast<const double2*>(src + strip_offset(g, be, face, e, lo_src));
-        *reinterpret_cast<double2*>(buf + e) = v;
-        *reinterpret_cast<double2*>(dst + strip_offset(g, be, face, e, lo_dst)) = v;
-    } else {
-        const double v0 = src[strip_offset(g, be, face, e, lo_src)];
-        buf[e] = v0;
-        dst[strip_offset(g, be, face, e, lo_dst)] = v0;
-        if (e + 1 < n) {
-            const double v1 = src[strip_offset(g, be, face, e + 1, lo_src)];
-            buf[e + 1] = v1;
-            dst[strip_offset(g, be, face, e + 1, lo_dst)] = v1;
+    if (axis == 0) {
+        const unsigned nrows = (unsigned)be.y * (unsigned)be.z;
+        // whole-sector stores of the ghost columns: rows start on 32-byte boundaries
+        const bool sector = OP != HALO_PACK && h <= 2 && g.xpad == 4 && (PX & 3) == 0 && ((face & 1) == 0 || (be.x & 3) == 0);
+        double v[kHaloUnits][2];
+        long long cell[kHaloUnits];
+#pragma unroll
+        for (int k = 0; k < kHaloUnits; ++k) {
+            const unsigned R = local + (unsigned)k * (unsigned)slots;
+            if (R >= nrows) continue;
+            const unsigned z = be.z == 1 ? 0u : R / (unsigned)be.y;
+            const unsigned y = R - z * (unsigned)be.y;
+            cell[k] = (long long)z * PXY + (long long)y * PX;
+            if (h <= 2) {
+#pragma unroll
+                for (int c = 0; c < 2; ++c)
+                    if (c < h) v[k][c] = OP == HALO_UNPACK ? buf[(long long)R * h + c] : src_blk[cell[k] + lo_src + c];
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < kHaloUnits; ++k) {
+            const unsigned R = local + (unsigned)k * (unsigned)slots;
+            if (R >= nrows) continue;
+            if (h <= 2) {
+                if (OP != HALO_UNPACK) {
+#pragma unroll
+                    for (int c = 0; c < 2; ++c)
+                        if (c < h) buf[(long long)R * h + c] = v[k][c];
+                }
+                if (OP != HALO_PACK) {
+                    if (sector) {
+                        double2* sec = reinterpret_cast<double2*>(own + cell[k] + ((face & 1) ? ext : -4));
+                        if (face & 1) {      // the ghosts are the first h cells of the sector
+                            sec[0] = make_double2(v[k][0], h == 2 ? v[k][1] : 0.0);
+                            sec[1] = make_double2(0.0, 0.0);
+                        } else {             // the last h
+                            sec[0] = make_double2(0.0, 0.0);
+                            sec[1] = h == 2 ? make_double2(v[k][0], v[k][1]) : make_double2(0.0, v[k][0]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 2; ++c)
+                            if (c < h) own[cell[k] + lo_dst + c] = v[k][c];
+                    }
+                }
+            } else {                         // wider strips (h <= 8): the row's cells, loads before stores
+                double w[8];
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    if (c < h) w[c] = OP == HALO_UNPACK ? buf[(long long)R * h + c] : src_blk[cell[k] + lo_src + c];
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    if (c >= h) continue;
+                    if (OP != HALO_UNPACK) buf[(long long)R * h + c] = w[c];
+                    if (OP != HALO_PACK) own[cell[k] + lo_dst + c] = w[c];
+                }
+            }
+        }
+        return;
+    }
+
+    // y and z faces: lines of be.x cells, contiguous in the block and in the buffer
+    const unsigned ex = (unsigned)be.x;
+    const bool vec = (ex & 1u) == 0 && (PX & 1) == 0;       // both sides 16-byte aligned
+    const unsigned V = vec ? ex >> 1 : ex;                    // units per line
+    const unsigned nlines = (unsigned)h * (unsigned)(axis == 1 ? be.z : be.y);
+    const unsigned TL = (unsigned)slots / V;                  // lines the pair's threads cover side by side
+    if (TL == 0) {
+        // a line longer than the pair's threads (tiny slots): threads stride over the units of the face
+        const unsigned nunits = V * nlines;
+        for (unsigned q = local; q < nunits; q += (unsigned)slots) {
+            const unsigned L = q / V, vi = q - L * V;
+            const unsigned a = axis == 1 ? L / (unsigned)h : L / (unsigned)be.y;
+            const unsigned r = axis == 1 ? L - a * h : L - a * be.y;
+            const long long so = axis == 1 ? (long long)a * PXY + (long long)(lo_src + (int)r) * PX
+                                           : (long long)r * PX + (long long)(lo_src + (int)a) * PXY;
+            const long long dn = axis == 1 ? (long long)a * PXY + (long long)(lo_dst + (int)r) * PX
+                                           : (long long)r * PX + (long long)(lo_dst + (int)a) * PXY;
+            const unsigned x0 = vec ? 2 * vi : vi;
+            for (unsigned c = 0; c < (vec ? 2u : 1u); ++c) {
+                const long long bi = (long long)L * ex + x0 + c;
+                const double w = OP == HALO_UNPACK ? buf[bi] : src_blk[so + x0 + c];
+                if (OP != HALO_UNPACK) buf[bi] = w;
+                if (OP != HALO_PACK) own[dn + x0 + c] = w;
+            }
+        }
+        return;
+    }
+    const unsigned L0 = local / V;
+    if (L0 >= TL) return;                                     // fewer than V threads left over
+    const unsigned vi = local - L0 * V;
+    const unsigned x0 = vec ? 2 * vi : vi;
+    double2 w2[kHaloUnits];
+    double w1[kHaloUnits];
+    long long dst_off[kHaloUnits], buf_off[kHaloUnits];
+    for (unsigned Lb = L0; Lb < nlines; Lb += kHaloUnits * TL) {
+#pragma unroll
+        for (int k = 0; k < kHaloUnits; ++k) {
+            const unsigned L = Lb + (unsigned)k * TL;
+            if (L >= nlines) continue;
+            // line -> (layer along the axis, position along the other axis)
+            unsigned a, r;
+            if (axis == 1) { a = h == 1 ? L : L / (unsigned)h; r = L - a * (unsigned)h; }      // a = z, r = layer
+            else { a = h == 1 ? 0u : L / (unsigned)be.y; r = L - a * (unsigned)be.y; }         // a = layer, r = y
+            const long long so = axis == 1 ? (long long)a * PXY + (long long)(lo_src + (int)r) * PX
+                                           : (long long)(lo_src + (int)a) * PXY + (long long)r * PX;
+            dst_off[k] = (axis == 1 ? (long long)a * PXY + (long long)(lo_dst + (int)r) * PX
+                                    : (long long)(lo_dst + (int)a) * PXY + (long long)r * PX) + x0;
+            buf_off[k] = (long long)L * ex + x0;
+            if (vec) w2[k] = OP == HALO_UNPACK ? *reinterpret_cast<const double2*>(buf + buf_off[k])
+                                               : *reinterpret_cast<const double2*>(src_blk + so + x0);
+            else w1[k] = OP == HALO_UNPACK ? buf[buf_off[k]] : src_blk[so + x0];
+        }
+#pragma unroll
+        for (int k = 0; k < kHaloUnits; ++k) {
+            const unsigned L = Lb + (unsigned)k * TL;
+            if (L >= nlines) continue;
+            if (vec) {
+                if (OP != HALO_UNPACK) *reinterpret_cast<double2*>(buf + buf_off[k]) = w2[k];
+                if (OP != HALO_PACK) *reinterpret_cast<double2*>(own + dst_off[k]) = w2[k];
+            } else {
+                if (OP != HALO_UNPACK) buf[buf_off[k]] = w1[k];
+                if (OP != HALO_PACK) own[dst_off[k]] = w1[k];
+            }
         }
     }
 }
@@ -907,6 +1007,7 @@ temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
                   double* __restrict__ partials, const JacGeom g, const int strips_x, const int strips_y,
                   const int rows_per_strip)
 {
+    if (solve_stopped(g)) return;
     extern __shared__ __align__(16) double2 t2_ring_mem[];   // [warp][u stages, then f stages][64]
     constexpr bool F_RING = temporal_f_ring(T, HAS_F);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;

@@ -43,6 +43,7 @@ __global__ void __launch_bounds__(kResThreads, 1)
 resident2d_kernel(const double* __restrict__ u, double* __restrict__ un, const double* __restrict__ f,
                   const JacGeom g, const int nsweeps, const int rows)
 {
+    if (solve_stopped(g)) return;      // every CTA of the cluster takes the same way out
     namespace cg = cooperative_groups;
     extern __shared__ __align__(16) double res_smem[];
     cg::cluster_group cluster = cg::this_cluster();

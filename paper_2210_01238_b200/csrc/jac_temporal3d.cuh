@@ -291,6 +291,7 @@ temporal3d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
                   double* __restrict__ partials, const JacGeom g, const int tiles_x, const int tiles_y,
                   const int tiles_z, const int zchunk)
 {
+    if (solve_stopped(g)) return;
     constexpr int NFS = t3_f_stages(T);
     constexpr int NUS = t3_u_stages(T);
     T3 c;

@@ -187,7 +187,7 @@ def test_launch_counts_per_schedule(jac):
         counts[mode] = J.launch_count() - c0
         J.close()
     assert counts["fused"] == 5
-    assert counts["exchange"] == 3 * 5
+    assert counts["exchange"] == 2 * 5
     assert counts["pertask"] == 5 * (2 * 34 + 12)
 
 
@@ -339,6 +339,48 @@ def test_residual_from_the_first_sweep_s_pass(jac, orc, n, b, h, mode, tsteps, h
     assert abs(J.residual() - B.residual()) <= RESID_TOL * B.residual()
     J.close()
     B.close()
+
+
+@pytest.mark.parametrize("mode", ["temporal", "fused", "exchange", "pertask", "resident", "wide"])
+def test_solve_stops_after_the_group_that_meets_the_tolerance(jac, orc, mode):
+    """Groups of 3 sweeps, the tolerance met in the middle of a batch of queued groups (and, with a
+    loose tolerance, in the very first group); a tolerance never met runs max_sweeps, the last
+    group shorter."""
+    n, b = (48, 40), (24, 20)
+    u0, f = _random_problem(n, 10)
+
+    def oracle_after(k):
+        B = orc.Blocked(n, b, 1, True)
+        B.set_u(u0)
+        B.set_f(f)
+        B.sweep(k - 1)
+        r = B.residual()
+        B.sweep(1)
+        out = B.get_u(), r
+        B.close()
+        return out
+
+    with jac.Jacobi(n, b, 1, True, mode) as J:
+        J.set_u(u0); J.set_f(f)
+        r0 = J.residual()
+    for tol, max_sweeps in ((0.12 * r0, 500), (10.0 * r0, 500), (0.0, 20)):
+        with jac.Jacobi(n, b, 1, True, mode) as J:
+            J.set_u(u0); J.set_f(f)
+            done, res = J.solve(max_sweeps, 3, tol)
+            got = J.get_u()
+            after = J.residual()
+        want_u, want_r = oracle_after(done)
+        assert res <= tol or done == max_sweeps
+        assert done % 3 == 0 or done == max_sweeps
+        assert abs(res - want_r) <= RESID_TOL * want_r
+        assert np.array_equal(got, want_u), (mode, tol, done)
+        assert after > 0
+        if tol == 10.0 * r0:
+            assert done == 3
+        if tol == 0.12 * r0:
+            assert done == 33          # the eleventh group: the third of the second batch of queued groups
+            prev_u, prev_r = oracle_after(done - 3)     # the group before had not met it yet
+            assert prev_r > tol
 
 
 def test_solve_stops_at_the_tolerance(jac, orc):
