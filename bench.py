@@ -551,6 +551,97 @@ def run_ours(args, w: inputs.Workload):
         dist.destroy_process_group()
 
 
+# ----------------------------------------------------------------------------- one domain over all ranks
+def run_sharded(args, w: inputs.Workload):
+    """--scaling strong: ONE job of the workload over all ranks.  The block grid is cut into slabs of
+    whole block planes along the slowest axis, one slab context per rank (paper_2210_01238_b200.sharded);
+    per sweep the faces on the cut planes travel to the neighbour ranks (NCCL send/recv between the
+    contexts' cut buffers) while the rest of each slab is updated, and a residual costs one all-reduce
+    of a double.  Every step copies the rank's part of the input in from pinned host memory and its
+    part of the solution back (the timed region is the whole step); value = all points x sweeps /
+    the slowest rank's time."""
+    import torch
+    import torch.distributed as dist
+    from paper_2210_01238_b200 import jac, sharded
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    stream = torch.cuda.current_stream()
+    sweeps = args.sweeps if args.sweeps > 0 else w.sweeps
+    every = w.residual_every if 0 < w.residual_every <= sweeps else sweeps
+    groups = [every] * (sweeps // every) + ([sweeps % every] if sweeps % every else [])
+    mode = "fused" if world > 1 else ("temporal" if args.mode == "auto" else args.mode)
+    u0, f = make_inputs(w)
+    sl = sharded.slab_slice(w.n, w.b, rank, world)
+    mine = torch.from_numpy(np.ascontiguousarray(u0[sl])).pin_memory()
+    out = torch.empty_like(mine).pin_memory()
+    J = sharded.slab_context(w.n, w.b, w.halo, w.has_f, mode, rank, world, stream=stream, flags=jac.FLAG_HOST_STAGING)
+    sharded.set_slab_boundary(J, w.ndim, rank, world, w.boundary())
+    if f is not None:
+        J.set_f(np.ascontiguousarray(f[sl]))
+    del u0, f
+
+    def sumsq():
+        return torch.tensor([J.residual_sumsq()], dtype=torch.float64, device="cuda")
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    norms = []
+
+    def step():
+        R = sharded.SlabRank(J, rank, world, dist, sumsq)
+        J.set_u_async(mine)
+        norms.clear()
+        for n_sw in groups:
+            R.sweep(n_sw)
+            norms.append(R.residual())
+        J.get_u_async(out)
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    l0 = J.launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step()
+    ev1.record(stream)
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    if world > 1:
+        ms = reduce_max_over_ranks(ms, "cuda")
+    launches = J.launch_count() - l0
+    J.close()
+    if rank == 0:
+        value = job_updates(w, sweeps) * args.steps / (ms * 1e-3) / 1e9
+        n_slab = sharded.slab_of(w.n, w.b, 0, world)[0]
+        cut_bytes = 8 * w.halo * int(np.prod(w.n[:-1]))
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+                "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+                "dtype": "f64", "data": "synthetic",
+                "config": {"workload": w.name, "grid": list(w.n), "block": list(w.b), "halo": w.halo, "has_f": w.has_f,
+                           "sweeps_per_step": sweeps, "residuals_per_step": len(groups), "schedule": mode,
+                           "slabs": world, "slab_of_rank_0": list(n_slab),
+                           "cut_bytes_per_sweep_per_direction": cut_bytes if world > 1 else 0},
+                "effective_gbs": value * w.bytes_per_point, "residual": norms[-1],
+                "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": int(mine.numel() * 8) * world,
+                        "d2h_bytes_per_step": int(mine.numel() * 8) * world + 8 * len(groups),
+                        "what": "the timed step itself: jac_set_u_async(pinned host) + sweeps + residuals + jac_get_u_async"},
+                "gpu_launches": int(launches), "roofline": None, "cpu_baseline": None}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 # ----------------------------------------------------------------------------- config 4
 def run_halo_microbenchmark(args):
     """Config 4 (halo pack/unpack microbenchmark): the library's timings per block size and halo
@@ -615,6 +706,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-others", action="store_true", help="skip the brief runs of the other schedules")
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="more than one GPU: weak = every rank runs a replica of the job; strong = one job, the "
+                         "block grid cut into one slab per rank")
     ap.add_argument("--n", type=int, default=0,
                     help="profiling aid: same recipe on an n^d grid (block size unchanged)")
     args = ap.parse_args()
@@ -629,6 +723,8 @@ def main():
         w = inputs.scaled(w, (args.n,) * w.ndim, name=f"{w.name}_at_{args.n}")
     if args.impl == "reference":
         run_reference(args, w)
+    elif args.scaling == "strong":
+        run_sharded(args, w)
     else:
         run_ours(args, w)
 

@@ -185,12 +185,13 @@ def _host_ptr(a: np.ndarray):
 class Jacobi:
     """One context of the library over a torch-owned workspace on the current CUDA device.
 
-    n, b: global / block interior points in (x, y[, z]) order.  Dense arrays are numpy float64
+    n, b: global / block interior points in (x, y[, z]) order.  ``workspace``: a uint8 CUDA tensor to
+    use instead of allocating one (256-byte aligned, ``workspace_bytes`` long).  Dense arrays are numpy float64
     of shape (ny, nx) / (nz, ny, nx), or torch CUDA float64 tensors of that shape for the
     ``*_device`` calls.
     """
 
-    def __init__(self, n, b, halo=1, has_f=False, mode="fused", tsteps=0, stream=None, flags=0):
+    def __init__(self, n, b, halo=1, has_f=False, mode="fused", tsteps=0, stream=None, flags=0, workspace=None):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("paper_2210_01238_b200.jac needs a CUDA device; there is no CPU path")
@@ -201,8 +202,14 @@ class Jacobi:
         self.desc = make_desc(n, b, halo, has_f, mode, tsteps, self.stream.cuda_stream, flags)
         self.layout = get_layout(self.desc)
         nbytes = workspace_bytes(self.desc)
-        with torch.cuda.stream(self.stream):
-            self.workspace = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        if workspace is not None:
+            # the caller's memory: a contiguous uint8 CUDA tensor of at least the size the library asks for
+            assert workspace.is_cuda and workspace.dtype == torch.uint8 and workspace.is_contiguous()
+            assert workspace.numel() >= nbytes and workspace.data_ptr() % 256 == 0
+            self.workspace = workspace
+        else:
+            with torch.cuda.stream(self.stream):
+                self.workspace = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
         self._ctx = C.c_void_p()
         self._call("jac_create", lib().jac_create(C.byref(self.desc), self.workspace.data_ptr(),
                                                   nbytes, C.byref(self._ctx)))
