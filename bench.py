@@ -703,6 +703,8 @@ def main():
                     help="schedule of jac_sweep; auto = the fastest one the library has for the workload")
     ap.add_argument("--tsteps", type=int, default=0)
     ap.add_argument("--sweeps", type=int, default=0, help="sweeps per step (default: the workload's)")
+    ap.add_argument("--residual-every", type=int, default=-1,
+                    help="residual norm after every N sweeps (default: the workload's; 0: only after the last sweep)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-others", action="store_true", help="skip the brief runs of the other schedules")
@@ -721,6 +723,9 @@ def main():
     w = inputs.CONFIGS[args.workload]
     if args.n:
         w = inputs.scaled(w, (args.n,) * w.ndim, name=f"{w.name}_at_{args.n}")
+    if args.residual_every >= 0:
+        import dataclasses
+        w = dataclasses.replace(w, residual_every=args.residual_every)
     if args.impl == "reference":
         run_reference(args, w)
     elif args.scaling == "strong":

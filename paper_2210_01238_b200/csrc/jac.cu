@@ -99,7 +99,7 @@ int temporal_rows_2d(const JacGeom& g, int T, bool has_f, int sms)
     return JAC_FORCE_ROWS;
 #endif
     const long long strips_x = ceil_div(g.nx, jac::temporal_strip_cols(T));
-    const int ctas_per_sm = ((T > 4 && jac::temporal_points(T) == 4) || jac::temporal_f_ring(T, has_f)) ? 2 : JAC_TOCC;
+    const int ctas_per_sm = jac::temporal_ctas_per_sm(T, has_f);
     const double capacity = (double)sms * ctas_per_sm * jac::kTemporalWarps;
     const double alpha = T > 4 ? 0.45 : 0.7;
     int best = 8;
@@ -108,7 +108,7 @@ int temporal_rows_2d(const JacGeom& g, int T, bool has_f, int sms)
         if (rows > g.ny && rows > 8) break;
         const double w = (double)(strips_x * ceil_div(g.ny, rows)) / capacity;
         const double rounds = w < 6.0 ? std::ceil(w - 1e-9) : w;
-        const double cost = (rows + 4 * T - 1) * (rounds + alpha);
+        const double cost = (rows + 2 * T) * (rounds + alpha);
         if (cost <= best_cost) {   // ties go to the longer strip (less redundant work)
             best_cost = cost;
             best = rows;
@@ -687,15 +687,18 @@ int usable(jac_ctx* c)
     return JAC_OK;
 }
 
-// Sweeps per launch when the caller leaves the choice to the library.  2D: 8 levels pay off only
-// without a right-hand side and on grids large enough to fill the GPU with 256-row strips
-// (measured: 16384^2 1668 vs 1320 GLUP/s; 4096^2 with f 236 vs 326); otherwise 4.  3D: 3.
+// Sweeps per launch when the caller leaves the choice to the library.  2D without a right-hand
+// side: 8 on grids large enough to fill the GPU with long strips (measured: 16384^2 1817 vs 1356
+// GLUP/s at 4), else 4 (4096^2: 1041 vs 1032).  2D with a right-hand side: 6 (4096^2: 702 GLUP/s
+// against 671 at 4 and 577 at 8, whose windows plus the f row no longer fit the registers; 8192^2:
+// 841 / 732 / 786).  3D: 3.
 int default_tsteps(const jac_desc& d)
 {
     if (d.tsteps > 0) return d.tsteps;
     if (d.ndim == 3) return 3;
+    if (d.has_f) return 6;
     const bool large = d.n[0] * d.n[1] >= (1LL << 26);
-    return (!d.has_f && large) ? 8 : 4;
+    return large ? 8 : 4;
 }
 
 // The dynamic shared memory a kernel may use is an attribute of the kernel on a device: set it the

@@ -710,12 +710,14 @@ dense_copy_kernel(double* __restrict__ blocks, double* __restrict__ dense, const
 // 2D temporal blocking: T sweeps per launch, in registers.
 //
 // A warp owns a strip 128 columns wide (4 consecutive points per lane) and streams it along
-// y.  Input row r enters at level 0; level s (s = 1..T) trails it and produces its row
-// r - 2s + 1 from rows r-2s, r-2s+1, r-2s+2 of level s-1, so a T-deep pipeline of 3-row
-// windows lives in registers (3*4*T doubles per lane).  Each level lags the one below by two
-// rows, so within one step no level waits for another (they are evaluated top level first):
-// the fp64 pipe always has 4*T independent points to work on.  West/east neighbours come from
-// the adjacent lanes by shuffle, so warps never synchronise with each other.  The two edge
+// y.  Input row r enters at level 0; in the same step level s (s = 1..T) produces its row r - s
+// from rows r-s-1, r-s, r-s+1 of level s-1, the last of which level s-1 has produced a moment
+// before.  Levels therefore run lowest first, and of each level only two rows are alive from one
+// step to the next (2*4*T doubles per lane; a pipeline whose levels lag by two rows and are
+// independent within a step keeps three, which at T = 8 leaves room for 8 warps per SM only).
+// Across the points of a row and across the warps of an SM there is independent work to cover
+// the latency of the chain of levels.  West/east neighbours come from the adjacent lanes by
+// shuffle, so warps never synchronise with each other.  The two edge
 // lanes of a warp lose one point of validity per level; lanes 1..30 (120 columns) are exact
 // after T <= 4 levels and are the ones stored.  Strips read across block borders directly
 // (the neighbour's interior is the halo), which is what an exchange before every sweep would
@@ -742,13 +744,21 @@ dense_copy_kernel(double* __restrict__ blocks, double* __restrict__ dense, const
 #endif
 constexpr int kTemporalWarps = JAC_TW;
 constexpr int kTemporalDepth = JAC_TD;
-// Right-hand side rows of the 2D temporal kernel: up to T = 4 they travel through a second
-// cp.async ring (a row is copied together with the u row of the same index and stays until the
-// top level has used it, DEPTH + 2T steps later); deeper pipelines read f through L1 instead.
+// Right-hand side rows of the 2D temporal kernel travel through a second cp.async ring: a row is
+// copied together with the u row of the same index and stays until the top level has used it,
+// DEPTH + T steps later (at most 16).
 constexpr int kTemporalFDepth = 16;
-__host__ __device__ constexpr bool temporal_f_ring(int T, bool has_f) { return has_f && T <= 4; }
+__host__ __device__ constexpr bool temporal_f_ring(int T, bool has_f) { return has_f && T + kTemporalDepth <= kTemporalFDepth; }
 __host__ __device__ constexpr int temporal_stages_per_warp(int T, bool has_f) {
     return kTemporalDepth + (temporal_f_ring(T, has_f) ? kTemporalFDepth : 0);
+}
+// CTAs per SM the register allocation aims for
+__host__ __device__ constexpr int temporal_ctas_per_sm(int T, bool has_f) {
+#ifdef JAC_T2_FORCE_MINB
+    return JAC_T2_FORCE_MINB;
+#else
+    return (T > 4 || has_f) ? 2 : JAC_TOCC;
+#endif
 }
 // A lane holds P consecutive points (4; the code also runs with 2, which halves the window
 // registers of deep pipelines but was measured slower).  A ring stage is one row of the strip: 16 P chunks of 16 bytes.
@@ -881,18 +891,17 @@ __device__ __forceinline__ RowN<P> take_row(const TemporalCtx& c, int r) {
 
 __host__ __device__ constexpr int slot3(int ph, int d) { return (((ph + d) % 3) + 3) % 3; }
 
-// One pipeline step: input row r arrives (phase PH = (r - r0) mod 3) and every level advances
-// one row.  EDGE = false is for steps in which no row and no column involved lies outside the
-// domain: no Dirichlet fix-up is compiled in.
-// level s of one step: row r - 2s + 1 from the window of level s - 1
+// level s of one step: row r - s from the window of level s - 1 (input row r has phase PH = (r - r0) mod 3).
+// EDGE = false is for steps in which no row and no column involved lies outside the domain: no
+// Dirichlet fix-up is compiled in.
 template <int T, bool HAS_F, int RES, int PH, bool EDGE, int s>
 __device__ __forceinline__ void temporal_level(RowN<temporal_points(T)> (&win)[T][3], const TemporalCtx& c,
                                                const JacGeom& g, int r, const RowCursor& out_cur, double& acc)
 {
     constexpr int P = temporal_points(T);
     using Row = RowN<P>;
-    constexpr bool F_RING = temporal_f_ring(T, HAS_F);
-    constexpr int d = -2 * s + 1;              // level s produces row r + d
+    static_assert(!HAS_F || temporal_f_ring(T, HAS_F), "the right-hand side travels through its ring");
+    constexpr int d = -s;                      // level s produces row r + d
     const int rs = r + d;
     const Row& S = win[s - 1][slot3(PH, d - 1)];
     const Row& M = win[s - 1][slot3(PH, d)];
@@ -902,22 +911,17 @@ __device__ __forceinline__ void temporal_level(RowN<temporal_points(T)> (&win)[T
     Row ff;
     if (HAS_F) {
         const bool ok = EDGE ? (rs >= 0 && rs < c.ny && !c.xout) : true;
-        if (ok && F_RING) {
-            // copied DEPTH + 2s - 1 steps ago; the warp-wide barriers of the steps in between
-            // made the other lanes' chunks visible
+        if (ok) {
+            // copied DEPTH + s steps ago; the warp-wide barriers of the steps in between made the
+            // other lanes' chunks visible
             const double2* fr = c.mine + (kTemporalDepth + ((rs - c.r0) & (kTemporalFDepth - 1))) *
                                              temporal_stage_chunks(P);
             ff = load_rown<P>(reinterpret_cast<const double*>(fr));
-        } else if (ok) {
-            // f of row rs: the output cursor points at row r - 2T + 1, i.e. (T - s) * 2 rows below rs
-            RowCursor fc = out_cur;
-#pragma unroll
-            for (int k = 0; k < 2 * (T - s); ++k) fc.advance(g, c.brs);
-            ff = load_rown<P>(c.fb + fc.off);
         } else {
             ff = fill_rown<P>(0.0);
         }
     }
+    constexpr bool MEASURES = (RES == kResBeforeLast && s == T) || (RES == kResOfInput && s == 1);
     Row o, res;
 #pragma unroll
     for (int q = 0; q < P; ++q) {
@@ -927,58 +931,52 @@ __device__ __forceinline__ void temporal_level(RowN<temporal_points(T)> (&win)[T
         if (HAS_F) sum = add_rn(sum, ff.v[q]);
         o.v[q] = mul_rn(sum, 0.25);
         // residual of the state this level reads (M is that state at this point)
-        if ((RES == kResBeforeLast && s == T) || (RES == kResOfInput && s == 1)) res.v[q] = sub_rn(sum, mul_rn(4.0, M.v[q]));
+        if (MEASURES) res.v[q] = sub_rn(sum, mul_rn(4.0, M.v[q]));
     }
     if (EDGE) {
         if (rs < 0) o = fill_rown<P>(c.c_my);
         if (rs >= c.ny) o = fill_rown<P>(c.c_py);
         if (c.xout) o = fill_rown<P>(c.cx);
     }
+    const bool in_strip = c.store_lane && rs >= c.Y0 && rs < c.Y1;
     if (s < T) {
         win[s][slot3(PH, d)] = o;
-    } else if (c.store_lane && rs >= c.Y0 && rs < c.Y1) {
+    } else if (in_strip) {
         store_rown<P>(c.ob + out_cur.off, o);
     }
     // the points of the strip's output region: every interior point is in exactly one, and every
     // level is exact there
-    if (((RES == kResBeforeLast && s == T) || (RES == kResOfInput && s == 1)) && c.store_lane && rs >= c.Y0 && rs < c.Y1) {
+    if (MEASURES && in_strip) {
 #pragma unroll
         for (int q = 0; q < P; ++q) acc = add_rn(acc, mul_rn(res.v[q], res.v[q]));
     }
 }
 
 template <int T, bool HAS_F, int RES, int PH, bool EDGE, int s>
-struct TemporalLevels {   // levels s, s - 1, ..., 2 (top level first)
+struct TemporalLevels {   // levels s, s + 1, ..., T (lowest first: each reads the row the one below has just made)
     static __device__ __forceinline__ void run(RowN<temporal_points(T)> (&win)[T][3], const TemporalCtx& c, const JacGeom& g, int r,
                                                const RowCursor& out_cur, double& acc) {
         temporal_level<T, HAS_F, RES, PH, EDGE, s>(win, c, g, r, out_cur, acc);
-        TemporalLevels<T, HAS_F, RES, PH, EDGE, s - 1>::run(win, c, g, r, out_cur, acc);
+        if constexpr (s < T) TemporalLevels<T, HAS_F, RES, PH, EDGE, s + 1>::run(win, c, g, r, out_cur, acc);
     }
 };
-template <int T, bool HAS_F, int RES, int PH, bool EDGE>
-struct TemporalLevels<T, HAS_F, RES, PH, EDGE, 1> {
-    static __device__ __forceinline__ void run(RowN<temporal_points(T)> (&)[T][3], const TemporalCtx&, const JacGeom&, int,
-                                               const RowCursor&, double&) {}
-};
 
-// One pipeline step: input row r arrives (phase PH = (r - r0) mod 3) and every level advances
-// one row.  Levels T..2 only need rows finished in earlier steps, so they run first and cover
-// the wait for the copy of row r; then the row is taken, its ring stage refilled, and level 1
-// runs.  EDGE = false is for steps in which no row and no column involved lies outside the
-// domain: no Dirichlet fix-up is compiled in.
+// One pipeline step: input row r arrives (phase PH = (r - r0) mod 3) and every level advances one
+// row, lowest first; then the ring stages that row r and f row r - T have left are refilled.
+// EDGE = false is for steps in which no row and no column involved lies outside the domain: no
+// Dirichlet fix-up is compiled in.
 template <int T, bool HAS_F, int RES, int PH, bool EDGE>
 __device__ __forceinline__ void temporal_step(RowN<temporal_points(T)> (&win)[T][3], const TemporalCtx& c, const JacGeom& g,
                                               int r, RowCursor& load_cur, RowCursor& out_cur, double& acc)
 {
     constexpr bool F_RING = temporal_f_ring(T, HAS_F);
-    TemporalLevels<T, HAS_F, RES, PH, EDGE, T>::run(win, c, g, r, out_cur, acc);
     cp_async_wait<kTemporalDepth - 1>();
     __syncwarp();                                    // the other lanes' chunks of row r have landed too
     win[0][PH] = take_row<temporal_points(T), EDGE>(c, r);
-    __syncwarp();                                    // everyone has read the stage before it is refilled
+    TemporalLevels<T, HAS_F, RES, PH, EDGE, 1>::run(win, c, g, r, out_cur, acc);
+    __syncwarp();                                    // everyone has read the stages before they are refilled
     issue_row<temporal_points(T), HAS_F, F_RING>(c, r + kTemporalDepth, load_cur);
     load_cur.advance(g, c.brs);
-    temporal_level<T, HAS_F, RES, PH, EDGE, 1>(win, c, g, r, out_cur, acc);
     out_cur.advance(g, c.brs);
 }
 
@@ -993,7 +991,7 @@ __device__ __forceinline__ void temporal_step_any(RowN<temporal_points(T)> (&win
                                                   int r, RowCursor& load_cur, RowCursor& out_cur, double& acc)
 {
     // warp-uniform: does this step see a row outside [0, ny) or a column outside [0, nx)?
-    const bool edge = c.edge_x || (r - 2 * T < 0) || (r >= c.ny);
+    const bool edge = c.edge_x || (r - T - 1 < 0) || (r >= c.ny);
     if (edge) temporal_step<T, HAS_F, RES, PH, true>(win, c, g, r, load_cur, out_cur, acc);
     else temporal_step<T, HAS_F, RES, PH, false>(win, c, g, r, load_cur, out_cur, acc);
 }
@@ -1001,8 +999,7 @@ __device__ __forceinline__ void temporal_step_any(RowN<temporal_points(T)> (&win
 // RES: the top level (kResBeforeLast) or the first level (kResOfInput) also accumulates the squared
 // residual of the state it reads; every warp writes its partial sum to partials[warp id].
 template <int T, bool HAS_F, int RES>
-__global__ void __launch_bounds__(kTemporalWarps * 32,
-                                  (((T > 4 && temporal_points(T) == 4) || temporal_f_ring(T, HAS_F)) ? 2 : JAC_TOCC))
+__global__ void __launch_bounds__(kTemporalWarps * 32, temporal_ctas_per_sm(T, HAS_F))
 temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const double* __restrict__ f,
                   double* __restrict__ partials, const JacGeom g, const int strips_x, const int strips_y,
                   const int rows_per_strip)
@@ -1047,7 +1044,7 @@ temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
     c.Y1 = min(c.ny, c.Y0 + rows_per_strip);
     c.r0 = c.Y0 - T;
     c.in_end = c.Y1 + T;
-    const int r_end = c.Y1 + 2 * T - 1;   // the top level trails the input by 2T - 1 rows
+    const int r_end = c.Y1 + T;           // the top level trails the input by T rows
 
     RowN<P> win[T][3];
 #pragma unroll
@@ -1057,7 +1054,7 @@ temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
 
     RowCursor load_cur, out_cur;
     load_cur.init(c.r0, g, c.brs);
-    out_cur.init(c.r0 - 2 * T + 1, g, c.brs);   // row produced by the top level in the first step
+    out_cur.init(c.r0 - T, g, c.brs);           // row produced by the top level in the first step
 
     // fill the ring with the first DEPTH rows
 #pragma unroll 1

@@ -286,7 +286,7 @@ def test_sweeps_per_launch_query(jac):
     cases = [(dict(n=(64, 64), b=(32, 32), mode="exchange"), 1),
              (dict(n=(64, 64), b=(32, 32), mode="temporal", tsteps=3), 3),
              (dict(n=(64, 64), b=(32, 32), mode="temporal"), 4),            # small grid: 4
-             (dict(n=(64, 64), b=(32, 32), mode="temporal", has_f=True), 4),
+             (dict(n=(64, 64), b=(32, 32), mode="temporal", has_f=True), 6),
              (dict(n=(16, 16, 16), b=(8, 8, 8), mode="temporal"), 3)]
     for kw, want in cases:
         with jac.Jacobi(**kw) as J:
