@@ -53,6 +53,9 @@ extern "C" {
 #define JAC_ECUDA    (-3)  /* a CUDA runtime call failed (sticky); see jac_last_cuda_error       */
 #define JAC_ENODEV   (-4)  /* no usable CUDA device                                              */
 #define JAC_ELIMIT   (-5)  /* problem larger than the fixed scratch of jac_residual_dense_static */
+#define JAC_ETIMEOUT (-6)  /* JAC_MODE_RESIDENT: a CTA gave up waiting for a neighbour's row (every
+                              device-side wait is bounded); the state is not to be trusted.  Reported
+                              by the next call that waits for the stream (sticky)                  */
 
 /* How jac_sweep schedules one iteration.  All modes leave bit-identical interiors. */
 #define JAC_MODE_FUSED    0 /* one launch per sweep over all blocks; across a face with a neighbour
@@ -80,8 +83,8 @@ extern "C" {
 #define JAC_MODE_RESIDENT 5 /* small 2D grids: all sweeps of a jac_sweep call in ONE launch of one
                                thread-block cluster (8 or 16 CTAs) that keeps the whole grid in
                                shared memory, slabs of rows per CTA, neighbouring slabs exchanging
-                               their edge rows through distributed shared memory, one cluster
-                               barrier per sweep.  Needs ndim == 2, b[0] and n[0] even and
+                               their edge rows through distributed shared memory, one
+                               row exchange per sweep (pairwise, through mbarriers).  Needs ndim == 2, b[0] and n[0] even and
                                (2*(r+2) + (has_f ? r : 0)) * (n[0]+4) * 8 bytes <= 227 KB for
                                r = ceil(n[1]/8) or ceil(n[1]/16) (e.g. 256 x 256 with f);
                                JAC_EINVAL otherwise, also when the device cannot co-schedule a

@@ -156,7 +156,7 @@ struct ResidentPlan {
     int cluster, rows;
     size_t smem;
 };
-constexpr size_t kMaxSmemPerCta = 227 * 1024;
+constexpr size_t kMaxSmemPerCta = 227 * 1024 - 64;   // dynamic shared memory beside the kernel's few static words
 
 int plan_resident(const JacGeom& g, bool has_f, int want_cluster, ResidentPlan* p)
 {
@@ -354,6 +354,7 @@ struct jac_ctx {
     cudaStream_t stream;
     int device;
     int cuda_err;       // sticky
+    bool timed_out;     // sticky: a resident launch gave up a wait
     long long launches;
 };
 
@@ -684,6 +685,7 @@ int usable(jac_ctx* c)
 {
     if (!c) return JAC_EINVAL;
     if (c->cuda_err) return JAC_ECUDA;
+    if (c->timed_out) return JAC_ETIMEOUT;
     return JAC_OK;
 }
 
@@ -822,7 +824,7 @@ int launch_resident_t(jac_ctx* c, const ResidentPlan& rp, const double* u, doubl
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    JAC_CK(c, cudaLaunchKernelEx(&cfg, kern, u, un, (const double*)c->f, c->g, nsweeps, rp.rows));
+    JAC_CK(c, cudaLaunchKernelEx(&cfg, kern, u, un, (const double*)c->f, c->g, nsweeps, rp.rows, reinterpret_cast<int*>(c->result + 4)));
     return check_launch(c);
 }
 
@@ -1037,6 +1039,20 @@ solve_check_kernel(const double* __restrict__ partials, const long long n, const
 }
 
 // fixed-order sum of the first nparts partial sums -> host, as a norm
+// has a resident launch given up a wait?  (call after the stream has been waited for)
+int check_timeout(jac_ctx* c)
+{
+    if (c->desc.mode != JAC_MODE_RESIDENT) return JAC_OK;
+    int flag = 0;
+    JAC_CK(c, cudaMemcpyAsync(&flag, c->result + 4, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+    JAC_CK(c, cudaStreamSynchronize(c->stream));
+    if (flag) {
+        c->timed_out = true;
+        return JAC_ETIMEOUT;
+    }
+    return JAC_OK;
+}
+
 int finish_norm(jac_ctx* c, long long nparts, double* host_out_l2)
 {
     jac::reduce_partials_kernel<<<1, 1024, 0, c->stream>>>(c->partials, nparts, c->result);
@@ -1045,6 +1061,7 @@ int finish_norm(jac_ctx* c, long long nparts, double* host_out_l2)
     double sum = 0.0;
     JAC_CK(c, cudaMemcpyAsync(&sum, c->result, sizeof(double), cudaMemcpyDeviceToHost, c->stream));
     JAC_CK(c, cudaStreamSynchronize(c->stream));
+    if ((rc = check_timeout(c))) return rc;
     *host_out_l2 = std::sqrt(sum);
     return JAC_OK;
 }
@@ -1248,6 +1265,7 @@ int jac_create(const jac_desc* desc, void* dev_workspace, size_t bytes, jac_ctx*
     c->stream = static_cast<cudaStream_t>(desc->stream);
     c->device = dev;
     c->cuda_err = 0;
+    c->timed_out = false;
     c->launches = 0;
     const cudaError_t e = cudaMemsetAsync(c->ws, 0, (size_t)L.total_bytes, c->stream);
     if (e != cudaSuccess) {
@@ -1329,7 +1347,8 @@ int jac_get_u(jac_ctx* c, double* host_dense)
     int rc = usable(c);
     if (rc) return rc;
     if (!host_dense) return JAC_EINVAL;
-    return blocks_to_host(c, c->u[c->cur], host_dense, true);
+    if ((rc = blocks_to_host(c, c->u[c->cur], host_dense, true))) return rc;
+    return check_timeout(c);
 }
 
 int jac_set_u_device(jac_ctx* c, const double* dev_dense)
@@ -1715,6 +1734,7 @@ const char* jac_strerror(int code)
         case JAC_ECUDA: return "CUDA runtime error";
         case JAC_ENODEV: return "no usable CUDA device";
         case JAC_ELIMIT: return "problem exceeds the fixed scratch of the no-allocation entry point";
+        case JAC_ETIMEOUT: return "a bounded device-side wait ran out";
         default: return "unknown error code";
     }
 }

@@ -4,11 +4,19 @@
 // A grid of a few hundred KB is bound by launch and pipeline latency, not by bandwidth: every
 // other schedule pays at least one launch per handful of sweeps and goes through L2 each time.
 // Here CTA c of the cluster owns a slab of `rows` consecutive grid rows in two shared-memory
-// buffers (plus the slab's right-hand side), sweeps from one buffer into the other, writes its
-// first and last new row straight into the neighbouring CTAs' halo rows through distributed
-// shared memory, and meets the other CTAs at one cluster barrier per sweep (arrive after the edge
-// rows, wait after the inner rows, so the barrier's latency is covered by work).  Global memory is
-// read once before the first sweep and written once after the last.
+// buffers (plus the slab's right-hand side) and sweeps from one buffer into the other.  Global
+// memory is read once before the first sweep and written once after the last.
+//
+// Neighbouring slabs only ever need each other's edge row, so they synchronise pairwise, not as a
+// cluster: a CTA computes its first and last new row first and sends them straight into the
+// neighbours' halo rows with st.async, which counts the bytes that have landed on an mbarrier in
+// the RECEIVING CTA; the receiver waits on its two mbarriers (one per side) after it has computed
+// its inner rows.  No fence, no cluster-wide barrier per sweep: the cluster barrier is used once
+// after the fill and once before the write-back.  Why a halo row can be overwritten safely: the
+// row a neighbour sends for sweep s + 1 can only leave after that neighbour has received this
+// CTA's row of sweep s, which each thread sends after it has read the halo cells it needs.
+// Every wait is bounded: a CTA that has polled kResMaxPolls times sets the error word, stops
+// waiting and runs to the end with whatever it has, so that all CTAs reach the final barrier.
 //
 // Slab layout (doubles): row pitch RP = nx + 4; grid column i sits at index i + 2 (so pairs of
 // columns are 16-byte aligned), the Dirichlet columns at 1 and nx + 2.  Local row 0 is the halo
@@ -25,6 +33,33 @@
 namespace jac {
 
 constexpr int kResThreads = 512;
+constexpr int kResMaxPolls = 1 << 22;     // mbarrier polls before a CTA gives up waiting
+
+// ---- mbarrier / distributed shared memory primitives (PTX) ---------------------------------
+__device__ __forceinline__ unsigned smem_addr(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
+    unsigned ok;
+    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// the address, in the cluster's shared window, of this CTA's shared address `local` in CTA `rank`
+__device__ __forceinline__ unsigned map_to_rank(unsigned local, unsigned rank) {
+    unsigned r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(r) : "r"(local), "r"(rank));
+    return r;
+}
+// 16 bytes into another CTA's shared memory; the bytes are counted on that CTA's mbarrier when they land
+__device__ __forceinline__ void send_pair(unsigned remote, unsigned remote_bar, double2 v) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f64 [%0], {%1, %2}, [%3];\n"
+                 ::"r"(remote), "d"(v.x), "d"(v.y), "r"(remote_bar) : "memory");
+}
 
 __host__ __device__ constexpr long long resident_pitch(long long nx) { return nx + 4; }
 // shared-memory bytes of one CTA whose slab has `rows` rows
@@ -41,7 +76,7 @@ __device__ __forceinline__ long long resident_offset(const JacGeom& g, long long
 template <bool HAS_F>
 __global__ void __launch_bounds__(kResThreads, 1)
 resident2d_kernel(const double* __restrict__ u, double* __restrict__ un, const double* __restrict__ f,
-                  const JacGeom g, const int nsweeps, const int rows)
+                  const JacGeom g, const int nsweeps, const int rows, int* __restrict__ timed_out)
 {
     if (solve_stopped(g)) return;      // every CTA of the cluster takes the same way out
     namespace cg = cooperative_groups;
@@ -57,6 +92,8 @@ resident2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
     const bool has_hi = rank + 1 < nranks && y0 + rows < ny; // a CTA above owns row y0 + rows
     double* const buf[2] = {res_smem, res_smem + (size_t)(rows + 2) * RP};
     double* fs = res_smem + (size_t)2 * (rows + 2) * RP;     // [rows][RP], same column placement
+    // arrival of the halo row below / above this slab in buffer 0 / 1: [side][buffer]
+    __shared__ __align__(8) unsigned long long halo_bar[2][2];
     const int tid = threadIdx.x;
     const int npairs = nx / 2;
 
@@ -81,25 +118,38 @@ resident2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
         if (HAS_F && l >= 1 && l <= mine)
             *reinterpret_cast<double2*>(fs + (l - 1) * RP + 2 + 2 * cp) = *reinterpret_cast<const double2*>(f + off);
     }
-    // where the neighbours keep the halo row that mirrors this slab's first / last row
-    // (A = the buffer being read, B = the one being written; they swap after every sweep)
-    double *lo_A = nullptr, *lo_B = nullptr, *hi_A = nullptr, *hi_B = nullptr;
+    // where the neighbours keep the halo row that mirrors this slab's first / last row, and the
+    // mbarrier that counts its arrival there, per buffer: this slab's first row goes to the upper
+    // halo row (rows + 1) of the CTA below, which is full (only the last owning CTA can be short)
+    unsigned lo_row[2] = {0, 0}, hi_row[2] = {0, 0}, lo_bar[2] = {0, 0}, hi_bar[2] = {0, 0};
     if (has_lo) {
-        // the CTA below is full (only the last owning CTA can be short): its upper halo is row rows + 1
-        lo_A = cluster.map_shared_rank(buf[0], rank - 1) + (size_t)(rows + 1) * RP;
-        lo_B = cluster.map_shared_rank(buf[1], rank - 1) + (size_t)(rows + 1) * RP;
+#pragma unroll
+        for (int w = 0; w < 2; ++w) {
+            lo_row[w] = map_to_rank(smem_addr(buf[w] + (size_t)(rows + 1) * RP), rank - 1);
+            lo_bar[w] = map_to_rank(smem_addr(&halo_bar[1][w]), rank - 1);     // it arrives from above, there
+        }
     }
     if (has_hi) {
-        hi_A = cluster.map_shared_rank(buf[0], rank + 1);
-        hi_B = cluster.map_shared_rank(buf[1], rank + 1);
+#pragma unroll
+        for (int w = 0; w < 2; ++w) {
+            hi_row[w] = map_to_rank(smem_addr(buf[w]), rank + 1);
+            hi_bar[w] = map_to_rank(smem_addr(&halo_bar[0][w]), rank + 1);     // from below, there
+        }
+    }
+    if (tid == 0) {
+#pragma unroll
+        for (int side = 0; side < 2; ++side)
+#pragma unroll
+            for (int w = 0; w < 2; ++w) mbar_init(smem_addr(&halo_bar[side][w]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
     cluster.sync();
 
     // ---- sweeps: A -> B.  The slab's first and last row go first: they are what the neighbours
-    // wait for, and the only rows that read this slab's halo rows.  Once they are written (here and
-    // into the neighbours' halo rows) the CTA arrives at the cluster barrier, computes its inner
-    // rows while the barrier completes, and waits before the next sweep.  The inner rows are
-    // marched through in segments (rows below and above a thread's pair stay in registers).
+    // wait for, and the only rows that read this slab's halo rows.  They are written here and sent
+    // into the neighbours' halo rows; then the inner rows are computed while those rows travel, and
+    // only then does the CTA wait for the two rows it is owed.  The inner rows are marched through
+    // in segments (rows below and above a thread's pair stay in registers).
     // The assignment of work to threads is the same in every sweep, so it is fixed here: a thread
     // owns the column pairs cp0, cp0 + pw, ... and row group `grp`; group 0 also computes edge row 1
     // and another group (the same one if there is only one) edge row `mine`.
@@ -112,8 +162,17 @@ resident2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
     const int l1 = grp < groups ? min(mine, l0 + segrows) : l0;
     const bool does_lo = grp == 0 && mine >= 1;
     const bool does_hi = grp == min(groups, 2) - 1 && mine >= 2;
-    double *A = buf[0], *B = buf[1];
+    const unsigned row_bytes = (unsigned)nx * (unsigned)sizeof(double);
+    bool gave_up = false;
     for (int s = 0; s < nsweeps; ++s) {
+        const int wb = (s + 1) & 1;                           // buffer written in this sweep
+        double* const A = buf[wb ^ 1];
+        double* const B = buf[wb];
+        // this sweep's incoming rows: one arrival (this one) plus the row's bytes complete a phase
+        if (tid == 0) {
+            if (has_lo) mbar_expect_tx(smem_addr(&halo_bar[0][wb]), row_bytes);
+            if (has_hi) mbar_expect_tx(smem_addr(&halo_bar[1][wb]), row_bytes);
+        }
 #pragma unroll 1
         for (int side = 0; side < 2; ++side) {
             if (side == 0 ? !does_lo : !does_hi) continue;
@@ -134,11 +193,11 @@ resident2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
                 }
                 const double2 o = make_double2(mul_rn(s0, 0.25), mul_rn(s1, 0.25));
                 *reinterpret_cast<double2*>(B + at) = o;
-                if (l == 1 && has_lo) *reinterpret_cast<double2*>(lo_B + 2 + 2 * cp) = o;
-                if (l == mine && has_hi) *reinterpret_cast<double2*>(hi_B + 2 + 2 * cp) = o;
+                const unsigned col = (unsigned)(2 + 2 * cp) * (unsigned)sizeof(double);
+                if (l == 1 && has_lo) send_pair(lo_row[wb] + col, lo_bar[wb], o);
+                if (l == mine && has_hi) send_pair(hi_row[wb] + col, hi_bar[wb], o);
             }
         }
-        cluster.barrier_arrive();   // release: this CTA's halo reads and edge-row writes are done
         if (l0 < l1) {
             for (int cp = cp0; cp < npairs; cp += pw) {
                 int at = l0 * RP + 2 + 2 * cp;
@@ -162,12 +221,27 @@ resident2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
                 }
             }
         }
-        __syncthreads();            // nobody in this CTA still reads A (the next sweep writes it)
-        cluster.barrier_wait();     // acquire: the neighbours' rows have arrived in B's halo rows
-        double* t = A; A = B; B = t;
-        t = lo_A; lo_A = lo_B; lo_B = t;
-        t = hi_A; hi_A = hi_B; hi_B = t;
+        // the neighbours' rows of this sweep (the k-th use of a buffer's mbarriers has parity k & 1)
+        const unsigned parity = (unsigned)(s >> 1) & 1u;
+        if (!gave_up) {
+#pragma unroll 1
+            for (int side = 0; side < 2; ++side) {
+                if (side == 0 ? !has_lo : !has_hi) continue;
+                const unsigned bar = smem_addr(&halo_bar[side][wb]);
+                int polls = 0;
+                while (!mbar_try_wait(bar, parity)) {
+                    if (++polls >= kResMaxPolls) {
+                        gave_up = true;
+                        *timed_out = 1;
+                        break;
+                    }
+                }
+            }
+        }
+        __syncthreads();            // this CTA's rows of B are complete, and nobody still reads A
     }
+    cluster.sync();                 // no row is still on its way to a CTA that is about to leave
+    double* const A = buf[nsweeps & 1];
 
     // ---- write the final state back
     for (int it = tid; it < mine * npairs; it += kResThreads) {

@@ -25,7 +25,7 @@ MODE_FUSED, MODE_PERTASK, MODE_TEMPORAL, MODE_EXCHANGE, MODE_WIDE, MODE_RESIDENT
 MODES = {"fused": MODE_FUSED, "pertask": MODE_PERTASK, "temporal": MODE_TEMPORAL,
          "exchange": MODE_EXCHANGE, "wide": MODE_WIDE, "resident": MODE_RESIDENT}
 
-OK, EINVAL, ENOMEM, ECUDA, ENODEV, ELIMIT = 0, -1, -2, -3, -4, -5
+OK, EINVAL, ENOMEM, ECUDA, ENODEV, ELIMIT, ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
 FLAG_HOST_STAGING, FLAG_CUT_LO, FLAG_CUT_HI = 1, 2, 4
 
 EXPORTS = [

@@ -36,7 +36,7 @@ def test_library_exports_every_declared_symbol(jac):
 
 def test_strerror(jac):
     assert jac.strerror(0) == "ok"
-    for code in (-1, -2, -3, -4, -5):
+    for code in (-1, -2, -3, -4, -5, -6):
         assert jac.strerror(code) not in ("ok", "unknown error code")
     assert jac.strerror(-99) == "unknown error code"
 
@@ -141,7 +141,7 @@ def test_host_staging_flag_adds_two_dense_arrays(jac, n, b, has_f):
         a, c = getattr(plain, name), getattr(L, name)
         assert (list(a) == list(c)) if hasattr(a, "__len__") else (a == c), name
     with pytest.raises(jac.JacError) as e:          # a flag bit the library does not know
-        jac.workspace_bytes(jac.make_desc(n, b, 1, has_f, flags=2))
+        jac.workspace_bytes(jac.make_desc(n, b, 1, has_f, flags=8))
     assert e.value.code == jac.EINVAL
 
 
