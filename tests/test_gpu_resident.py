@@ -83,3 +83,22 @@ def test_resident_refusals(jac):
         with pytest.raises(jac.JacError) as e:
             jac.Jacobi(n, b, 1, False, "resident")
         assert e.value.code == jac.EINVAL
+
+
+def test_a_given_up_wait_is_reported_and_sticks(jac):
+    """The status word a CTA raises when it has polled its mbarrier to the limit is what the host
+    looks at after it has waited for the stream: raise it by hand (no kernel is made to wait) and the
+    next such call returns JAC_ETIMEOUT, as does every call after it."""
+    import ctypes as C
+    import torch
+    with jac.Jacobi((64, 64), (64, 64), 1, False, "resident") as J:
+        J.sweep(3)
+        assert J.residual() >= 0.0
+        word = int(J.layout.off_scratch) // 8 + int(J.layout.partials) + 4
+        J.stream.synchronize()
+        J.workspace.view(torch.int32)[2 * word] = 1
+        out = C.c_double(0.0)
+        L = jac.lib()
+        assert L.jac_residual(J._ctx, C.byref(out)) == jac.ETIMEOUT
+        assert L.jac_sweep(J._ctx, 1) == jac.ETIMEOUT
+        assert "wait" in jac.strerror(jac.ETIMEOUT)
