@@ -389,6 +389,23 @@ int jac_launch_count(const jac_ctx *ctx, int64_t *host_out);
 /* cudaError_t value of the failure that made the context sticky (0 if none). */
 int jac_last_cuda_error(const jac_ctx *ctx);
 
+/* Out-of-bounds evidence of a CHECKED BUILD of the library (compiled with -DJAC_CHECK_BOUNDS: every
+ * global-memory access of the kernels is first compared with the array it belongs to; an access
+ * outside is skipped and the first one recorded; nothing traps).  Waits for the stream, then HOST
+ * outputs: *host_checked = 1 if this build makes the checks, else 0; *host_record = 0 if no access
+ * has left its array since the context was created, else kernel id << 56 | array << 52 | byte
+ * offset from the array's start (low 52 bits, two's complement) of the first one (arrays: 0 the
+ * solution arrays and f, 1 the send buffers, 2 the reduction scratch).  For tests; the ordinary
+ * build always reports 0, 0. */
+int jac_debug_bounds(jac_ctx *ctx, int *host_checked, uint64_t *host_record);
+
+/* Test aid for the checked build: from now on the kernels of this context hold their accesses to
+ * `array` (0, 1, 2 as above) against a range that ends `bytes` before the array's real end, so
+ * that accesses which are in fact legitimate get flagged and skipped -- the way to see the check,
+ * the record and the skipping at work without a single access outside the workspace.  No effect on
+ * the ordinary build.  Errors: JAC_EINVAL for a bad array or more bytes than the array has. */
+int jac_debug_shrink_bounds(jac_ctx *ctx, int array, int64_t bytes);
+
 /* Static, NUL-terminated description of an error code. */
 const char *jac_strerror(int code);
 

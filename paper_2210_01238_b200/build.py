@@ -13,6 +13,7 @@ PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libjac.so"
+CHECKED_LIB = PKG / "libjac_checked.so"      # the same library with every kernel address checked (tests)
 SOURCES = [CSRC / "jac.cu", CSRC / "jac_static.cu"]
 HEADERS = [ROOT / "include" / "jac.h", *sorted(CSRC.glob("*.h")), *sorted(CSRC.glob("*.cuh"))]
 
@@ -30,6 +31,15 @@ def needs_build() -> bool:
         return True
     t = LIB.stat().st_mtime
     return any(p.stat().st_mtime > t for p in [*SOURCES, *HEADERS, Path(__file__)])
+
+
+def build_checked(force: bool = False) -> Path:
+    """The checked build (-DJAC_CHECK_BOUNDS): kernels compare every global address with its array."""
+    if not force and CHECKED_LIB.exists():
+        t = CHECKED_LIB.stat().st_mtime
+        if not any(p.stat().st_mtime > t for p in [*SOURCES, *HEADERS, Path(__file__)]):
+            return CHECKED_LIB
+    return build(out=CHECKED_LIB, defines=["JAC_CHECK_BOUNDS"])
 
 
 def build(force: bool = False, verbose: bool = False, out: Path | None = None, defines=()) -> Path:
@@ -54,3 +64,5 @@ def build(force: bool = False, verbose: bool = False, out: Path | None = None, d
 
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    if "--checked" in sys.argv:
+        print(build_checked(force="--force" in sys.argv))

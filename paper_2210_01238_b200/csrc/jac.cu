@@ -1267,6 +1267,14 @@ int jac_create(const jac_desc* desc, void* dev_workspace, size_t bytes, jac_ctx*
     c->cuda_err = 0;
     c->timed_out = false;
     c->launches = 0;
+    // the ranges a checked build holds every global access against, and its record word
+    c->g.chk_lo[0] = c->ws + L.off_u[0];
+    c->g.chk_hi[0] = c->ws + L.off_send;
+    c->g.chk_lo[1] = c->ws + L.off_send;
+    c->g.chk_hi[1] = c->ws + L.off_scratch;
+    c->g.chk_lo[2] = c->ws + L.off_scratch;
+    c->g.chk_hi[2] = c->ws + L.off_scratch + (L.partials + 32) * (long long)sizeof(double);
+    c->g.chk_rec = reinterpret_cast<unsigned long long*>(c->result + 5);
     const cudaError_t e = cudaMemsetAsync(c->ws, 0, (size_t)L.total_bytes, c->stream);
     if (e != cudaSuccess) {
         delete c;
@@ -1724,6 +1732,29 @@ int jac_launch_count(const jac_ctx* c, int64_t* host_out)
 }
 
 int jac_last_cuda_error(const jac_ctx* c) { return c ? c->cuda_err : 0; }
+
+int jac_debug_shrink_bounds(jac_ctx* c, int array, int64_t bytes)
+{
+    if (!c || array < 0 || array > 2 || bytes < 0 || bytes > c->g.chk_hi[array] - c->g.chk_lo[array]) return JAC_EINVAL;
+    c->g.chk_hi[array] -= bytes;
+    return JAC_OK;
+}
+
+int jac_debug_bounds(jac_ctx* c, int* host_checked, uint64_t* host_record)
+{
+    if (!c || !host_checked || !host_record) return JAC_EINVAL;
+    if (!jac::kChecksBounds) {
+        *host_checked = 0;
+        *host_record = 0;
+        return JAC_OK;
+    }
+    unsigned long long rec = 0;
+    JAC_CK(c, cudaMemcpyAsync(&rec, c->g.chk_rec, sizeof(rec), cudaMemcpyDeviceToHost, c->stream));
+    JAC_CK(c, cudaStreamSynchronize(c->stream));
+    *host_checked = jac::kChecksBounds ? 1 : 0;
+    *host_record = rec;
+    return JAC_OK;
+}
 
 const char* jac_strerror(int code)
 {

@@ -36,4 +36,10 @@ struct JacGeom {
     // jac_solve: where a call that has met its tolerance raises a flag; the sweep and halo kernels of
     // the call's later groups look at it first and return at once (null outside jac_solve)
     const int* stop;
+    // Checked build (JAC_CHECK_BOUNDS): the byte ranges a kernel's global accesses must stay inside --
+    // [0] the solution arrays and f, [1] the send buffers, [2] the reduction scratch -- and the word
+    // that records the first access outside them (which is then skipped).  Unused otherwise.
+    const char* chk_lo[3];
+    const char* chk_hi[3];
+    unsigned long long* chk_rec;
 };

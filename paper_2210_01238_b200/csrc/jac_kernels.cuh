@@ -36,6 +36,45 @@ __device__ __forceinline__ bool solve_stopped(const JacGeom& g) { return g.stop 
 // ask for a line to be brought into L2
 __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];\n" ::"l"(p)); }
 
+// ---------------------------------------------------------------------------------------
+// Checked build.  compute-sanitizer is not always at hand; compiled with -DJAC_CHECK_BOUNDS every
+// global-memory access of the kernels first compares its address range with the array it belongs
+// to (JacGeom::chk_lo / chk_hi).  An access outside is NOT made: the first one is recorded in
+// *JacGeom::chk_rec -- kernel id in bits 56..63, array in bits 52..55, the byte offset from the
+// array's start (two's complement, low 52 bits) below -- loads return 0, and the kernel carries
+// on.  Nothing traps and nothing hangs; jac_debug_bounds reads the record.  In the ordinary build
+// in_bounds() is the constant true and the checks compile to nothing.
+// ---------------------------------------------------------------------------------------
+enum : int { CHK_FIELD = 0, CHK_SEND = 1, CHK_SCRATCH = 2 };
+enum : int { KID_SWEEP2D = 1, KID_SWEEP3D = 2, KID_REDUCE = 3, KID_HALO = 4, KID_CUT = 5, KID_HALO_WIDE = 6,
+             KID_FILL_BOUNDARY = 7, KID_DENSE_COPY = 8, KID_TEMPORAL2D = 9, KID_TEMPORAL3D = 10, KID_RESIDENT = 11 };
+#ifdef JAC_CHECK_BOUNDS
+constexpr bool kChecksBounds = true;
+__device__ __forceinline__ bool in_bounds(const JacGeom& g, const void* p, int bytes, int which, int kid) {
+    const char* a = static_cast<const char*>(p);
+    if (a >= g.chk_lo[which] && a + bytes <= g.chk_hi[which]) return true;
+    const unsigned long long off = (unsigned long long)(a - g.chk_lo[which]) & ((1ULL << 52) - 1);
+    atomicCAS(g.chk_rec, 0ULL, ((unsigned long long)kid << 56) | ((unsigned long long)which << 52) | off);
+    return false;
+}
+#else
+constexpr bool kChecksBounds = false;
+__device__ __forceinline__ constexpr bool in_bounds(const JacGeom&, const void*, int, int, int) { return true; }
+#endif
+// global loads and stores that go through the check
+__device__ __forceinline__ double g_ld(const JacGeom& g, const double* p, int which, int kid) {
+    return in_bounds(g, p, 8, which, kid) ? *p : 0.0;
+}
+__device__ __forceinline__ void g_st(const JacGeom& g, double* p, double v, int which, int kid) {
+    if (in_bounds(g, p, 8, which, kid)) *p = v;
+}
+__device__ __forceinline__ double2 g_ld2(const JacGeom& g, const double* p, int which, int kid) {
+    return in_bounds(g, p, 16, which, kid) ? *reinterpret_cast<const double2*>(p) : make_double2(0.0, 0.0);
+}
+__device__ __forceinline__ void g_st2(const JacGeom& g, double* p, double2 v, int which, int kid) {
+    if (in_bounds(g, p, 16, which, kid)) *reinterpret_cast<double2*>(p) = v;
+}
+
 // NV consecutive doubles held by one thread (NV = 1 or 2; NV = 2 uses one 128-bit access).
 template <int NV> struct Vec { double v[NV]; };
 
@@ -51,6 +90,14 @@ template <int NV> __device__ __forceinline__ void store_vec(double* p, const Vec
 template <> __device__ __forceinline__ void store_vec<1>(double* p, const Vec<1>& a) { *p = a.v[0]; }
 template <> __device__ __forceinline__ void store_vec<2>(double* p, const Vec<2>& a) {
     *reinterpret_cast<double2*>(p) = make_double2(a.v[0], a.v[1]);
+}
+
+template <int NV> __device__ __forceinline__ Vec<NV> g_load_vec(const JacGeom& g, const double* p, int kid) {
+    if (!in_bounds(g, p, 8 * NV, CHK_FIELD, kid)) { Vec<NV> z; for (int q = 0; q < NV; ++q) z.v[q] = 0.0; return z; }
+    return load_vec<NV>(p);
+}
+template <int NV> __device__ __forceinline__ void g_store_vec(const JacGeom& g, double* p, const Vec<NV>& a, int kid) {
+    if (in_bounds(g, p, 8 * NV, CHK_FIELD, kid)) store_vec<NV>(p, a);
 }
 
 // Sum of a per-thread value over the CTA in a fixed order: lanes by shuffle, then warps in
@@ -154,8 +201,8 @@ sweep2d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
         // whole warp waits for DRAM in every row
         const bool far_w = op_pulls(OP) && off_w != -1, far_e = op_pulls(OP) && off_e != NV;
 
-        Vec<NV> S = load_vec<NV>(ub + (j0 == 0 ? off_s0 : (long long)(j0 - 1) * PX));
-        Vec<NV> Cc = load_vec<NV>(ub + (long long)j0 * PX);
+        Vec<NV> S = g_load_vec<NV>(g, ub + (j0 == 0 ? off_s0 : (long long)(j0 - 1) * PX), KID_SWEEP2D);
+        Vec<NV> Cc = g_load_vec<NV>(g, ub + (long long)j0 * PX, KID_SWEEP2D);
 #pragma unroll 4
         for (int j = j0; j < j1; ++j) {
             const long long ro = (long long)j * PX;
@@ -163,11 +210,11 @@ sweep2d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
                 if (far_w) prefetch_l2(ub + ro + 8 * PX + off_w);
                 if (far_e) prefetch_l2(ub + ro + 8 * PX + off_e);
             }
-            const Vec<NV> N = load_vec<NV>(ub + ro + ((op_pulls(OP) && j + 1 == g.by) ? off_n1 : PX));
-            const double w = ub[ro + off_w];
-            const double e = ub[ro + off_e];
+            const Vec<NV> N = g_load_vec<NV>(g, ub + ro + ((op_pulls(OP) && j + 1 == g.by) ? off_n1 : PX), KID_SWEEP2D);
+            const double w = g_ld(g, ub + ro + off_w, CHK_FIELD, KID_SWEEP2D);
+            const double e = g_ld(g, ub + ro + off_e, CHK_FIELD, KID_SWEEP2D);
             Vec<NV> ff;
-            if (HAS_F) ff = load_vec<NV>(fb + ro);
+            if (HAS_F) ff = g_load_vec<NV>(g, fb + ro, KID_SWEEP2D);
             Vec<NV> o;
 #pragma unroll
             for (int q = 0; q < NV; ++q) {
@@ -182,14 +229,14 @@ sweep2d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
                 if (op_stores(OP)) o.v[q] = mul_rn(s, 0.25);
                 if (op_ext(OP) && !(xin[q] && gy0 + j >= 0 && gy0 + j < g.ny)) o.v[q] = Cc.v[q];
             }
-            if (op_stores(OP)) store_vec<NV>(ob + ro, o);
+            if (op_stores(OP)) g_store_vec<NV>(g, ob + ro, o, KID_SWEEP2D);
             S = Cc;
             Cc = N;
         }
     }
     if (op_sums(OP)) {
         const double total = block_sum(acc);
-        if (threadIdx.x == 0) partials[blockIdx.x] = total;
+        if (threadIdx.x == 0) g_st(g, partials + blockIdx.x, total, CHK_SCRATCH, KID_SWEEP2D);
     }
 }
 
@@ -257,8 +304,8 @@ sweep3d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
         // far west / east neighbours (the next block's column): asked for a few planes ahead, as in 2D
         const bool far_w = op_pulls(OP) && off_w != -1, far_e = op_pulls(OP) && off_e != NV;
 
-        Vec<NV> D = load_vec<NV>(ub + (k0 == 0 ? off_d0 : (long long)(k0 - 1) * PXY));
-        Vec<NV> Cc = load_vec<NV>(ub + (long long)k0 * PXY);
+        Vec<NV> D = g_load_vec<NV>(g, ub + (k0 == 0 ? off_d0 : (long long)(k0 - 1) * PXY), KID_SWEEP3D);
+        Vec<NV> Cc = g_load_vec<NV>(g, ub + (long long)k0 * PXY, KID_SWEEP3D);
 #pragma unroll 2
         for (int k = k0; k < k1; ++k) {
             const long long po = (long long)k * PXY;
@@ -266,13 +313,13 @@ sweep3d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
                 if (far_w) prefetch_l2(ub + po + 4 * PXY + off_w);
                 if (far_e) prefetch_l2(ub + po + 4 * PXY + off_e);
             }
-            const Vec<NV> U = load_vec<NV>(ub + po + ((op_pulls(OP) && k + 1 == g.bz) ? off_u1 : PXY));
-            const Vec<NV> S = load_vec<NV>(ub + po + off_s);
-            const Vec<NV> N = load_vec<NV>(ub + po + off_n);
-            const double w = ub[po + off_w];
-            const double e = ub[po + off_e];
+            const Vec<NV> U = g_load_vec<NV>(g, ub + po + ((op_pulls(OP) && k + 1 == g.bz) ? off_u1 : PXY), KID_SWEEP3D);
+            const Vec<NV> S = g_load_vec<NV>(g, ub + po + off_s, KID_SWEEP3D);
+            const Vec<NV> N = g_load_vec<NV>(g, ub + po + off_n, KID_SWEEP3D);
+            const double w = g_ld(g, ub + po + off_w, CHK_FIELD, KID_SWEEP3D);
+            const double e = g_ld(g, ub + po + off_e, CHK_FIELD, KID_SWEEP3D);
             Vec<NV> ff;
-            if (HAS_F) ff = load_vec<NV>(fb + po);
+            if (HAS_F) ff = g_load_vec<NV>(g, fb + po, KID_SWEEP3D);
             Vec<NV> o;
 #pragma unroll
             for (int q = 0; q < NV; ++q) {
@@ -288,14 +335,14 @@ sweep3d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
                 if (op_stores(OP)) o.v[q] = mul_rn(s, c6);
                 if (op_ext(OP) && !(xyin[q] && gz0 + k >= 0 && gz0 + k < g.nz)) o.v[q] = Cc.v[q];
             }
-            if (op_stores(OP)) store_vec<NV>(ob + po, o);
+            if (op_stores(OP)) g_store_vec<NV>(g, ob + po, o, KID_SWEEP3D);
             D = Cc;
             Cc = U;
         }
     }
     if (op_sums(OP)) {
         const double total = block_sum(acc);
-        if (threadIdx.x == 0 && threadIdx.y == 0) partials[blockIdx.x] = total;
+        if (threadIdx.x == 0 && threadIdx.y == 0) g_st(g, partials + blockIdx.x, total, CHK_SCRATCH, KID_SWEEP3D);
     }
 }
 
@@ -458,7 +505,7 @@ halo_kernel(double* __restrict__ u, double* __restrict__ send, const JacGeom g,
             if (h <= 2) {
 #pragma unroll
                 for (int c = 0; c < 2; ++c)
-                    if (c < h) v[k][c] = OP == HALO_UNPACK ? buf[(long long)R * h + c] : src_blk[cell[k] + lo_src + c];
+                    if (c < h) v[k][c] = OP == HALO_UNPACK ? g_ld(g, buf + (long long)R * h + c, CHK_SEND, KID_HALO) : g_ld(g, src_blk + cell[k] + lo_src + c, CHK_FIELD, KID_HALO);
             }
         }
 #pragma unroll
@@ -469,34 +516,34 @@ halo_kernel(double* __restrict__ u, double* __restrict__ send, const JacGeom g,
                 if (OP != HALO_UNPACK) {
 #pragma unroll
                     for (int c = 0; c < 2; ++c)
-                        if (c < h) buf[(long long)R * h + c] = v[k][c];
+                        if (c < h) g_st(g, buf + (long long)R * h + c, v[k][c], CHK_SEND, KID_HALO);
                 }
                 if (OP != HALO_PACK) {
                     if (sector) {
-                        double2* sec = reinterpret_cast<double2*>(own + cell[k] + ((face & 1) ? ext : -4));
+                        double* sec = own + cell[k] + ((face & 1) ? ext : -4);
                         if (face & 1) {      // the ghosts are the first h cells of the sector
-                            sec[0] = make_double2(v[k][0], h == 2 ? v[k][1] : 0.0);
-                            sec[1] = make_double2(0.0, 0.0);
+                            g_st2(g, sec, make_double2(v[k][0], h == 2 ? v[k][1] : 0.0), CHK_FIELD, KID_HALO);
+                            g_st2(g, sec + 2, make_double2(0.0, 0.0), CHK_FIELD, KID_HALO);
                         } else {             // the last h
-                            sec[0] = make_double2(0.0, 0.0);
-                            sec[1] = h == 2 ? make_double2(v[k][0], v[k][1]) : make_double2(0.0, v[k][0]);
+                            g_st2(g, sec, make_double2(0.0, 0.0), CHK_FIELD, KID_HALO);
+                            g_st2(g, sec + 2, h == 2 ? make_double2(v[k][0], v[k][1]) : make_double2(0.0, v[k][0]), CHK_FIELD, KID_HALO);
                         }
                     } else {
 #pragma unroll
                         for (int c = 0; c < 2; ++c)
-                            if (c < h) own[cell[k] + lo_dst + c] = v[k][c];
+                            if (c < h) g_st(g, own + cell[k] + lo_dst + c, v[k][c], CHK_FIELD, KID_HALO);
                     }
                 }
             } else {                         // wider strips (h <= 8): the row's cells, loads before stores
                 double w[8];
 #pragma unroll
                 for (int c = 0; c < 8; ++c)
-                    if (c < h) w[c] = OP == HALO_UNPACK ? buf[(long long)R * h + c] : src_blk[cell[k] + lo_src + c];
+                    if (c < h) w[c] = OP == HALO_UNPACK ? g_ld(g, buf + (long long)R * h + c, CHK_SEND, KID_HALO) : g_ld(g, src_blk + cell[k] + lo_src + c, CHK_FIELD, KID_HALO);
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
                     if (c >= h) continue;
-                    if (OP != HALO_UNPACK) buf[(long long)R * h + c] = w[c];
-                    if (OP != HALO_PACK) own[cell[k] + lo_dst + c] = w[c];
+                    if (OP != HALO_UNPACK) g_st(g, buf + (long long)R * h + c, w[c], CHK_SEND, KID_HALO);
+                    if (OP != HALO_PACK) g_st(g, own + cell[k] + lo_dst + c, w[c], CHK_FIELD, KID_HALO);
                 }
             }
         }
@@ -523,9 +570,9 @@ halo_kernel(double* __restrict__ u, double* __restrict__ send, const JacGeom g,
             const unsigned x0 = vec ? 2 * vi : vi;
             for (unsigned c = 0; c < (vec ? 2u : 1u); ++c) {
                 const long long bi = (long long)L * ex + x0 + c;
-                const double w = OP == HALO_UNPACK ? buf[bi] : src_blk[so + x0 + c];
-                if (OP != HALO_UNPACK) buf[bi] = w;
-                if (OP != HALO_PACK) own[dn + x0 + c] = w;
+                const double w = OP == HALO_UNPACK ? g_ld(g, buf + bi, CHK_SEND, KID_HALO) : g_ld(g, src_blk + so + x0 + c, CHK_FIELD, KID_HALO);
+                if (OP != HALO_UNPACK) g_st(g, buf + bi, w, CHK_SEND, KID_HALO);
+                if (OP != HALO_PACK) g_st(g, own + dn + x0 + c, w, CHK_FIELD, KID_HALO);
             }
         }
         return;
@@ -551,20 +598,20 @@ halo_kernel(double* __restrict__ u, double* __restrict__ send, const JacGeom g,
             dst_off[k] = (axis == 1 ? (long long)a * PXY + (long long)(lo_dst + (int)r) * PX
                                     : (long long)(lo_dst + (int)a) * PXY + (long long)r * PX) + x0;
             buf_off[k] = (long long)L * ex + x0;
-            if (vec) w2[k] = OP == HALO_UNPACK ? *reinterpret_cast<const double2*>(buf + buf_off[k])
-                                               : *reinterpret_cast<const double2*>(src_blk + so + x0);
-            else w1[k] = OP == HALO_UNPACK ? buf[buf_off[k]] : src_blk[so + x0];
+            if (vec) w2[k] = OP == HALO_UNPACK ? g_ld2(g, buf + buf_off[k], CHK_SEND, KID_HALO)
+                                               : g_ld2(g, src_blk + so + x0, CHK_FIELD, KID_HALO);
+            else w1[k] = OP == HALO_UNPACK ? g_ld(g, buf + buf_off[k], CHK_SEND, KID_HALO) : g_ld(g, src_blk + so + x0, CHK_FIELD, KID_HALO);
         }
 #pragma unroll
         for (int k = 0; k < kHaloUnits; ++k) {
             const unsigned L = Lb + (unsigned)k * TL;
             if (L >= nlines) continue;
             if (vec) {
-                if (OP != HALO_UNPACK) *reinterpret_cast<double2*>(buf + buf_off[k]) = w2[k];
-                if (OP != HALO_PACK) *reinterpret_cast<double2*>(own + dst_off[k]) = w2[k];
+                if (OP != HALO_UNPACK) g_st2(g, buf + buf_off[k], w2[k], CHK_SEND, KID_HALO);
+                if (OP != HALO_PACK) g_st2(g, own + dst_off[k], w2[k], CHK_FIELD, KID_HALO);
             } else {
-                if (OP != HALO_UNPACK) buf[buf_off[k]] = w1[k];
-                if (OP != HALO_PACK) own[dst_off[k]] = w1[k];
+                if (OP != HALO_UNPACK) g_st(g, buf + buf_off[k], w1[k], CHK_SEND, KID_HALO);
+                if (OP != HALO_PACK) g_st(g, own + dst_off[k], w1[k], CHK_FIELD, KID_HALO);
             }
         }
     }
@@ -594,16 +641,17 @@ cut_kernel(double* __restrict__ u, double* __restrict__ buf, const JacGeom g, co
     const int lo = UNPACK ? ((face & 1) ? ext : -g.h) : ((face & 1) ? ext - g.h : 0);
     double* ub = u + blk * g.block_stride + g.origin;
     double* bp = buf + m * slot;
-    if ((be.x & 1) == 0) {
-        double2* cell = reinterpret_cast<double2*>(ub + strip_offset(g, be, face, e, lo));
+    // (the block side goes through the checked-build test; the plane may be another context's buffer)
+    if ((be.x & 1) == 0 && (g.PX & 1) == 0) {
+        double* cell = ub + strip_offset(g, be, face, e, lo);
         double2* sl = reinterpret_cast<double2*>(bp + e);
-        if (UNPACK) *cell = *sl; else *sl = *cell;
+        if (UNPACK) g_st2(g, cell, *sl, CHK_FIELD, KID_CUT); else *sl = g_ld2(g, cell, CHK_FIELD, KID_CUT);
     } else {
         double* c0 = ub + strip_offset(g, be, face, e, lo);
-        if (UNPACK) *c0 = bp[e]; else bp[e] = *c0;
+        if (UNPACK) g_st(g, c0, bp[e], CHK_FIELD, KID_CUT); else bp[e] = g_ld(g, c0, CHK_FIELD, KID_CUT);
         if (e + 1 < n) {
             double* c1 = ub + strip_offset(g, be, face, e + 1, lo);
-            if (UNPACK) *c1 = bp[e + 1]; else bp[e + 1] = *c1;
+            if (UNPACK) g_st(g, c1, bp[e + 1], CHK_FIELD, KID_CUT); else bp[e + 1] = g_ld(g, c1, CHK_FIELD, KID_CUT);
         }
     }
 }
@@ -646,8 +694,10 @@ halo_wide_kernel(double* __restrict__ arr, double* __restrict__ send, const JacG
         const unsigned k = q / wy; y = (int)(q - k * wy) - h; z = (int)k + lo;
     }
     double* cell = arr + (long long)blk * g.block_stride + g.origin + z * g.PXY + y * g.PX + x;
-    if (UNPACK) *cell = send[(long long)bp.nb * g.send_stride + g.face_off[face ^ 1] + e];
-    else send[(long long)blk * g.send_stride + g.face_off[face] + e] = *cell;
+    if (UNPACK) g_st(g, cell, g_ld(g, send + (long long)bp.nb * g.send_stride + g.face_off[face ^ 1] + e, CHK_SEND, KID_HALO_WIDE),
+                     CHK_FIELD, KID_HALO_WIDE);
+    else g_st(g, send + (long long)blk * g.send_stride + g.face_off[face] + e, g_ld(g, cell, CHK_FIELD, KID_HALO_WIDE),
+              CHK_SEND, KID_HALO_WIDE);
 }
 
 // Dirichlet value into the ghost strip of `face` of every block on that domain face, in both
@@ -678,8 +728,8 @@ fill_boundary_kernel(double* __restrict__ u0, double* __restrict__ u1, const Jac
     for (long long e = (long long)chunk * blockDim.x + threadIdx.x; e < n;
          e += (long long)chunks * blockDim.x) {
         const long long off = base + strip_offset(g, be, face, e, lo);
-        u0[off] = value;
-        u1[off] = value;
+        g_st(g, u0 + off, value, CHK_FIELD, KID_FILL_BOUNDARY);
+        g_st(g, u1 + off, value, CHK_FIELD, KID_FILL_BOUNDARY);
     }
 }
 
@@ -702,8 +752,8 @@ dense_copy_kernel(double* __restrict__ blocks, double* __restrict__ dense, const
     const long long bxi = gi / g.bx;
     double* bp = blocks + row_off + bxi * g.block_stride + (gi - bxi * g.bx);
     double* dp = dense + row * g.nx + gi;
-    if (TO_BLOCKS) store_vec<NV>(bp, load_vec<NV>(dp));
-    else store_vec<NV>(dp, load_vec<NV>(bp));
+    if (TO_BLOCKS) g_store_vec<NV>(g, bp, load_vec<NV>(dp), KID_DENSE_COPY);
+    else store_vec<NV>(dp, g_load_vec<NV>(g, bp, KID_DENSE_COPY));
 }
 
 // ---------------------------------------------------------------------------------------
@@ -822,6 +872,9 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src)
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem_src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+__device__ __forceinline__ void g_cp_async16(const JacGeom& g, void* smem_dst, const double* gmem_src, int kid) {
+    if (in_bounds(g, gmem_src, 16, CHK_FIELD, kid)) cp_async16(smem_dst, gmem_src);
+}
 template <int N> __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
 }
@@ -860,16 +913,16 @@ struct TemporalCtx {
 // right-hand side, f row r goes into the f ring (F_RING: stages follow the u stages of the warp),
 // or is at least requested into L2 for the loads that follow DEPTH steps later.
 template <int P, bool HAS_F, bool F_RING>
-__device__ __forceinline__ void issue_row(const TemporalCtx& c, int r, const RowCursor& cur) {
+__device__ __forceinline__ void issue_row(const TemporalCtx& c, const JacGeom& g, int r, const RowCursor& cur) {
     constexpr int SC = temporal_stage_chunks(P);
     if (r >= 0 && r < c.ny && r < c.in_end) {
         const int st = ((r - c.r0) % kTemporalDepth) * SC;
-        if (c.copy_a) cp_async16(c.dst_a + st, c.src_a + cur.off);
-        if (P == 4 && c.copy_b) cp_async16(c.dst_b + st, c.src_b + cur.off);
+        if (c.copy_a) g_cp_async16(g, c.dst_a + st, c.src_a + cur.off, KID_TEMPORAL2D);
+        if (P == 4 && c.copy_b) g_cp_async16(g, c.dst_b + st, c.src_b + cur.off, KID_TEMPORAL2D);
         if (F_RING) {
             const int fs = (kTemporalDepth + ((r - c.r0) % kTemporalFDepth)) * SC;
-            if (c.copy_a) cp_async16(c.dst_a + fs, c.src_a + c.fdelta + cur.off);
-            if (P == 4 && c.copy_b) cp_async16(c.dst_b + fs, c.src_b + c.fdelta + cur.off);
+            if (c.copy_a) g_cp_async16(g, c.dst_a + fs, c.src_a + c.fdelta + cur.off, KID_TEMPORAL2D);
+            if (P == 4 && c.copy_b) g_cp_async16(g, c.dst_b + fs, c.src_b + c.fdelta + cur.off, KID_TEMPORAL2D);
         } else if (HAS_F && !c.xout) {
             prefetch_line(c.fb + cur.off);
         }
@@ -942,7 +995,7 @@ __device__ __forceinline__ void temporal_level(RowN<temporal_points(T)> (&win)[T
     if (s < T) {
         win[s][slot3(PH, d)] = o;
     } else if (in_strip) {
-        store_rown<P>(c.ob + out_cur.off, o);
+        if (in_bounds(g, c.ob + out_cur.off, 8 * P, CHK_FIELD, KID_TEMPORAL2D)) store_rown<P>(c.ob + out_cur.off, o);
     }
     // the points of the strip's output region: every interior point is in exactly one, and every
     // level is exact there
@@ -975,7 +1028,7 @@ __device__ __forceinline__ void temporal_step(RowN<temporal_points(T)> (&win)[T]
     win[0][PH] = take_row<temporal_points(T), EDGE>(c, r);
     TemporalLevels<T, HAS_F, RES, PH, EDGE, 1>::run(win, c, g, r, out_cur, acc);
     __syncwarp();                                    // everyone has read the stages before they are refilled
-    issue_row<temporal_points(T), HAS_F, F_RING>(c, r + kTemporalDepth, load_cur);
+    issue_row<temporal_points(T), HAS_F, F_RING>(c, g, r + kTemporalDepth, load_cur);
     load_cur.advance(g, c.brs);
     out_cur.advance(g, c.brs);
 }
@@ -1059,7 +1112,7 @@ temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
     // fill the ring with the first DEPTH rows
 #pragma unroll 1
     for (int k = 0; k < kTemporalDepth; ++k) {
-        issue_row<P, HAS_F, F_RING>(c, c.r0 + k, load_cur);
+        issue_row<P, HAS_F, F_RING>(c, g, c.r0 + k, load_cur);
         load_cur.advance(g, c.brs);
     }
 
@@ -1073,7 +1126,7 @@ temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
     if (RES != kResNone) {
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) acc = add_rn(acc, __shfl_down_sync(0xffffffffu, acc, off));
-        if (lane == 0) partials[wid] = acc;
+        if (lane == 0) g_st(g, partials + wid, acc, CHK_SCRATCH, KID_TEMPORAL2D);
     }
 }
 

@@ -114,9 +114,9 @@ resident2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
         const int gy = y0 + l - 1;
         if (mine == 0 || (l == 0 && !has_lo) || (l == mine + 1 && !has_hi)) continue;
         const long long off = resident_offset(g, 2 * cp, gy);
-        *reinterpret_cast<double2*>(buf[0] + l * RP + 2 + 2 * cp) = *reinterpret_cast<const double2*>(u + off);
+        *reinterpret_cast<double2*>(buf[0] + l * RP + 2 + 2 * cp) = g_ld2(g, u + off, CHK_FIELD, KID_RESIDENT);
         if (HAS_F && l >= 1 && l <= mine)
-            *reinterpret_cast<double2*>(fs + (l - 1) * RP + 2 + 2 * cp) = *reinterpret_cast<const double2*>(f + off);
+            *reinterpret_cast<double2*>(fs + (l - 1) * RP + 2 + 2 * cp) = g_ld2(g, f + off, CHK_FIELD, KID_RESIDENT);
     }
     // where the neighbours keep the halo row that mirrors this slab's first / last row, and the
     // mbarrier that counts its arrival there, per buffer: this slab's first row goes to the upper
@@ -246,8 +246,8 @@ resident2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
     // ---- write the final state back
     for (int it = tid; it < mine * npairs; it += kResThreads) {
         const int l = it / npairs + 1, cp = it - (l - 1) * npairs;
-        *reinterpret_cast<double2*>(un + resident_offset(g, 2 * cp, y0 + l - 1)) =
-            *reinterpret_cast<const double2*>(A + l * RP + 2 + 2 * cp);
+        g_st2(g, un + resident_offset(g, 2 * cp, y0 + l - 1), *reinterpret_cast<const double2*>(A + l * RP + 2 + 2 * cp),
+              CHK_FIELD, KID_RESIDENT);
     }
 }
 

@@ -133,7 +133,7 @@ __device__ __forceinline__ void t3_issue(const T3& c, const JacGeom& g, const do
         for (int r = 0; r < kT3Rows; ++r) {
             double cval = 0.0;
             if (EDGE && t3_outside(c, g, p, r, &cval)) sts_pair(st + r * kT3Cols, pair_of(cval));
-            else cp_async16(st + r * kT3Cols, u + cur.off + c.row_off[r]);
+            else g_cp_async16(g, st + r * kT3Cols, u + cur.off + c.row_off[r], KID_TEMPORAL3D);
         }
     }
     if (HAS_F) {
@@ -143,7 +143,7 @@ __device__ __forceinline__ void t3_issue(const T3& c, const JacGeom& g, const do
 #pragma unroll
             for (int r = 0; r < kT3Rows; ++r) {
                 double cval = 0.0;
-                if (!(EDGE && t3_outside(c, g, q, r, &cval))) cp_async16(st + r * kT3Cols, f + f_off + c.row_off[r]);
+                if (!(EDGE && t3_outside(c, g, q, r, &cval))) g_cp_async16(g, st + r * kT3Cols, f + f_off + c.row_off[r], KID_TEMPORAL3D);
             }
         }
     }
@@ -212,7 +212,7 @@ __device__ __forceinline__ void t3_upper_levels(Rows2 (&win)[kT3MaxT][3], const 
             t3_level<HAS_F, EDGE, RES == kResBeforeLast>(c, g, D, M, U, below, above, q, fp, o, live, acc);
 #pragma unroll
             for (int r = 0; r < kT3Rows; ++r)
-                if (live[r]) sts_pair(un + out_cur.off + c.row_off[r], o.row[r]);
+                if (live[r]) g_st2(g, un + out_cur.off + c.row_off[r], make_double2(o.row[r].v[0], o.row[r].v[1]), CHK_FIELD, KID_TEMPORAL3D);
         } else {
             Rows2& o = win[s][slot3(PH, -s)];
             const bool none[kT3Rows] = {false, false};
@@ -267,7 +267,7 @@ __device__ __forceinline__ void t3_step(Rows2 (&win)[kT3MaxT][3], const T3& c, c
         t3_level<HAS_F, EDGE, RES != kResNone>(c, g, D, M, U, below, above, q, fp, o, live, acc);
 #pragma unroll
         for (int r = 0; r < kT3Rows; ++r)
-            if (live[r]) sts_pair(un + out_cur.off + c.row_off[r], o.row[r]);
+            if (live[r]) g_st2(g, un + out_cur.off + c.row_off[r], make_double2(o.row[r].v[0], o.row[r].v[1]), CHK_FIELD, KID_TEMPORAL3D);
     } else {
         Rows2& o = win[1][slot3(PH, -1)];
         // the residual of the state the launch reads: over the tile's output cells, which every
@@ -414,7 +414,7 @@ temporal3d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
     if (RES != kResNone) {
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) acc = add_rn(acc, __shfl_down_sync(0xffffffffu, acc, off));
-        if (lane == 0) partials[(long long)blockIdx.x * kT3Warps + warp] = acc;
+        if (lane == 0) g_st(g, partials + (long long)blockIdx.x * kT3Warps + warp, acc, CHK_SCRATCH, KID_TEMPORAL3D);
     }
 }
 

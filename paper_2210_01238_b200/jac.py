@@ -37,7 +37,7 @@ EXPORTS = [
     "jac_sweep_residual", "jac_solve", "jac_exchange_wide", "jac_get_wide_buffer",
     "jac_set_u_async", "jac_get_u_async", "jac_residual_async", "jac_exchange_halos",
     "jac_pack_cut", "jac_unpack_cut", "jac_sweep_begin", "jac_sweep_end", "jac_cut_info",
-    "jac_residual_sumsq_async", "jac_residual_sweep_async",
+    "jac_residual_sumsq_async", "jac_residual_sweep_async", "jac_debug_bounds", "jac_debug_shrink_bounds",
 ]
 
 
@@ -106,6 +106,8 @@ def lib() -> C.CDLL:
         L.jac_launch_count.argtypes = [vp, C.POINTER(C.c_int64)]
         L.jac_sweeps_per_launch.argtypes = [vp, C.POINTER(C.c_int)]
         L.jac_last_cuda_error.argtypes = [vp]
+        L.jac_debug_bounds.argtypes = [vp, C.POINTER(C.c_int), C.POINTER(C.c_uint64)]
+        L.jac_debug_shrink_bounds.argtypes = [vp, C.c_int, C.c_int64]
         L.jac_strerror.argtypes = [C.c_int]
         L.jac_residual_dense_static.argtypes = [C.c_int, C.POINTER(C.c_int64), vp, vp,
                                                 C.POINTER(C.c_double), vp, dp]
@@ -222,11 +224,24 @@ class Jacobi:
                 detail = f" [cudaError {lib().jac_last_cuda_error(self._ctx)}]"
             raise JacError(rc, what + detail)
 
+    def bounds_record(self):
+        """(does this build of the library check its kernels' addresses, record of the first access
+        outside its array or 0) -- see ``jac_debug_bounds``."""
+        checked, rec = C.c_int(0), C.c_uint64(0)
+        self._call("jac_debug_bounds", lib().jac_debug_bounds(self._ctx, C.byref(checked), C.byref(rec)))
+        return bool(checked.value), int(rec.value)
+
     def close(self):
         if getattr(self, "_ctx", None):
+            # a checked build (JAC_LIB pointing at one) speaks up when a context is closed
+            checked, rec = C.c_int(0), C.c_uint64(0)
+            rc = lib().jac_debug_bounds(self._ctx, C.byref(checked), C.byref(rec))
             lib().jac_destroy(self._ctx)
             self._ctx = C.c_void_p()
             self.workspace = None
+            if rc == OK and checked.value and rec.value:
+                raise JacError(EINVAL, f"a kernel reached outside its array: kernel {rec.value >> 56}, array "
+                                       f"{(rec.value >> 52) & 15}, byte offset {rec.value & ((1 << 52) - 1):#x}")
 
     def __del__(self):
         try:
