@@ -103,7 +103,9 @@ extern "C" {
                                    array is free and overlaps whatever is queued on the caller's
                                    stream (the previous job's sweeps and copy out); the caller's
                                    stream waits for it before it touches the blocks.  For callers
-                                   that stream jobs through a context from pinned host memory     */
+                                   that stream jobs through a context from page-locked (pinned or
+                                   registered) host memory; pageable host arrays are still accepted
+                                   and take the per-block copies on the caller's stream            */
 
 #define JAC_FLAG_CUT_LO 2       /* the context is one SLAB of a larger domain that is cut into slabs of  */
 #define JAC_FLAG_CUT_HI 4       /* whole block planes along the slowest axis (y in 2D, z in 3D), one slab

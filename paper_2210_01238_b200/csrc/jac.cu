@@ -671,14 +671,29 @@ int staged_out(jac_ctx* c, double* arr, double* host, bool wait)
     return JAC_OK;
 }
 
-// dense host array <-> blocks, by whichever route the context has
+// is this host memory page-locked (allocated or registered with CUDA)?  Only then is a copy on a
+// stream of the library's own ordered by the events around it: the runtime moves pageable memory
+// through a staging buffer of its own, on its own schedule.
+bool is_pinned(const void* host)
+{
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, host) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return at.type == cudaMemoryTypeHost;
+}
+
+// dense host array <-> blocks, by whichever route the context has (the staging arrays serve
+// page-locked host memory; pageable memory takes the per-block copies on the caller's stream)
 int host_to_blocks(jac_ctx* c, double* arr, const double* host, bool wait)
 {
-    return c->stage_in ? staged_in(c, arr, host, wait) : copy_dense_host(c, arr, const_cast<double*>(host), true, wait);
+    return (c->stage_in && is_pinned(host)) ? staged_in(c, arr, host, wait)
+                                            : copy_dense_host(c, arr, const_cast<double*>(host), true, wait);
 }
 int blocks_to_host(jac_ctx* c, double* arr, double* host, bool wait)
 {
-    return c->stage_out ? staged_out(c, arr, host, wait) : copy_dense_host(c, arr, host, false, wait);
+    return (c->stage_out && is_pinned(host)) ? staged_out(c, arr, host, wait) : copy_dense_host(c, arr, host, false, wait);
 }
 
 int usable(jac_ctx* c)
@@ -1291,6 +1306,14 @@ int jac_create(const jac_desc* desc, void* dev_workspace, size_t bytes, jac_ctx*
             cudaEventCreateWithFlags(&c->ev_in_ready, cudaEventDisableTiming) != cudaSuccess ||
             cudaEventCreateWithFlags(&c->ev_in_free, cudaEventDisableTiming) != cudaSuccess ||
             cudaEventCreateWithFlags(&c->ev_out_done, cudaEventDisableTiming) != cudaSuccess) {
+            cudaGetLastError();
+            release_copy_objects(c);
+            delete c;
+            return JAC_ECUDA;
+        }
+        // the copy stream must not run ahead of the clearing of the workspace queued above on the
+        // caller's stream: the staging array counts as free only once that has been done
+        if (cudaEventRecord(c->ev_in_free, c->stream) != cudaSuccess) {
             cudaGetLastError();
             release_copy_objects(c);
             delete c;

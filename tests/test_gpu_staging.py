@@ -80,3 +80,19 @@ def test_jobs_queued_back_to_back_from_pinned_memory(jac, orc):
     assert np.array_equal(outs[2].numpy(), w2)
     for got, want in zip(norms.tolist(), (r0, r1, r2)):
         assert abs(got - want) <= 1e-10 * want
+
+
+def test_first_copy_in_does_not_overtake_the_clearing_of_the_workspace(jac):
+    """jac_create clears the workspace on the caller's stream; a copy in from pinned memory right
+    after it runs on the context's own stream and must still come after that clearing.  With a
+    workspace of a few GB the clearing takes long enough for a copy that overtook it to lose data:
+    at u = 0 the residual norm is the norm of f, to the last bit of the reduction."""
+    import torch
+    n, b = (384, 384, 384), (128, 128, 128)
+    f = np.random.default_rng(9).standard_normal((n[2], n[1], n[0]))
+    fp = torch.from_numpy(f).pin_memory()
+    with jac.Jacobi(n, b, 1, True, "temporal", flags=jac.FLAG_HOST_STAGING) as J:
+        J._call("jac_set_f", jac.lib().jac_set_f(J._ctx, fp.data_ptr()))
+        got = J.residual()
+    want = float(np.sqrt(np.sum(f * f)))
+    assert abs(got - want) <= 1e-12 * want
