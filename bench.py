@@ -48,20 +48,25 @@ L2_BYTES = 126e6
 # launch (a smaller case of the same workload, named beside each entry), scaled to the workload by
 # its points -- traffic is proportional to the points: every strip or tile reads and writes its own
 # part of the grid once per launch.
-SWEEP_SOURCES = ("jac_kernels.cuh", "jac_geom.h", "jac.cu")
+SWEEP_SOURCES = ("jac_kernels.cuh", "jac_temporal3d.cuh", "jac_resident.cuh", "jac_geom.h", "jac.cu")
+CAPTURE_SHA = "cf9d99d95184a8b9"
 NCU_TRAFFIC = {
     # profiles/temporal2d_eigenmode_8192.md
-    ("temporal", 8, 2, False): {"bytes_per_point_per_launch": (592.426752e6 + 492.332288e6) / 8192 ** 2,
-                                "src": SWEEP_SOURCES, "src_sha": "6926e351d1db4903"},
-    ("temporal", 4, 2, False): {"bytes_per_point_per_launch": (606.767616e6 + 489.245952e6) / 8192 ** 2,
-                                "src": SWEEP_SOURCES, "src_sha": "6926e351d1db4903"},
+    ("temporal", 8, 2, False): {"bytes_per_point_per_launch": (607.570432e6 + 493.969152e6) / 8192 ** 2},
+    ("temporal", 4, 2, False): {"bytes_per_point_per_launch": (618.106880e6 + 491.452160e6) / 8192 ** 2},
+    # profiles/temporal2d_poisson_4096.md (config 2 itself; its arrays are about the size of L2)
+    ("temporal", 6, 2, True): {"bytes_per_point_per_launch": (322.013440e6 + 103.846144e6) / 4096 ** 2},
     # profiles/temporal3d_poisson_512.md
-    ("temporal", 2, 3, True): {"bytes_per_point_per_launch": (2.497970e9 + 1.048288e9) / 512 ** 3,
-                               "src": SWEEP_SOURCES, "src_sha": "6926e351d1db4903"},
+    ("temporal", 3, 3, True): {"bytes_per_point_per_launch": (2.473455e9 + 1.048308e9) / 512 ** 3},
+    ("temporal", 2, 3, True): {"bytes_per_point_per_launch": (2.355331e9 + 1.051190e9) / 512 ** 3},
     # profiles/exchange_schedule_eigenmode_8192.md (the update launch alone)
-    ("exchange", 1, 2, False): {"bytes_per_point_per_launch": (574.306816e6 + 495.150336e6) / 8192 ** 2,
-                                "src": SWEEP_SOURCES, "src_sha": "6926e351d1db4903"},
+    ("exchange", 1, 2, False): {"bytes_per_point_per_launch": (574.191104e6 + 495.439872e6) / 8192 ** 2},
+    ("exchange", 1, 3, True): {"bytes_per_point_per_launch": (2.370626e9 + 1.049313e9) / 512 ** 3},
+    # profiles/resident_heated_edge_256.md (config 1 itself: the grid is read once, the result stays in L2)
+    ("resident", 0, 2, False): {"bytes_per_point_per_launch": 578.816e3 / 256 ** 2},
 }
+for _rec in NCU_TRAFFIC.values():
+    _rec.update(src=SWEEP_SOURCES, src_sha=CAPTURE_SHA)
 KERNEL_NAMES = {("temporal", 2): "temporal2d_kernel", ("temporal", 3): "temporal3d_kernel", ("fused", 2): "sweep2d_kernel (update pulling neighbour interiors)",
                 ("exchange", 2): "sweep2d_kernel", ("pertask", 2): "sweep2d_kernel (one launch per block)",
                 ("fused", 3): "sweep3d_kernel (update pulling neighbour interiors)", ("exchange", 3): "sweep3d_kernel",
