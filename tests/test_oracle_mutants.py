@@ -45,6 +45,11 @@ MUTANTS = {
     "dirichlet_of_remainder_block_at_full_size_position": (
         "if (face & 1) { lo[axis] = ext[axis]; hi[axis] = ext[axis] + s->h; }",
         "if (face & 1) { lo[axis] = s->b[axis]; hi[axis] = s->b[axis] + s->h; }", 1),
+    "cut_pack_takes_the_ghost_layers": ("strip_range(s, blk0 + m, face, 0, lo, hi);", "strip_range(s, blk0 + m, face, 1, lo, hi);", 1),
+    "cut_unpack_fills_the_interior_strip": ("strip_range(s, blk0 + m, face, 1, lo, hi);\n        const double *buf = in",
+                                            "strip_range(s, blk0 + m, face, 0, lo, hi);\n        const double *buf = in", 1),
+    "cut_plane_of_the_wrong_end": ("*blk0 = side ? (s->g[sa] - 1) * *count : 0;", "*blk0 = side ? 0 : (s->g[sa] - 1) * *count;", 1),
+    "cut_slots_overlap": ("double *buf = out + m * s->face_elems[face];", "double *buf = out + m * (s->face_elems[face] - 1);", 1),
     "update_runs_over_the_full_block_size": (
         "        for (int64_t k = 0; k < ext[2]; ++k)\n            for (int64_t j = 0; j < ext[1]; ++j)\n"
         "                for (int64_t i = 0; i < ext[0]; ++i) {\n                    const int64_t p = pad_index(s, i, j, k);",
@@ -70,7 +75,8 @@ def test_planted_mistake_is_caught(name, tmp_path):
                         str(ROOT / "tests" / "test_oracle_sweep.py"),
                         str(ROOT / "tests" / "test_oracle_blocks.py"),
                         str(ROOT / "tests" / "test_oracle_wide.py"),
-                        str(ROOT / "tests" / "test_oracle_remainder.py")],
+                        str(ROOT / "tests" / "test_oracle_remainder.py"),
+                        str(ROOT / "tests" / "test_oracle_slabs.py")],
                        cwd=ROOT, env=env, capture_output=True, text=True)
     assert r.returncode == 1, f"mutant {name} survived the pins:\n{r.stdout[-2000:]}"
     assert "failed" in r.stdout
