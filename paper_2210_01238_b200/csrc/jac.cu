@@ -255,6 +255,8 @@ int build_geometry(const jac_desc* d, JacGeom* g, jac_layout* L)
         if (d->ndim == 2 && (b[0] % 4 != 0 || n[0] % 4 != 0)) return JAC_EINVAL;
         if (d->ndim == 3 && (b[0] % 2 != 0 || n[0] % 2 != 0 || d->tsteps > jac::kT3MaxT || n[2] >= (1LL << 30)))
             return JAC_EINVAL;
+        // the 3D kernel keeps row offsets inside one z-layer of blocks in 32 bits
+        if (d->ndim == 3 && g->block_stride * g->gx * g->gy >= (1LL << 31)) return JAC_EINVAL;
     }
     if (d->mode == JAC_MODE_RESIDENT) {
         ResidentPlan rp;
@@ -732,7 +734,7 @@ int ensure_dynamic_smem(jac_ctx* c, size_t smem)
     return JAC_OK;
 }
 
-// T sweeps in one launch (3D, tiles of 64 x 32 streamed along z).  RES (jac::kRes*): the launch also
+// T sweeps in one launch (3D, tiles of 64 x 24 streamed along z).  RES (jac::kRes*): the launch also
 // leaves per-warp partial sums of the squared residual of the state before its last sweep, or of
 // the state it reads.
 template <int T, bool HAS_F, int RES>
