@@ -49,7 +49,7 @@ L2_BYTES = 126e6
 # its points -- traffic is proportional to the points: every strip or tile reads and writes its own
 # part of the grid once per launch.
 SWEEP_SOURCES = ("jac_kernels.cuh", "jac_temporal3d.cuh", "jac_resident.cuh", "jac_geom.h", "jac.cu")
-CAPTURE_SHA = "cf9d99d95184a8b9"
+CAPTURE_SHA = "e844179aae10ebde"
 NCU_TRAFFIC = {
     # profiles/temporal2d_eigenmode_8192.md
     ("temporal", 8, 2, False): {"bytes_per_point_per_launch": (607.570432e6 + 493.969152e6) / 8192 ** 2},
@@ -57,8 +57,8 @@ NCU_TRAFFIC = {
     # profiles/temporal2d_poisson_4096.md (config 2 itself; its arrays are about the size of L2)
     ("temporal", 6, 2, True): {"bytes_per_point_per_launch": (322.013440e6 + 103.846144e6) / 4096 ** 2},
     # profiles/temporal3d_poisson_512.md
-    ("temporal", 3, 3, True): {"bytes_per_point_per_launch": (2.473455e9 + 1.048308e9) / 512 ** 3},
-    ("temporal", 2, 3, True): {"bytes_per_point_per_launch": (2.355331e9 + 1.051190e9) / 512 ** 3},
+    ("temporal", 3, 3, True): {"bytes_per_point_per_launch": (2.503104e9 + 1.050502e9) / 512 ** 3},
+    ("temporal", 2, 3, True): {"bytes_per_point_per_launch": (2.415353e9 + 1.050802e9) / 512 ** 3},
     # profiles/exchange_schedule_eigenmode_8192.md (the update launch alone)
     ("exchange", 1, 2, False): {"bytes_per_point_per_launch": (574.191104e6 + 495.439872e6) / 8192 ** 2},
     ("exchange", 1, 3, True): {"bytes_per_point_per_launch": (2.370626e9 + 1.049313e9) / 512 ** 3},
