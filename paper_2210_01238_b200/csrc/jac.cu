@@ -1292,6 +1292,8 @@ int jac_create(const jac_desc* desc, void* dev_workspace, size_t bytes, jac_ctx*
     c->g.chk_lo[2] = c->ws + L.off_scratch;
     c->g.chk_hi[2] = c->ws + L.off_scratch + (L.partials + 32) * (long long)sizeof(double);
     c->g.chk_rec = reinterpret_cast<unsigned long long*>(c->result + 5);
+    c->g.quarter = 0.25;
+    c->g.sixth = 1.0 / 6.0;
     const cudaError_t e = cudaMemsetAsync(c->ws, 0, (size_t)L.total_bytes, c->stream);
     if (e != cudaSuccess) {
         delete c;

@@ -27,6 +27,9 @@ struct JacGeom {
     long long face_off[6];
     long long send_stride;
     double bval[6];
+    // 1/4 and 1/6 (correctly rounded), for kernels that want the stencil's factor as an operand
+    // from the constant bank instead of a literal they would have to build in registers
+    double quarter, sixth;
     // wide exchange: a wide face is h layers along its axis and the whole padded extent
     // (b + 2h) along the other axes
     long long wface_elems[6];

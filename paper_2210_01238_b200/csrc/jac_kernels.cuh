@@ -982,7 +982,7 @@ __device__ __forceinline__ void temporal_level(RowN<temporal_points(T)> (&win)[T
         const double E = (q == P - 1) ? e : M.v[q + 1];
         double sum = add_rn(add_rn(W, E), add_rn(S.v[q], N.v[q]));
         if (HAS_F) sum = add_rn(sum, ff.v[q]);
-        o.v[q] = mul_rn(sum, 0.25);
+        o.v[q] = mul_rn(sum, g.quarter);
         // residual of the state this level reads (M is that state at this point)
         if (MEASURES) res.v[q] = sub_rn(sum, mul_rn(4.0, M.v[q]));
     }

@@ -175,7 +175,7 @@ __device__ __forceinline__ void t3_level(const T3& c, const JacGeom& g, const Ro
                                          const double* fplane /* this lane's pair in row 0 of the warp, f plane q */,
                                          Rows& out, unsigned live, double& acc)
 {
-    const double c6 = 1.0 / 6.0;
+    const double c6 = g.sixth;
 #pragma unroll
     for (int r = 0; r < kT3Rows; ++r) {
         const Pair& S = (r == 0) ? below : M.row[r - 1];
