@@ -903,6 +903,49 @@ int choose_resident_cluster(jac_ctx* c)
     return JAC_EINVAL;
 }
 
+// Relative cost of one temporal launch of depth t: a pass over memory plus t levels, per output
+// column (2D: a strip stores 120 of its 128 columns up to t = 4 and 112 beyond, so t = 5 pays for
+// halo lanes that t = 8 would use too).  Fitted to launch times on 4096^2 with f (0.107 / 0.135 /
+// 0.1425 ms at t = 4 / 5 / 6), 16384^2 without (0.750 / 1.141 ms at t = 4 / 8) and 1024^3 with f
+// (5.11 / 6.13 / 7.65 ms at t = 1 / 2 / 3).
+double temporal_launch_cost(int ndim, bool has_f, int t)
+{
+    if (ndim == 3) return t == 1 ? 5.11 : t == 2 ? 6.13 : 7.65;
+    return ((has_f ? 2.0 : 3.7) + t) * 120.0 / jac::temporal_strip_cols(t);
+}
+
+// Depths of the launches that make up nsweeps sweeps at depth <= T: as few launches as the depth
+// allows (a launch of one sweep costs most of what a launch of T does); all but the last few at
+// full depth, and the last (up to four) share what is left in the cheapest way by the cost above
+// -- ten sweeps at T = 6 run as 6 + 4, not 5 + 5; ten at T = 3 as 3 + 3 + 2 + 2.
+void temporal_depths(int nsweeps, int T, int ndim, bool has_f, std::vector<int>* depths)
+{
+    depths->clear();
+    const int launches = (nsweeps + T - 1) / T;
+    const int m = std::min(launches, 4);
+    for (int k = 0; k < launches - m; ++k) depths->push_back(T);
+    const int tail = nsweeps - (launches - m) * T;
+    int best[4] = {0, 0, 0, 0}, cur[4] = {0, 0, 0, 0};
+    double best_cost = 1e300;
+    // non-increasing depths cur[0] >= cur[1] >= ... summing to tail
+    auto rec = [&](auto&& self, int k, int left, int cap, double cost) -> void {
+        if (k == m) {
+            if (left == 0 && cost < best_cost - 1e-12) {
+                best_cost = cost;
+                std::copy(cur, cur + 4, best);
+            }
+            return;
+        }
+        for (int t = std::min(cap, left - (m - k - 1)); t >= 1; --t) {
+            if ((long long)t * (m - k) < left) break;   // the rest cannot be covered by depths <= t
+            cur[k] = t;
+            self(self, k + 1, left - t, t, cost + temporal_launch_cost(ndim, has_f, t));
+        }
+    };
+    rec(rec, 0, tail, T, 0.0);
+    for (int k = 0; k < m; ++k) depths->push_back(best[k]);
+}
+
 // nsweeps iterations in the context's schedule.  res (jac::kRes*): one launch also leaves partial
 // sums of the squared residual in the scratch (*nparts of them) -- kResBeforeLast: the last sweep,
 // of the state it reads; kResOfInput: the first sweep, of the state the call starts from.
@@ -955,12 +998,11 @@ int run_sweeps(jac_ctx* c, int nsweeps, int res, long long* nparts)
             if (res) *nparts = sweep_parts;
             break;
         case JAC_MODE_TEMPORAL: {
-            // as few launches as the depth allows, and those of equal depth up to one sweep: a
-            // launch of one sweep costs most of what a launch of T does
             const int T = default_tsteps(c->desc);
-            const int launches = (nsweeps + T - 1) / T;
+            std::vector<int> depths;
+            temporal_depths(nsweeps, T, g.ndim, c->desc.has_f != 0, &depths);
             for (int k = 0, left = nsweeps; left > 0; ++k) {
-                const int t = nsweeps / launches + (k < nsweeps % launches ? 1 : 0);
+                const int t = depths[(size_t)k];
                 const int r = (res == jac::kResBeforeLast && left == t) ? jac::kResBeforeLast
                               : (res == jac::kResOfInput && k == 0)     ? jac::kResOfInput
                                                                         : jac::kResNone;
