@@ -1073,9 +1073,6 @@ int run_sweeps(jac_ctx* c, int nsweeps, int res, long long* nparts)
     return JAC_OK;
 }
 
-// the square root of one device double, in place (correctly rounded, as std::sqrt on the host)
-__global__ void sqrt_in_place_kernel(double* v) { *v = sqrt(*v); }
-
 // End of one group of jac_solve's sweeps, on the device: the group's partial sums are added in the
 // usual fixed order, the norm and the sweeps done so far are recorded, and once the norm has met
 // the tolerance a flag goes up that turns every later launch of the call into a no-op.
@@ -1114,7 +1111,7 @@ int check_timeout(jac_ctx* c)
 
 int finish_norm(jac_ctx* c, long long nparts, double* host_out_l2)
 {
-    jac::reduce_partials_kernel<<<1, 1024, 0, c->stream>>>(c->partials, nparts, c->result);
+    jac::reduce_partials_kernel<<<1, 1024, 0, c->stream>>>(c->partials, nparts, c->result, false);
     int rc = check_launch(c);
     if (rc) return rc;
     double sum = 0.0;
@@ -1703,12 +1700,8 @@ int residual_queued(jac_ctx* c, double* host_out, bool norm)
     if (has_cuts(c) && (!c->cut_fresh || c->in_sweep)) return JAC_EINVAL;
     if (!c->ghosts_fresh && (rc = (c->desc.mode == JAC_MODE_PERTASK ? do_exchange(c) : do_exchange_fused(c)))) return rc;
     if ((rc = launch_sweep<jac::OP_RESIDUAL>(c, c->u[c->cur], nullptr, 0, c->g.nblocks))) return rc;
-    jac::reduce_partials_kernel<<<1, 1024, 0, c->stream>>>(c->partials, c->g.nblocks * c->tile.ctas_per_block, c->result);
+    jac::reduce_partials_kernel<<<1, 1024, 0, c->stream>>>(c->partials, c->g.nblocks * c->tile.ctas_per_block, c->result, norm);
     if ((rc = check_launch(c))) return rc;
-    if (norm) {
-        sqrt_in_place_kernel<<<1, 1, 0, c->stream>>>(c->result);
-        if ((rc = check_launch(c))) return rc;
-    }
     JAC_CK(c, cudaMemcpyAsync(host_out, c->result, sizeof(double), cudaMemcpyDeviceToHost, c->stream));
     return JAC_OK;
 }
@@ -1730,9 +1723,7 @@ int jac_residual_sweep_async(jac_ctx* c, int nsweeps, double* host_out_l2)
     }
     long long nparts = 0;
     if ((rc = run_sweeps(c, nsweeps, jac::kResOfInput, &nparts))) return rc;
-    jac::reduce_partials_kernel<<<1, 1024, 0, c->stream>>>(c->partials, nparts, c->result);
-    if ((rc = check_launch(c))) return rc;
-    sqrt_in_place_kernel<<<1, 1, 0, c->stream>>>(c->result);
+    jac::reduce_partials_kernel<<<1, 1024, 0, c->stream>>>(c->partials, nparts, c->result, true);
     if ((rc = check_launch(c))) return rc;
     JAC_CK(c, cudaMemcpyAsync(host_out_l2, c->result, sizeof(double), cudaMemcpyDeviceToHost, c->stream));
     return JAC_OK;

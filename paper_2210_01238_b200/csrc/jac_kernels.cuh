@@ -346,14 +346,15 @@ sweep3d_kernel(const double* __restrict__ u, double* __restrict__ un, const doub
     }
 }
 
-// Second pass of the residual: one CTA adds the per-CTA partials in a fixed order.
+// Second pass of the residual: one CTA adds the per-CTA partials in a fixed order and leaves the
+// sum, or (root) its square root, the norm.
 __global__ void __launch_bounds__(1024)
-reduce_partials_kernel(const double* __restrict__ partials, const long long n, double* __restrict__ out)
+reduce_partials_kernel(const double* __restrict__ partials, const long long n, double* __restrict__ out, const bool root)
 {
     double acc = 0.0;
     for (long long i = threadIdx.x; i < n; i += blockDim.x) acc = add_rn(acc, partials[i]);
     const double total = block_sum(acc);
-    if (threadIdx.x == 0) *out = total;
+    if (threadIdx.x == 0) *out = root ? sqrt(total) : total;
 }
 
 // ---------------------------------------------------------------------------------------
