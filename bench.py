@@ -303,19 +303,19 @@ def run_ours(args, w: inputs.Workload):
 
     def one_job(J, pairs=None):
         """The sweeps of one step with the residual norm after every group (queued, nothing waits).
-        The norm after group k comes out of the first sweep of group k + 1, which reads that state
-        anyway (jac_residual_sweep_async); only the last one needs a pass of its own."""
-        for k, n_sw in enumerate(groups):
-            if pairs is not None:
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(J.stream)
-            if k == 0:
-                J.sweep(n_sw)
-            else:
-                J.residual_sweep_async(n_sw, norms[k - 1:k])
-            if pairs is not None:
-                b.record(J.stream)
-                pairs.append((a, b))
+        The norm after group k comes out of the sweep that reads that state anyway, the first of
+        group k + 1 (jac_sweep_norms_async; the temporal schedule does not even cut its launches
+        there); only the last one needs a pass of its own."""
+        if pairs is not None:
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(J.stream)
+        if len(groups) > 1:
+            J.sweep_norms_async(sweeps, every, norms)
+        else:
+            J.sweep(sweeps)
+        if pairs is not None:
+            b.record(J.stream)
+            pairs.append((a, b))
         J.residual_async(norms[len(groups) - 1:])
 
     def time_schedule(J, mode, tsteps, steps, warmup, sample_clocks):
@@ -345,7 +345,9 @@ def run_ours(args, w: inputs.Workload):
         ms_total = max_over_ranks(ev0.elapsed_time(ev1))
         per_step = sorted(sum(a.elapsed_time(b) for a, b in pairs) for pairs in step_pairs)
         sweep_ms = sum(per_step)
-        if mode == "temporal":
+        if mode == "temporal" and every >= tsteps:
+            n_launch = -(-sweeps // tsteps)          # launches run across the points where a norm is due
+        elif mode == "temporal":
             n_launch = sum(-(-n_sw // tsteps) for n_sw in groups)
         else:
             n_launch = len(groups) if mode == "resident" else sweeps
@@ -423,11 +425,10 @@ def run_ours(args, w: inputs.Workload):
 
         def e2e_step(Jc, out, nrm):
             Jc.set_u_async(host_in)
-            for k, n_sw in enumerate(groups):
-                if k == 0:
-                    Jc.sweep(n_sw)
-                else:
-                    Jc.residual_sweep_async(n_sw, nrm[k - 1:k])
+            if len(groups) > 1:
+                Jc.sweep_norms_async(sweeps, every, nrm)
+            else:
+                Jc.sweep(sweeps)
             Jc.residual_async(nrm[len(groups) - 1:])
             Jc.get_u_async(out)
 
@@ -465,7 +466,7 @@ def run_ours(args, w: inputs.Workload):
 
         one_steps = max(3, min(args.steps, 6))
         one = e2e_record(run_pipeline(1, one_steps), one_steps,
-                         "one context, steps queued back to back on one stream: jac_set_u_async(pinned host) + jac_sweep (jac_residual_sweep_async from the second group on) + "
+                         "one context, steps queued back to back on one stream: jac_set_u_async(pinned host) + jac_sweep (jac_sweep_norms_async when the workload names a residual cadence) + "
                          "jac_residual_async after the last group + jac_get_u_async(pinned host)")
         e2e = one
         # several contexts on as many streams, steps going round them: the copy in of one step, the
@@ -477,7 +478,7 @@ def run_ours(args, w: inputs.Workload):
             pipe_steps = max(2 * depth, args.steps)
             e2e = e2e_record(run_pipeline(depth, pipe_steps), pipe_steps,
                              f"{depth} contexts on {depth} streams, steps going round them; every step is jac_set_u_async(pinned "
-                             "host) + jac_sweep (jac_residual_sweep_async from the second group on) + jac_residual_async + jac_get_u_async(pinned host); timed by the host "
+                             "host) + jac_sweep (jac_sweep_norms_async when the workload names a residual cadence) + jac_residual_async + jac_get_u_async(pinned host); timed by the host "
                              "clock between synchronisations of all streams")
             e2e["one_context"] = one
         bound_ms = 2 * nbytes / 55e9 * 1e3

@@ -290,6 +290,21 @@ int jac_sweep_residual(jac_ctx *ctx, int nsweeps, double *host_out_l2);
  * fixed iteration count.) */
 int jac_residual_sweep_async(jac_ctx *ctx, int nsweeps, double *host_out_l2);
 
+/* nsweeps sweeps of a job that monitors the residual every `every` sweeps: host_out_l2[m - 1]
+ * receives the L2 residual norm of the state after m * every sweeps, for every m >= 1 with
+ * m * every < nsweeps (the state after the last sweep is read by no sweep of the call: jac_residual
+ * or jac_residual_async gives its norm).  Each norm is what jac_residual would return at that
+ * point, up to summation order (<= 1e-10 relative), and comes out of the sweep that reads the
+ * state, as in jac_residual_sweep_async.  In JAC_MODE_TEMPORAL with every >= the sweeps per launch
+ * the launches are not cut where a norm is due: a launch of T sweeps holds the states after
+ * 0 .. T - 1 of its sweeps in its levels, and the level that reads the wanted state measures it,
+ * so 50 sweeps at T = 3 with a norm every 10 run as 16 launches of depth 3 and one of 2, not as
+ * 5 x (3 + 3 + 2 + 2).  Other schedules, and every < T, run group by group.  Nothing waits: the
+ * norms are written (pinned memory: (nsweeps - 1) / every doubles) as the stream gets there.
+ * nsweeps >= 1, every >= 1; host_out_l2 may be NULL when no norm falls inside the call.  Not for
+ * slab contexts.  (Not in the paper, which runs a fixed iteration count.) */
+int jac_sweep_norms_async(jac_ctx *ctx, int nsweeps, int every, double *host_out_l2);
+
 /* Iterate until converged: runs sweeps in groups of check_every (each group as
  * jac_sweep_residual does) until the lagged residual norm is <= tol or max_sweeps sweeps have run.
  * The comparison with tol is made on the device: several groups are queued at a time without

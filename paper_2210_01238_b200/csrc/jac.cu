@@ -734,9 +734,9 @@ int ensure_dynamic_smem(jac_ctx* c, size_t smem)
     return JAC_OK;
 }
 
-// T sweeps in one launch (3D, tiles of 64 x 24 streamed along z).  RES (jac::kRes*): the launch also
-// leaves per-warp partial sums of the squared residual of the state before its last sweep, or of
-// the state it reads.
+// T sweeps in one launch (3D, tiles of 64 x 24 streamed along z).  RES = 1..T: level RES also leaves
+// per-warp partial sums of the squared residual of the state it reads (the one after RES - 1 sweeps
+// of the launch); 0: none.
 template <int T, bool HAS_F, int RES>
 int launch_temporal3d_t(jac_ctx* c, const double* u, double* un, long long* nparts)
 {
@@ -748,37 +748,13 @@ int launch_temporal3d_t(jac_ctx* c, const double* u, double* un, long long* npar
     if (rc) return rc;
     kern<<<(unsigned)t.ctas, jac::kT3Warps * 32, smem, c->stream>>>(u, un, c->f, c->partials, c->g, t.a, t.b, t.c,
                                                                    t.chunk);
-    if (RES != jac::kResNone) *nparts = t.warps;
+    if (RES != 0) *nparts = t.warps;
     return check_launch(c);
 }
 
-template <int T, int RES>
-int launch_temporal3d(jac_ctx* c, const double* u, double* un, long long* nparts)
-{
-    return c->desc.has_f ? launch_temporal3d_t<T, true, RES>(c, u, un, nparts)
-                         : launch_temporal3d_t<T, false, RES>(c, u, un, nparts);
-}
-
-template <int RES>
-int launch_temporal3d_r(jac_ctx* c, int t, const double* u, double* un, long long* nparts)
-{
-    switch (t) {
-        case 1: return launch_temporal3d<1, RES>(c, u, un, nparts);
-        case 2: return launch_temporal3d<2, RES>(c, u, un, nparts);
-        default: return launch_temporal3d<3, RES>(c, u, un, nparts);
-    }
-}
-
-int launch_temporal3d_n(jac_ctx* c, int t, const double* u, double* un, int res, long long* nparts)
-{
-    if (res == jac::kResBeforeLast) return launch_temporal3d_r<jac::kResBeforeLast>(c, t, u, un, nparts);
-    if (res == jac::kResOfInput) return launch_temporal3d_r<jac::kResOfInput>(c, t, u, un, nparts);
-    return launch_temporal3d_r<jac::kResNone>(c, t, u, un, nparts);
-}
-
-// T sweeps in one launch (2D, register-streaming temporal blocking)
+// T sweeps in one launch (2D, register-streaming temporal blocking); RES as above
 template <int T, bool HAS_F, int RES>
-int launch_temporal_t(jac_ctx* c, const double* u, double* un, long long* nparts)
+int launch_temporal2d_t(jac_ctx* c, const double* u, double* un, long long* nparts)
 {
     const TemporalGrid t = temporal_grid_2d(c->g, T, HAS_F, c->sms);
     constexpr auto kern = jac::temporal2d_kernel<T, HAS_F, RES>;
@@ -789,37 +765,65 @@ int launch_temporal_t(jac_ctx* c, const double* u, double* un, long long* nparts
     }
     kern<<<(unsigned)t.ctas, jac::kTemporalWarps * 32, smem, c->stream>>>(u, un, c->f, c->partials, c->g, t.a, t.b,
                                                                          t.chunk);
-    if (RES != jac::kResNone) *nparts = t.warps;
+    if (RES != 0) *nparts = t.warps;
     return check_launch(c);
 }
 
-template <int T, int RES>
-int launch_temporal(jac_ctx* c, const double* u, double* un, long long* nparts)
+// the run-time depth t and measuring level (0..t) picked out of the compiled ones
+template <int NDIM, int T, int RES>
+int launch_temporal_tr(jac_ctx* c, const double* u, double* un, long long* nparts)
 {
-    return c->desc.has_f ? launch_temporal_t<T, true, RES>(c, u, un, nparts)
-                         : launch_temporal_t<T, false, RES>(c, u, un, nparts);
-}
-
-template <int RES>
-int launch_temporal_r(jac_ctx* c, int t, const double* u, double* un, long long* nparts)
-{
-    switch (t) {
-        case 1: return launch_temporal<1, RES>(c, u, un, nparts);
-        case 2: return launch_temporal<2, RES>(c, u, un, nparts);
-        case 3: return launch_temporal<3, RES>(c, u, un, nparts);
-        case 4: return launch_temporal<4, RES>(c, u, un, nparts);
-        case 5: return launch_temporal<5, RES>(c, u, un, nparts);
-        case 6: return launch_temporal<6, RES>(c, u, un, nparts);
-        case 7: return launch_temporal<7, RES>(c, u, un, nparts);
-        default: return launch_temporal<8, RES>(c, u, un, nparts);
+    if constexpr (RES > T) {
+        return JAC_EINVAL;
+    } else if constexpr (NDIM == 2) {
+        return c->desc.has_f ? launch_temporal2d_t<T, true, RES>(c, u, un, nparts)
+                             : launch_temporal2d_t<T, false, RES>(c, u, un, nparts);
+    } else {
+        return c->desc.has_f ? launch_temporal3d_t<T, true, RES>(c, u, un, nparts)
+                             : launch_temporal3d_t<T, false, RES>(c, u, un, nparts);
     }
 }
 
-int launch_temporal_n(jac_ctx* c, int t, const double* u, double* un, int res, long long* nparts)
+template <int NDIM, int T>
+int launch_temporal_level(jac_ctx* c, int level, const double* u, double* un, long long* nparts)
 {
-    if (res == jac::kResBeforeLast) return launch_temporal_r<jac::kResBeforeLast>(c, t, u, un, nparts);
-    if (res == jac::kResOfInput) return launch_temporal_r<jac::kResOfInput>(c, t, u, un, nparts);
-    return launch_temporal_r<jac::kResNone>(c, t, u, un, nparts);
+    switch (level) {
+        case 0: return launch_temporal_tr<NDIM, T, 0>(c, u, un, nparts);
+        case 1: return launch_temporal_tr<NDIM, T, 1>(c, u, un, nparts);
+        case 2: return launch_temporal_tr<NDIM, T, 2>(c, u, un, nparts);
+        case 3: return launch_temporal_tr<NDIM, T, 3>(c, u, un, nparts);
+        case 4: return launch_temporal_tr<NDIM, T, 4>(c, u, un, nparts);
+        case 5: return launch_temporal_tr<NDIM, T, 5>(c, u, un, nparts);
+        case 6: return launch_temporal_tr<NDIM, T, 6>(c, u, un, nparts);
+        case 7: return launch_temporal_tr<NDIM, T, 7>(c, u, un, nparts);
+        case 8: return launch_temporal_tr<NDIM, T, 8>(c, u, un, nparts);
+        default: return JAC_EINVAL;
+    }
+}
+
+// one temporal launch of depth t whose level `level` (1..t; 0: none) measures the residual
+int launch_temporal_n(jac_ctx* c, int t, const double* u, double* un, int level, long long* nparts)
+{
+    if (level < 0 || level > t) return JAC_EINVAL;
+    if (c->g.ndim == 3) {
+        switch (t) {
+            case 1: return launch_temporal_level<3, 1>(c, level, u, un, nparts);
+            case 2: return launch_temporal_level<3, 2>(c, level, u, un, nparts);
+            case 3: return launch_temporal_level<3, 3>(c, level, u, un, nparts);
+            default: return JAC_EINVAL;
+        }
+    }
+    switch (t) {
+        case 1: return launch_temporal_level<2, 1>(c, level, u, un, nparts);
+        case 2: return launch_temporal_level<2, 2>(c, level, u, un, nparts);
+        case 3: return launch_temporal_level<2, 3>(c, level, u, un, nparts);
+        case 4: return launch_temporal_level<2, 4>(c, level, u, un, nparts);
+        case 5: return launch_temporal_level<2, 5>(c, level, u, un, nparts);
+        case 6: return launch_temporal_level<2, 6>(c, level, u, un, nparts);
+        case 7: return launch_temporal_level<2, 7>(c, level, u, un, nparts);
+        case 8: return launch_temporal_level<2, 8>(c, level, u, un, nparts);
+        default: return JAC_EINVAL;
+    }
 }
 
 // nsweeps sweeps in ONE launch of one thread-block cluster that keeps the grid in shared memory
@@ -1003,12 +1007,11 @@ int run_sweeps(jac_ctx* c, int nsweeps, int res, long long* nparts)
             temporal_depths(nsweeps, T, g.ndim, c->desc.has_f != 0, &depths);
             for (int k = 0, left = nsweeps; left > 0; ++k) {
                 const int t = depths[(size_t)k];
-                const int r = (res == jac::kResBeforeLast && left == t) ? jac::kResBeforeLast
-                              : (res == jac::kResOfInput && k == 0)     ? jac::kResOfInput
-                                                                        : jac::kResNone;
-                rc = (g.ndim == 2) ? launch_temporal_n(c, t, c->u[c->cur], c->u[c->cur ^ 1], r, nparts)
-                                   : launch_temporal3d_n(c, t, c->u[c->cur], c->u[c->cur ^ 1], r, nparts);
-                if (rc) return rc;
+                // the level that measures: the top one of the last launch, the first one of the first
+                const int level = (res == jac::kResBeforeLast && left == t) ? t
+                                  : (res == jac::kResOfInput && k == 0)     ? 1
+                                                                            : 0;
+                if ((rc = launch_temporal_n(c, t, c->u[c->cur], c->u[c->cur ^ 1], level, nparts))) return rc;
                 c->cur ^= 1;
                 left -= t;
             }
@@ -1726,6 +1729,52 @@ int jac_residual_sweep_async(jac_ctx* c, int nsweeps, double* host_out_l2)
     jac::reduce_partials_kernel<<<1, 1024, 0, c->stream>>>(c->partials, nparts, c->result, true);
     if ((rc = check_launch(c))) return rc;
     JAC_CK(c, cudaMemcpyAsync(host_out_l2, c->result, sizeof(double), cudaMemcpyDeviceToHost, c->stream));
+    return JAC_OK;
+}
+
+int jac_sweep_norms_async(jac_ctx* c, int nsweeps, int every, double* host_out_l2)
+{
+    int rc = usable(c);
+    if (rc) return rc;
+    if (nsweeps < 1 || every < 1 || has_cuts(c)) return JAC_EINVAL;
+    const int nnorms = (nsweeps - 1) / every;
+    if (nnorms > 0 && !host_out_l2) return JAC_EINVAL;
+    const int T = default_tsteps(c->desc);
+    if (c->desc.mode == JAC_MODE_TEMPORAL && nnorms > 0 && every >= T) {
+        // The state after j sweeps is what sweep j + 1 reads: level j - a + 1 of the launch that starts
+        // after a sweeps.  So the launches need not end where a norm is due; they keep the depths the
+        // whole run would have, and at most one level of a launch measures (every >= T).
+        std::vector<int> depths;
+        temporal_depths(nsweeps, T, c->g.ndim, c->desc.has_f != 0, &depths);
+        int a = 0;
+        for (const int t : depths) {
+            int j = (a + every - 1) / every * every;     // the first multiple of `every` not below a
+            if (j == 0) j = every;
+            const int level = j < a + t ? j - a + 1 : 0;
+            long long nparts = 0;
+            if ((rc = launch_temporal_n(c, t, c->u[c->cur], c->u[c->cur ^ 1], level, &nparts))) return rc;
+            c->cur ^= 1;
+            c->ghosts_fresh = false;
+            c->packed_current = false;
+            if (level) {
+                jac::reduce_partials_kernel<<<1, 1024, 0, c->stream>>>(c->partials, nparts, c->result, true);
+                if ((rc = check_launch(c))) return rc;
+                JAC_CK(c, cudaMemcpyAsync(host_out_l2 + (j / every - 1), c->result, sizeof(double),
+                                          cudaMemcpyDeviceToHost, c->stream));
+            }
+            a += t;
+        }
+        return JAC_OK;
+    }
+    // every other case group by group: the norm of the state a group starts from comes out of the
+    // group's first sweep
+    int done = std::min(every, nsweeps);
+    if ((rc = run_sweeps(c, done, jac::kResNone, nullptr))) return rc;
+    for (int k = 0; done < nsweeps; ++k) {
+        const int n = std::min(every, nsweeps - done);
+        if ((rc = jac_residual_sweep_async(c, n, host_out_l2 + k))) return rc;
+        done += n;
+    }
     return JAC_OK;
 }
 

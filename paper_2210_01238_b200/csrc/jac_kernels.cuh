@@ -20,10 +20,12 @@ __host__ __device__ constexpr bool op_pulls(int op) { return op == OP_UPDATE_PUL
 __host__ __device__ constexpr bool op_sums(int op) { return op == OP_RESIDUAL || op == OP_UPDATE_RES || op == OP_UPDATE_PULL_RES; }
 __host__ __device__ constexpr bool op_ext(int op) { return op == OP_UPDATE_EXT; }
 
-// which state a temporal launch also measures the residual of (RES template argument)
+// which state a run of sweeps also measures the residual of (host side)
 enum : int { kResNone = 0,        // none
-             kResBeforeLast = 1,  // the state before the last sweep of the launch (its top level reads it)
-             kResOfInput = 2 };   // the state the launch reads (its first level reads it)
+             kResBeforeLast = 1,  // the state before the last sweep
+             kResOfInput = 2 };   // the state the run starts from
+// A temporal kernel takes the level that measures as its RES template argument: level s (1..T) reads
+// the state after s - 1 sweeps of the launch and accumulates that state's squared residual; 0: none.
 
 __device__ __forceinline__ double add_rn(double a, double b) { return __dadd_rn(a, b); }
 __device__ __forceinline__ double sub_rn(double a, double b) { return __dsub_rn(a, b); }
@@ -975,7 +977,7 @@ __device__ __forceinline__ void temporal_level(RowN<temporal_points(T)> (&win)[T
             ff = fill_rown<P>(0.0);
         }
     }
-    constexpr bool MEASURES = (RES == kResBeforeLast && s == T) || (RES == kResOfInput && s == 1);
+    constexpr bool MEASURES = RES == s;
     Row o, res;
 #pragma unroll
     for (int q = 0; q < P; ++q) {
@@ -1050,8 +1052,8 @@ __device__ __forceinline__ void temporal_step_any(RowN<temporal_points(T)> (&win
     else temporal_step<T, HAS_F, RES, PH, false>(win, c, g, r, load_cur, out_cur, acc);
 }
 
-// RES: the top level (kResBeforeLast) or the first level (kResOfInput) also accumulates the squared
-// residual of the state it reads; every warp writes its partial sum to partials[warp id].
+// RES: level RES (1..T; 0: none) also accumulates the squared residual of the state it reads, the one
+// after RES - 1 sweeps of the launch; every warp writes its partial sum to partials[warp id].
 template <int T, bool HAS_F, int RES>
 __global__ void __launch_bounds__(kTemporalWarps * 32, temporal_ctas_per_sm(T, HAS_F))
 temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const double* __restrict__ f,
@@ -1124,7 +1126,7 @@ temporal2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
         if (r + 2 < r_end) temporal_step_any<T, HAS_F, RES, 2>(win, c, g, r + 2, load_cur, out_cur, acc);
     }
     cp_async_wait<0>();
-    if (RES != kResNone) {
+    if (RES != 0) {
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) acc = add_rn(acc, __shfl_down_sync(0xffffffffu, acc, off));
         if (lane == 0) g_st(g, partials + wid, acc, CHK_SCRATCH, KID_TEMPORAL2D);

@@ -240,13 +240,13 @@ __device__ __forceinline__ void t3_levels(Rows (&win)[kT3MaxT][3], const T3& c, 
     if constexpr (s == T) {
         Rows o;
         const unsigned live = t3_live_rows(c, q);
-        t3_level<HAS_F, EDGE, (T == 1 ? RES != kResNone : RES == kResBeforeLast)>(c, g, D, M, U, below, above, q, fp, o, live, acc);
+        t3_level<HAS_F, EDGE, RES == T>(c, g, D, M, U, below, above, q, fp, o, live, acc);
         t3_store(c, g, un, out_off, o, live);
     } else {
         Rows& o = win[s][slot3(PH, -s)];
-        // level 1 can also give the residual of the state the launch reads: over the tile's output
-        // cells, which every interior point is in exactly once, and where level 1 is exact
-        constexpr bool RES_HERE = s == 1 && RES == kResOfInput;
+        // a level below the top can also give the residual of the state it reads: over the tile's
+        // output cells, which every interior point is in exactly once, and where every level is exact
+        constexpr bool RES_HERE = s == RES;
         const unsigned live = RES_HERE ? t3_live_rows(c, q) : 0u;
         t3_level<HAS_F, EDGE, RES_HERE>(c, g, D, M, U, below, above, q, fp, o, live, acc);
         // the warp's first and last row are what other warps read
@@ -268,9 +268,8 @@ __device__ __forceinline__ void t3_step(Rows (&win)[kT3MaxT][3], const T3& c, co
     t3_levels<T, HAS_F, RES, PH, EDGE, 1>(win, c, g, un, p, out_off, acc);
 }
 
-// RES: partials[CTA * 8 + warp] gets the warp's sum of squared residuals over exactly the points
-// the warp stores -- of the state before the last sweep of the launch (kResBeforeLast) or of the
-// state the launch reads (kResOfInput).
+// RES (1..T; 0: none): partials[CTA * 12 + warp] gets the warp's sum of squared residuals over exactly
+// the points the warp stores -- of the state level RES reads, the one after RES - 1 sweeps of the launch.
 template <int T, bool HAS_F, int RES>
 __global__ void __launch_bounds__(kT3Warps * 32, 1)
 temporal3d_kernel(const double* __restrict__ u, double* __restrict__ un, const double* __restrict__ f,
@@ -392,7 +391,7 @@ temporal3d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
 #undef JAC_T3_STEP
 #undef JAC_T3_ISSUE
     cp_async_wait<0>();
-    if (RES != kResNone) {
+    if (RES != 0) {
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) acc = add_rn(acc, __shfl_down_sync(0xffffffffu, acc, off));
         if (lane == 0) g_st(g, partials + (long long)blockIdx.x * kT3Warps + warp, acc, CHK_SCRATCH, KID_TEMPORAL3D);

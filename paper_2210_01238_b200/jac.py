@@ -38,6 +38,7 @@ EXPORTS = [
     "jac_set_u_async", "jac_get_u_async", "jac_residual_async", "jac_exchange_halos",
     "jac_pack_cut", "jac_unpack_cut", "jac_sweep_begin", "jac_sweep_end", "jac_cut_info",
     "jac_residual_sumsq_async", "jac_residual_sweep_async", "jac_debug_bounds", "jac_debug_shrink_bounds",
+    "jac_sweep_norms_async",
 ]
 
 
@@ -102,6 +103,7 @@ def lib() -> C.CDLL:
         L.jac_residual.argtypes = [vp, dp]
         L.jac_sweep_residual.argtypes = [vp, C.c_int, dp]
         L.jac_residual_sweep_async.argtypes = [vp, C.c_int, vp]
+        L.jac_sweep_norms_async.argtypes = [vp, C.c_int, C.c_int, vp]
         L.jac_solve.argtypes = [vp, C.c_int, C.c_int, C.c_double, C.POINTER(C.c_int), dp]
         L.jac_launch_count.argtypes = [vp, C.POINTER(C.c_int64)]
         L.jac_sweeps_per_launch.argtypes = [vp, C.POINTER(C.c_int)]
@@ -444,6 +446,17 @@ class Jacobi:
         assert out.numel() == 1
         self._call("jac_residual_sweep_async",
                    lib().jac_residual_sweep_async(self._ctx, int(nsweeps), self._pinned_ptr(out)))
+        return out
+
+    def sweep_norms_async(self, nsweeps: int, every: int, out=None):
+        """nsweeps sweeps; the pinned tensor ``out`` receives, when the stream gets there, the residual
+        norms of the states after every, 2 * every, ... (< nsweeps) sweeps: (nsweeps - 1) // every values."""
+        need = (int(nsweeps) - 1) // int(every) if nsweeps >= 1 and every >= 1 else 0
+        if need > 0:
+            assert out is not None and out.numel() >= need
+        ptr = self._pinned_ptr(out) if out is not None else None
+        self._call("jac_sweep_norms_async",
+                   lib().jac_sweep_norms_async(self._ctx, int(nsweeps), int(every), ptr))
         return out
 
     def solve(self, max_sweeps: int, check_every: int, tol: float):

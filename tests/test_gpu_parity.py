@@ -341,6 +341,48 @@ def test_residual_from_the_first_sweep_s_pass(jac, orc, n, b, h, mode, tsteps, h
     B.close()
 
 
+# (n, b, mode, tsteps, nsweeps, every): norms due inside launches (every > T, no multiple of T), at
+# launch borders (every = T), every < T (group by group), nothing due (nsweeps <= every)
+NORM_CASES = [((120, 40), (60, 20), "temporal", 3, 23, 5), ((256, 100), (64, 25), "temporal", 8, 50, 10),
+              ((256, 100), (64, 25), "temporal", 6, 31, 10), ((1100, 200), (220, 50), "temporal", 4, 17, 4),
+              ((36, 24), (12, 8), "temporal", 4, 9, 2), ((36, 24), (12, 8), "temporal", 0, 7, 7),
+              ((36, 24), (12, 8), "fused", 0, 11, 3), ((36, 24), (12, 8), "exchange", 0, 7, 2),
+              ((64, 48), (64, 48), "resident", 0, 9, 4),
+              ((40, 36, 30), (20, 12, 10), "temporal", 3, 22, 5), ((40, 36, 30), (20, 12, 10), "temporal", 2, 9, 3),
+              ((40, 36, 30), (20, 12, 10), "temporal", 3, 10, 3), ((24, 18, 12), (8, 6, 4), "fused", 0, 7, 3)]
+
+
+@pytest.mark.parametrize("n,b,mode,tsteps,nsweeps,every", NORM_CASES)
+@pytest.mark.parametrize("has_f", [False, True])
+def test_norms_every_k_sweeps_from_the_sweeps_own_passes(jac, orc, n, b, mode, tsteps, nsweeps, every, has_f):
+    """jac_sweep_norms_async: the norm of the state after every, 2 * every, ... sweeps equals the oracle's
+    residual at that point, whichever level of whichever launch measures it, and the sweeps themselves
+    leave the oracle's bits."""
+    import torch
+    J, B = _setup_pair(jac, orc, n, b, 1, has_f, mode, seed=9, tsteps=tsteps)
+    need = (nsweeps - 1) // every
+    out = torch.full((max(need, 1) + 1,), -7.0, dtype=torch.float64).pin_memory()
+    J.sweep_norms_async(nsweeps, every, out if need else None)
+    torch.cuda.synchronize()
+    want = []
+    done = 0
+    while done < nsweeps:
+        k = min(every, nsweeps - done)
+        B.sweep(k)
+        done += k
+        if done < nsweeps:
+            want.append(B.residual())
+    assert len(want) == need
+    for m in range(need):
+        assert abs(float(out[m]) - want[m]) <= RESID_TOL * want[m], (m, float(out[m]), want[m])
+    assert float(out[need]) == -7.0                       # nothing written past the norms that are due
+    _assert_sweep_close(J.get_u(), B.get_u())
+    r, w = J.residual(), B.residual()
+    assert abs(r - w) <= RESID_TOL * w
+    J.close()
+    B.close()
+
+
 @pytest.mark.parametrize("mode", ["temporal", "fused", "exchange", "pertask", "resident", "wide"])
 def test_solve_stops_after_the_group_that_meets_the_tolerance(jac, orc, mode):
     """Groups of 3 sweeps, the tolerance met in the middle of a batch of queued groups (and, with a
