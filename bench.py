@@ -49,21 +49,21 @@ L2_BYTES = 126e6
 # its points -- traffic is proportional to the points: every strip or tile reads and writes its own
 # part of the grid once per launch.
 SWEEP_SOURCES = ("jac_kernels.cuh", "jac_temporal3d.cuh", "jac_resident.cuh", "jac_geom.h", "jac.cu")
-CAPTURE_SHA = "980f7b371eefd455"
+CAPTURE_SHA = "7211b707c087a97f"
 NCU_TRAFFIC = {
     # profiles/temporal2d_eigenmode_8192.md
-    ("temporal", 8, 2, False): {"bytes_per_point_per_launch": (606.670336e6 + 494.481152e6) / 8192 ** 2},
-    ("temporal", 4, 2, False): {"bytes_per_point_per_launch": (617.931520e6 + 489.596928e6) / 8192 ** 2},
+    ("temporal", 8, 2, False): {"bytes_per_point_per_launch": (606.731520e6 + 494.180608e6) / 8192 ** 2},
+    ("temporal", 4, 2, False): {"bytes_per_point_per_launch": (617.857024e6 + 489.936640e6) / 8192 ** 2},
     # profiles/temporal2d_poisson_4096.md (config 2 itself; its arrays are about the size of L2)
-    ("temporal", 6, 2, True): {"bytes_per_point_per_launch": (321.993216e6 + 103.352320e6) / 4096 ** 2},
+    ("temporal", 6, 2, True): {"bytes_per_point_per_launch": (321.955584e6 + 102.860032e6) / 4096 ** 2},
     # profiles/temporal3d_poisson_512.md
-    ("temporal", 3, 3, True): {"bytes_per_point_per_launch": (2.513648e9 + 1.050928e9) / 512 ** 3},
-    ("temporal", 2, 3, True): {"bytes_per_point_per_launch": (2.447557e9 + 1.049917e9) / 512 ** 3},
+    ("temporal", 3, 3, True): {"bytes_per_point_per_launch": (2.498106e9 + 1.050876e9) / 512 ** 3},
+    ("temporal", 2, 3, True): {"bytes_per_point_per_launch": (2.445537e9 + 1.049933e9) / 512 ** 3},
     # profiles/exchange_schedule_eigenmode_8192.md (the update launch alone)
-    ("exchange", 1, 2, False): {"bytes_per_point_per_launch": (574.191104e6 + 493.950720e6) / 8192 ** 2},
-    ("exchange", 1, 3, True): {"bytes_per_point_per_launch": (2.370614e9 + 1.048733e9) / 512 ** 3},
+    ("exchange", 1, 2, False): {"bytes_per_point_per_launch": (574.266624e6 + 494.105088e6) / 8192 ** 2},
+    ("exchange", 1, 3, True): {"bytes_per_point_per_launch": (2.370183e9 + 1.048935e9) / 512 ** 3},
     # profiles/resident_heated_edge_256.md (config 1 itself: the grid is read once, the result stays in L2)
-    ("resident", 0, 2, False): {"bytes_per_point_per_launch": 579.584e3 / 256 ** 2},
+    ("resident", 0, 2, False): {"bytes_per_point_per_launch": 579.328e3 / 256 ** 2},
 }
 for _rec in NCU_TRAFFIC.values():
     _rec.update(src=SWEEP_SOURCES, src_sha=CAPTURE_SHA)
