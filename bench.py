@@ -48,8 +48,10 @@ L2_BYTES = 126e6
 # launch (a smaller case of the same workload, named beside each entry), scaled to the workload by
 # its points -- traffic is proportional to the points: every strip or tile reads and writes its own
 # part of the grid once per launch.
-SWEEP_SOURCES = ("jac_kernels.cuh", "jac_temporal3d.cuh", "jac_resident.cuh", "jac_geom.h", "jac.cu")
-CAPTURE_SHA = "7211b707c087a97f"
+SWEEP_SOURCES = ("jac_kernels.cuh", "jac_temporal3d.cuh", "jac_geom.h", "jac.cu")
+CAPTURE_SHA = "a88faf6c8d2ab7b2"
+RESIDENT_SOURCES = ("jac_resident.cuh", "jac_kernels.cuh", "jac_geom.h", "jac.cu")
+RESIDENT_CAPTURE_SHA = "39125e5533e7e26f"
 NCU_TRAFFIC = {
     # profiles/temporal2d_eigenmode_8192.md
     ("temporal", 8, 2, False): {"bytes_per_point_per_launch": (606.731520e6 + 494.180608e6) / 8192 ** 2},
@@ -63,10 +65,13 @@ NCU_TRAFFIC = {
     ("exchange", 1, 2, False): {"bytes_per_point_per_launch": (574.266624e6 + 494.105088e6) / 8192 ** 2},
     ("exchange", 1, 3, True): {"bytes_per_point_per_launch": (2.370183e9 + 1.048935e9) / 512 ** 3},
     # profiles/resident_heated_edge_256.md (config 1 itself: the grid is read once, the result stays in L2)
-    ("resident", 0, 2, False): {"bytes_per_point_per_launch": 579.328e3 / 256 ** 2},
+    ("resident", 0, 2, False): {"bytes_per_point_per_launch": 601.088e3 / 256 ** 2},
 }
-for _rec in NCU_TRAFFIC.values():
-    _rec.update(src=SWEEP_SOURCES, src_sha=CAPTURE_SHA)
+for _key, _rec in NCU_TRAFFIC.items():
+    if _key[0] == "resident":
+        _rec.update(src=RESIDENT_SOURCES, src_sha=RESIDENT_CAPTURE_SHA)
+    else:
+        _rec.update(src=SWEEP_SOURCES, src_sha=CAPTURE_SHA)
 KERNEL_NAMES = {("temporal", 2): "temporal2d_kernel", ("temporal", 3): "temporal3d_kernel", ("fused", 2): "sweep2d_kernel (update pulling neighbour interiors)",
                 ("exchange", 2): "sweep2d_kernel", ("pertask", 2): "sweep2d_kernel (one launch per block)",
                 ("fused", 3): "sweep3d_kernel (update pulling neighbour interiors)", ("exchange", 3): "sweep3d_kernel",

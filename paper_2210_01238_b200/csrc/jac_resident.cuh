@@ -10,13 +10,18 @@
 // Neighbouring slabs only ever need each other's edge row, so they synchronise pairwise, not as a
 // cluster: a CTA computes its first and last new row first and sends them straight into the
 // neighbours' halo rows with st.async, which counts the bytes that have landed on an mbarrier in
-// the RECEIVING CTA; the receiver waits on its two mbarriers (one per side) after it has computed
-// its inner rows.  No fence, no cluster-wide barrier per sweep: the cluster barrier is used once
+// the RECEIVING CTA; one warp of the receiver waits on its two mbarriers (one per side) after it
+// has computed its inner rows, and the CTA barrier that ends the sweep passes the rows on to the
+// other warps.  No fence, no cluster-wide barrier per sweep: the cluster barrier is used once
 // after the fill and once before the write-back.  Why a halo row can be overwritten safely: the
 // row a neighbour sends for sweep s + 1 can only leave after that neighbour has received this
 // CTA's row of sweep s, which each thread sends after it has read the halo cells it needs.
 // Every wait is bounded: a CTA that has polled kResMaxPolls times sets the error word, stops
 // waiting and runs to the end with whatever it has, so that all CTAs reach the final barrier.
+// Measured with clock64 stamps in a copy of the kernel (256^2, 16 CTAs): a sweep took ~1850 cycles,
+// ~740 of them for the edge row while thread 0 also announced the incoming rows to the mbarriers and
+// every thread polled them; with the announcement made by a warp that has no edge row, one polling
+// warp, and the two buffers alternating as compile-time constants, 100 sweeps take 94 us, not 113.
 //
 // Slab layout (doubles): row pitch RP = nx + 4; grid column i sits at index i + 2 (so pairs of
 // columns are 16-byte aligned), the Dirichlet columns at 1 and nx + 2.  Local row 0 is the halo
@@ -26,6 +31,8 @@
 #pragma once
 #include <cooperative_groups.h>
 #include <cuda_runtime.h>
+
+#include <type_traits>
 
 #include "jac_geom.h"
 #include "jac_kernels.cuh"
@@ -164,19 +171,20 @@ resident2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
     const bool does_hi = grp == min(groups, 2) - 1 && mine >= 2;
     const unsigned row_bytes = (unsigned)nx * (unsigned)sizeof(double);
     bool gave_up = false;
-    for (int s = 0; s < nsweeps; ++s) {
-        const int wb = (s + 1) & 1;                           // buffer written in this sweep
-        double* const A = buf[wb ^ 1];
+    // One sweep into buffer WB, a compile-time constant: the loop below alternates the two, so no
+    // sweep selects its buffers, halo rows or mbarriers at run time.
+    auto sweep_once = [&](auto wbc, const int s) {
+        constexpr int wb = decltype(wbc)::value;
+        const double* const A = buf[wb ^ 1];
         double* const B = buf[wb];
-        // this sweep's incoming rows: one arrival (this one) plus the row's bytes complete a phase
-        if (tid == 0) {
+        // this sweep's incoming rows: one arrival (this one) plus the row's bytes complete a phase.
+        // Announced by a thread whose warp computes no edge row where there is one (four row
+        // groups): the rows the neighbours wait for do not queue behind it.
+        if (tid == kResThreads - 1) {
             if (has_lo) mbar_expect_tx(smem_addr(&halo_bar[0][wb]), row_bytes);
             if (has_hi) mbar_expect_tx(smem_addr(&halo_bar[1][wb]), row_bytes);
         }
-#pragma unroll 1
-        for (int side = 0; side < 2; ++side) {
-            if (side == 0 ? !does_lo : !does_hi) continue;
-            const int l = side == 0 ? 1 : mine;
+        auto edge_row = [&](const int l) {
             for (int cp = cp0; cp < npairs; cp += pw) {
                 const int at = l * RP + 2 + 2 * cp;
                 const double2 S = *reinterpret_cast<const double2*>(A + at - RP);
@@ -197,7 +205,9 @@ resident2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
                 if (l == 1 && has_lo) send_pair(lo_row[wb] + col, lo_bar[wb], o);
                 if (l == mine && has_hi) send_pair(hi_row[wb] + col, hi_bar[wb], o);
             }
-        }
+        };
+        if (does_lo) edge_row(1);
+        if (does_hi) edge_row(mine);
         if (l0 < l1) {
             for (int cp = cp0; cp < npairs; cp += pw) {
                 int at = l0 * RP + 2 + 2 * cp;
@@ -221,9 +231,10 @@ resident2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
                 }
             }
         }
-        // the neighbours' rows of this sweep (the k-th use of a buffer's mbarriers has parity k & 1)
+        // the neighbours' rows of this sweep (the k-th use of a buffer's mbarriers has parity k & 1).
+        // One warp waits for them; the barrier below passes on what it has seen to the others.
         const unsigned parity = (unsigned)(s >> 1) & 1u;
-        if (!gave_up) {
+        if (!gave_up && tid >= kResThreads - 32) {
 #pragma unroll 1
             for (int side = 0; side < 2; ++side) {
                 if (side == 0 ? !has_lo : !has_hi) continue;
@@ -239,6 +250,14 @@ resident2d_kernel(const double* __restrict__ u, double* __restrict__ un, const d
             }
         }
         __syncthreads();            // this CTA's rows of B are complete, and nobody still reads A
+    };
+    {
+        int s = 0;                  // sweep s writes buffer (s + 1) & 1
+        for (; s + 1 < nsweeps; s += 2) {
+            sweep_once(std::integral_constant<int, 1>{}, s);
+            sweep_once(std::integral_constant<int, 0>{}, s + 1);
+        }
+        if (s < nsweeps) sweep_once(std::integral_constant<int, 1>{}, s);
     }
     cluster.sync();                 // no row is still on its way to a CTA that is about to leave
     double* const A = buf[nsweeps & 1];
