@@ -73,7 +73,7 @@ def test_parity_tests_pass_under_the_checked_build(checked_lib):
     suites with all addresses checked.  A context that recorded a violation raises when it is closed."""
     env = dict(os.environ, JAC_LIB=str(checked_lib))
     sel = ("test_sweep_matches_oracle or test_pack_and_unpack or test_temporal_blocking or fused_residual or "
-           "first_sweep or solve_stops or remainder or wide or resident or slab_contexts or cut_planes")
+           "first_sweep or norms_every or solve_stops or remainder or wide or resident or slab_contexts or cut_planes")
     r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-m", "gpu", "-k", sel,
                         "tests/test_gpu_parity.py", "tests/test_gpu_remainder.py", "tests/test_gpu_wide.py",
                         "tests/test_gpu_resident.py", "tests/test_gpu_slabs.py", "tests/test_gpu_staging.py"],

@@ -102,6 +102,9 @@ def test_nothing_outside_the_entitled_cells_is_written(jac, n, b, h, has_f, mode
     J.sweep_residual(3)
     out = torch.zeros(1, dtype=torch.float64).pin_memory()
     J.residual_sweep_async(4, out)
+    norms = torch.zeros(4, dtype=torch.float64).pin_memory()
+    J.sweep_norms_async(9, 2, norms)
+    J.sweep_norms_async(17, 8, norms)
     J.solve(7, 2, 0.0)
     J.get_u()
     J.stream.synchronize()
