@@ -49,23 +49,23 @@ L2_BYTES = 126e6
 # its points -- traffic is proportional to the points: every strip or tile reads and writes its own
 # part of the grid once per launch.
 SWEEP_SOURCES = ("jac_kernels.cuh", "jac_temporal3d.cuh", "jac_geom.h", "jac.cu")
-CAPTURE_SHA = "a88faf6c8d2ab7b2"
+CAPTURE_SHA = "22367cf9d08cf954"
 RESIDENT_SOURCES = ("jac_resident.cuh", "jac_kernels.cuh", "jac_geom.h", "jac.cu")
-RESIDENT_CAPTURE_SHA = "39125e5533e7e26f"
+RESIDENT_CAPTURE_SHA = "5bebd6c06a175820"
 NCU_TRAFFIC = {
     # profiles/temporal2d_eigenmode_8192.md
-    ("temporal", 8, 2, False): {"bytes_per_point_per_launch": (606.731520e6 + 494.180608e6) / 8192 ** 2},
-    ("temporal", 4, 2, False): {"bytes_per_point_per_launch": (617.857024e6 + 489.936640e6) / 8192 ** 2},
+    ("temporal", 8, 2, False): {"bytes_per_point_per_launch": (606.869248e6 + 494.355200e6) / 8192 ** 2},
+    ("temporal", 4, 2, False): {"bytes_per_point_per_launch": (617.974528e6 + 489.620224e6) / 8192 ** 2},
     # profiles/temporal2d_poisson_4096.md (config 2 itself; its arrays are about the size of L2)
-    ("temporal", 6, 2, True): {"bytes_per_point_per_launch": (321.955584e6 + 102.860032e6) / 4096 ** 2},
+    ("temporal", 6, 2, True): {"bytes_per_point_per_launch": (322.085632e6 + 103.113216e6) / 4096 ** 2},
     # profiles/temporal3d_poisson_512.md
-    ("temporal", 3, 3, True): {"bytes_per_point_per_launch": (2.498106e9 + 1.050876e9) / 512 ** 3},
-    ("temporal", 2, 3, True): {"bytes_per_point_per_launch": (2.445537e9 + 1.049933e9) / 512 ** 3},
+    ("temporal", 3, 3, True): {"bytes_per_point_per_launch": (2.514893e9 + 1.050443e9) / 512 ** 3},
+    ("temporal", 2, 3, True): {"bytes_per_point_per_launch": (2.447718e9 + 1.050805e9) / 512 ** 3},
     # profiles/exchange_schedule_eigenmode_8192.md (the update launch alone)
-    ("exchange", 1, 2, False): {"bytes_per_point_per_launch": (574.266624e6 + 494.105088e6) / 8192 ** 2},
-    ("exchange", 1, 3, True): {"bytes_per_point_per_launch": (2.370183e9 + 1.048935e9) / 512 ** 3},
+    ("exchange", 1, 2, False): {"bytes_per_point_per_launch": (574.175488e6 + 494.808576e6) / 8192 ** 2},
+    ("exchange", 1, 3, True): {"bytes_per_point_per_launch": (2.370464e9 + 1.048717e9) / 512 ** 3},
     # profiles/resident_heated_edge_256.md (config 1 itself: the grid is read once, the result stays in L2)
-    ("resident", 0, 2, False): {"bytes_per_point_per_launch": 601.088e3 / 256 ** 2},
+    ("resident", 0, 2, False): {"bytes_per_point_per_launch": 600.832e3 / 256 ** 2},
 }
 for _key, _rec in NCU_TRAFFIC.items():
     if _key[0] == "resident":

@@ -1746,6 +1746,12 @@ int jac_sweep_norms_async(jac_ctx* c, int nsweeps, int every, double* host_out_l
         // whole run would have, and at most one level of a launch measures (every >= T).
         std::vector<int> depths;
         temporal_depths(nsweeps, T, c->g.ndim, c->desc.has_f != 0, &depths);
+        // The norms collect in the status words 8 .. 31 of the scratch and travel to the host 24 at a
+        // time: a copy of 8 bytes after every measuring launch would put a gap into the stream each
+        // time (a hundred of them in a job of 1000 sweeps with a norm every 10).
+        constexpr int kNormRing = 24;
+        double* const ring = c->result + 8;
+        int pending = 0, copied = 0;
         int a = 0;
         for (const int t : depths) {
             int j = (a + every - 1) / every * every;     // the first multiple of `every` not below a
@@ -1757,13 +1763,21 @@ int jac_sweep_norms_async(jac_ctx* c, int nsweeps, int every, double* host_out_l
             c->ghosts_fresh = false;
             c->packed_current = false;
             if (level) {
-                jac::reduce_partials_kernel<<<1, 1024, 0, c->stream>>>(c->partials, nparts, c->result, true);
+                // norm number j / every - 1 = copied + pending: they are due in order
+                jac::reduce_partials_kernel<<<1, 1024, 0, c->stream>>>(c->partials, nparts, ring + pending, true);
                 if ((rc = check_launch(c))) return rc;
-                JAC_CK(c, cudaMemcpyAsync(host_out_l2 + (j / every - 1), c->result, sizeof(double),
-                                          cudaMemcpyDeviceToHost, c->stream));
+                if (++pending == kNormRing) {
+                    JAC_CK(c, cudaMemcpyAsync(host_out_l2 + copied, ring, pending * sizeof(double),
+                                              cudaMemcpyDeviceToHost, c->stream));
+                    copied += pending;
+                    pending = 0;
+                }
             }
             a += t;
         }
+        if (pending)
+            JAC_CK(c, cudaMemcpyAsync(host_out_l2 + copied, ring, pending * sizeof(double), cudaMemcpyDeviceToHost,
+                                      c->stream));
         return JAC_OK;
     }
     // every other case group by group: the norm of the state a group starts from comes out of the

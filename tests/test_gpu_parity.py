@@ -342,10 +342,11 @@ def test_residual_from_the_first_sweep_s_pass(jac, orc, n, b, h, mode, tsteps, h
 
 
 # (n, b, mode, tsteps, nsweeps, every): norms due inside launches (every > T, no multiple of T), at
-# launch borders (every = T), every < T (group by group), nothing due (nsweeps <= every)
+# launch borders (every = T), every < T (group by group), nothing due (nsweeps <= every), many norms
 NORM_CASES = [((120, 40), (60, 20), "temporal", 3, 23, 5), ((256, 100), (64, 25), "temporal", 8, 50, 10),
               ((256, 100), (64, 25), "temporal", 6, 31, 10), ((1100, 200), (220, 50), "temporal", 4, 17, 4),
               ((36, 24), (12, 8), "temporal", 4, 9, 2), ((36, 24), (12, 8), "temporal", 0, 7, 7),
+              ((120, 40), (60, 20), "temporal", 2, 110, 2),      # 54 norms: more than travel in one copy
               ((36, 24), (12, 8), "fused", 0, 11, 3), ((36, 24), (12, 8), "exchange", 0, 7, 2),
               ((64, 48), (64, 48), "resident", 0, 9, 4),
               ((40, 36, 30), (20, 12, 10), "temporal", 3, 22, 5), ((40, 36, 30), (20, 12, 10), "temporal", 2, 9, 3),
